@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the STA+GSTA forward pass:  python bench.py --gpus N --steps K --warmup W [--workload cfg3]
+
+One "step" is one laser_forward call (projections, fused segment attention, GSTA) over one batch of seeded
+synthetic inputs of a named configuration.  Prints ONE JSON line (rank 0).
+
+  value        user x candidate scores per second, whole job, inputs resident in HBM
+  e2e          the same metric through laser_forward_host with pinned HOST buffers (H2D + D2H in the timed region)
+  roofline     the dominant kernel's algorithmic work / its CUDA-event duration, against the measured peak
+  cpu_baseline the float64 numpy oracle timed on this machine's host cores on a bounded sample of the same workload
+
+--impl reference times the oracle alone (there is no reference implementation to install for this paper).
+With torchrun (N > 1) every rank runs the same configuration on its own batch (seed offset = rank); users are
+independent, so there is no data-path collective: only the barrier and the max-over-ranks of the device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "user x candidate scores/sec for STA+GSTA fwd"
+UNIT = "scores/s"
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ----------------------------------------------------------------------------------------------------- helpers
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK)
+    p["_source"] = "fallback"
+    return p
+
+
+def algorithmic_work(w):
+    """Algorithmic flops / bytes of one step (valid items only; 2 flops per multiply-accumulate)."""
+    s = w.spec
+    lens = w.lengths.astype(np.int64)
+    ncand = (w.cand_offsets[1:] - w.cand_offsets[:-1]).astype(np.int64)
+    nseg = -(-lens // s.S)
+    esz = 4 if s.dtype == "f32" else 2
+    proj = 2 * int(lens.sum()) * s.d * (s.d_qk + s.d)
+    attn = 2 * int((lens * ncand).sum()) * (s.d_qk + s.d)
+    gates = int((lens * ncand).sum()) * s.H
+    gsta = s.M * int((ncand * (6 * s.d * s.d + 4 * s.H * nseg * s.d)).sum())
+    io_bytes = (int(lens.sum()) * s.d + 2 * int(ncand.sum()) * s.d) * esz
+    return {"proj_flops": proj, "attn_flops": attn, "gate_evals": gates, "gsta_flops": gsta, "io_bytes": io_bytes,
+            "valid_items": int(lens.sum()), "scores": int(ncand.sum())}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(w, budget_users=None):
+    """Users forming a bounded sample for the CPU oracle (a prefix of the batch), sized by a rough cost model so
+    that the run takes on the order of 10-30 s."""
+    s = w.spec
+    cost = w.lengths.astype(np.float64) * 0 + s.L  # the oracle projects and gates all L rows of a user
+    ncand = (w.cand_offsets[1:] - w.cand_offsets[:-1]).astype(np.float64)
+    per_user = cost * (ncand * s.H * 40.0 + s.d * (s.d_qk + s.d) * 2.0) + ncand * s.M * s.n_seg * 4.0 * s.d * s.d
+    target = 4e10 if budget_users is None else None   # ~ flop-equivalents for roughly 10-30 s of numpy float64
+    users, acc = [], 0.0
+    for u in range(s.U):
+        if budget_users is not None and len(users) >= budget_users:
+            break
+        if target is not None and users and acc + per_user[u] > target:
+            break
+        users.append(u)
+        acc += per_user[u]
+    return users
+
+
+def time_oracle(w, users):
+    from oracle import laser_oracle
+    s = w.spec
+    t0 = time.perf_counter()
+    laser_oracle.forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H, w.gamma, w.tau,
+                         users=users, return_hprime=False)
+    dt = time.perf_counter() - t0
+    scores = int(sum(int(w.cand_offsets[u + 1] - w.cand_offsets[u]) for u in users))
+    return dt, scores
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ----------------------------------------------------------------------------------------------------- arms
+def run_reference(args, rank, world):
+    """The oracle as it stands, on the host cores; each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    from workloads import make_workload
+    w = make_workload(args.workload)
+    users = oracle_sample(w)
+    # shrink the sample so that warmup + steps stay within a few minutes
+    dt0, sc0 = time_oracle(w, users[:1])
+    per_user = max(dt0, 1e-3)
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    users = users[:max(1, min(len(users), int(budget / per_user)))]
+    for _ in range(args.warmup):
+        time_oracle(w, users)
+    tot_t, tot_s = 0.0, 0
+    for _ in range(args.steps):
+        dt, sc = time_oracle(w, users)
+        tot_t += dt
+        tot_s += sc
+    value = tot_s / tot_t
+    sample = f"users 0..{len(users) - 1} of {w.spec.U} of {w.spec.name} per step ({tot_s // max(1, args.steps)} scores)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.spec.name, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def dominant_kernel_roofline(w, prof, peaks):
+    """Roofline entry for the kernel with the largest share of the step."""
+    work = algorithmic_work(w)
+    if not prof:
+        return None
+    name, ms = max(prof.items(), key=lambda kv: kv[1])
+    sec = ms * 1e-3
+    src = "of measured" if peaks["_source"] == "measured" else "of fallback"
+    if name.startswith("stream"):
+        achieved = work["io_bytes"] / sec / 1e9
+        peak = peaks["hbm_gbs"]
+        return {"kernel": name, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": src, "ms": ms,
+                "frac_of_nominal": achieved / NOMINAL["hbm_gbs"]}
+    if name.startswith("sta"):
+        flops = work["attn_flops"]
+    elif name.startswith("proj"):
+        flops = work["proj_flops"]
+    else:
+        flops = work["gsta_flops"]
+    achieved = flops / sec / 1e12
+    peak = peaks["bf16_tflops"]
+    return {"kernel": name, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": achieved / peak, "traffic": None, "peak_source": src, "ms": ms,
+            "frac_of_nominal": achieved / NOMINAL["bf16_tflops"],
+            "gate_evals_per_s": work["gate_evals"] / sec if name.startswith("sta") else None}
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2602_11562_b200 as P
+    from workloads import make_workload
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    P.load_library()   # fails loudly if the CUDA library is missing
+    peaks = load_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = make_workload(args.workload, seed_offset=rank)
+    s = w.spec
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device=dev)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device=dev)
+    z = torch.empty((b.cfg.total_cands, s.d), dtype=b.items.dtype, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    def step():
+        P.laser_forward(b.cfg, *b.args(), b.Wg, z=z, workspace=ws, stream=stream)
+
+    # parity on sampled users before any timing (rank 0 only; the oracle runs on the host)
+    parity = None
+    cpu_base = None
+    if rank == 0:
+        step()
+        assert P.laser_check_status(ws) == 0
+        users = oracle_sample(w)
+        dt, scores = time_oracle(w, users)
+        from oracle import laser_oracle
+        _, z_ref = laser_oracle.forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
+                                        w.gamma, w.tau, users=users[:2], return_hprime=False)
+        rows = np.arange(int(w.cand_offsets[0]), int(w.cand_offsets[min(2, len(users))]))
+        got = z.float().cpu().numpy().astype(np.float64)[rows]
+        err = float(np.max(np.abs(got - z_ref[rows]) / np.maximum(1.0, np.abs(z_ref[rows])))) if rows.size else 0.0
+        tol = 1e-4 if s.dtype == "f32" else 2e-2
+        if not (err <= tol):
+            raise SystemExit(f"parity failure before timing: z error {err:.3e} > {tol}")
+        parity = {"z_err": err, "tol": tol, "users_checked": min(2, len(users))}
+        cpu_base = {"value": scores / dt, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+                    "sample": f"users 0..{len(users) - 1} of {s.U} ({scores} scores) of {s.name}, {dt:.1f} s"}
+
+    for _ in range(max(3, args.warmup)):
+        flush.fill_(1)
+        step()
+    launches_per_step = P.laser_last_launch_count()
+
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for e0, e1 in evs:
+        flush.fill_(1)          # evict the previous step's data from L2 (outside the timed bracket)
+        e0.record(stream)
+        step()
+        e1.record(stream)
+    barrier()
+    dev_ms = sum(e0.elapsed_time(e1) for e0, e1 in evs)
+
+    # per-kernel durations (CUDA events recorded by the library around each launch), same step, same flush
+    P.laser_profile_enable(True)
+    prof = {}
+    for _ in range(args.steps):
+        flush.fill_(1)
+        step()
+        for name, ms in P.laser_profile_read():
+            prof[name] = prof.get(name, 0.0) + ms / args.steps
+    P.laser_profile_enable(False)
+
+    # end to end: pinned host buffers in, z out, through laser_forward_host
+    hb = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device="cpu", pin_host=True)
+    hws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device=dev)
+    z_h = torch.empty((hb.cfg.total_cands, s.d), dtype=hb.items.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (hb.items, hb.lengths, hb.cands, hb.cand_offsets, hb.Wq, hb.Wk,
+                                                    hb.Wv, hb.Wg))
+    d2h = z_h.numel() * z_h.element_size()
+    for _ in range(2):
+        P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, hws, stream=stream, blocking=True)
+    barrier()
+    e2e_steps = max(1, min(args.steps, 20))
+    t0 = time.perf_counter()
+    ee = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e2e_steps)]
+    for e0, e1 in ee:
+        e0.record(stream)
+        P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, hws, stream=stream, blocking=False)
+        e1.record(stream)
+    barrier()
+    e2e_ms = sum(e0.elapsed_time(e1) for e0, e1 in ee)
+    clocks = sampler.stop()
+
+    if world > 1:
+        t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dev_ms, e2e_ms = float(t[0]), float(t[1])
+        n_scores = torch.tensor([w.N], dtype=torch.float64, device=dev)
+        dist.all_reduce(n_scores)
+        total_scores = float(n_scores[0])
+    else:
+        total_scores = float(w.N)
+
+    if rank == 0:
+        ms_per_step = dev_ms / args.steps
+        work = algorithmic_work(w)
+        roof = dominant_kernel_roofline(w, prof, peaks)
+        line = {"metric": METRIC, "value": total_scores / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32" if s.dtype == "f32" else "bf16", "data": "synthetic",
+                "config": {"workload": s.name, "users": s.U, "cands_per_user": s.C, "L": s.L, "d": s.d, "heads": s.H,
+                           "d_qk": s.d_qk, "seg_size": s.S, "gsta_layers": s.M, "valid_items": work["valid_items"],
+                           "l2": "flushed between timed steps (256 MB write)", "parallelism": f"dp{world} by user"},
+                "e2e": {"value": total_scores / (e2e_ms / e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps},
+                "gpu_launches": launches_per_step * args.steps,
+                "clocks": clocks,
+                "roofline": roof,
+                "kernels_ms": prof,
+                "cpu_baseline": cpu_base,
+                "parity": parity,
+                "work": work}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

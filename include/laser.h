@@ -1,0 +1,167 @@
+/*
+ * laser.h -- C ABI of the B200 (sm_100a) forward pass of LASER's Segmented Target Attention (STA)
+ * followed by Global Stacked Target Attention (GSTA).
+ *
+ * What is computed (paper sections "Fine-grained Target-aware Compression", "Global Target Attention over
+ * Compressed Sequence" and "Global Attention with Segmented Aggregation"):
+ *
+ *   STA   For user u with items x_0..x_{len-1} in R^d and each of its candidates t in R^d:
+ *           q = t W_q,  k_n = x_n W_k,  v_n = x_n W_v                                   (Eq. 4 / Eq. 8-9)
+ *           alpha_{n,h} = Sigmoid(q_h . k_{n,h} / gamma)          one gate per item and head   (Eq. 5 / Eq. 10)
+ *           s_i[head h] = sum over the items n of segment i (n < len) of alpha_{n,h} v_{n,h}   (Eq. 11-12)
+ *         Segment i holds items [i*S, (i+1)*S) (Eq. 3); L' = ceil(L / S); H' = [s_0 .. s_{L'-1}] in R^{L' x d}.
+ *   GSTA  t_0 = t;  for l = 1..M, per head: a = softmax_j((t_{l-1} W_q^l)_h . (s_j W_k^l)_h / tau) over the
+ *         non-empty segments j, o_l[head h] = sum_j a_j (s_j W_v^l)_h,  t_l = t_{l-1} + o_l;  z = t_M.   (Eq. 7)
+ *
+ * Conventions where the paper gives none: heads split the columns of W_q, W_k ([d, d_qk]) and of W_v and
+ * the GSTA weights ([d, d]) into H contiguous slices, head outputs are concatenated, there is no output
+ * projection and no bias; an item at or beyond a user's length contributes exactly nothing (whatever the
+ * padded rows contain, as long as it is finite); a segment without valid items yields a zero row of H' and
+ * takes no part in the GSTA softmax; a user of length 0 yields H' = 0 and z = t.  No FFN / LayerNorm
+ * (Eq. 6) sits between the two stages.
+ *
+ * General rules for every entry point
+ *   - Unless stated otherwise every pointer is a DEVICE pointer to memory owned by the caller; the library
+ *     never allocates, frees or keeps a pointer after the call returns, and never synchronises (except
+ *     laser_check_status and laser_forward_host's final wait when `blocking` is non-zero).
+ *   - All arrays are dense row-major with the innermost index contiguous; base pointers must be 16-byte
+ *     aligned.  Floating-point arrays (items, candidates, weights, H', z) all have the config's dtype.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t cast to void*; NULL = the legacy default stream).
+ *   - Return value: LASER_OK, or a negative laser_status for an error the host can see (bad argument,
+ *     unsupported shape, workspace too small, a CUDA launch error).  Nothing is launched after such an
+ *     error.  Errors that only the device can see (a length outside [0, L], candidate offsets that are not
+ *     non-decreasing within [0, N], a bounded wait that ran out) are written to a status word at the
+ *     start of the workspace, make the affected kernels skip the offending work, and are returned by
+ *     laser_check_status.
+ *   - Weights are right-multiplied: y = x W, W stored [in, out].
+ *   - There is no CPU fallback: a shape outside the supported envelope returns LASER_ERR_UNSUPPORTED.
+ *   - Calls that use the same workspace must not overlap on the GPU; distinct workspaces may run
+ *     concurrently on distinct streams.
+ */
+#ifndef LASER_H_
+#define LASER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LASER_API __attribute__((visibility("default")))
+#else
+#define LASER_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { LASER_F32 = 0, LASER_BF16 = 1 } laser_dtype;
+
+typedef enum {
+  LASER_OK = 0,
+  LASER_ERR_INVALID_ARG = -1,
+  LASER_ERR_UNSUPPORTED = -2,
+  LASER_ERR_WORKSPACE = -3,
+  LASER_ERR_CUDA = -4,
+  LASER_ERR_TIMEOUT = -5,   /* a bounded device-side wait gave up (device-reported) */
+  LASER_ERR_BAD_INPUT = -6  /* a length or candidate offset out of range (device-reported) */
+} laser_status;
+
+/* Which kernels carry the path.  AUTO picks: F32 -> SIMT; BF16 -> STREAM when no user has more than one
+ * candidate, otherwise TENSOR. */
+typedef enum {
+  LASER_PATH_AUTO = 0,
+  LASER_PATH_SIMT = 1,    /* FP32-ALU kernels, fp32 arithmetic for either dtype (the only F32 path)       */
+  LASER_PATH_TENSOR = 2,  /* BF16: tcgen05 / TMEM / TMA kernels, bf16 operands, fp32 accumulation         */
+  LASER_PATH_STREAM = 3   /* BF16, at most one candidate per user: one HBM-streaming pass over the items  */
+} laser_path;
+
+typedef struct laser_config {
+  int32_t num_users;          /* U >= 0                                                                   */
+  int32_t max_len;            /* L >= 1: rows of each user's item block (its row stride)                  */
+  int32_t d_model;            /* d: embedding width of items, candidates, H' and z                        */
+  int32_t d_qk;               /* STA query/key width, = num_heads * d_qh (the paper's d_q; 16 per head)   */
+  int32_t num_heads;          /* H >= 1, divides d_model and d_qk                                         */
+  int32_t seg_size;           /* S >= 1, the paper's w;  L' = ceil(L / S)                                 */
+  int32_t num_gsta_layers;    /* M >= 0, the paper's L_stack                                              */
+  int32_t dtype;              /* laser_dtype                                                              */
+  int32_t total_cands;        /* N = cand_offsets[U]                                                      */
+  int32_t max_cands_per_user; /* an upper bound of cand_offsets[u+1] - cand_offsets[u] (sizes launch grids) */
+  int32_t path;               /* laser_path                                                               */
+  float sta_gamma;            /* gamma of Eq. 5;  <= 0 selects sqrt(d_qk / H)                             */
+  float gsta_scale;           /* tau, the divisor of Eq. 7;  <= 0 selects sqrt(d / H)                     */
+} laser_config;
+
+/* Bytes of device scratch that laser_sta_forward / laser_gsta_forward / laser_forward need for `cfg`
+ * (the maximum over the three; includes room for an internal H' when laser_forward is not given one).
+ * Returns 0 if cfg is NULL or invalid.  Host-only, launches nothing. */
+LASER_API size_t laser_workspace_bytes(const laser_config* cfg);
+
+/* STA (Eq. 3-5 in the global form Eq. 8-12).
+ *   items        [U, L, d]   item embeddings; rows >= lengths[u] of user u are ignored (must be finite)
+ *   lengths      [U] int32   valid prefix length of each user, 0..L
+ *   cands        [N, d]      candidate (target) embeddings
+ *   cand_offsets [U+1] int32 user u owns candidates [cand_offsets[u], cand_offsets[u+1])
+ *   Wq, Wk       [d, d_qk];  Wv [d, d]
+ *   Hprime       [N, L', d]  OUT: every row is written (zero rows for empty segments)
+ *   workspace    device scratch of at least laser_workspace_bytes(cfg) bytes, 256-byte aligned
+ */
+LASER_API int laser_sta_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                      const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* GSTA (Eq. 7 and the residual update t_l = t_{l-1} + o_l), M = cfg->num_gsta_layers layers over a
+ * caller-supplied H'.
+ *   Hprime  [N, L', d]    segment vectors (rows of empty segments are not read)
+ *   Wgsta   [M, 3, d, d]  per layer W_q^l, W_k^l, W_v^l
+ *   z       [N, d]        OUT
+ */
+LASER_API int laser_gsta_forward(const laser_config* cfg, const void* Hprime, const int32_t* lengths,
+                       const int32_t* cand_offsets, const void* cands, const void* Wgsta, void* z,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* STA followed by GSTA.  Hprime may be NULL (H' is then kept in the workspace or never materialised);
+ * when non-NULL it receives the same values laser_sta_forward would write. */
+LASER_API int laser_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                  const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
+                  void* Hprime, void* z, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Device scratch laser_forward_host needs: laser_workspace_bytes(cfg) plus staging for every input and z. */
+LASER_API size_t laser_host_workspace_bytes(const laser_config* cfg);
+
+/* laser_forward for callers whose data lives in HOST memory (the end-to-end path): copies the inputs to
+ * the device, runs laser_forward without H' output, copies z back.
+ *   items_h, lengths_h, cands_h, cand_offsets_h, Wq_h, Wk_h, Wv_h, Wgsta_h : HOST pointers, same shapes
+ *       and dtype as above (pinned memory makes the copies asynchronous; pageable memory also works)
+ *   z_h        HOST pointer, OUT [N, d]
+ *   workspace  DEVICE scratch of at least laser_host_workspace_bytes(cfg) bytes
+ *   blocking   non-zero: wait for the stream and return the device status too; zero: return after enqueue
+ *              (z_h is valid once the stream has drained)
+ */
+LASER_API int laser_forward_host(const laser_config* cfg, const void* items_h, const int32_t* lengths_h,
+                       const void* cands_h, const int32_t* cand_offsets_h, const void* Wq_h, const void* Wk_h,
+                       const void* Wv_h, const void* Wgsta_h, void* z_h, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream, int blocking);
+
+/* Waits for `cuda_stream`, reads the device status word at the start of `workspace` and returns it
+ * (LASER_OK, LASER_ERR_TIMEOUT, LASER_ERR_BAD_INPUT) or LASER_ERR_CUDA if the stream reports an error. */
+LASER_API int laser_check_status(const void* workspace, void* cuda_stream);
+
+/* Number of kernels the last successful call on this host thread enqueued (launch accounting for benchmarks). */
+LASER_API int laser_last_launch_count(void);
+
+/* Per-kernel timing for benchmarks (state is per host thread).  laser_profile_enable(1) makes every later
+ * forward call on this thread bracket each of its kernel launches with CUDA events recorded on the call's
+ * stream (the first such call creates the events); laser_profile_enable(0) turns that off again.
+ * laser_profile_read waits for the last profiled call's kernels and writes, for up to `max_kernels` of them
+ * in launch order, the duration in milliseconds to ms_out[i] (HOST) and a static name to names_out[i] (HOST);
+ * it returns how many entries it wrote, or a negative laser_status. */
+LASER_API int laser_profile_enable(int on);
+LASER_API int laser_profile_read(int max_kernels, float* ms_out, const char** names_out);
+
+/* Static description of a laser_status value. */
+LASER_API const char* laser_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LASER_H_ */

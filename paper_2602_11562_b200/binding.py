@@ -1,0 +1,263 @@
+"""ctypes binding of liblaser.so: same names as the C entry points, torch tensors in place of raw pointers.
+
+Only marshalling happens here (pointer extraction, shape / dtype / contiguity checks, workspace and output
+allocation through torch).  Every arithmetic step of the path runs inside the library's CUDA kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_STREAM = 0, 1, 2, 3
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+_LIB: Optional[ctypes.CDLL] = None
+
+
+class LaserError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__(f"{where}: {laser_status_string(status)} (status {status})")
+
+
+class LaserConfig(ctypes.Structure):
+    """Mirror of `laser_config` in include/laser.h."""
+    _fields_ = [
+        ("num_users", ctypes.c_int32), ("max_len", ctypes.c_int32), ("d_model", ctypes.c_int32),
+        ("d_qk", ctypes.c_int32), ("num_heads", ctypes.c_int32), ("seg_size", ctypes.c_int32),
+        ("num_gsta_layers", ctypes.c_int32), ("dtype", ctypes.c_int32), ("total_cands", ctypes.c_int32),
+        ("max_cands_per_user", ctypes.c_int32), ("path", ctypes.c_int32),
+        ("sta_gamma", ctypes.c_float), ("gsta_scale", ctypes.c_float),
+    ]
+
+    @property
+    def n_seg(self) -> int:
+        return -(-self.max_len // self.seg_size)
+
+    def torch_dtype(self):
+        return torch.float32 if self.dtype == DTYPE_F32 else torch.bfloat16
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaser.so")
+
+
+def load_library() -> ctypes.CDLL:
+    """Load liblaser.so (built by `python -m paper_2602_11562_b200.build`). There is no fallback."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2602_11562_b200.build` "
+                           "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(path)
+    vp, i32p, cfgp, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(LaserConfig), ctypes.c_size_t
+    lib.laser_workspace_bytes.restype = sz
+    lib.laser_workspace_bytes.argtypes = [cfgp]
+    lib.laser_host_workspace_bytes.restype = sz
+    lib.laser_host_workspace_bytes.argtypes = [cfgp]
+    lib.laser_sta_forward.restype = ctypes.c_int
+    lib.laser_sta_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, sz, vp]
+    lib.laser_gsta_forward.restype = ctypes.c_int
+    lib.laser_gsta_forward.argtypes = [cfgp, vp, i32p, i32p, vp, vp, vp, vp, sz, vp]
+    lib.laser_forward.restype = ctypes.c_int
+    lib.laser_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.laser_forward_host.restype = ctypes.c_int
+    lib.laser_forward_host.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.c_int]
+    lib.laser_check_status.restype = ctypes.c_int
+    lib.laser_check_status.argtypes = [vp, vp]
+    lib.laser_last_launch_count.restype = ctypes.c_int
+    lib.laser_last_launch_count.argtypes = []
+    lib.laser_profile_enable.restype = ctypes.c_int
+    lib.laser_profile_enable.argtypes = [ctypes.c_int]
+    lib.laser_profile_read.restype = ctypes.c_int
+    lib.laser_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_char_p)]
+    lib.laser_status_string.restype = ctypes.c_char_p
+    lib.laser_status_string.argtypes = [ctypes.c_int]
+    _LIB = lib
+    return lib
+
+
+def make_config(*, num_users, max_len, d_model, d_qk, num_heads, seg_size, num_gsta_layers, dtype, total_cands,
+                max_cands_per_user, path=PATH_AUTO, sta_gamma=0.0, gsta_scale=0.0) -> LaserConfig:
+    if isinstance(dtype, str):
+        dtype = {"f32": DTYPE_F32, "bf16": DTYPE_BF16}[dtype]
+    return LaserConfig(num_users, max_len, d_model, d_qk, num_heads, seg_size, num_gsta_layers, dtype, total_cands,
+                       max_cands_per_user, path, float(sta_gamma), float(gsta_scale))
+
+
+def laser_status_string(status: int) -> str:
+    return load_library().laser_status_string(int(status)).decode()
+
+
+def laser_workspace_bytes(cfg: LaserConfig) -> int:
+    return int(load_library().laser_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_host_workspace_bytes(cfg: LaserConfig) -> int:
+    return int(load_library().laser_host_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_last_launch_count() -> int:
+    return int(load_library().laser_last_launch_count())
+
+
+def laser_profile_enable(on: bool) -> None:
+    load_library().laser_profile_enable(1 if on else 0)
+
+
+def laser_profile_read(max_kernels: int = 16):
+    """[(kernel name, milliseconds)] of the last profiled call on this thread, in launch order."""
+    ms = (ctypes.c_float * max_kernels)()
+    names = (ctypes.c_char_p * max_kernels)()
+    n = load_library().laser_profile_read(max_kernels, ms, names)
+    _check(min(n, 0), "laser_profile_read")
+    return [(names[i].decode(), float(ms[i])) for i in range(n)]
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _workspace(cfg: LaserConfig, workspace, device, host: bool = False) -> torch.Tensor:
+    need = laser_host_workspace_bytes(cfg) if host else laser_workspace_bytes(cfg)
+    if need == 0:
+        raise LaserError(-1, "laser_workspace_bytes (invalid or unsupported configuration)")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise LaserError(rc, where)
+
+
+def laser_sta_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime=None, workspace=None, stream=None):
+    """STA: returns H' [N, L', d]. All tensors live on the GPU; see include/laser.h for shapes."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    ws = _workspace(cfg, workspace, items.device)
+    if Hprime is None:
+        Hprime = torch.empty((cfg.total_cands, cfg.n_seg, cfg.d_model), dtype=dt, device=items.device)
+    rc = lib.laser_sta_forward(ctypes.byref(cfg), _dev(items, dt, "items"), _dev(lengths, torch.int32, "lengths"),
+                               _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                               _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Hprime, dt, "Hprime"),
+                               ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_sta_forward")
+    return Hprime
+
+
+def laser_gsta_forward(cfg, Hprime, lengths, cand_offsets, cands, Wgsta, z=None, workspace=None, stream=None):
+    """GSTA over a given H': returns z [N, d]."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    ws = _workspace(cfg, workspace, Hprime.device)
+    if z is None:
+        z = torch.empty((cfg.total_cands, cfg.d_model), dtype=dt, device=Hprime.device)
+    rc = lib.laser_gsta_forward(ctypes.byref(cfg), _dev(Hprime, dt, "Hprime"), _dev(lengths, torch.int32, "lengths"),
+                                _dev(cand_offsets, torch.int32, "cand_offsets"), _dev(cands, dt, "cands"),
+                                _dev(Wgsta, dt, "Wgsta"), _dev(z, dt, "z"), ws.data_ptr(), ws.numel(),
+                                _stream_ptr(stream))
+    _check(rc, "laser_gsta_forward")
+    return z
+
+
+def laser_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, Hprime=None, z=None, workspace=None,
+                  stream=None, want_hprime=False):
+    """STA + GSTA: returns z, or (H', z) when want_hprime / an Hprime buffer is given."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    ws = _workspace(cfg, workspace, items.device)
+    if z is None:
+        z = torch.empty((cfg.total_cands, cfg.d_model), dtype=dt, device=items.device)
+    if Hprime is None and want_hprime:
+        Hprime = torch.empty((cfg.total_cands, cfg.n_seg, cfg.d_model), dtype=dt, device=items.device)
+    rc = lib.laser_forward(ctypes.byref(cfg), _dev(items, dt, "items"), _dev(lengths, torch.int32, "lengths"),
+                           _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                           _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Wgsta, dt, "Wgsta"),
+                           None if Hprime is None else _dev(Hprime, dt, "Hprime"), _dev(z, dt, "z"),
+                           ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_forward")
+    return (Hprime, z) if Hprime is not None else z
+
+
+def _host(t: torch.Tensor, dtype, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError(f"{name}: expected a contiguous CPU tensor of {dtype}")
+    return t.data_ptr()
+
+
+def laser_forward_host(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, z, workspace, stream=None,
+                       blocking=True):
+    """End-to-end call on HOST tensors (ideally pinned): H2D copies, forward, D2H copy of z, inside the library."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    rc = lib.laser_forward_host(ctypes.byref(cfg), _host(items, dt, "items"), _host(lengths, torch.int32, "lengths"),
+                                _host(cands, dt, "cands"), _host(cand_offsets, torch.int32, "cand_offsets"),
+                                _host(Wq, dt, "Wq"), _host(Wk, dt, "Wk"), _host(Wv, dt, "Wv"),
+                                _host(Wgsta, dt, "Wgsta"), _host(z, dt, "z"), workspace.data_ptr(), workspace.numel(),
+                                _stream_ptr(stream), 1 if blocking else 0)
+    _check(rc, "laser_forward_host")
+    return z
+
+
+def laser_check_status(workspace: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream and returns the device-side status word (0 = ok)."""
+    return int(load_library().laser_check_status(workspace.data_ptr(), _stream_ptr(stream)))
+
+
+@dataclass
+class DeviceBatch:
+    """A workload's arrays as device tensors of the configuration dtype, plus the matching laser_config."""
+    cfg: LaserConfig
+    items: torch.Tensor
+    lengths: torch.Tensor
+    cands: torch.Tensor
+    cand_offsets: torch.Tensor
+    Wq: torch.Tensor
+    Wk: torch.Tensor
+    Wv: torch.Tensor
+    Wg: torch.Tensor
+
+    @staticmethod
+    def from_numpy(*, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wg, S, H, M, dtype, gamma=0.0, tau=0.0,
+                   path=PATH_AUTO, device="cuda", pin_host=False) -> "DeviceBatch":
+        import numpy as np
+        dt = torch.float32 if dtype in ("f32", DTYPE_F32) else torch.bfloat16
+        U, L, d = items.shape
+        offs = np.asarray(cand_offsets, dtype=np.int64)
+        N = int(offs[-1])
+        maxc = int(np.max(offs[1:] - offs[:-1])) if U > 0 else 0
+        cfg = make_config(num_users=U, max_len=L, d_model=d, d_qk=Wq.shape[1], num_heads=H, seg_size=S,
+                          num_gsta_layers=M, dtype=DTYPE_F32 if dt == torch.float32 else DTYPE_BF16, total_cands=N,
+                          max_cands_per_user=maxc, path=path, sta_gamma=gamma, gsta_scale=tau)
+
+        def up(a, tdt):
+            t = torch.from_numpy(np.ascontiguousarray(a)).to(tdt)
+            if device == "cpu":
+                return t.pin_memory() if pin_host else t
+            return t.to(device)
+
+        return DeviceBatch(cfg, up(items, dt), up(np.asarray(lengths, dtype=np.int32), torch.int32), up(cands, dt),
+                           up(np.asarray(cand_offsets, dtype=np.int32), torch.int32), up(Wq, dt), up(Wk, dt),
+                           up(Wv, dt), up(Wg, dt))
+
+    @staticmethod
+    def from_workload(w, path=PATH_AUTO, device="cuda", pin_host=False) -> "DeviceBatch":
+        s = w.spec
+        return DeviceBatch.from_numpy(items=w.items, lengths=w.lengths, cands=w.cands, cand_offsets=w.cand_offsets,
+                                      Wq=w.Wq, Wk=w.Wk, Wv=w.Wv, Wg=w.Wg, S=s.S, H=s.H, M=s.M, dtype=s.dtype,
+                                      gamma=w.gamma, tau=w.tau, path=path, device=device, pin_host=pin_host)
+
+    def args(self):
+        return (self.items, self.lengths, self.cands, self.cand_offsets, self.Wq, self.Wk, self.Wv)

@@ -1,0 +1,332 @@
+// extern "C" entry points: argument validation, path selection, workspace carve-up, dispatch.
+#include <math.h>
+#include <string.h>
+
+#include "laser_common.cuh"
+
+namespace laser {
+
+constexpr int kMaxProfiled = 16;
+static thread_local int g_launches = 0;
+static thread_local bool g_profile = false;
+static thread_local int g_prof_n = 0;
+static thread_local const char* g_prof_name[kMaxProfiled];
+static thread_local cudaEvent_t g_prof_ev[2 * kMaxProfiled];
+static thread_local bool g_prof_ev_made = false;
+
+void reset_launch_count() { g_launches = 0; g_prof_n = 0; }
+
+LaunchScope::LaunchScope(const char* name, cudaStream_t st) : st_(st), slot_(-1) {
+  ++g_launches;
+  if (!g_profile || g_prof_n >= kMaxProfiled) return;
+  if (!g_prof_ev_made) {
+    for (int i = 0; i < 2 * kMaxProfiled; ++i)
+      if (cudaEventCreate(&g_prof_ev[i]) != cudaSuccess) return;
+    g_prof_ev_made = true;
+  }
+  slot_ = g_prof_n++;
+  g_prof_name[slot_] = name;
+  cudaEventRecord(g_prof_ev[2 * slot_], st_);
+}
+LaunchScope::~LaunchScope() {
+  if (slot_ >= 0) cudaEventRecord(g_prof_ev[2 * slot_ + 1], st_);
+}
+
+static int resolve_path(const Plan& p, int requested) {
+  if (requested == LASER_PATH_AUTO) {
+    if (p.dtype == LASER_F32) return LASER_PATH_SIMT;
+    if (p.maxC <= 1 && stream_supported(p)) return LASER_PATH_STREAM;
+    if (tensor_supported(p)) return LASER_PATH_TENSOR;
+    return LASER_PATH_SIMT;
+  }
+  if (requested == LASER_PATH_SIMT) return LASER_PATH_SIMT;
+  if (requested == LASER_PATH_TENSOR) return tensor_supported(p) ? (int)LASER_PATH_TENSOR : (int)LASER_ERR_UNSUPPORTED;
+  if (requested == LASER_PATH_STREAM) return (p.maxC <= 1 && stream_supported(p)) ? (int)LASER_PATH_STREAM : (int)LASER_ERR_UNSUPPORTED;
+  return LASER_ERR_INVALID_ARG;
+}
+
+int make_plan(const laser_config* c, Plan* p) {
+  if (!c || !p) return LASER_ERR_INVALID_ARG;
+  memset(p, 0, sizeof(*p));
+  if (c->num_users < 0 || c->max_len < 1 || c->d_model < 1 || c->d_qk < 1 || c->num_heads < 1 || c->seg_size < 1 ||
+      c->num_gsta_layers < 0 || c->total_cands < 0 || c->max_cands_per_user < 0)
+    return LASER_ERR_INVALID_ARG;
+  if (c->dtype != LASER_F32 && c->dtype != LASER_BF16) return LASER_ERR_INVALID_ARG;
+  if (c->d_model % c->num_heads || c->d_qk % c->num_heads) return LASER_ERR_INVALID_ARG;
+  if (c->max_cands_per_user > c->total_cands) return LASER_ERR_INVALID_ARG;
+  if (c->total_cands > 0 && (c->max_cands_per_user == 0 || c->num_users == 0)) return LASER_ERR_INVALID_ARG;
+  p->U = c->num_users; p->L = c->max_len; p->d = c->d_model; p->dqk = c->d_qk; p->H = c->num_heads;
+  p->S = c->seg_size; p->M = c->num_gsta_layers; p->dtype = c->dtype; p->N = c->total_cands;
+  p->maxC = c->max_cands_per_user;
+  p->Lp = (p->L + p->S - 1) / p->S;
+  p->dqh = p->dqk / p->H; p->dvh = p->d / p->H;
+  const float gamma = c->sta_gamma > 0.f ? c->sta_gamma : sqrtf((float)p->dqh);
+  const float tau = c->gsta_scale > 0.f ? c->gsta_scale : sqrtf((float)p->dvh);
+  p->inv_gamma = 1.f / gamma; p->inv_tau = 1.f / tau;
+  p->esize = p->dtype == LASER_F32 ? 4 : 2;
+  if ((size_t)p->N * p->Lp * p->d >= ((size_t)1 << 40)) return LASER_ERR_UNSUPPORTED;
+
+  const int path = resolve_path(*p, c->path);
+  if (path < 0) return path;
+  p->path = path;
+
+  size_t off = 0;
+  p->off_status = off; off = align_up(off + kStatusWords * sizeof(int));
+  p->off_hp = off; off = align_up(off + (size_t)p->N * p->Lp * p->d * p->esize);
+  if (path == LASER_PATH_SIMT) {
+    p->off_q = off; off = align_up(off + (size_t)p->N * p->dqk * sizeof(float));
+    p->off_k = off; off = align_up(off + (size_t)p->U * p->L * p->dqk * sizeof(float));
+    p->off_v = off; off = align_up(off + (size_t)p->U * p->L * p->d * sizeof(float));
+  } else if (path == LASER_PATH_TENSOR) {
+    tensor_geometry(*p, &p->tg);
+    const TensorGeom& g = p->tg;
+    const size_t q_tiles = (size_t)g.cand_tiles_max;
+    p->off_tq = off; off = align_up(off + q_tiles * 128 * p->dqk * 2);
+    p->off_tk = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->dqk * 2);
+    p->off_tv = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->d * 2);
+    p->off_tsv = off; off = align_up(off + (size_t)p->U * p->Lp * p->d * sizeof(float));
+    p->off_twork = off; off = align_up(off + ((size_t)p->U * 4 + 64) * sizeof(int));
+    p->off_tcount = off; off = align_up(off + 64 * sizeof(int));
+  } else if (path == LASER_PATH_STREAM) {
+    p->off_su = off; off = align_up(off + (size_t)p->U * (p->H * p->d + p->H * p->H * p->d + 8) * sizeof(float));
+  }
+  p->total = off;
+  return LASER_OK;
+}
+
+static bool aligned16(const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; }
+
+static int check_ptrs(std::initializer_list<const void*> ptrs) {
+  for (const void* q : ptrs) {
+    if (!q) return LASER_ERR_INVALID_ARG;
+    if (!aligned16(q)) return LASER_ERR_INVALID_ARG;
+  }
+  return LASER_OK;
+}
+
+static int check_ws(const Plan& p, const void* ws, size_t bytes) {
+  if (!ws) return LASER_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & (kAlign - 1)) return LASER_ERR_INVALID_ARG;
+  if (bytes < p.total) return LASER_ERR_WORKSPACE;
+  return LASER_OK;
+}
+
+static int clear_status(const Plan& p, char* ws, cudaStream_t st) {
+  LASER_CUDA_OK(cudaMemsetAsync(ws + p.off_status, 0, kStatusWords * sizeof(int), st));
+  return LASER_OK;
+}
+
+static int run_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hp, char* ws,
+                   cudaStream_t st) {
+  switch (p.path) {
+    case LASER_PATH_SIMT: return simt_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+    case LASER_PATH_TENSOR: return tensor_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+    default: return LASER_ERR_UNSUPPORTED;
+  }
+}
+
+static int run_gsta(const Plan& p, const void* Hp, const int32_t* lengths, const int32_t* cand_offsets,
+                    const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st) {
+  switch (p.path) {
+    case LASER_PATH_SIMT: return simt_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+    case LASER_PATH_TENSOR: return tensor_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+    default: return LASER_ERR_UNSUPPORTED;
+  }
+}
+
+static int forward_impl(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                        const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wg,
+                        void* Hprime, void* z, char* ws, cudaStream_t st) {
+  int rc = clear_status(p, ws, st);
+  if (rc != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  if (p.path == LASER_PATH_STREAM)
+    return stream_forward(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wg, Hprime, z, ws, st);
+  void* Hp = Hprime ? Hprime : (void*)(ws + p.off_hp);
+  rc = run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+  if (rc != LASER_OK) return rc;
+  return run_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+}
+
+}  // namespace laser
+
+using namespace laser;
+
+extern "C" {
+
+size_t laser_workspace_bytes(const laser_config* cfg) {
+  Plan p;
+  if (make_plan(cfg, &p) != LASER_OK) return 0;
+  return p.total;
+}
+
+int laser_sta_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                      const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (p.path == LASER_PATH_STREAM) return LASER_ERR_UNSUPPORTED;   // the streaming path only exists fused
+  if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({items, cands, Wq, Wk, Wv, Hprime})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  return run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
+}
+
+int laser_gsta_forward(const laser_config* cfg, const void* Hprime, const int32_t* lengths,
+                       const int32_t* cand_offsets, const void* cands, const void* Wgsta, void* z, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (p.path == LASER_PATH_STREAM) return LASER_ERR_UNSUPPORTED;
+  if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({Hprime, cands, z})) != LASER_OK) return rc;
+  if (p.N > 0 && p.M > 0 && (rc = check_ptrs({Wgsta})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  return run_gsta(p, Hprime, lengths, cand_offsets, cands, Wgsta, z, ws, st);
+}
+
+int laser_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                  const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
+                  void* Hprime, void* z, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({items, cands, Wq, Wk, Wv, z})) != LASER_OK) return rc;
+  if (p.N > 0 && p.M > 0 && (rc = check_ptrs({Wgsta})) != LASER_OK) return rc;
+  if (Hprime && !aligned16(Hprime)) return LASER_ERR_INVALID_ARG;
+  return forward_impl(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, Hprime, z,
+                      static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
+}
+
+namespace {
+struct HostStage {
+  size_t items, lengths, cands, offs, wq, wk, wv, wg, z, total;
+  size_t b_items, b_lengths, b_cands, b_offs, b_wq, b_wk, b_wv, b_wg, b_z;
+};
+HostStage host_stage(const Plan& p) {
+  HostStage s;
+  s.b_items = (size_t)p.U * p.L * p.d * p.esize;
+  s.b_lengths = (size_t)p.U * sizeof(int32_t);
+  s.b_cands = (size_t)p.N * p.d * p.esize;
+  s.b_offs = (size_t)(p.U + 1) * sizeof(int32_t);
+  s.b_wq = s.b_wk = (size_t)p.d * p.dqk * p.esize;
+  s.b_wv = (size_t)p.d * p.d * p.esize;
+  s.b_wg = (size_t)p.M * 3 * p.d * p.d * p.esize;
+  s.b_z = (size_t)p.N * p.d * p.esize;
+  size_t off = p.total;
+  s.items = off; off = align_up(off + s.b_items);
+  s.lengths = off; off = align_up(off + s.b_lengths);
+  s.cands = off; off = align_up(off + s.b_cands);
+  s.offs = off; off = align_up(off + s.b_offs);
+  s.wq = off; off = align_up(off + s.b_wq);
+  s.wk = off; off = align_up(off + s.b_wk);
+  s.wv = off; off = align_up(off + s.b_wv);
+  s.wg = off; off = align_up(off + s.b_wg);
+  s.z = off; off = align_up(off + s.b_z);
+  s.total = off;
+  return s;
+}
+}  // namespace
+
+size_t laser_host_workspace_bytes(const laser_config* cfg) {
+  Plan p;
+  if (make_plan(cfg, &p) != LASER_OK) return 0;
+  return host_stage(p).total;
+}
+
+int laser_forward_host(const laser_config* cfg, const void* items_h, const int32_t* lengths_h, const void* cands_h,
+                       const int32_t* cand_offsets_h, const void* Wq_h, const void* Wk_h, const void* Wv_h,
+                       const void* Wgsta_h, void* z_h, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                       int blocking) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
+  const HostStage s = host_stage(p);
+  if (workspace_bytes < s.total) return LASER_ERR_WORKSPACE;
+  if (!lengths_h || !cand_offsets_h) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (!items_h || !cands_h || !Wq_h || !Wk_h || !Wv_h || !z_h || (p.M > 0 && !Wgsta_h)))
+    return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  auto h2d = [&](size_t off, const void* src, size_t bytes) -> cudaError_t {
+    if (!bytes) return cudaSuccess;
+    return cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, st);
+  };
+  LASER_CUDA_OK(h2d(s.lengths, lengths_h, s.b_lengths));
+  LASER_CUDA_OK(h2d(s.offs, cand_offsets_h, s.b_offs));
+  if (p.N > 0) {
+    LASER_CUDA_OK(h2d(s.items, items_h, s.b_items));
+    LASER_CUDA_OK(h2d(s.cands, cands_h, s.b_cands));
+    LASER_CUDA_OK(h2d(s.wq, Wq_h, s.b_wq));
+    LASER_CUDA_OK(h2d(s.wk, Wk_h, s.b_wk));
+    LASER_CUDA_OK(h2d(s.wv, Wv_h, s.b_wv));
+    LASER_CUDA_OK(h2d(s.wg, Wgsta_h, s.b_wg));
+  }
+  rc = forward_impl(p, ws + s.items, reinterpret_cast<const int32_t*>(ws + s.lengths), ws + s.cands,
+                    reinterpret_cast<const int32_t*>(ws + s.offs), ws + s.wq, ws + s.wk, ws + s.wv, ws + s.wg, nullptr,
+                    ws + s.z, ws, st);
+  if (rc != LASER_OK) return rc;
+  if (s.b_z) LASER_CUDA_OK(cudaMemcpyAsync(z_h, ws + s.z, s.b_z, cudaMemcpyDeviceToHost, st));
+  if (blocking) return laser_check_status(workspace, cuda_stream);
+  return LASER_OK;
+}
+
+int laser_check_status(const void* workspace, void* cuda_stream) {
+  if (!workspace) return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return LASER_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LASER_ERR_CUDA;
+  return word;
+}
+
+int laser_last_launch_count(void) { return g_launches; }
+
+int laser_profile_enable(int on) {
+  g_profile = on != 0;
+  return LASER_OK;
+}
+
+int laser_profile_read(int max_kernels, float* ms_out, const char** names_out) {
+  if (max_kernels < 0 || (max_kernels > 0 && (!ms_out || !names_out))) return LASER_ERR_INVALID_ARG;
+  const int n = g_prof_n < max_kernels ? g_prof_n : max_kernels;
+  for (int i = 0; i < n; ++i) {
+    if (cudaEventSynchronize(g_prof_ev[2 * i + 1]) != cudaSuccess) return LASER_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms_out[i], g_prof_ev[2 * i], g_prof_ev[2 * i + 1]) != cudaSuccess) return LASER_ERR_CUDA;
+    names_out[i] = g_prof_name[i];
+  }
+  return n;
+}
+
+const char* laser_status_string(int status) {
+  switch (status) {
+    case LASER_OK: return "ok";
+    case LASER_ERR_INVALID_ARG: return "invalid argument";
+    case LASER_ERR_UNSUPPORTED: return "shape or path not supported";
+    case LASER_ERR_WORKSPACE: return "workspace too small";
+    case LASER_ERR_CUDA: return "CUDA runtime error";
+    case LASER_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case LASER_ERR_BAD_INPUT: return "a length or candidate offset is out of range";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+// Shared host-side plan (validated configuration + workspace carve-up) and small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "laser.h"
+
+namespace laser {
+
+constexpr int kStatusWords = 64;          // int32 words reserved at the start of every workspace
+constexpr size_t kAlign = 256;
+
+// Tile geometry of the tensor-core path (defined by laser_tensor.cu, used by the plan for sizing).
+struct TensorGeom {
+  int IT;        // items per tile (multiple of 16, <= 128)
+  int NT;        // tiles per segment
+  int n_tiles;   // tiles per user = L' * NT
+  int cand_tiles_max;  // upper bound on 128-candidate tiles over all users
+};
+
+struct Plan {
+  int U, L, d, dqk, H, S, M, dtype, N, maxC, path;
+  int Lp, dqh, dvh;
+  float inv_gamma, inv_tau;
+  size_t esize;
+  // workspace byte offsets
+  size_t off_status;
+  size_t off_q, off_k, off_v;      // SIMT: fp32 Q [N,dqk], K [U,L,dqk], V [U,L,d]
+  size_t off_hp;                   // internal H' [N,Lp,d] in the I/O dtype
+  // tensor path
+  TensorGeom tg;
+  size_t off_tq, off_tk, off_tv, off_tsv, off_twork, off_tcount;
+  // stream path
+  size_t off_su;
+  size_t total;
+};
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+// Validates cfg and fills the plan. Returns LASER_OK or a negative status.
+int make_plan(const laser_config* cfg, Plan* p);
+
+// Launch accounting (thread-local).  Every kernel launch sits inside a LaunchScope: it counts the launch and, when
+// profiling is enabled through laser_profile_enable, brackets it with CUDA events on the launching stream.
+void reset_launch_count();
+class LaunchScope {
+ public:
+  LaunchScope(const char* name, cudaStream_t st);
+  ~LaunchScope();
+ private:
+  cudaStream_t st_;
+  int slot_;
+};
+
+// --- per-path launchers (each returns LASER_OK / LASER_ERR_*) -------------------------------------------------------
+int simt_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+             const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
+int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
+              const void* Wg, void* z, char* ws, cudaStream_t st);
+
+bool tensor_supported(const Plan& p);
+void tensor_geometry(const Plan& p, TensorGeom* g);
+int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
+int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
+                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st);
+
+bool stream_supported(const Plan& p);
+int stream_forward(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wg,
+                   void* Hprime, void* z, char* ws, cudaStream_t st);
+
+// --- device helpers ---------------------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ void report_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+#define LASER_CUDA_OK(expr)                          \
+  do {                                               \
+    cudaError_t _e = (expr);                         \
+    if (_e != cudaSuccess) return LASER_ERR_CUDA;    \
+  } while (0)
+
+}  // namespace laser

@@ -1,0 +1,158 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 oracle, element by element.
+
+Bar: max |g - r| / max(1, |r|) <= 1e-4 for fp32 and <= 2e-2 for bf16 (fp32 accumulation), on H' and on z."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_11562_b200 as P
+from oracle import laser_oracle
+from workloads import make_custom, make_workload, round_to_dtype
+
+from _util import TOL, cand_rows, err_metric, oracle_forward, to_np
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"simt": P.PATH_SIMT, "tensor": P.PATH_TENSOR, "stream": P.PATH_STREAM, "auto": P.PATH_AUTO}
+
+
+def _path_available(batch_cfg) -> bool:
+    return P.laser_workspace_bytes(batch_cfg) > 0
+
+
+def run_forward(w, path, want_hprime=True):
+    b = P.DeviceBatch.from_workload(w, path=PATHS[path])
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    out = P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=ws, want_hprime=want_hprime)
+    assert P.laser_check_status(ws) == 0
+    return out
+
+
+def check_against_oracle(w, path, users=None, what=("hp", "z")):
+    tol = TOL[w.spec.dtype]
+    Hp_ref, z_ref = oracle_forward(w, users=users)
+    Hp, z = run_forward(w, path)
+    rows = slice(None) if users is None else cand_rows(w, users)
+    e_hp = err_metric(to_np(Hp)[rows], Hp_ref[rows])
+    e_z = err_metric(to_np(z)[rows], z_ref[rows])
+    assert e_hp <= tol, f"H' error {e_hp:.3e} > {tol}"
+    assert e_z <= tol, f"z error {e_z:.3e} > {tol}"
+    return e_hp, e_z
+
+
+SMALL = [
+    # U, C, L, d, H, S, M, d_qh, lengths
+    dict(U=1, C=16, L=256, d=32, H=1, S=32, M=1, d_qh=16, lengths=None),
+    dict(U=3, C=5, L=70, d=32, H=2, S=16, M=2, d_qh=16, lengths=[70, 33, 1]),        # ragged, L % S != 0
+    dict(U=2, C=37, L=96, d=64, H=4, S=24, M=2, d_qh=16, lengths=[0, 96]),           # an empty user, S % 16 != 0
+    dict(U=2, C=3, L=48, d=64, H=2, S=48, M=3, d_qh=16, lengths=[48, 20]),           # one segment (S = L)
+    dict(U=4, C=1, L=100, d=64, H=2, S=10, M=1, d_qh=16, lengths=[100, 9, 10, 11]),  # one candidate per user, S = 10
+    dict(U=1, C=130, L=300, d=128, H=4, S=100, M=2, d_qh=16, lengths=[250]),         # >128 candidates, S = 100
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_small_shapes_simt(case, dtype):
+    kw = dict(SMALL[case])
+    # N(0,1) embeddings (the fp32 configuration's distribution) for d = 32; N(0,1/d) for wider d, where N(0,1)
+    # inputs give GSTA logits of magnitude ~50 whose fp32 rounding alone exceeds 1e-4 after the softmax
+    std = "one" if (dtype == "f32" and kw["d"] <= 32) else "inv_sqrt_d"
+    w = make_custom(dtype=dtype, seed=100 + case, emb_std=std, **kw)
+    check_against_oracle(w, "simt")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stage_entry_points_simt(dtype):
+    """laser_sta_forward and laser_gsta_forward on their own: GSTA is fed the oracle's H' (rounded to the dtype)."""
+    w = make_custom(U=2, C=9, L=80, d=64, H=4, S=16, M=2, dtype=dtype, seed=5, lengths=[80, 41])
+    s = w.spec
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_SIMT)
+    Hp = P.laser_sta_forward(b.cfg, *b.args())
+    Hp_ref = laser_oracle.sta_forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, s.S, s.H, w.gamma)
+    assert err_metric(to_np(Hp), Hp_ref) <= TOL[dtype]
+    Hp_in = round_to_dtype(Hp_ref.astype(np.float32), dtype)
+    z_ref = laser_oracle.gsta_forward(Hp_in, w.lengths, w.cand_offsets, w.cands, w.Wg, s.S, s.H, w.tau)
+    z = P.laser_gsta_forward(b.cfg, torch.from_numpy(Hp_in).to(b.items.dtype).cuda(), b.lengths, b.cand_offsets,
+                             b.cands, b.Wg)
+    assert err_metric(to_np(z), z_ref) <= TOL[dtype]
+
+
+def test_cfg1_tiny_fp32_full():
+    w = make_workload("cfg1")
+    e_hp, e_z = check_against_oracle(w, "auto")
+    assert max(e_hp, e_z) <= 1e-4
+
+
+def test_cfg2_serving_bf16_full_simt():
+    check_against_oracle(make_workload("cfg2"), "simt")
+
+
+def test_uneven_candidate_counts_and_users_without_candidates():
+    w = make_custom(U=4, C=4, L=64, d=32, H=2, S=16, M=1, dtype="f32", seed=3, lengths=[64, 10, 0, 33])
+    offs = np.array([0, 7, 7, 8, 16], dtype=np.int32)       # 7, 0, 1, 8 candidates
+    w.cand_offsets = offs
+    check_against_oracle(w, "simt")
+
+
+def test_padding_rows_never_influence_outputs_and_runs_are_deterministic():
+    w = make_custom(U=2, C=6, L=64, d=32, H=2, S=16, M=2, dtype="bf16", seed=8, lengths=[40, 5])
+    Hp1, z1 = run_forward(w, "simt")
+    Hp1b, z1b = run_forward(w, "simt")
+    assert torch.equal(Hp1, Hp1b) and torch.equal(z1, z1b)
+    w.items[0, 40:] = -123.0
+    w.items[1, 5:] = 0.015625
+    Hp2, z2 = run_forward(w, "simt")
+    assert torch.equal(Hp1, Hp2) and torch.equal(z1, z2)
+
+
+def test_no_candidates_is_a_no_op():
+    w = make_custom(U=2, C=0, L=32, d=32, H=1, S=8, M=1, dtype="f32", seed=1, lengths=[32, 3])
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_SIMT)
+    z = P.laser_forward(b.cfg, *b.args(), b.Wg)
+    assert tuple(z.shape) == (0, 32)
+
+
+def test_device_detected_bad_inputs_are_reported_not_faulted():
+    w = make_custom(U=2, C=3, L=32, d=32, H=1, S=8, M=1, dtype="f32", seed=1, lengths=[32, 3])
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_SIMT)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    bad_len = torch.tensor([33, 3], dtype=torch.int32, device="cuda")       # beyond L
+    P.laser_forward(b.cfg, b.items, bad_len, b.cands, b.cand_offsets, b.Wq, b.Wk, b.Wv, b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == -6
+    bad_off = torch.tensor([0, 9, 6], dtype=torch.int32, device="cuda")     # beyond N, decreasing
+    P.laser_forward(b.cfg, b.items, b.lengths, b.cands, bad_off, b.Wq, b.Wk, b.Wv, b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == -6
+    P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=ws)                   # the status word is cleared per call
+    assert P.laser_check_status(ws) == 0
+
+
+def test_host_detected_errors():
+    w = make_custom(U=1, C=2, L=32, d=32, H=1, S=8, M=1, dtype="f32", seed=1, lengths=[32])
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_SIMT)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.LaserError) as ei:
+        P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=small)
+    assert ei.value.status == -3
+    with pytest.raises(TypeError):
+        P.laser_forward(b.cfg, b.items.double(), b.lengths, b.cands, b.cand_offsets, b.Wq, b.Wk, b.Wv, b.Wg)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = make_custom(U=3, C=4, L=64, d=32, H=2, S=16, M=2, dtype="bf16", seed=21, lengths=[64, 17, 40])
+    z_dev = run_forward(w, "auto", want_hprime=False)
+    hb = P.DeviceBatch.from_workload(w, device="cpu", pin_host=True)
+    ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
+    z_h = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype).pin_memory()
+    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
+    assert torch.equal(z_h, z_dev.cpu())
+
+
+# ------------------------------------------------------------------ full-size configurations, sampled users
+@pytest.mark.parametrize("name,n_users", [("cfg3", 3), ("cfg4", 2), ("cfg5", 48)])
+def test_full_size_configs_sampled_users(name, n_users):
+    w = make_workload(name)
+    rng = np.random.default_rng(0)
+    order = np.argsort(w.lengths)
+    users = sorted({int(order[0]), int(order[-1]), *rng.choice(w.spec.U, size=n_users, replace=False).tolist()})
+    check_against_oracle(w, "auto", users=users)

@@ -1,0 +1,64 @@
+"""CPU-side checks of the C-ABI library: it builds, loads, exports every declared symbol, and its host-side
+argument validation answers without touching a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2602_11562_b200 as P
+from paper_2602_11562_b200 import build as laser_build
+
+
+@pytest.fixture(scope="module")
+def lib():
+    laser_build.build()
+    return P.load_library()
+
+
+def test_exports_every_declared_symbol(lib, repo_root):
+    hdr = open(os.path.join(repo_root, "include", "laser.h")).read()
+    names = re.findall(r"LASER_API\s+[\w\s\*]+?\b(laser_\w+)\s*\(", hdr)
+    assert len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_config_struct_matches_header(repo_root):
+    hdr = open(os.path.join(repo_root, "include", "laser.h")).read()
+    body = re.search(r"typedef struct laser_config \{(.*?)\} laser_config;", hdr, re.S).group(1)
+    fields = re.findall(r"^\s*(int32_t|float)\s+(\w+);", body, re.M)
+    assert [f[1] for f in fields] == [f[0] for f in P.LaserConfig._fields_]
+    assert ctypes.sizeof(P.LaserConfig) == 4 * len(fields)
+
+
+def _cfg(**kw):
+    base = dict(num_users=2, max_len=64, d_model=32, d_qk=16, num_heads=2, seg_size=16, num_gsta_layers=1,
+                dtype="f32", total_cands=6, max_cands_per_user=3)
+    base.update(kw)
+    return P.make_config(**base)
+
+
+def test_workspace_query_and_validation(lib):
+    assert P.laser_workspace_bytes(_cfg()) > 0
+    assert P.laser_host_workspace_bytes(_cfg()) > P.laser_workspace_bytes(_cfg())
+    assert P.laser_workspace_bytes(_cfg(num_heads=3)) == 0          # H must divide d and d_qk
+    assert P.laser_workspace_bytes(_cfg(seg_size=0)) == 0
+    assert P.laser_workspace_bytes(_cfg(dtype=7)) == 0
+    assert P.laser_workspace_bytes(_cfg(max_cands_per_user=9)) == 0  # larger than total
+    assert P.laser_workspace_bytes(_cfg(path=P.PATH_TENSOR)) == 0    # tensor path is bf16-only
+    # host-detectable errors come back as negative statuses before anything is launched
+    cfg = _cfg()
+    null = ctypes.c_void_p(0)
+    rc = lib.laser_forward(ctypes.byref(cfg), null, null, null, null, null, null, null, null, null, null, null, 0, null)
+    assert rc == -1
+    assert P.laser_status_string(rc) == "invalid argument"
+    assert "workspace" in P.laser_status_string(-3)
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2602_11562_b200 import binding
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "library_path", lambda: str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.load_library()
