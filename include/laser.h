@@ -125,6 +125,30 @@ LASER_API int laser_forward(const laser_config* cfg, const void* items, const in
                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
                   void* Hprime, void* z, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* STA without any workspace argument, for callers that cannot allocate device memory (no counterpart in the
+ * paper: this is a deployment convenience of this library).  Think of a plug-in inside a serving process
+ * whose GPU memory belongs entirely to the host framework's pool, or of a request thread that must never hit
+ * cudaMalloc's device-wide synchronisation: such a caller has inputs and an output buffer, but no scratch.
+ * This entry point computes exactly what laser_sta_forward computes with path = LASER_PATH_SIMT, and keeps
+ * the fp32 Q / K / V scratch in an array compiled into the library (LASER_STATIC_SCRATCH_BYTES per GPU that
+ * loads the library, held until the process exits).  It never calls cudaMalloc / cudaFree or any allocating
+ * routine.
+ *   - Size limit: 256 + 4*(N*d_qk + U*L*(d_qk + d)) bytes (each term rounded up to 256) must fit in
+ *     LASER_STATIC_SCRATCH_BYTES, otherwise LASER_ERR_WORKSPACE is returned and nothing is launched.
+ *   - cfg->path is ignored; items .. Hprime are as for laser_sta_forward.
+ *   - status_out: optional DEVICE int32; if non-NULL the device-side status word of this call (LASER_OK or
+ *     LASER_ERR_BAD_INPUT) is copied to it on the stream after the kernels.
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents (only the status
+ *     word is cleared per call): two calls that overlap on the GPU (different streams or threads) race.
+ *     Serialise them on one stream or with events. */
+#define LASER_STATIC_SCRATCH_BYTES (8u << 20)
+LASER_API int laser_sta_forward_static(const laser_config* cfg, const void* items, const int32_t* lengths,
+                                       const void* cands, const int32_t* cand_offsets, const void* Wq,
+                                       const void* Wk, const void* Wv, void* Hprime, int32_t* status_out,
+                                       void* cuda_stream);
+
 /* Device scratch laser_forward_host needs: laser_workspace_bytes(cfg) plus staging for every input and z. */
 LASER_API size_t laser_host_workspace_bytes(const laser_config* cfg);
 

@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     laser_workspace_bytes,
     laser_host_workspace_bytes,
     laser_sta_forward,
+    laser_sta_forward_static,
     laser_gsta_forward,
     laser_forward,
     laser_forward_host,

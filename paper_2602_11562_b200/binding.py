@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
     lib.laser_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.laser_forward_host.restype = ctypes.c_int
     lib.laser_forward_host.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.c_int]
+    lib.laser_sta_forward_static.restype = ctypes.c_int
+    lib.laser_sta_forward_static.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp]
     lib.laser_check_status.restype = ctypes.c_int
     lib.laser_check_status.argtypes = [vp, vp]
     lib.laser_last_launch_count.restype = ctypes.c_int
@@ -157,6 +159,22 @@ def laser_sta_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hpri
                                _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Hprime, dt, "Hprime"),
                                ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     _check(rc, "laser_sta_forward")
+    return Hprime
+
+
+def laser_sta_forward_static(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, status_out=None,
+                             stream=None):
+    """STA through the entry point that needs no workspace: for callers that cannot allocate device memory (all
+    scratch lives in a fixed array inside the library).  The caller supplies every buffer, including the output
+    Hprime [N, L', d] and, optionally, a one-element int32 device tensor that receives the device-side status."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    rc = lib.laser_sta_forward_static(ctypes.byref(cfg), _dev(items, dt, "items"),
+                                      _dev(lengths, torch.int32, "lengths"), _dev(cands, dt, "cands"),
+                                      _dev(cand_offsets, torch.int32, "cand_offsets"), _dev(Wq, dt, "Wq"),
+                                      _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Hprime, dt, "Hprime"),
+                                      None if status_out is None else _dev(status_out, torch.int32, "status_out"),
+                                      _stream_ptr(stream))
+    _check(rc, "laser_sta_forward_static")
     return Hprime
 
 
