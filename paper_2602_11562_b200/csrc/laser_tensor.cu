@@ -1,10 +1,777 @@
-// Tensor-core (tcgen05 / TMEM / TMA) path.  Placeholder until the kernels land: reports "not supported".
+// Tensor-core path (bf16 operands, fp32 accumulation) for sm_100a: tcgen05.mma with TMEM accumulators, bulk-TMA
+// staging through mbarrier rings, warp-specialised roles.
+//
+//   tc_prep_kernel   validates lengths / offsets, builds the unit and candidate-tile prefix arrays, zeroes the segment
+//                    value sums, and writes the transposed weight images in UMMA canonical layout.
+//   tc_proj_kernel   Eq. 8-9: K = X W_k, V = X W_v (and Q = T W_q / (2 gamma)) on the tensor cores.  Outputs are written
+//                    tile by tile in exactly the shared-memory layout the attention kernel's MMAs consume, so that
+//                    kernel stages them with plain bulk copies.  Also accumulates SV = sum of valid V rows per segment.
+//   tc_sta_kernel    Eq. 10-12 fused: per (user, 128-candidate tile, segment) and head,
+//                      scores = Q_h K_h^T (MMA, TMEM)  ->  P' = tanh(scores) (registers)  ->  O_h += P' V_h (MMA, TMEM)
+//                    and H' = (SV + O) / 2.  Uses Sigmoid(x) = 1/2 + 1/2 tanh(x/2): the 1/2 term is the candidate-
+//                    independent sum SV, the tanh term needs one transcendental and nothing else per gate.  Masked
+//                    items have zero K and V rows, so they contribute exactly nothing.  No score ever leaves the SM.
 #include "laser_common.cuh"
+#include "laser_ptx.cuh"
+
 namespace laser {
-bool tensor_supported(const Plan&) { return false; }
-void tensor_geometry(const Plan&, TensorGeom* g) { g->IT = 16; g->NT = 1; g->n_tiles = 0; g->cand_tiles_max = 0; }
-int tensor_sta(const Plan&, const void*, const int32_t*, const void*, const int32_t*, const void*, const void*,
-               const void*, void*, char*, cudaStream_t) { return LASER_ERR_UNSUPPORTED; }
-int tensor_gsta(const Plan&, const void*, const int32_t*, const int32_t*, const void*, const void*, void*, char*,
-                cudaStream_t) { return LASER_ERR_UNSUPPORTED; }
+namespace {
+
+using bf16 = __nv_bfloat16;
+using namespace ptx;
+
+constexpr int kCandTile = 128;        // candidates per tile = MMA M = TMEM lanes
+constexpr int kProjThreads = 128;
+constexpr int kProjTmemCols = 256;    // K / Q accumulator at column 0, V^T accumulator at column 128
+constexpr int kStaThreads = 512;
+constexpr int kStaTmemCols = 512;
+constexpr int kKvStages = 4;
+
+struct TcParams {
+  int U, L, d, dqk, H, S, Lp, N, dqh, dvh, maxC;
+  int IT, NT, NTG, NG, n_tiles;       // items per tile, tiles per segment, tiles per projection unit, units per segment
+  int cand_tiles_max;
+  float q_scale;                      // 1 / (2 gamma)
+  const bf16 *items, *cands, *Wq, *Wk, *Wv;
+  const int *lengths, *cand_offsets;
+  bf16 *Qblk, *Kblk, *Vtblk;
+  float* SV;                          // [U, Lp, d] sum of the valid (bf16-rounded) V rows of each segment
+  int *unit_start, *tile_off;         // [U+1] prefix of attention units / candidate tiles per user
+  int* counters;                      // [0] attention units, [1] candidate tiles, [2] projection ticket
+  bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
+  int* status;
+  bf16* Hp;
+};
+
+// Sanitised view of one user: invalid lengths / offsets behave like an empty user (and are reported by tc_prep_kernel).
+struct UserShape {
+  int len, c0, nc, nseg, ctiles;
+};
+__device__ __forceinline__ UserShape user_shape(const TcParams& P, int u) {
+  UserShape s;
+  int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
+  const bool bad = len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+  s.len = bad ? 0 : len;
+  s.c0 = bad ? 0 : c0;
+  s.nc = bad ? 0 : c1 - c0;
+  s.nseg = (s.len + P.S - 1) / P.S;
+  s.ctiles = (s.nc + kCandTile - 1) / kCandTile;
+  return s;
+}
+
+// Canonical K-major (no swizzle) element offset of (row, k) in a [rows x kdim] operand: 8x8-element core matrices of
+// 64 contiguous elements, core matrices of one 8-row group adjacent along k.
+__device__ __forceinline__ int canon_off(int row, int k, int kdim) {
+  return ((row >> 3) * (kdim >> 3) + (k >> 3)) * 64 + (row & 7) * 8 + (k & 7);
+}
+
+// ------------------------------------------------------------------------------------------------------- prep
+__global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0) {
+    __shared__ int sa[1024], sb[1024];
+    const int per = (P.U + 1023) / 1024;
+    const int u0 = min(tid * per, P.U), u1 = min(u0 + per, P.U);
+    int a = 0, b = 0;
+    bool bad = false;
+    for (int u = u0; u < u1; ++u) {
+      const int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
+      bad |= len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+      const UserShape s = user_shape(P, u);
+      a += s.ctiles;
+      b += s.ctiles * s.nseg;
+    }
+    if (bad) report_status(P.status, LASER_ERR_BAD_INPUT);
+    sa[tid] = a;
+    sb[tid] = b;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+      int va = 0, vb = 0;
+      if (tid >= off) { va = sa[tid - off]; vb = sb[tid - off]; }
+      __syncthreads();
+      sa[tid] += va;
+      sb[tid] += vb;
+      __syncthreads();
+    }
+    int pa = sa[tid] - a, pb = sb[tid] - b;   // exclusive prefixes
+    for (int u = u0; u < u1; ++u) {
+      const UserShape s = user_shape(P, u);
+      P.tile_off[u] = pa;
+      P.unit_start[u] = pb;
+      pa += s.ctiles;
+      pb += s.ctiles * s.nseg;
+    }
+    if (tid == 1023) {
+      P.tile_off[P.U] = sa[1023];
+      P.unit_start[P.U] = sb[1023];
+      P.counters[0] = sb[1023];
+      P.counters[1] = sa[1023];
+      P.counters[2] = 0;
+    }
+    return;
+  }
+  // remaining blocks: weight images and SV zero fill, grid-stride
+  const int nthreads = (gridDim.x - 1) * blockDim.x;
+  const int g = (blockIdx.x - 1) * blockDim.x + tid;
+  const int nK = P.dqk * P.d;
+  for (int i = g; i < nK; i += nthreads) {       // i = k * dqk + j  (coalesced read of W[k][j])
+    const int k = i / P.dqk, j = i - k * P.dqk;
+    const int o = canon_off(j, k, P.d);
+    P.imgK[o] = P.Wk[i];
+    P.imgQ[o] = P.Wq[i];
+  }
+  const int nV = kCandTile * P.d;
+  for (int i = g; i < nV; i += nthreads) {       // i = k * 128 + j ; rows j >= d are zero
+    const int k = i / kCandTile, j = i - k * kCandTile;
+    P.imgV[canon_off(j, k, P.d)] = j < P.d ? P.Wv[(size_t)k * P.d + j] : __float2bfloat16_rn(0.f);
+  }
+  const size_t nS = (size_t)P.U * P.Lp * P.d;
+  for (size_t i = g; i < nS; i += nthreads) P.SV[i] = 0.f;
+}
+
+// H' rows of segments without valid items are zero rows (only needed when the caller wants H').
+__global__ void __launch_bounds__(256) tc_zero_empty_kernel(TcParams P) {
+  const int u = blockIdx.y, seg = blockIdx.x;
+  const UserShape s = user_shape(P, u);
+  if (seg < s.nseg || s.nc == 0) return;
+  const int vec = P.d / 8;   // 16-byte chunks per row
+  for (int i = threadIdx.x; i < s.nc * vec; i += blockDim.x) {
+    const int c = i / vec, q = i - c * vec;
+    *reinterpret_cast<uint4*>(P.Hp + ((size_t)(s.c0 + c) * P.Lp + seg) * P.d + q * 8) = make_uint4(0, 0, 0, 0);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------- projection
+struct ProjSmem {
+  bf16 *imgK, *imgQ, *imgV, *X;
+};
+
+__global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ uint64_t bar_img, bar_mma;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_ticket;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int d = P.d, dqk = P.dqk;
+  bf16* imgK = reinterpret_cast<bf16*>(smem_raw);
+  bf16* imgQ = imgK + dqk * d;
+  bf16* imgV = imgQ + dqk * d;
+  bf16* X = imgV + kCandTile * d;
+
+  if (tid == 0) {
+    mbar_init(&bar_img, 1);
+    mbar_init(&bar_mma, 1);
+    s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&s_tmem, kProjTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+
+  if (tid == 0) {
+    const uint32_t bK = dqk * d * 2, bV = kCandTile * d * 2;
+    mbar_arrive_expect_tx(&bar_img, 2 * bK + bV);
+    bulk_g2s(imgK, P.imgK, bK, &bar_img);
+    bulk_g2s(imgQ, P.imgQ, bK, &bar_img);
+    bulk_g2s(imgV, P.imgV, bV, &bar_img);
+  }
+  bool ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
+
+  const int n_item_units = P.U * P.Lp * P.NG;
+  const int total_units = n_item_units + P.cand_tiles_max;
+  const int n_ctiles = P.counters[1];
+  const uint32_t sbo = (d >> 3) * 128, lbo = 128;
+  const uint32_t tmem_lane = tmem + ((uint32_t)(warp * 32) << 16);
+  uint32_t mma_phase = 0;
+
+  while (ok) {
+    __syncthreads();                       // previous unit fully drained (TMEM read, X consumed, s_ticket read)
+    if (tid == 0) s_ticket = atomicAdd(&P.counters[2], 1);
+    __syncthreads();
+    const int t = s_ticket;
+    if (t >= total_units) break;
+
+    // ---- decode the unit
+    bool is_item = t < n_item_units;
+    int u = 0, seg = 0, t0 = 0, rows = 0, jt = 0;
+    UserShape us;
+    if (is_item) {
+      u = t / (P.Lp * P.NG);
+      const int rem = t - u * (P.Lp * P.NG);
+      seg = rem / P.NG;
+      t0 = (rem - seg * P.NG) * P.NTG;
+      us = user_shape(P, u);
+      if (seg >= us.nseg) continue;
+      const int seg_items = min(P.S, us.len - seg * P.S);
+      if (t0 * P.IT >= seg_items) continue;                 // a tile group beyond the segment's valid items
+      const int t1 = min(P.NT, t0 + P.NTG);
+      rows = (t1 - t0) * P.IT;
+    } else {
+      const int ct = t - n_item_units;
+      if (ct >= n_ctiles) continue;
+      int lo = 0, hi = P.U;                                  // tile_off[lo] <= ct < tile_off[hi]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (P.tile_off[mid] <= ct) lo = mid; else hi = mid;
+      }
+      u = lo;
+      us = user_shape(P, u);
+      jt = ct - P.tile_off[u];
+      rows = kCandTile;
+    }
+
+    // ---- stage the rows into the canonical K-major layout (16-byte chunks; 8 lanes cover one core matrix)
+    {
+      const int chunks_per_row = d >> 3;
+      const int total = rows * chunks_per_row;
+      for (int q = tid; q < total; q += kProjThreads) {
+        const int r = ((q / (8 * chunks_per_row)) << 3) + (q & 7);
+        const int c = (q >> 3) % chunks_per_row;
+        const bf16* src;
+        uint32_t nbytes = 16;
+        if (is_item) {
+          const int tt = t0 + r / P.IT, rr = r % P.IT;
+          const int n = seg * P.S + tt * P.IT + rr;
+          if (n < P.L) src = P.items + ((size_t)u * P.L + n) * d + c * 8;
+          else { src = P.items; nbytes = 0; }
+        } else {
+          const int ci = jt * kCandTile + r;
+          if (ci < us.nc) src = P.cands + (size_t)(us.c0 + ci) * d + c * 8;
+          else { src = P.cands; nbytes = 0; }
+        }
+        cp_async16(X + ((r >> 3) * chunks_per_row + c) * 64 + (r & 7) * 8, src, nbytes);
+      }
+      cp_async_wait_all();
+      fence_proxy_async_smem();
+    }
+    __syncthreads();
+
+    // ---- MMAs (one thread issues)
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t xa = smem_u32(X);
+      const int ksteps = d >> 4;
+      const uint32_t wa = smem_u32(is_item ? imgK : imgQ);
+      const uint32_t id1 = idesc_bf16(128, dqk);
+      for (int ks = 0; ks < ksteps; ++ks)
+        mma_ss(tmem, smem_desc(xa + ks * 256, lbo, sbo), smem_desc(wa + ks * 256, lbo, sbo), id1, ks > 0);
+      if (is_item) {
+        const uint32_t va = smem_u32(imgV);
+        const uint32_t id2 = idesc_bf16(128, rows);
+        for (int ks = 0; ks < ksteps; ++ks)
+          mma_ss(tmem + 128, smem_desc(va + ks * 256, lbo, sbo), smem_desc(xa + ks * 256, lbo, sbo), id2, ks > 0);
+      }
+      tc_commit(&bar_mma);
+    }
+    ok = __syncthreads_and(mbar_wait(&bar_mma, mma_phase, abortp));
+    mma_phase ^= 1;
+    if (!ok) break;
+    tc_fence_after();
+
+    // ---- epilogue 1: K (or Q) rows.  TMEM lane = row of the unit; 16 columns per load.
+    if (warp * 32 < rows) {
+      const int r = tid;
+      const float scale = is_item ? 1.f : P.q_scale;
+      bool valid;
+      bf16* dst_tile;
+      int rr, tile_rows;
+      if (is_item) {
+        const int tt = t0 + r / P.IT;
+        rr = r % P.IT;
+        const int pos = tt * P.IT + rr;
+        valid = r < rows && pos < P.S && seg * P.S + pos < us.len;
+        dst_tile = P.Kblk + ((size_t)u * P.n_tiles + seg * P.NT + tt) * ((size_t)P.IT * dqk);
+        tile_rows = P.IT;
+      } else {
+        rr = r;
+        valid = jt * kCandTile + r < us.nc;
+        dst_tile = P.Qblk + (size_t)(P.tile_off[u] + jt) * (kCandTile * dqk);
+        tile_rows = kCandTile;
+      }
+      const int cpr = P.dqh >> 3;   // 8-element chunks per head row
+      for (int c16 = 0; c16 < dqk; c16 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_lane + c16, v);
+        tc_wait_ld();
+        if (r < rows) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int col = c16 + half * 8;
+            const int h = col / P.dqh, c = (col - h * P.dqh) >> 3;
+            uint4 o;
+            if (valid) {
+              o.x = pack_bf16x2(__uint_as_float(v[half * 8 + 0]) * scale, __uint_as_float(v[half * 8 + 1]) * scale);
+              o.y = pack_bf16x2(__uint_as_float(v[half * 8 + 2]) * scale, __uint_as_float(v[half * 8 + 3]) * scale);
+              o.z = pack_bf16x2(__uint_as_float(v[half * 8 + 4]) * scale, __uint_as_float(v[half * 8 + 5]) * scale);
+              o.w = pack_bf16x2(__uint_as_float(v[half * 8 + 6]) * scale, __uint_as_float(v[half * 8 + 7]) * scale);
+            } else {
+              o = make_uint4(0, 0, 0, 0);
+            }
+            bf16* dst = dst_tile + (size_t)h * tile_rows * P.dqh + ((rr >> 3) * cpr + c) * 64 + (rr & 7) * 8;
+            *reinterpret_cast<uint4*>(dst) = o;
+          }
+        }
+      }
+    }
+    // ---- epilogue 2: V^T.  TMEM lane = value feature j; columns = rows of the unit.
+    if (is_item && warp * 32 < d) {
+      const int j = tid;
+      const int h = j / P.dvh, jj = j - h * P.dvh;
+      const int npr = P.dvh >> 3;   // 8-row groups per head
+      float sv = 0.f;
+      for (int c16 = 0; c16 < rows; c16 += 16) {
+        uint32_t v[16];
+        tmem_ld16(tmem_lane + 128 + c16, v);
+        tc_wait_ld();
+        if (j < d) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int r0 = c16 + half * 8;
+            const int tt = t0 + r0 / P.IT, rr0 = r0 % P.IT;
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float a = __uint_as_float(v[half * 8 + 2 * e]), b = __uint_as_float(v[half * 8 + 2 * e + 1]);
+              const int pa = tt * P.IT + rr0 + 2 * e, pb = pa + 1;
+              if (!(pa < P.S && seg * P.S + pa < us.len)) a = 0.f;
+              if (!(pb < P.S && seg * P.S + pb < us.len)) b = 0.f;
+              pk[e] = pack_bf16x2(a, b);
+              sv += __uint_as_float(pk[e] << 16) + __uint_as_float(pk[e] & 0xFFFF0000u);
+            }
+            bf16* dst = P.Vtblk + ((size_t)u * P.n_tiles + seg * P.NT + tt) * ((size_t)P.IT * d) +
+                        (size_t)h * P.IT * P.dvh + ((rr0 >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
+            *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      }
+      if (j < d) atomicAdd(&P.SV[((size_t)u * P.Lp + seg) * d + j], sv);
+    }
+    tc_fence_before();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kProjTmemCols);
+  if (tid == 0 && s_abort) report_status(P.status, LASER_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------------- attention
+// Walks the attention units (user, candidate tile, segment) of a contiguous id range in order.
+struct UnitWalker {
+  int u, j, seg;
+  UserShape us;
+  __device__ void init(const TcParams& P, int id) {
+    int lo = 0, hi = P.U;   // unit_start[lo] <= id < unit_start[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (P.unit_start[mid] <= id) lo = mid; else hi = mid;
+    }
+    u = lo;
+    us = user_shape(P, u);
+    const int local = id - P.unit_start[u];
+    j = local / us.nseg;
+    seg = local - j * us.nseg;
+  }
+  __device__ void next(const TcParams& P) {
+    if (++seg < us.nseg) return;
+    seg = 0;
+    if (++j < us.ctiles) return;
+    j = 0;
+    do {
+      ++u;
+      if (u >= P.U) return;
+      us = user_shape(P, u);
+    } while (us.nseg == 0 || us.ctiles == 0);
+  }
+  // tiles of the current segment that hold at least one valid item
+  __device__ int ntiles(const TcParams& P) const {
+    const int seg_items = min(P.S, us.len - seg * P.S);
+    return min(P.NT, (seg_items + P.IT - 1) / P.IT);
+  }
+};
+
+struct StaBars {
+  uint64_t q_full[2], q_empty[2];
+  uint64_t kv_full[kKvStages], kv_empty[kKvStages];
+  uint64_t s_full[2], p_full[2], p_empty[2];
+  uint64_t o_full[2], o_empty[2];
+  uint64_t done;
+};
+
+__global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ StaBars bars;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int d = P.d, dqk = P.dqk, IT = P.IT, H = P.H;
+  const uint32_t q_bytes = kCandTile * dqk * 2, k_bytes = IT * dqk * 2, v_bytes = IT * d * 2;
+  uint8_t* Qs = smem_raw;                         // [2][q_bytes]
+  uint8_t* Ks = Qs + 2 * q_bytes;                 // [kKvStages][k_bytes]
+  uint8_t* Vs = Ks + kKvStages * k_bytes;         // [kKvStages][v_bytes]
+
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars.q_full[i], 1);
+      mbar_init(&bars.q_empty[i], 1);
+      mbar_init(&bars.s_full[i], 1);
+      mbar_init(&bars.p_full[i], 4);
+      mbar_init(&bars.p_empty[i], 1);
+      mbar_init(&bars.o_full[i], 1);
+      mbar_init(&bars.o_empty[i], 4);
+    }
+    for (int i = 0; i < kKvStages; ++i) {
+      mbar_init(&bars.kv_full[i], 1);
+      mbar_init(&bars.kv_empty[i], 1);
+    }
+    mbar_init(&bars.done, 1);
+    s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 2) {
+    tmem_alloc(&s_tmem, kStaTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+
+  // TMEM columns: O[2] (d each), S[2] (IT each, fp32 scores), P[2] (IT/2 each, packed bf16 pairs)
+  const uint32_t colO = 0, colS = 2 * d, colP = 2 * d + 2 * IT;
+
+  // this block's contiguous range of units
+  const int n_units = P.counters[0];
+  const int G = gridDim.x, b = blockIdx.x;
+  const int unit_lo = (int)(((long long)n_units * b) / G);
+  const int unit_hi = (int)(((long long)n_units * (b + 1)) / G);
+  const int my_units = unit_hi - unit_lo;
+
+  if (my_units > 0) {
+    if (warp == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      if (lane == 0) {
+        UnitWalker w;
+        w.init(P, unit_lo);
+        int pu = -1, pj = -1;
+        uint32_t qcount = 0, kvcount = 0;
+        bool ok = true;
+        for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+          if (w.u != pu || w.j != pj) {
+            const int qs = qcount & 1;
+            ok = mbar_wait(&bars.q_empty[qs], ((qcount >> 1) & 1) ^ 1, abortp);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&bars.q_full[qs], q_bytes);
+            bulk_g2s(Qs + qs * q_bytes, P.Qblk + (size_t)(P.tile_off[w.u] + w.j) * (kCandTile * dqk), q_bytes,
+                     &bars.q_full[qs]);
+            ++qcount;
+            pu = w.u;
+            pj = w.j;
+          }
+          const int nt = w.ntiles(P);
+          for (int t = 0; t < nt && ok; ++t) {
+            const int st = kvcount % kKvStages;
+            ok = mbar_wait(&bars.kv_empty[st], ((kvcount / kKvStages) & 1) ^ 1, abortp);
+            if (!ok) break;
+            const size_t tile = (size_t)w.u * P.n_tiles + w.seg * P.NT + t;
+            mbar_arrive_expect_tx(&bars.kv_full[st], k_bytes + v_bytes);
+            bulk_g2s(Ks + st * k_bytes, P.Kblk + tile * ((size_t)IT * dqk), k_bytes, &bars.kv_full[st]);
+            bulk_g2s(Vs + st * v_bytes, P.Vtblk + tile * ((size_t)IT * d), v_bytes, &bars.kv_full[st]);
+            ++kvcount;
+          }
+        }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ MMA issuer
+      if (lane == 0) {
+        const uint32_t id1 = idesc_bf16(128, IT);        // scores: 128 candidates x IT items, K = dqh
+        const uint32_t id2 = idesc_bf16(128, P.dvh);     // O_h: 128 candidates x dvh, K = IT items
+        const uint32_t qk_sbo = (P.dqh >> 3) * 128;      // 8-row groups of a [rows x dqh] head block
+        const uint32_t v_lbo = (P.dvh >> 3) * 128;       // V^T head block: k-chunks (8 items) are dvh/8 core matrices apart
+        const int ks1 = P.dqh >> 4, ks2 = IT >> 4;
+
+        // cursor 1 issues the score MMAs two gate-units ahead of cursor 2, which issues the P'V MMAs
+        UnitWalker w1, w2;
+        w1.init(P, unit_lo);
+        w2.init(P, unit_lo);
+        int it1 = 0, t1 = 0, h1 = 0, nt1 = w1.ntiles(P);
+        int it2 = 0, t2 = 0, h2 = 0, nt2 = w2.ntiles(P);
+        uint32_t q1 = 0, kv1 = 0, kv2 = 0, g1 = 0, g2 = 0, seg2 = 0;
+        int pu1 = -1, pj1 = -1;
+        bool ok = true;
+
+        auto issue1 = [&]() {
+          if (it1 >= my_units || !ok) return;
+          if (t1 == 0 && h1 == 0 && (w1.u != pu1 || w1.j != pj1)) {
+            if (pu1 >= 0) { tc_commit(&bars.q_empty[(q1 - 1) & 1]); }
+            ok = mbar_wait(&bars.q_full[q1 & 1], (q1 >> 1) & 1, abortp);
+            if (!ok) return;
+            ++q1;
+            pu1 = w1.u;
+            pj1 = w1.j;
+          }
+          const int st = kv1 % kKvStages;
+          if (h1 == 0) {
+            ok = mbar_wait(&bars.kv_full[st], (kv1 / kKvStages) & 1, abortp);
+            if (!ok) return;
+          }
+          tc_fence_after();
+          const uint32_t qa = smem_u32(Qs + ((q1 - 1) & 1) * q_bytes) + h1 * (kCandTile * P.dqh * 2);
+          const uint32_t ka = smem_u32(Ks + st * k_bytes) + h1 * (IT * P.dqh * 2);
+          const uint32_t dS = tmem + colS + (g1 & 1) * IT;
+          for (int ks = 0; ks < ks1; ++ks)
+            mma_ss(dS, smem_desc(qa + ks * 256, 128, qk_sbo), smem_desc(ka + ks * 256, 128, qk_sbo), id1, ks > 0);
+          tc_commit(&bars.s_full[g1 & 1]);
+          ++g1;
+          if (++h1 == H) {
+            h1 = 0;
+            ++kv1;
+            if (++t1 == nt1) {
+              t1 = 0;
+              ++it1;
+              w1.next(P);
+              if (it1 < my_units) nt1 = w1.ntiles(P);
+            }
+          }
+        };
+
+        issue1();
+        issue1();
+        while (it2 < my_units && ok) {
+          const int pb = g2 & 1;
+          ok = mbar_wait(&bars.p_full[pb], (g2 >> 1) & 1, abortp);
+          if (!ok) break;
+          issue1();                                        // scores of gate-unit g2 + 2 reuse the buffer just drained
+          if (!ok) break;
+          const int ob = seg2 & 1;
+          if (t2 == 0 && h2 == 0) {
+            ok = mbar_wait(&bars.o_empty[ob], ((seg2 >> 1) & 1) ^ 1, abortp);
+            if (!ok) break;
+          }
+          tc_fence_after();
+          const int st = kv2 % kKvStages;
+          const uint32_t va = smem_u32(Vs + st * v_bytes) + h2 * (IT * P.dvh * 2);
+          const uint32_t dO = tmem + colO + ob * d + h2 * P.dvh;
+          const uint32_t aP = tmem + colP + pb * (IT >> 1);
+          for (int ks = 0; ks < ks2; ++ks)
+            mma_ts(dO, aP + ks * 8, smem_desc(va + ks * 2 * v_lbo, v_lbo, 128), id2, (t2 > 0 || ks > 0) ? 1u : 0u);
+          tc_commit(&bars.p_empty[pb]);
+          ++g2;
+          if (++h2 == H) {
+            h2 = 0;
+            tc_commit(&bars.kv_empty[st]);
+            ++kv2;
+            if (++t2 == nt2) {
+              t2 = 0;
+              tc_commit(&bars.o_full[ob]);
+              ++seg2;
+              ++it2;
+              w2.next(P);
+              if (it2 < my_units) nt2 = w2.ntiles(P);
+            }
+          }
+        }
+        // every MMA issued by this thread has completed once `done` flips
+        tc_commit(&bars.done);
+        mbar_wait(&bars.done, 0, abortp);
+      }
+    } else if (warp >= 8) {
+      // ------------------------------------------------------------------ gate warps: P' = tanh(scores)
+      const int wg = (warp - 8) >> 2;                       // warpgroup 0 / 1 owns score and P buffer 0 / 1
+      const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+      const uint32_t tS = tmem + lane_base + colS + wg * IT;
+      const uint32_t tP = tmem + lane_base + colP + wg * (IT >> 1);
+      UnitWalker w;
+      w.init(P, unit_lo);
+      uint32_t g = 0, k = 0;
+      bool ok = true;
+      for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+        const int n_sub = w.ntiles(P) * H;
+        for (int s = 0; s < n_sub && ok; ++s, ++g) {
+          if ((int)(g & 1) != wg) continue;
+          ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], k & 1, abortp));
+          if (!ok) break;
+          ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_empty[wg], (k & 1) ^ 1, abortp));
+          if (!ok) break;
+          tc_fence_after();
+          int c = 0;
+          for (; c + 32 <= IT; c += 32) {
+            uint32_t v[32], o[16];
+            tmem_ld32(tS + c, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e)
+              o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+            tmem_st16(tP + (c >> 1), o);
+          }
+          if (c < IT) {   // 16-column tail
+            uint32_t v[16], o[8];
+            tmem_ld16(tS + c, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+            tmem_st8(tP + (c >> 1), o);
+          }
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.p_full[wg]);
+          ++k;
+        }
+      }
+    } else if (warp >= 4) {
+      // ------------------------------------------------------------------ epilogue: H' = (SV + O) / 2
+      const int q = warp - 4;
+      const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+      const int m = q * 32 + lane;
+      UnitWalker w;
+      w.init(P, unit_lo);
+      bool ok = true;
+      for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+        const int ob = it & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], (it >> 1) & 1, abortp));
+        if (!ok) break;
+        tc_fence_after();
+        const int ci = w.j * kCandTile + m;
+        const bool valid = ci < w.us.nc;
+        const float* sv = P.SV + ((size_t)w.u * P.Lp + w.seg) * d;
+        bf16* out = P.Hp + ((size_t)(w.us.c0 + (valid ? ci : 0)) * P.Lp + w.seg) * d;
+        for (int c = 0; c < d; c += 16) {
+          uint32_t v[16];
+          tmem_ld16(tmem + lane_base + colO + ob * d + c, v);
+          tc_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const float4 s0 = __ldg(reinterpret_cast<const float4*>(sv + c + half * 8));
+              const float4 s1 = __ldg(reinterpret_cast<const float4*>(sv + c + half * 8 + 4));
+              uint4 o;
+              o.x = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 0]) + s0.x), 0.5f * (__uint_as_float(v[half * 8 + 1]) + s0.y));
+              o.y = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 2]) + s0.z), 0.5f * (__uint_as_float(v[half * 8 + 3]) + s0.w));
+              o.z = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 4]) + s1.x), 0.5f * (__uint_as_float(v[half * 8 + 5]) + s1.y));
+              o.w = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 6]) + s1.z), 0.5f * (__uint_as_float(v[half * 8 + 7]) + s1.w));
+              *reinterpret_cast<uint4*>(out + c + half * 8) = o;
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tmem, kStaTmemCols);
+  if (tid == 0 && s_abort) report_status(P.status, LASER_ERR_TIMEOUT);
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                     const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hp, char* ws) {
+  TcParams P;
+  P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
+  P.dqh = p.dqh; P.dvh = p.dvh; P.maxC = p.maxC;
+  P.IT = p.tg.IT; P.NT = p.tg.NT; P.n_tiles = p.tg.n_tiles; P.cand_tiles_max = p.tg.cand_tiles_max;
+  P.NTG = P.IT <= 64 ? (128 / P.IT < P.NT ? 128 / P.IT : P.NT) : 1;
+  P.NG = (P.NT + P.NTG - 1) / P.NTG;
+  P.q_scale = 0.5f * p.inv_gamma;
+  P.items = (const bf16*)items; P.cands = (const bf16*)cands;
+  P.Wq = (const bf16*)Wq; P.Wk = (const bf16*)Wk; P.Wv = (const bf16*)Wv;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.Qblk = (bf16*)(ws + p.off_tq); P.Kblk = (bf16*)(ws + p.off_tk); P.Vtblk = (bf16*)(ws + p.off_tv);
+  P.SV = (float*)(ws + p.off_tsv);
+  P.unit_start = (int*)(ws + p.off_twork);
+  P.tile_off = P.unit_start + (p.U + 1);
+  P.counters = (int*)(ws + p.off_tcount);
+  P.imgK = (bf16*)(ws + p.off_timg);
+  P.imgQ = P.imgK + (size_t)p.dqk * p.d;
+  P.imgV = P.imgQ + (size_t)p.dqk * p.d;
+  P.status = (int*)(ws + p.off_status);
+  P.Hp = (bf16*)Hp;
+  return P;
+}
+
+}  // namespace
+
+bool tensor_supported(const Plan& p) {
+  if (p.dtype != LASER_BF16) return false;
+  if (p.d % 16 || p.d < 16 || p.d > 128) return false;
+  if (p.dqh % 16 || p.dqk > 128) return false;
+  if (p.dvh % 16) return false;
+  TensorGeom g;
+  tensor_geometry(p, &g);
+  if ((long long)p.U * g.n_tiles >= (1ll << 30)) return false;
+  if ((long long)p.U * p.Lp * 4 >= (1ll << 30)) return false;
+  return true;
+}
+
+void tensor_geometry(const Plan& p, TensorGeom* g) {
+  const int it_max = p.d > 64 ? 64 : 128;   // TMEM: 2 d (outputs) + 3 IT (scores, packed gates) <= 512 columns
+  g->NT = (p.S + it_max - 1) / it_max;
+  const int per = (p.S + g->NT - 1) / g->NT;
+  g->IT = (per + 15) / 16 * 16;
+  g->n_tiles = p.Lp * g->NT;
+  const long long a = (long long)p.N / kCandTile + p.U;
+  const long long b = (long long)p.U * ((p.maxC + kCandTile - 1) / kCandTile);
+  g->cand_tiles_max = (int)(a < b ? a : b);
+}
+
+int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+  if (p.N == 0 || p.U == 0) return LASER_OK;
+  const bool user_wants_hp = Hprime != (void*)(ws + p.off_hp);
+  TcParams P = make_params(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws);
+  const int sms = sm_count();
+  {
+    LaunchScope ls("tc_prep", st);
+    tc_prep_kernel<<<1 + 32, 1024, 0, st>>>(P);
+  }
+  {
+    const size_t smem = ((size_t)2 * p.dqk * p.d + 2 * (size_t)kCandTile * p.d) * 2;
+    LASER_CUDA_OK(cudaFuncSetAttribute(tc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LaunchScope ls("tc_proj", st);
+    tc_proj_kernel<<<2 * sms, kProjThreads, smem, st>>>(P);
+  }
+  if (user_wants_hp) {
+    LaunchScope ls("tc_zero_empty", st);
+    tc_zero_empty_kernel<<<dim3(p.Lp, p.U), 256, 0, st>>>(P);
+  }
+  {
+    const size_t smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * P.IT * (p.dqk + p.d) * 2;
+    if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+    LASER_CUDA_OK(cudaFuncSetAttribute(tc_sta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LaunchScope ls("sta_tc", st);
+    tc_sta_kernel<<<sms, kStaThreads, smem, st>>>(P);
+  }
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
+                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st) {
+  return simt_gsta(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st);
+}
+
 }  // namespace laser

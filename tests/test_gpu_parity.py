@@ -62,6 +62,45 @@ def test_small_shapes_simt(case, dtype):
     check_against_oracle(w, "simt")
 
 
+TENSOR = [
+    dict(U=1, C=128, L=128, d=64, H=4, S=64, M=1, d_qh=16, lengths=[128]),               # one full tile, 2 segments
+    dict(U=2, C=200, L=512, d=64, H=4, S=64, M=2, d_qh=16, lengths=[512, 301]),          # ragged, partial candidate tile
+    dict(U=3, C=130, L=700, d=128, H=4, S=128, M=2, d_qh=16, lengths=[700, 129, 0]),     # two item tiles per segment
+    dict(U=2, C=300, L=1000, d=64, H=4, S=100, M=2, d_qh=16, lengths=[1000, 250]),       # S = 100 -> 112-row tiles
+    dict(U=5, C=1, L=300, d=32, H=2, S=10, M=1, d_qh=16, lengths=[300, 9, 10, 11, 0]),   # S = 10, one candidate
+    dict(U=2, C=40, L=520, d=64, H=2, S=260, M=1, d_qh=32, lengths=[520, 300]),          # S > 128, d_qh = 32
+    dict(U=1, C=16, L=48, d=16, H=1, S=48, M=1, d_qh=16, lengths=[40]),                  # smallest widths, S = L
+]
+
+
+@pytest.mark.parametrize("case", range(len(TENSOR)))
+def test_small_shapes_tensor_path(case):
+    w = make_custom(dtype="bf16", seed=200 + case, **TENSOR[case])
+    check_against_oracle(w, "tensor")
+
+
+def test_tensor_path_padding_rows_and_determinism():
+    w = make_custom(U=2, C=150, L=256, d=64, H=4, S=64, M=2, dtype="bf16", seed=9, lengths=[130, 5])
+    Hp1, z1 = run_forward(w, "tensor")
+    Hp1b, z1b = run_forward(w, "tensor")
+    assert torch.equal(Hp1, Hp1b) and torch.equal(z1, z1b)
+    w.items[0, 130:] = -123.0
+    w.items[1, 5:] = 0.015625
+    Hp2, z2 = run_forward(w, "tensor")
+    assert torch.equal(Hp1, Hp2) and torch.equal(z1, z2)
+
+
+def test_tensor_path_reports_bad_inputs():
+    w = make_custom(U=2, C=3, L=64, d=64, H=4, S=16, M=1, dtype="bf16", seed=1, lengths=[64, 3])
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    bad_len = torch.tensor([65, 3], dtype=torch.int32, device="cuda")
+    P.laser_forward(b.cfg, b.items, bad_len, b.cands, b.cand_offsets, b.Wq, b.Wk, b.Wv, b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == -6
+    P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_stage_entry_points_simt(dtype):
     """laser_sta_forward and laser_gsta_forward on their own: GSTA is fed the oracle's H' (rounded to the dtype)."""
