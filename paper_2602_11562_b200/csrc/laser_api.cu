@@ -88,8 +88,10 @@ int make_plan(const laser_config* c, Plan* p) {
     p->off_twork = off; off = align_up(off + ((size_t)p->U + 1) * 2 * sizeof(int));
     p->off_tcount = off; off = align_up(off + 64 * sizeof(int));
     p->off_timg = off; off = align_up(off + ((size_t)2 * p->dqk * p->d + (size_t)128 * p->d) * 2);
+    if (gsta_mma_supported(*p)) { p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p)); }
   } else if (path == LASER_PATH_STREAM) {
-    p->off_su = off; off = align_up(off + (size_t)p->U * (p->H * p->d + p->H * p->H * p->d + 8) * sizeof(float));
+    p->off_su = off; off = align_up(off + stream_scratch_bytes(*p));
+    p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p));
   }
   p->total = off;
   return LASER_OK;
@@ -123,6 +125,7 @@ static int run_sta(const Plan& p, const void* items, const int32_t* lengths, con
   switch (p.path) {
     case LASER_PATH_SIMT: return simt_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
     case LASER_PATH_TENSOR: return tensor_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+    case LASER_PATH_STREAM: return stream_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
     default: return LASER_ERR_UNSUPPORTED;
   }
 }
@@ -132,6 +135,7 @@ static int run_gsta(const Plan& p, const void* Hp, const int32_t* lengths, const
   switch (p.path) {
     case LASER_PATH_SIMT: return simt_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
     case LASER_PATH_TENSOR: return tensor_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+    case LASER_PATH_STREAM: return gsta_mma(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
     default: return LASER_ERR_UNSUPPORTED;
   }
 }
@@ -142,8 +146,6 @@ static int forward_impl(const Plan& p, const void* items, const int32_t* lengths
   int rc = clear_status(p, ws, st);
   if (rc != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
-  if (p.path == LASER_PATH_STREAM)
-    return stream_forward(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wg, Hprime, z, ws, st);
   void* Hp = Hprime ? Hprime : (void*)(ws + p.off_hp);
   rc = run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
   if (rc != LASER_OK) return rc;
@@ -169,7 +171,6 @@ int laser_sta_forward(const laser_config* cfg, const void* items, const int32_t*
   Plan p;
   int rc = make_plan(cfg, &p);
   if (rc != LASER_OK) return rc;
-  if (p.path == LASER_PATH_STREAM) return LASER_ERR_UNSUPPORTED;   // the streaming path only exists fused
   if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
   if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
   if (p.N > 0 && (rc = check_ptrs({items, cands, Wq, Wk, Wv, Hprime})) != LASER_OK) return rc;
@@ -187,7 +188,6 @@ int laser_gsta_forward(const laser_config* cfg, const void* Hprime, const int32_
   Plan p;
   int rc = make_plan(cfg, &p);
   if (rc != LASER_OK) return rc;
-  if (p.path == LASER_PATH_STREAM) return LASER_ERR_UNSUPPORTED;
   if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
   if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
   if (p.N > 0 && (rc = check_ptrs({Hprime, cands, z})) != LASER_OK) return rc;

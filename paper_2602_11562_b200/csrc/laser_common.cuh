@@ -33,6 +33,7 @@ struct Plan {
   // tensor path
   TensorGeom tg;
   size_t off_tq, off_tk, off_tv, off_tsv, off_twork, off_tcount, off_timg;
+  size_t off_gimg;                 // GSTA weight images in MMA fragment order (bf16 paths)
   // stream path
   size_t off_su;
   size_t total;
@@ -68,10 +69,17 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
                 const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st);
 
+// Fused warp-MMA GSTA kernel for bf16 (laser_gsta.cu); needs gsta_mma_image_bytes(p) of scratch at off_gimg.
+bool gsta_mma_supported(const Plan& p);
+size_t gsta_mma_image_bytes(const Plan& p);
+int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
+             const void* Wg, void* z, char* ws, cudaStream_t st);
+
+// One-candidate-per-user STA (laser_stream.cu); needs stream_scratch_bytes(p) of scratch at off_su.  Its GSTA is gsta_mma.
 bool stream_supported(const Plan& p);
-int stream_forward(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
-                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wg,
-                   void* Hprime, void* z, char* ws, cudaStream_t st);
+size_t stream_scratch_bytes(const Plan& p);
+int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
 
 // --- device helpers ---------------------------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -1,7 +1,362 @@
-// One-candidate-per-user HBM-streaming path.  Placeholder until the kernel lands: reports "not supported".
+// One-candidate-per-user path (bf16): a single pass over each user's raw item rows, bound by HBM bandwidth.
+//
+// With one target per user, materialising K = X W_k and V = X W_v (Eq. 9) would cost 2 d (d_qk + d) flops per
+// 2 d-byte item row and make the pass compute bound.  Both projections are therefore folded out of the item loop
+// (exact in real arithmetic):
+//
+//   gate      q_h . k_{n,h} / gamma = x_n . u_h          with  u_h = W_k[:, head h] (t W_q)_h / gamma   in R^d
+//   segment   s_i[head h] = sum_n g_{n,h} (x_n W_v)[head h] = r_{i,h} W_v[:, head h]   with  r_{i,h} = sum_n g_{n,h} x_n
+//
+// so the item loop only needs the 2 H dot products x_n . u_h and the 2 H d multiply-adds of r += g x per row
+// (Eq. 10-12), and W_v is applied once per segment afterwards.
+//
+//   stream_pre_kernel    u [U, H, d] (fp32) for every user, and the fragment-ordered image of W_v
+//   stream_sta_kernel    one block per user; every warp owns whole segments, streams their rows through a private
+//                        cp.async ring (16 rows per stage, 128-bit copies, padded rows) and feeds them twice to
+//                        warp-level MMAs: scores = U X^T (rows = heads), then R += G X.  u, the gates and r are
+//                        split into bf16 high and low parts that occupy MMA rows h and h + 8, so the fp32 values
+//                        survive the bf16 operands to about 16 bits.  After the item loop the block multiplies all
+//                        its segment sums by W_v (MMA, rows = segments) and writes H'.
+//   GSTA                 the shared fused GSTA kernel (laser_gsta.cu) on that H'.
 #include "laser_common.cuh"
+#include "laser_mma.cuh"
+
 namespace laser {
-bool stream_supported(const Plan&) { return false; }
-int stream_forward(const Plan&, const void*, const int32_t*, const void*, const int32_t*, const void*, const void*,
-                   const void*, const void*, void*, void*, char*, cudaStream_t) { return LASER_ERR_UNSUPPORTED; }
+namespace {
+
+using bf16 = __nv_bfloat16;
+using namespace mma;
+
+constexpr int kSW = 4;            // warps per block
+constexpr int kSThreads = kSW * 32;
+constexpr int kSRows = 16;        // item rows per stage (one MMA k / n step)
+constexpr int kSStages = 4;       // ring depth per warp
+constexpr int kPreUsers = 8;      // users per block of the pre kernel
+
+struct StreamParams {
+  int U, L, d, dqk, H, S, Lp, N;
+  float inv_gamma;
+  const bf16 *items, *cands, *Wq, *Wk, *Wv;
+  const int *lengths, *cand_offsets;
+  float* u;                       // [U, H, d]
+  uint4* imgv;                    // W_v as MMA B fragments: [d/16 k-tiles][d/16 column pairs][32 lanes]
+  bf16* Hp;                       // [N, Lp, d]
+  int zero_empty;                 // write zero rows for segments without valid items
+  int* status;
+};
+
+// Candidate of user u, or -1 when it has none (or its offsets / length are invalid).
+__device__ __forceinline__ int user_candidate(const StreamParams& P, int u, int* len_out) {
+  const int c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1], len = P.lengths[u];
+  if (c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > 1 || len < 0 || len > P.L) {
+    report_status(P.status, LASER_ERR_BAD_INPUT);
+    return -1;
+  }
+  *len_out = len;
+  return c1 > c0 ? c0 : -1;
+}
+
+__global__ void __launch_bounds__(128) stream_pre_kernel(StreamParams P, int user_blocks) {
+  const int tid = threadIdx.x;
+  const int d = P.d, dqk = P.dqk, H = P.H, dqh = dqk / H;
+  if ((int)blockIdx.x >= user_blocks) {
+    // W_v image: entry (kt, p, lane) = {b0, b1 of column tile 2p, b0, b1 of column tile 2p+1}, B[k][n] = W_v[k][n]
+    const int D16 = d >> 4, total = D16 * D16 * 32;
+    const uint16_t* W = reinterpret_cast<const uint16_t*>(P.Wv);
+    for (int i = (blockIdx.x - user_blocks) * blockDim.x + tid; i < total; i += (gridDim.x - user_blocks) * blockDim.x) {
+      const int lane = i & 31, p = (i >> 5) % D16, kt = (i >> 5) / D16;
+      const int g = lane >> 2, t = lane & 3;
+      uint32_t v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int n = (2 * p + (q >> 1)) * 8 + g, k = kt * 16 + 2 * t + (q & 1) * 8;
+        v[q] = (uint32_t)W[(size_t)k * d + n] | ((uint32_t)W[(size_t)(k + 1) * d + n] << 16);
+      }
+      P.imgv[i] = make_uint4(v[0], v[1], v[2], v[3]);
+    }
+    return;
+  }
+  extern __shared__ float sm[];
+  float* ts = sm;                      // [kPreUsers][d]
+  float* qs = ts + kPreUsers * d;      // [kPreUsers][dqk]
+  __shared__ int cand_s[kPreUsers];
+  const int u0 = blockIdx.x * kPreUsers;
+  if (tid < kPreUsers) {
+    int len = 0;
+    cand_s[tid] = u0 + tid < P.U ? user_candidate(P, u0 + tid, &len) : -1;
+  }
+  __syncthreads();
+  for (int i = tid; i < kPreUsers * d; i += blockDim.x) {
+    const int uu = i / d, c = cand_s[uu];
+    ts[i] = c >= 0 ? __bfloat162float(P.cands[(size_t)c * d + (i - uu * d)]) : 0.f;
+  }
+  __syncthreads();
+  for (int a = tid; a < dqk; a += blockDim.x) {        // q = t W_q / gamma   (Eq. 4 / Eq. 8)
+    float acc[kPreUsers] = {};
+    for (int i = 0; i < d; ++i) {
+      const float w = __bfloat162float(P.Wq[(size_t)i * dqk + a]);
+#pragma unroll
+      for (int uu = 0; uu < kPreUsers; ++uu) acc[uu] = fmaf(ts[uu * d + i], w, acc[uu]);
+    }
+#pragma unroll
+    for (int uu = 0; uu < kPreUsers; ++uu) qs[uu * dqk + a] = acc[uu] * P.inv_gamma;
+  }
+  __syncthreads();
+  for (int i = tid; i < d; i += blockDim.x) {          // u_h[i] = sum_{a in head h} W_k[i][a] q[a]
+    for (int h = 0; h < H; ++h) {
+      float acc[kPreUsers] = {};
+      for (int a = h * dqh; a < (h + 1) * dqh; ++a) {
+        const float w = __bfloat162float(P.Wk[(size_t)i * dqk + a]);
+#pragma unroll
+        for (int uu = 0; uu < kPreUsers; ++uu) acc[uu] = fmaf(w, qs[uu * dqk + a], acc[uu]);
+      }
+#pragma unroll
+      for (int uu = 0; uu < kPreUsers; ++uu)
+        if (u0 + uu < P.U) P.u[((size_t)(u0 + uu) * H + h) * d + i] = acc[uu];
+    }
+  }
+}
+
+__device__ __forceinline__ float sigmoid_fast(float x) {
+  // 1 / (1 + e^-x); e^-x overflowing to +inf gives exactly 0
+  return __frcp_rn(1.f + __expf(-x));
+}
+
+template <int D16>
+__global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
+  constexpr int d = D16 * 16;
+  constexpr int RS = 2 * d + 16;                 // bytes per staged row (the padding keeps ldmatrix conflict-free)
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int H = P.H, dvh = d / H;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int u = blockIdx.x;
+  int len = 0;
+  const int cand = user_candidate(P, u, &len);
+  if (cand < 0) return;
+  const int nv = (len + P.S - 1) / P.S;          // non-empty segments
+  const int Lp16 = (P.Lp + 15) & ~15;
+  uint8_t* Rhi = smem;                           // [Lp16][H] rows: bf16 high part of r_{i,h}
+  uint8_t* Rlo = Rhi + (size_t)Lp16 * H * RS;    // same shape: bf16 low part
+  uint8_t* ring = Rlo + (size_t)Lp16 * H * RS + (size_t)warp * kSStages * kSRows * RS;
+
+  if (nv > 0) {
+    // A fragments of U: row h = high part of u_h, row h + 8 = low part
+    uint32_t ua[D16][4];
+    {
+      const float* up = P.u + ((size_t)u * H + g) * d;
+#pragma unroll
+      for (int kt = 0; kt < D16; ++kt) {
+        ua[kt][0] = ua[kt][1] = ua[kt][2] = ua[kt][3] = 0u;
+        if (g < H) {
+          const float2 x0 = *reinterpret_cast<const float2*>(up + kt * 16 + 2 * t);
+          const float2 x1 = *reinterpret_cast<const float2*>(up + kt * 16 + 2 * t + 8);
+          ua[kt][0] = pack2(x0.x, x0.y);
+          ua[kt][1] = pack2(x0.x - bf16_lo(ua[kt][0]), x0.y - bf16_hi(ua[kt][0]));
+          ua[kt][2] = pack2(x1.x, x1.y);
+          ua[kt][3] = pack2(x1.x - bf16_lo(ua[kt][2]), x1.y - bf16_hi(ua[kt][2]));
+        }
+      }
+    }
+    const bf16* xu = P.items + (size_t)u * P.L * d;
+
+    // fetch cursor over this warp's (segment, 16-row group) sequence
+    int f_seg = warp, f_grp = 0;
+    bool f_valid = warp < nv;
+    auto groups_of = [&](int seg) { return (min(P.S, len - seg * P.S) + kSRows - 1) / kSRows; };
+    auto issue = [&](int stage) {
+      const int seg_end = min((f_seg + 1) * P.S, len);
+      const int n0 = f_seg * P.S + f_grp * kSRows;
+      const uint32_t dst = smem_addr(ring + (size_t)stage * kSRows * RS);
+#pragma unroll
+      for (int i = 0; i < D16; ++i) {
+        const int piece = i * 32 + lane;
+        const int r = piece / (2 * D16), q = piece - r * (2 * D16);
+        const bool ok = n0 + r < seg_end;        // rows past the segment (or the valid prefix) are staged as zeros
+        cp16(dst + r * RS + q * 16, ok ? (const void*)(xu + (size_t)(n0 + r) * d + q * 8) : (const void*)P.items,
+             ok ? 16u : 0u);
+      }
+      if (++f_grp >= groups_of(f_seg)) {
+        f_grp = 0;
+        f_seg += kSW;
+        if (f_seg >= nv) f_valid = false;
+      }
+    };
+#pragma unroll
+    for (int s = 0; s < kSStages - 1; ++s) {
+      if (f_valid) issue(s);
+      cp_commit();
+    }
+
+    int stage = 0;
+    const uint32_t off1 = ((lane & 7) + ((lane >> 4) & 1) * 8) * RS + ((lane >> 3) & 1) * 16;   // [item][k] operand
+    const uint32_t off2 = ((lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16;         // [item][col], transposed
+    for (int seg = warp; seg < nv; seg += kSW) {
+      float racc[2 * D16][4];
+#pragma unroll
+      for (int j = 0; j < 2 * D16; ++j) racc[j][0] = racc[j][1] = racc[j][2] = racc[j][3] = 0.f;
+      const int ngrp = groups_of(seg);
+      for (int grp = 0; grp < ngrp; ++grp) {
+        cp_wait<kSStages - 2>();
+        __syncwarp();
+        if (f_valid) issue((stage + kSStages - 1) % kSStages);
+        cp_commit();
+        const uint32_t sb = smem_addr(ring + (size_t)stage * kSRows * RS);
+        // scores (Eq. 10 before the sigmoid): rows = heads (high / low parts), columns = the 16 items
+        float sc[2][4] = {};
+#pragma unroll
+        for (int kt = 0; kt < D16; ++kt) {
+          uint32_t b[4];
+          ldsm_x4(b, sb + off1 + kt * 32);
+          mma16816(sc[0], ua[kt][0], ua[kt][1], ua[kt][2], ua[kt][3], b[0], b[1]);
+          mma16816(sc[1], ua[kt][0], ua[kt][1], ua[kt][2], ua[kt][3], b[2], b[3]);
+        }
+        // gates; a zero row has score 0, gate 1/2 and contributes 1/2 * 0 = 0, so no mask is needed here
+        uint32_t ga[4] = {0u, 0u, 0u, 0u};
+        if (g < H) {
+#pragma unroll
+          for (int nt = 0; nt < 2; ++nt) {
+            const float g0 = sigmoid_fast(sc[nt][0] + sc[nt][2]), g1 = sigmoid_fast(sc[nt][1] + sc[nt][3]);
+            ga[2 * nt] = pack2(g0, g1);
+            ga[2 * nt + 1] = pack2(g0 - bf16_lo(ga[2 * nt]), g1 - bf16_hi(ga[2 * nt]));
+          }
+        }
+        // r += G X  (Eq. 11-12 with the value projection postponed): rows = heads, k = items, columns = d
+#pragma unroll
+        for (int jp = 0; jp < D16; ++jp) {
+          uint32_t b[4];
+          ldsm_x4_t(b, sb + off2 + jp * 32);
+          mma16816(racc[2 * jp], ga[0], ga[1], ga[2], ga[3], b[0], b[1]);
+          mma16816(racc[2 * jp + 1], ga[0], ga[1], ga[2], ga[3], b[2], b[3]);
+        }
+        stage = (stage + 1) % kSStages;
+      }
+      if (g < H) {
+#pragma unroll
+        for (int j = 0; j < 2 * D16; ++j) {
+          const float r0 = racc[j][0] + racc[j][2], r1 = racc[j][1] + racc[j][3];
+          const uint32_t hi = pack2(r0, r1);
+          const uint32_t lo = pack2(r0 - bf16_lo(hi), r1 - bf16_hi(hi));
+          const size_t o = (size_t)(seg * H + g) * RS + (j * 8 + 2 * t) * 2;
+          *reinterpret_cast<uint32_t*>(Rhi + o) = hi;
+          *reinterpret_cast<uint32_t*>(Rlo + o) = lo;
+        }
+      }
+    }
+    cp_wait<0>();
+  }
+  __syncthreads();
+
+  // s_i[head h] = r_{i,h} W_v[:, head h]: one unit = (16 segments, head)
+  {
+    const int NP = dvh >> 4;                      // 16-column pairs per head
+    const int units = ((nv + 15) >> 4) * H;
+    const uint32_t arow = (lane & 7) + ((lane >> 3) & 1) * 8, akc = lane >> 4;
+    for (int unit = warp; unit < units; unit += kSW) {
+      const int mt = unit / H, h = unit - mt * H;
+      float acc[2 * D16][4];
+#pragma unroll
+      for (int j = 0; j < 2 * D16; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
+#pragma unroll
+      for (int kt = 0; kt < D16; ++kt) {
+        uint32_t ah[4], al[4];
+        const size_t o = (size_t)((mt * 16 + arow) * H + h) * RS + (kt * 2 + akc) * 16;
+        ldsm_x4(ah, smem_addr(Rhi + o));
+        ldsm_x4(al, smem_addr(Rlo + o));
+#pragma unroll
+        for (int p = 0; p < D16; ++p) {
+          if (p < NP) {
+            const uint4 b = __ldg(P.imgv + (kt * D16 + h * NP + p) * 32 + lane);
+            mma16816(acc[2 * p], ah[0], ah[1], ah[2], ah[3], b.x, b.y);
+            mma16816(acc[2 * p], al[0], al[1], al[2], al[3], b.x, b.y);
+            mma16816(acc[2 * p + 1], ah[0], ah[1], ah[2], ah[3], b.z, b.w);
+            mma16816(acc[2 * p + 1], al[0], al[1], al[2], al[3], b.z, b.w);
+          }
+        }
+      }
+      const int s0 = mt * 16 + g, s1 = s0 + 8;
+#pragma unroll
+      for (int j = 0; j < 2 * D16; ++j) {
+        if (j < 2 * NP) {
+          const int col = h * dvh + j * 8 + 2 * t;
+          if (s0 < nv) *reinterpret_cast<uint32_t*>(P.Hp + ((size_t)cand * P.Lp + s0) * d + col) = pack2(acc[j][0], acc[j][1]);
+          if (s1 < nv) *reinterpret_cast<uint32_t*>(P.Hp + ((size_t)cand * P.Lp + s1) * d + col) = pack2(acc[j][2], acc[j][3]);
+        }
+      }
+    }
+  }
+  if (P.zero_empty) {
+    const int vec = d / 8;
+    for (int i = tid; i < (P.Lp - nv) * vec; i += kSThreads) {
+      const int seg = nv + i / vec, q = i % vec;
+      *reinterpret_cast<uint4*>(P.Hp + ((size_t)cand * P.Lp + seg) * d + q * 8) = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+size_t stream_smem_bytes(int d, int H, int Lp) {
+  const size_t RS = 2 * (size_t)d + 16;
+  const size_t Lp16 = ((size_t)Lp + 15) & ~(size_t)15;
+  return 2 * Lp16 * H * RS + (size_t)kSW * kSStages * kSRows * RS;
+}
+
+template <int D16>
+int launch_stream(const StreamParams& P, cudaStream_t st) {
+  const size_t smem = stream_smem_bytes(P.d, P.H, P.Lp);
+  LASER_CUDA_OK(cudaFuncSetAttribute(stream_sta_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LaunchScope ls("stream_sta", st);
+  stream_sta_kernel<D16><<<P.U, kSThreads, smem, st>>>(P);
+  return LASER_OK;
+}
+
+}  // namespace
+
+bool stream_supported(const Plan& p) {
+  if (p.dtype != LASER_BF16 || p.maxC > 1) return false;
+  if (p.d % 16 || p.d < 16 || p.d > 128) return false;
+  if (p.H > 8 || p.dvh % 16) return false;
+  if (!gsta_mma_supported(p)) return false;
+  return stream_smem_bytes(p.d, p.H, p.Lp) <= 110 * 1024;
+}
+
+size_t stream_scratch_bytes(const Plan& p) {
+  return align_up((size_t)p.U * p.H * p.d * sizeof(float)) + align_up((size_t)p.d * p.d * 2);
+}
+
+int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+  if (p.N == 0 || p.U == 0) return LASER_OK;
+  StreamParams P;
+  P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
+  P.inv_gamma = p.inv_gamma;
+  P.items = (const bf16*)items; P.cands = (const bf16*)cands;
+  P.Wq = (const bf16*)Wq; P.Wk = (const bf16*)Wk; P.Wv = (const bf16*)Wv;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.u = reinterpret_cast<float*>(ws + p.off_su);
+  P.imgv = reinterpret_cast<uint4*>(ws + p.off_su + align_up((size_t)p.U * p.H * p.d * sizeof(float)));
+  P.Hp = (bf16*)Hprime;
+  P.zero_empty = Hprime != (void*)(ws + p.off_hp);
+  P.status = reinterpret_cast<int*>(ws + p.off_status);
+  {
+    const int user_blocks = (p.U + kPreUsers - 1) / kPreUsers;
+    const size_t smem = (size_t)kPreUsers * (p.d + p.dqk) * sizeof(float);
+    LaunchScope ls("stream_pre", st);
+    stream_pre_kernel<<<user_blocks + 4, 128, smem, st>>>(P, user_blocks);
+  }
+  int rc;
+  switch (p.d / 16) {
+    case 1: rc = launch_stream<1>(P, st); break;
+    case 2: rc = launch_stream<2>(P, st); break;
+    case 3: rc = launch_stream<3>(P, st); break;
+    case 4: rc = launch_stream<4>(P, st); break;
+    case 5: rc = launch_stream<5>(P, st); break;
+    case 6: rc = launch_stream<6>(P, st); break;
+    case 7: rc = launch_stream<7>(P, st); break;
+    case 8: rc = launch_stream<8>(P, st); break;
+    default: return LASER_ERR_UNSUPPORTED;
+  }
+  if (rc != LASER_OK) return rc;
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
 }  // namespace laser

@@ -771,6 +771,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
 
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
                 const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st) {
+  if (gsta_mma_supported(p)) return gsta_mma(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st);
   return simt_gsta(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st);
 }
 

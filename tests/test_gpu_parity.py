@@ -117,6 +117,40 @@ def test_stage_entry_points_simt(dtype):
     assert err_metric(to_np(z), z_ref) <= TOL[dtype]
 
 
+GSTA_CASES = [
+    # U, C, L, d, H, S, M, lengths: the GSTA kernel alone, fed the oracle's H' rounded to bf16
+    dict(U=2, C=9, L=80, d=64, H=4, S=16, M=2, lengths=[80, 41]),                 # 18 candidates: a ragged 16-group
+    dict(U=3, C=21, L=1200, d=64, H=4, S=10, M=2, lengths=[1200, 333, 0]),        # 120 segments: four 32-vector chunks
+    dict(U=2, C=16, L=520, d=128, H=8, S=8, M=3, lengths=[520, 257]),             # 8 heads, 65 segments, three layers
+    dict(U=4, C=5, L=96, d=16, H=1, S=32, M=1, lengths=[96, 1, 33, 0]),           # narrowest width, one head
+    dict(U=2, C=33, L=100, d=48, H=3, S=25, M=2, lengths=[100, 26]),              # d = 48: three 16-wide heads
+    dict(U=1, C=40, L=64, d=32, H=2, S=64, M=0, lengths=[64]),                    # no layers: z = t
+]
+
+
+@pytest.mark.parametrize("case", range(len(GSTA_CASES)))
+def test_gsta_kernel_alone_tensor_path(case):
+    kw = GSTA_CASES[case]
+    w = make_custom(dtype="bf16", seed=300 + case, d_qh=16, **kw)
+    s = w.spec
+    offs = w.cand_offsets
+    if case == 0:                                           # uneven candidate counts across users
+        offs = np.array([0, 13, 18], dtype=np.int32)
+        w.cand_offsets = offs
+    Hp_ref = laser_oracle.sta_forward(w.items, w.lengths, w.cands, offs, w.Wq, w.Wk, w.Wv, s.S, s.H, w.gamma)
+    Hp_in = round_to_dtype(Hp_ref.astype(np.float32), "bf16")
+    for u in range(s.U):                                    # rows of empty segments must never be read
+        nv = -(-int(w.lengths[u]) // s.S)
+        Hp_in[int(offs[u]):int(offs[u + 1]), nv:, :] = np.float32("nan")
+    z_ref = laser_oracle.gsta_forward(np.nan_to_num(Hp_in), w.lengths, offs, w.cands, w.Wg, s.S, s.H, w.tau)
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    z = P.laser_gsta_forward(b.cfg, torch.from_numpy(Hp_in).to(torch.bfloat16).cuda(), b.lengths, b.cand_offsets,
+                             b.cands, b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    assert err_metric(to_np(z), z_ref) <= TOL["bf16"]
+
+
 def test_cfg1_tiny_fp32_full():
     w = make_workload("cfg1")
     e_hp, e_z = check_against_oracle(w, "auto")
