@@ -315,7 +315,7 @@ bool stream_supported(const Plan& p) {
   if (p.d % 16 || p.d < 16 || p.d > 128) return false;
   if (p.H > 8 || p.dvh % 16) return false;
   if (!gsta_mma_supported(p)) return false;
-  return stream_smem_bytes(p.d, p.H, p.Lp) <= 110 * 1024;
+  return stream_smem_bytes(p.d, p.H, p.Lp) <= 200 * 1024;
 }
 
 size_t stream_scratch_bytes(const Plan& p) {

@@ -117,6 +117,47 @@ def test_stage_entry_points_simt(dtype):
     assert err_metric(to_np(z), z_ref) <= TOL[dtype]
 
 
+STREAM = [
+    # one candidate per user: U, L, d, H, S, M, d_qh, lengths
+    dict(U=5, L=300, d=64, H=2, S=64, M=1, d_qh=16, lengths=[300, 64, 65, 1, 0]),        # ragged, an empty user
+    dict(U=3, L=1000, d=64, H=2, S=10, M=1, d_qh=16, lengths=[1000, 9, 500]),            # S = 10: 100 short segments
+    dict(U=4, L=260, d=128, H=4, S=100, M=2, d_qh=16, lengths=[260, 100, 101, 37]),      # S = 100, two GSTA layers
+    dict(U=2, L=96, d=16, H=1, S=96, M=1, d_qh=16, lengths=[96, 40]),                    # narrowest width, S = L
+    dict(U=6, L=128, d=32, H=2, S=16, M=3, d_qh=32, lengths=[128, 17, 16, 15, 0, 77]),   # d_qh = 32, three layers
+    dict(U=3, L=200, d=128, H=8, S=33, M=1, d_qh=16, lengths=[200, 34, 66]),             # eight heads, odd segment size
+]
+
+
+@pytest.mark.parametrize("case", range(len(STREAM)))
+def test_small_shapes_stream_path(case):
+    w = make_custom(dtype="bf16", seed=400 + case, C=1, **STREAM[case])
+    check_against_oracle(w, "stream")
+
+
+def test_stream_path_users_without_candidate_padding_rows_and_determinism():
+    w = make_custom(U=4, C=1, L=192, d=64, H=2, S=32, M=1, dtype="bf16", seed=11, lengths=[192, 50, 70, 3])
+    w.cand_offsets = np.array([0, 1, 1, 2, 3], dtype=np.int32)     # user 1 has no candidate
+    w.cands = w.cands[:3].copy()
+    e_hp, e_z = check_against_oracle(w, "stream")
+    Hp1, z1 = run_forward(w, "stream")
+    Hp1b, z1b = run_forward(w, "stream")
+    assert torch.equal(Hp1, Hp1b) and torch.equal(z1, z1b)
+    w.items[1, :] = -55.0
+    w.items[2, 70:] = 0.125
+    w.items[3, 3:] = -123.0
+    Hp2, z2 = run_forward(w, "stream")
+    assert torch.equal(Hp1, Hp2) and torch.equal(z1, z2)
+
+
+def test_stream_path_is_tighter_than_the_bf16_bound():
+    """The folded one-candidate path keeps fp32-grade intermediates: its H' differs from the oracle only by the
+    final rounding to bf16 (relative 2^-9), far inside the 2e-2 bound of the tensor-core path."""
+    w = make_custom(U=8, C=1, L=512, d=64, H=2, S=64, M=1, dtype="bf16", seed=12)
+    Hp_ref, _ = oracle_forward(w)
+    Hp, _ = run_forward(w, "stream")
+    assert err_metric(to_np(Hp), Hp_ref) <= 4e-3
+
+
 GSTA_CASES = [
     # U, C, L, d, H, S, M, lengths: the GSTA kernel alone, fed the oracle's H' rounded to bf16
     dict(U=2, C=9, L=80, d=64, H=4, S=16, M=2, lengths=[80, 41]),                 # 18 candidates: a ragged 16-group
