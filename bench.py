@@ -201,7 +201,7 @@ def dominant_kernel_roofline(w, prof, peaks):
                 "frac_of_nominal": achieved / NOMINAL["hbm_gbs"]}
     if name.startswith("sta"):
         flops = work["attn_flops"]
-    elif name.startswith("proj"):
+    elif "proj" in name:
         flops = work["proj_flops"]
     else:
         flops = work["gsta_flops"]

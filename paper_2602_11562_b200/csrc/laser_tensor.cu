@@ -23,7 +23,8 @@ using namespace ptx;
 constexpr int kCandTile = 128;        // candidates per tile = MMA M = TMEM lanes
 constexpr int kProjThreads = 128;
 constexpr int kProjTmemCols = 256;    // K / Q accumulator at column 0, V^T accumulator at column 128
-constexpr int kStaThreads = 512;
+constexpr int kGateGroups = 4;        // gate warpgroups; each owns one score / gate buffer in TMEM
+constexpr int kStaThreads = (8 + 4 * kGateGroups) * 32;
 constexpr int kStaTmemCols = 512;
 constexpr int kKvStages = 4;
 
@@ -31,6 +32,7 @@ struct TcParams {
   int U, L, d, dqk, H, S, Lp, N, dqh, dvh, maxC;
   int IT, NT, NTG, NG, n_tiles;       // items per tile, tiles per segment, tiles per projection unit, units per segment
   int cand_tiles_max;
+  int n_obuf;                         // output accumulators in TMEM (2 when they fit beside the gate buffers, else 1)
   float q_scale;                      // 1 / (2 gamma)
   const bf16 *items, *cands, *Wq, *Wk, *Wv;
   const int *lengths, *cand_offsets;
@@ -364,10 +366,16 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
 }
 
 // ------------------------------------------------------------------------------------------------------- attention
-// Walks the attention units (user, candidate tile, segment) of a contiguous id range in order.
+// Walks the attention units (user, candidate tile, segment) of a contiguous id range in order.  The user's shape is
+// cached, so a step inside one user costs a few integer instructions.
 struct UnitWalker {
   int u, j, seg;
-  UserShape us;
+  int nseg, ctiles, c0, nc, last_tiles;
+  __device__ void load_user(const TcParams& P) {
+    const UserShape s = user_shape(P, u);
+    nseg = s.nseg; ctiles = s.ctiles; c0 = s.c0; nc = s.nc;
+    last_tiles = s.nseg > 0 ? min(P.NT, (s.len - (s.nseg - 1) * P.S + P.IT - 1) / P.IT) : 0;
+  }
   __device__ void init(const TcParams& P, int id) {
     int lo = 0, hi = P.U;   // unit_start[lo] <= id < unit_start[hi]
     while (hi - lo > 1) {
@@ -375,42 +383,48 @@ struct UnitWalker {
       if (P.unit_start[mid] <= id) lo = mid; else hi = mid;
     }
     u = lo;
-    us = user_shape(P, u);
+    load_user(P);
     const int local = id - P.unit_start[u];
-    j = local / us.nseg;
-    seg = local - j * us.nseg;
+    j = local / nseg;
+    seg = local - j * nseg;
   }
   __device__ void next(const TcParams& P) {
-    if (++seg < us.nseg) return;
+    if (++seg < nseg) return;
     seg = 0;
-    if (++j < us.ctiles) return;
+    if (++j < ctiles) return;
     j = 0;
     do {
       ++u;
       if (u >= P.U) return;
-      us = user_shape(P, u);
-    } while (us.nseg == 0 || us.ctiles == 0);
+      load_user(P);
+    } while (nseg == 0 || ctiles == 0);
   }
   // tiles of the current segment that hold at least one valid item
-  __device__ int ntiles(const TcParams& P) const {
-    const int seg_items = min(P.S, us.len - seg * P.S);
-    return min(P.NT, (seg_items + P.IT - 1) / P.IT);
-  }
+  __device__ int ntiles(const TcParams& P) const { return seg == nseg - 1 ? last_tiles : P.NT; }
 };
 
 struct StaBars {
   uint64_t q_full[2], q_empty[2];
   uint64_t kv_full[kKvStages], kv_empty[kKvStages];
-  uint64_t s_full[2], p_full[2], p_empty[2];
+  uint64_t s_full[kGateGroups], p_full[kGateGroups], sp_free[kGateGroups];
   uint64_t o_full[2], o_empty[2];
-  uint64_t done;
+  uint64_t done[2];
 };
 
+// Roles of the 24 warps of a block (one block per SM):
+//   warp 0      bulk-copy producer: Q tile per (user, candidate tile), K / V^T tile per item tile, through mbarrier rings
+//   warp 1      score issuer:  S = Q_h K_h^T for every (item tile, head) into that gate-unit's TMEM buffer
+//   warp 2      TMEM allocation
+//   warp 3      value issuer:  O_h += P' V_h, with P' read from TMEM
+//   warps 4-7   epilogue: H' = (SV + O) / 2 per finished segment
+//   warps 8-23  four gate warpgroups: P' = tanh(S), written over S in place
+// Gate-unit g (counting (tile, head) pairs of this block) lives in buffer g % 4 and is handled by warpgroup g % 4.
 __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ StaBars bars;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
+  __shared__ __align__(16) float sv_s[4][2][128];   // per epilogue warp, double-buffered: SV row of the segment
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d = P.d, dqk = P.dqk, IT = P.IT, H = P.H;
@@ -423,17 +437,19 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.q_full[i], 1);
       mbar_init(&bars.q_empty[i], 1);
-      mbar_init(&bars.s_full[i], 1);
-      mbar_init(&bars.p_full[i], 4);
-      mbar_init(&bars.p_empty[i], 1);
       mbar_init(&bars.o_full[i], 1);
       mbar_init(&bars.o_empty[i], 4);
+      mbar_init(&bars.done[i], 1);
+    }
+    for (int i = 0; i < kGateGroups; ++i) {
+      mbar_init(&bars.s_full[i], 1);
+      mbar_init(&bars.p_full[i], 4);
+      mbar_init(&bars.sp_free[i], 1);
     }
     for (int i = 0; i < kKvStages; ++i) {
       mbar_init(&bars.kv_full[i], 1);
       mbar_init(&bars.kv_empty[i], 1);
     }
-    mbar_init(&bars.done, 1);
     s_abort = 0;
     fence_mbar_init();
   }
@@ -447,8 +463,10 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
 
-  // TMEM columns: O[2] (d each), S[2] (IT each, fp32 scores), P[2] (IT/2 each, packed bf16 pairs)
-  const uint32_t colO = 0, colS = 2 * d, colP = 2 * d + 2 * IT;
+  // TMEM columns: O[n_obuf] (d each), then one buffer of IT columns per gate warpgroup.  A buffer first holds the fp32
+  // scores of one (tile, head); its warpgroup overwrites them in place with the packed bf16 gates (IT/2 columns).
+  const int n_obuf = P.n_obuf;
+  const uint32_t colO = 0, colSP = n_obuf * d;
 
   // this block's contiguous range of units
   const int n_units = P.counters[0];
@@ -459,12 +477,12 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
 
   if (my_units > 0) {
     if (warp == 0) {
-      // ------------------------------------------------------------------ TMA producer
+      // ------------------------------------------------------------------ bulk-copy producer
       if (lane == 0) {
         UnitWalker w;
         w.init(P, unit_lo);
         int pu = -1, pj = -1;
-        uint32_t qcount = 0, kvcount = 0;
+        uint32_t qcount = 0, st = 0, kv_par = 1;      // kv_par: parity that means "stage st is free"
         bool ok = true;
         for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
           if (w.u != pu || w.j != pj) {
@@ -479,131 +497,124 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
             pj = w.j;
           }
           const int nt = w.ntiles(P);
+          const size_t tile0 = (size_t)w.u * P.n_tiles + w.seg * P.NT;
           for (int t = 0; t < nt && ok; ++t) {
-            const int st = kvcount % kKvStages;
-            ok = mbar_wait(&bars.kv_empty[st], ((kvcount / kKvStages) & 1) ^ 1, abortp);
+            ok = mbar_wait(&bars.kv_empty[st], kv_par, abortp);
             if (!ok) break;
-            const size_t tile = (size_t)w.u * P.n_tiles + w.seg * P.NT + t;
             mbar_arrive_expect_tx(&bars.kv_full[st], k_bytes + v_bytes);
-            bulk_g2s(Ks + st * k_bytes, P.Kblk + tile * ((size_t)IT * dqk), k_bytes, &bars.kv_full[st]);
-            bulk_g2s(Vs + st * v_bytes, P.Vtblk + tile * ((size_t)IT * d), v_bytes, &bars.kv_full[st]);
-            ++kvcount;
+            bulk_g2s(Ks + st * k_bytes, P.Kblk + (tile0 + t) * ((size_t)IT * dqk), k_bytes, &bars.kv_full[st]);
+            bulk_g2s(Vs + st * v_bytes, P.Vtblk + (tile0 + t) * ((size_t)IT * d), v_bytes, &bars.kv_full[st]);
+            if (++st == kKvStages) { st = 0; kv_par ^= 1; }
           }
         }
       }
     } else if (warp == 1) {
-      // ------------------------------------------------------------------ MMA issuer
+      // ------------------------------------------------------------------ score issuer
       if (lane == 0) {
-        const uint32_t id1 = idesc_bf16(128, IT);        // scores: 128 candidates x IT items, K = dqh
-        const uint32_t id2 = idesc_bf16(128, P.dvh);     // O_h: 128 candidates x dvh, K = IT items
+        const uint32_t id1 = idesc_bf16(128, IT);        // 128 candidates x IT items, K = dqh
         const uint32_t qk_sbo = (P.dqh >> 3) * 128;      // 8-row groups of a [rows x dqh] head block
-        const uint32_t v_lbo = (P.dvh >> 3) * 128;       // V^T head block: k-chunks (8 items) are dvh/8 core matrices apart
-        const int ks1 = P.dqh >> 4, ks2 = IT >> 4;
-
-        // cursor 1 issues the score MMAs two gate-units ahead of cursor 2, which issues the P'V MMAs
-        UnitWalker w1, w2;
-        w1.init(P, unit_lo);
-        w2.init(P, unit_lo);
-        int it1 = 0, t1 = 0, h1 = 0, nt1 = w1.ntiles(P);
-        int it2 = 0, t2 = 0, h2 = 0, nt2 = w2.ntiles(P);
-        uint32_t q1 = 0, kv1 = 0, kv2 = 0, g1 = 0, g2 = 0, seg2 = 0;
-        int pu1 = -1, pj1 = -1;
+        const int ks1 = P.dqh >> 4;
+        const uint64_t q_desc0 = smem_desc(smem_u32(Qs), 128, qk_sbo);
+        const uint64_t k_desc0 = smem_desc(smem_u32(Ks), 128, qk_sbo);
+        const uint32_t q_head = (kCandTile * P.dqh * 2) >> 4, k_head = (IT * P.dqh * 2) >> 4;   // descriptor units
+        UnitWalker w;
+        w.init(P, unit_lo);
+        int pu = -1, pj = -1;
+        uint32_t qcount = 0, st = 0, kv_par = 0, gb = 0, sp_par = 1;
+        uint64_t q_desc = q_desc0;
         bool ok = true;
-
-        auto issue1 = [&]() {
-          if (it1 >= my_units || !ok) return;
-          if (t1 == 0 && h1 == 0 && (w1.u != pu1 || w1.j != pj1)) {
-            if (pu1 >= 0) { tc_commit(&bars.q_empty[(q1 - 1) & 1]); }
-            ok = mbar_wait(&bars.q_full[q1 & 1], (q1 >> 1) & 1, abortp);
-            if (!ok) return;
-            ++q1;
-            pu1 = w1.u;
-            pj1 = w1.j;
-          }
-          const int st = kv1 % kKvStages;
-          if (h1 == 0) {
-            ok = mbar_wait(&bars.kv_full[st], (kv1 / kKvStages) & 1, abortp);
-            if (!ok) return;
-          }
-          tc_fence_after();
-          const uint32_t qa = smem_u32(Qs + ((q1 - 1) & 1) * q_bytes) + h1 * (kCandTile * P.dqh * 2);
-          const uint32_t ka = smem_u32(Ks + st * k_bytes) + h1 * (IT * P.dqh * 2);
-          const uint32_t dS = tmem + colS + (g1 & 1) * IT;
-          for (int ks = 0; ks < ks1; ++ks)
-            mma_ss(dS, smem_desc(qa + ks * 256, 128, qk_sbo), smem_desc(ka + ks * 256, 128, qk_sbo), id1, ks > 0);
-          tc_commit(&bars.s_full[g1 & 1]);
-          ++g1;
-          if (++h1 == H) {
-            h1 = 0;
-            ++kv1;
-            if (++t1 == nt1) {
-              t1 = 0;
-              ++it1;
-              w1.next(P);
-              if (it1 < my_units) nt1 = w1.ntiles(P);
-            }
-          }
-        };
-
-        issue1();
-        issue1();
-        while (it2 < my_units && ok) {
-          const int pb = g2 & 1;
-          ok = mbar_wait(&bars.p_full[pb], (g2 >> 1) & 1, abortp);
-          if (!ok) break;
-          issue1();                                        // scores of gate-unit g2 + 2 reuse the buffer just drained
-          if (!ok) break;
-          const int ob = seg2 & 1;
-          if (t2 == 0 && h2 == 0) {
-            ok = mbar_wait(&bars.o_empty[ob], ((seg2 >> 1) & 1) ^ 1, abortp);
+        for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+          if (w.u != pu || w.j != pj) {
+            if (pu >= 0) tc_commit(&bars.q_empty[(qcount - 1) & 1]);   // every score MMA on the old Q tile is issued
+            ok = mbar_wait(&bars.q_full[qcount & 1], (qcount >> 1) & 1, abortp);
             if (!ok) break;
+            q_desc = q_desc0 + (uint64_t)((qcount & 1) * (q_bytes >> 4));
+            ++qcount;
+            pu = w.u;
+            pj = w.j;
           }
-          tc_fence_after();
-          const int st = kv2 % kKvStages;
-          const uint32_t va = smem_u32(Vs + st * v_bytes) + h2 * (IT * P.dvh * 2);
-          const uint32_t dO = tmem + colO + ob * d + h2 * P.dvh;
-          const uint32_t aP = tmem + colP + pb * (IT >> 1);
-          for (int ks = 0; ks < ks2; ++ks)
-            mma_ts(dO, aP + ks * 8, smem_desc(va + ks * 2 * v_lbo, v_lbo, 128), id2, (t2 > 0 || ks > 0) ? 1u : 0u);
-          tc_commit(&bars.p_empty[pb]);
-          ++g2;
-          if (++h2 == H) {
-            h2 = 0;
-            tc_commit(&bars.kv_empty[st]);
-            ++kv2;
-            if (++t2 == nt2) {
-              t2 = 0;
-              tc_commit(&bars.o_full[ob]);
-              ++seg2;
-              ++it2;
-              w2.next(P);
-              if (it2 < my_units) nt2 = w2.ntiles(P);
+          const int nt = w.ntiles(P);
+          for (int t = 0; t < nt && ok; ++t) {
+            ok = mbar_wait(&bars.kv_full[st], kv_par, abortp);
+            if (!ok) break;
+            const uint64_t k_desc = k_desc0 + (uint64_t)(st * (k_bytes >> 4));
+            for (int h = 0; h < H; ++h) {
+              ok = mbar_wait(&bars.sp_free[gb], sp_par, abortp);   // P'V of the unit that used this buffer is done
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t dS = tmem + colSP + gb * IT;
+              for (int ks = 0; ks < ks1; ++ks)
+                mma_ss(dS, q_desc + h * q_head + ks * 16, k_desc + h * k_head + ks * 16, id1, ks > 0);
+              tc_commit(&bars.s_full[gb]);
+              if (++gb == kGateGroups) { gb = 0; sp_par ^= 1; }
             }
+            if (++st == kKvStages) { st = 0; kv_par ^= 1; }
           }
         }
-        // every MMA issued by this thread has completed once `done` flips
-        tc_commit(&bars.done);
-        mbar_wait(&bars.done, 0, abortp);
+        tc_commit(&bars.done[0]);
+        mbar_wait(&bars.done[0], 0, abortp);
+      }
+    } else if (warp == 3) {
+      // ------------------------------------------------------------------ value issuer
+      if (lane == 0) {
+        const uint32_t id2 = idesc_bf16(128, P.dvh);     // 128 candidates x dvh, K = IT items
+        const uint32_t v_lbo = (P.dvh >> 3) * 128;       // V^T head block: k-chunks (8 items) are dvh/8 core matrices apart
+        const int ks2 = IT >> 4;
+        const uint64_t v_desc0 = smem_desc(smem_u32(Vs), v_lbo, 128);
+        const uint32_t v_head = (IT * P.dvh * 2) >> 4, v_step = (2 * v_lbo) >> 4;
+        UnitWalker w;
+        w.init(P, unit_lo);
+        uint32_t st = 0, gb = 0, p_par = 0, ob = 0, o_par = 1;
+        bool ok = true;
+        for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+          const int nt = w.ntiles(P);
+          const uint32_t dO0 = tmem + colO + ob * d;
+          for (int t = 0; t < nt && ok; ++t) {
+            const uint64_t v_desc = v_desc0 + (uint64_t)(st * (v_bytes >> 4));
+            for (int h = 0; h < H; ++h) {
+              ok = mbar_wait(&bars.p_full[gb], p_par, abortp);
+              if (!ok) break;
+              if (t == 0 && h == 0) {
+                ok = mbar_wait(&bars.o_empty[ob], o_par, abortp);
+                if (!ok) break;
+              }
+              tc_fence_after();
+              const uint32_t aP = tmem + colSP + gb * IT;
+              const uint32_t dO = dO0 + h * P.dvh;
+              const uint64_t vd = v_desc + h * v_head;
+#pragma unroll 4
+              for (int ks = 0; ks < ks2; ++ks) mma_ts(dO, aP + ks * 8, vd + ks * v_step, id2, (t | ks) != 0);
+              tc_commit(&bars.sp_free[gb]);
+              if (++gb == kGateGroups) { gb = 0; p_par ^= 1; }
+            }
+            tc_commit(&bars.kv_empty[st]);   // the scores of this tile were consumed before its gates were written
+            if (++st == kKvStages) st = 0;
+          }
+          tc_commit(&bars.o_full[ob]);
+          if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
+        }
+        tc_commit(&bars.done[1]);
+        mbar_wait(&bars.done[1], 0, abortp);
       }
     } else if (warp >= 8) {
-      // ------------------------------------------------------------------ gate warps: P' = tanh(scores)
-      const int wg = (warp - 8) >> 2;                       // warpgroup 0 / 1 owns score and P buffer 0 / 1
+      // ------------------------------------------------------------------ gate warps: P' = tanh(scores), in place
+      const int wg = (warp - 8) >> 2;                       // warpgroup wg owns buffer wg
       const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + lane_base + colS + wg * IT;
-      const uint32_t tP = tmem + lane_base + colP + wg * (IT >> 1);
+      const uint32_t tS = tmem + lane_base + colSP + wg * IT;
       UnitWalker w;
       w.init(P, unit_lo);
-      uint32_t g = 0, k = 0;
+      uint32_t g = 0, par = 0;
       bool ok = true;
       for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
         const int n_sub = w.ntiles(P) * H;
         for (int s = 0; s < n_sub && ok; ++s, ++g) {
-          if ((int)(g & 1) != wg) continue;
-          ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], k & 1, abortp));
+          if ((int)(g % kGateGroups) != wg) continue;
+          ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], par, abortp));
           if (!ok) break;
-          ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_empty[wg], (k & 1) ^ 1, abortp));
-          if (!ok) break;
+          par ^= 1;
           tc_fence_after();
+          // columns [c, c+32) of the scores become columns [c/2, c/2+16) of the gates: always inside the part of the
+          // buffer that has already been read
           int c = 0;
           for (; c + 32 <= IT; c += 32) {
             uint32_t v[32], o[16];
@@ -612,7 +623,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
 #pragma unroll
             for (int e = 0; e < 16; ++e)
               o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
-            tmem_st16(tP + (c >> 1), o);
+            tmem_st16(tS + (c >> 1), o);
           }
           if (c < IT) {   // 16-column tail
             uint32_t v[16], o[8];
@@ -621,13 +632,12 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
 #pragma unroll
             for (int e = 0; e < 8; ++e)
               o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
-            tmem_st8(tP + (c >> 1), o);
+            tmem_st8(tS + (c >> 1), o);
           }
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.p_full[wg]);
-          ++k;
         }
       }
     } else if (warp >= 4) {
@@ -637,25 +647,40 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
       const int m = q * 32 + lane;
       UnitWalker w;
       w.init(P, unit_lo);
+      uint32_t ob = 0, o_par = 0;
       bool ok = true;
-      for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
-        const int ob = it & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], (it >> 1) & 1, abortp));
+      // the SV row of the next segment is fetched into registers one unit ahead and handed over through shared memory
+      float sv_reg[4];
+      auto fetch_sv = [&](const UnitWalker& ww) {
+        const float* sv = P.SV + ((size_t)ww.u * P.Lp + ww.seg) * d;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sv_reg[i] = lane + 32 * i < d ? __ldg(sv + lane + 32 * i) : 0.f;
+      };
+      fetch_sv(w);
+      for (int it = 0; it < my_units && ok; ++it) {
+        float* svb = sv_s[q][it & 1];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) svb[lane + 32 * i] = sv_reg[i];
+        UnitWalker wn = w;
+        wn.next(P);
+        if (it + 1 < my_units) fetch_sv(wn);
+        __syncwarp();
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], o_par, abortp));
         if (!ok) break;
         tc_fence_after();
         const int ci = w.j * kCandTile + m;
-        const bool valid = ci < w.us.nc;
-        const float* sv = P.SV + ((size_t)w.u * P.Lp + w.seg) * d;
-        bf16* out = P.Hp + ((size_t)(w.us.c0 + (valid ? ci : 0)) * P.Lp + w.seg) * d;
+        const bool valid = ci < w.nc;
+        bf16* out = P.Hp + ((size_t)(w.c0 + (valid ? ci : 0)) * P.Lp + w.seg) * d;
+        const uint32_t tO = tmem + lane_base + colO + ob * d;
         for (int c = 0; c < d; c += 16) {
           uint32_t v[16];
-          tmem_ld16(tmem + lane_base + colO + ob * d + c, v);
+          tmem_ld16(tO + c, v);
           tc_wait_ld();
           if (valid) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-              const float4 s0 = __ldg(reinterpret_cast<const float4*>(sv + c + half * 8));
-              const float4 s1 = __ldg(reinterpret_cast<const float4*>(sv + c + half * 8 + 4));
+              const float4 s0 = *reinterpret_cast<const float4*>(svb + c + half * 8);
+              const float4 s1 = *reinterpret_cast<const float4*>(svb + c + half * 8 + 4);
               uint4 o;
               o.x = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 0]) + s0.x), 0.5f * (__uint_as_float(v[half * 8 + 1]) + s0.y));
               o.y = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 2]) + s0.z), 0.5f * (__uint_as_float(v[half * 8 + 3]) + s0.w));
@@ -668,6 +693,8 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
+        if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
+        w = wn;
       }
     }
   }
@@ -694,6 +721,7 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.dqh = p.dqh; P.dvh = p.dvh; P.maxC = p.maxC;
   P.IT = p.tg.IT; P.NT = p.tg.NT; P.n_tiles = p.tg.n_tiles; P.cand_tiles_max = p.tg.cand_tiles_max;
+  P.n_obuf = 2 * p.d + kGateGroups * P.IT <= kStaTmemCols ? 2 : 1;
   P.NTG = P.IT <= 64 ? (128 / P.IT < P.NT ? 128 / P.IT : P.NT) : 1;
   P.NG = (P.NT + P.NTG - 1) / P.NTG;
   P.q_scale = 0.5f * p.inv_gamma;
@@ -728,7 +756,8 @@ bool tensor_supported(const Plan& p) {
 }
 
 void tensor_geometry(const Plan& p, TensorGeom* g) {
-  const int it_max = p.d > 64 ? 64 : 128;   // TMEM: 2 d (outputs) + 3 IT (scores, packed gates) <= 512 columns
+  // TMEM: one or two output accumulators (d columns each) + kGateGroups score / gate buffers (IT columns each) <= 512
+  const int it_max = ((512 - p.d) / kGateGroups) / 16 * 16 > 128 ? 128 : ((512 - p.d) / kGateGroups) / 16 * 16;
   g->NT = (p.S + it_max - 1) / it_max;
   const int per = (p.S + g->NT - 1) / g->NT;
   g->IT = (per + 15) / 16 * 16;
