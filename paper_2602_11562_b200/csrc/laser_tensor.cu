@@ -24,7 +24,7 @@ constexpr int kCandTile = 128;        // candidates per tile = MMA M = TMEM lane
 constexpr int kProjThreads = 128;
 constexpr int kProjTmemCols = 256;    // K / Q accumulator at column 0, V^T accumulator at column 128
 constexpr int kGateGroups = 4;        // gate warpgroups; each owns one score / gate buffer in TMEM
-constexpr int kStaThreads = (8 + 4 * kGateGroups) * 32;
+constexpr int kStaThreads = (9 + 4 * kGateGroups) * 32;
 constexpr int kStaTmemCols = 512;
 constexpr int kKvStages = 4;
 
@@ -370,11 +370,12 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
 // cached, so a step inside one user costs a few integer instructions.
 struct UnitWalker {
   int u, j, seg;
-  int nseg, ctiles, c0, nc, last_tiles;
+  int nseg, ctiles, c0, nc, last_items, last_tiles;
   __device__ void load_user(const TcParams& P) {
     const UserShape s = user_shape(P, u);
     nseg = s.nseg; ctiles = s.ctiles; c0 = s.c0; nc = s.nc;
-    last_tiles = s.nseg > 0 ? min(P.NT, (s.len - (s.nseg - 1) * P.S + P.IT - 1) / P.IT) : 0;
+    last_items = s.nseg > 0 ? s.len - (s.nseg - 1) * P.S : 0;       // items of the last non-empty segment
+    last_tiles = min(P.NT, (last_items + P.IT - 1) / P.IT);
   }
   __device__ void init(const TcParams& P, int id) {
     int lo = 0, hi = P.U;   // unit_start[lo] <= id < unit_start[hi]
@@ -401,24 +402,37 @@ struct UnitWalker {
   }
   // tiles of the current segment that hold at least one valid item
   __device__ int ntiles(const TcParams& P) const { return seg == nseg - 1 ? last_tiles : P.NT; }
+  // columns of tile t that can hold a non-zero gate: its valid items rounded up to the MMA k-step (16)
+  __device__ int tile_cols(const TcParams& P, int t) const {
+    const int items = min(P.IT, (seg == nseg - 1 ? last_items : P.S) - t * P.IT);
+    return (items + 15) & ~15;
+  }
 };
 
 struct StaBars {
   uint64_t q_full[2], q_empty[2];
   uint64_t kv_full[kKvStages], kv_empty[kKvStages];
-  uint64_t s_full[kGateGroups], p_full[kGateGroups], sp_free[kGateGroups];
+  uint64_t s_full[kGateGroups], s_free[kGateGroups], p_full[kGateGroups], p_free[kGateGroups];
   uint64_t o_full[2], o_empty[2];
-  uint64_t done[2];
+  uint64_t done[kGateGroups];
 };
 
-// Roles of the 24 warps of a block (one block per SM):
-//   warp 0      bulk-copy producer: Q tile per (user, candidate tile), K / V^T tile per item tile, through mbarrier rings
-//   warp 1      score issuer:  S = Q_h K_h^T for every (item tile, head) into that gate-unit's TMEM buffer
-//   warp 2      TMEM allocation
-//   warp 3      value issuer:  O_h += P' V_h, with P' read from TMEM
-//   warps 4-7   epilogue: H' = (SV + O) / 2 per finished segment
-//   warps 8-23  four gate warpgroups: P' = tanh(S), written over S in place
-// Gate-unit g (counting (tile, head) pairs of this block) lives in buffer g % 4 and is handled by warpgroup g % 4.
+constexpr int kProducerWarp = 8 + 4 * kGateGroups;
+constexpr int kItMax = 64;                          // items per tile: one 64-column fp32 score buffer per warpgroup
+constexpr uint32_t kColS = 0;                       // TMEM: scores  [kGateGroups][kItMax] fp32
+constexpr uint32_t kColP = kGateGroups * kItMax;    //       gates   [kGateGroups][kItMax / 2] packed bf16 pairs
+constexpr uint32_t kColO = kColP + kGateGroups * (kItMax / 2);   // outputs [n_obuf][d] fp32
+
+// Roles of the 25 warps of a block (one block per SM):
+//   warps 0-3   MMA issuers, one per gate warpgroup (the warp runs the loop, one elected lane issues)
+//   warps 4-7   epilogue: H' = (SV + O) / 2 per finished segment, staged in shared memory, written by bulk stores
+//   warps 8-23  four gate warpgroups: P' = tanh(S)
+//   warp 24     bulk-copy producer (Q tile per (user, candidate tile), K / V^T tile per item tile, mbarrier rings) and
+//               TMEM allocation
+// A gate-unit is one (item tile, head).  Head h always belongs to warpgroup / issuer h % 4, which owns one score buffer
+// and one gate buffer in TMEM.  Per unit: the issuer writes S = Q_h K_h^T; the warpgroup reads it (releasing the score
+// buffer for the issuer's next unit as soon as the last column is in registers), writes P' = tanh(S) as packed bf16; the
+// issuer accumulates O_h += P' V_h.  All MMAs into a head's accumulator come from one thread, in order.
 __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ StaBars bars;
@@ -428,32 +442,36 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d = P.d, dqk = P.dqk, IT = P.IT, H = P.H;
+  const int n_groups = H < kGateGroups ? H : kGateGroups;     // warpgroups / issuers that own at least one head
   const uint32_t q_bytes = kCandTile * dqk * 2, k_bytes = IT * dqk * 2, v_bytes = IT * d * 2;
+  const uint32_t out_row = d * 2 + 16;            // bytes per staged output row (padding spreads the banks)
   uint8_t* Qs = smem_raw;                         // [2][q_bytes]
   uint8_t* Ks = Qs + 2 * q_bytes;                 // [kKvStages][k_bytes]
   uint8_t* Vs = Ks + kKvStages * k_bytes;         // [kKvStages][v_bytes]
+  uint8_t* Os = Vs + kKvStages * v_bytes;         // [2][kCandTile][out_row]  staged H' rows
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.q_full[i], 1);
-      mbar_init(&bars.q_empty[i], 1);
-      mbar_init(&bars.o_full[i], 1);
+      mbar_init(&bars.q_empty[i], n_groups);      // every issuer releases the old Q tile
+      mbar_init(&bars.o_full[i], n_groups);       // every issuer finishes its heads of the segment
       mbar_init(&bars.o_empty[i], 4);
-      mbar_init(&bars.done[i], 1);
     }
     for (int i = 0; i < kGateGroups; ++i) {
       mbar_init(&bars.s_full[i], 1);
+      mbar_init(&bars.s_free[i], 4);
       mbar_init(&bars.p_full[i], 4);
-      mbar_init(&bars.sp_free[i], 1);
+      mbar_init(&bars.p_free[i], 1);
+      mbar_init(&bars.done[i], 1);
     }
     for (int i = 0; i < kKvStages; ++i) {
       mbar_init(&bars.kv_full[i], 1);
-      mbar_init(&bars.kv_empty[i], 1);
+      mbar_init(&bars.kv_empty[i], H);            // one arrival per (tile, head)
     }
     s_abort = 0;
     fence_mbar_init();
   }
-  if (warp == 2) {
+  if (warp == kProducerWarp) {
     tmem_alloc(&s_tmem, kStaTmemCols);
     tmem_relinquish();
   }
@@ -462,11 +480,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
-
-  // TMEM columns: O[n_obuf] (d each), then one buffer of IT columns per gate warpgroup.  A buffer first holds the fp32
-  // scores of one (tile, head); its warpgroup overwrites them in place with the packed bf16 gates (IT/2 columns).
   const int n_obuf = P.n_obuf;
-  const uint32_t colO = 0, colSP = n_obuf * d;
 
   // this block's contiguous range of units
   const int n_units = P.counters[0];
@@ -476,7 +490,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   const int my_units = unit_hi - unit_lo;
 
   if (my_units > 0) {
-    if (warp == 0) {
+    if (warp == kProducerWarp) {
       // ------------------------------------------------------------------ bulk-copy producer
       if (lane == 0) {
         UnitWalker w;
@@ -508,136 +522,181 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           }
         }
       }
-    } else if (warp == 1) {
-      // ------------------------------------------------------------------ score issuer
-      if (lane == 0) {
-        const uint32_t id1 = idesc_bf16(128, IT);        // 128 candidates x IT items, K = dqh
+    } else if (warp < kGateGroups) {
+      // ------------------------------------------------------------------ MMA issuer of warpgroup `warp`
+      // The whole warp runs the loop, so that addresses and descriptors stay warp-uniform; one elected lane issues.
+      if (warp < n_groups) {
+        const int wgi = warp;
+        const bool leader = elect_one();
+        const uint32_t id1 = idesc_bf16(128, IT);        // scores: 128 candidates x IT items, K = dqh
+        const uint32_t id2 = idesc_bf16(128, P.dvh);     // O_h: 128 candidates x dvh, K = the tile's items
         const uint32_t qk_sbo = (P.dqh >> 3) * 128;      // 8-row groups of a [rows x dqh] head block
+        const uint32_t v_lbo = (P.dvh >> 3) * 128;       // V^T head block: k-chunks (8 items) are dvh/8 core matrices apart
         const int ks1 = P.dqh >> 4;
         const uint64_t q_desc0 = smem_desc(smem_u32(Qs), 128, qk_sbo);
         const uint64_t k_desc0 = smem_desc(smem_u32(Ks), 128, qk_sbo);
-        const uint32_t q_head = (kCandTile * P.dqh * 2) >> 4, k_head = (IT * P.dqh * 2) >> 4;   // descriptor units
-        UnitWalker w;
-        w.init(P, unit_lo);
-        int pu = -1, pj = -1;
-        uint32_t qcount = 0, st = 0, kv_par = 0, gb = 0, sp_par = 1;
+        const uint64_t v_desc0 = smem_desc(smem_u32(Vs), v_lbo, 128);
+        const uint32_t q_head = (kCandTile * P.dqh * 2) >> 4, k_head = (IT * P.dqh * 2) >> 4;   // in 16-byte units
+        const uint32_t v_head = (IT * P.dvh * 2) >> 4, v_step = (2 * v_lbo) >> 4;
+        const uint32_t tS = tmem + kColS + wgi * kItMax, tP = tmem + kColP + wgi * (kItMax / 2);
+
+        struct Cursor {
+          UnitWalker w;
+          int it, t, h, nt;
+          uint32_t st, kv_par;                            // K / V stage of the current tile and its "full" parity
+        };
+        auto advance = [&](Cursor& c) -> bool {           // to this issuer's next gate-unit; false past the end
+          c.h += kGateGroups;
+          if (c.h < H) return true;
+          c.h = wgi;
+          if (++c.st == kKvStages) { c.st = 0; c.kv_par ^= 1; }
+          if (++c.t < c.nt) return true;
+          c.t = 0;
+          if (++c.it >= my_units) return false;
+          c.w.next(P);
+          c.nt = c.w.ntiles(P);
+          return true;
+        };
+        auto wait_all = [&](uint64_t* bar, uint32_t parity) {
+          return __all_sync(0xffffffffu, mbar_wait(bar, parity, abortp)) != 0;
+        };
+        int qu = -1, qj = -1;
+        uint32_t qcount = 0, sf_par = 0, p_par = 0, ob = 0, o_par = 1;
         uint64_t q_desc = q_desc0;
         bool ok = true;
-        for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
-          if (w.u != pu || w.j != pj) {
-            if (pu >= 0) tc_commit(&bars.q_empty[(qcount - 1) & 1]);   // every score MMA on the old Q tile is issued
-            ok = mbar_wait(&bars.q_full[qcount & 1], (qcount >> 1) & 1, abortp);
-            if (!ok) break;
+
+        auto issue_scores = [&](const Cursor& c) {
+          if (c.w.u != qu || c.w.j != qj) {               // first unit on a new candidate tile
+            if (qu >= 0 && leader) tc_commit(&bars.q_empty[(qcount - 1) & 1]);   // my score MMAs on the old Q tile are issued
+            ok = wait_all(&bars.q_full[qcount & 1], (qcount >> 1) & 1);
+            if (!ok) return;
             q_desc = q_desc0 + (uint64_t)((qcount & 1) * (q_bytes >> 4));
             ++qcount;
-            pu = w.u;
-            pj = w.j;
+            qu = c.w.u;
+            qj = c.w.j;
           }
-          const int nt = w.ntiles(P);
-          for (int t = 0; t < nt && ok; ++t) {
-            ok = mbar_wait(&bars.kv_full[st], kv_par, abortp);
-            if (!ok) break;
-            const uint64_t k_desc = k_desc0 + (uint64_t)(st * (k_bytes >> 4));
-            for (int h = 0; h < H; ++h) {
-              ok = mbar_wait(&bars.sp_free[gb], sp_par, abortp);   // P'V of the unit that used this buffer is done
-              if (!ok) break;
-              tc_fence_after();
-              const uint32_t dS = tmem + colSP + gb * IT;
-              for (int ks = 0; ks < ks1; ++ks)
-                mma_ss(dS, q_desc + h * q_head + ks * 16, k_desc + h * k_head + ks * 16, id1, ks > 0);
-              tc_commit(&bars.s_full[gb]);
-              if (++gb == kGateGroups) { gb = 0; sp_par ^= 1; }
-            }
-            if (++st == kKvStages) { st = 0; kv_par ^= 1; }
+          ok = wait_all(&bars.kv_full[c.st], c.kv_par);
+          if (!ok) return;
+          tc_fence_after();
+          const uint64_t qd = q_desc + c.h * q_head, kd = k_desc0 + (uint64_t)(c.st * (k_bytes >> 4) + c.h * k_head);
+          if (leader) {
+            for (int ks = 0; ks < ks1; ++ks) mma_ss(tS, qd + ks * 16, kd + ks * 16, id1, ks > 0);
+            tc_commit(&bars.s_full[wgi]);
           }
-        }
-        tc_commit(&bars.done[0]);
-        mbar_wait(&bars.done[0], 0, abortp);
-      }
-    } else if (warp == 3) {
-      // ------------------------------------------------------------------ value issuer
-      if (lane == 0) {
-        const uint32_t id2 = idesc_bf16(128, P.dvh);     // 128 candidates x dvh, K = IT items
-        const uint32_t v_lbo = (P.dvh >> 3) * 128;       // V^T head block: k-chunks (8 items) are dvh/8 core matrices apart
-        const int ks2 = IT >> 4;
-        const uint64_t v_desc0 = smem_desc(smem_u32(Vs), v_lbo, 128);
-        const uint32_t v_head = (IT * P.dvh * 2) >> 4, v_step = (2 * v_lbo) >> 4;
-        UnitWalker w;
-        w.init(P, unit_lo);
-        uint32_t st = 0, gb = 0, p_par = 0, ob = 0, o_par = 1;
-        bool ok = true;
-        for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
-          const int nt = w.ntiles(P);
-          const uint32_t dO0 = tmem + colO + ob * d;
-          for (int t = 0; t < nt && ok; ++t) {
-            const uint64_t v_desc = v_desc0 + (uint64_t)(st * (v_bytes >> 4));
-            for (int h = 0; h < H; ++h) {
-              ok = mbar_wait(&bars.p_full[gb], p_par, abortp);
-              if (!ok) break;
-              if (t == 0 && h == 0) {
-                ok = mbar_wait(&bars.o_empty[ob], o_par, abortp);
-                if (!ok) break;
-              }
-              tc_fence_after();
-              const uint32_t aP = tmem + colSP + gb * IT;
-              const uint32_t dO = dO0 + h * P.dvh;
-              const uint64_t vd = v_desc + h * v_head;
+          __syncwarp();
+        };
+        auto issue_values = [&](const Cursor& c) {
+          ok = wait_all(&bars.p_full[wgi], p_par);
+          if (!ok) return;
+          p_par ^= 1;
+          if (c.t == 0 && c.h == wgi) {                   // my first unit of the segment: the accumulator must be drained
+            ok = wait_all(&bars.o_empty[ob], o_par);
+            if (!ok) return;
+          }
+          tc_fence_after();
+          const uint32_t dO = tmem + kColO + ob * d + c.h * P.dvh;
+          const uint64_t vd = v_desc0 + (uint64_t)(c.st * (v_bytes >> 4) + c.h * v_head);
+          const int ks2 = c.w.tile_cols(P, c.t) >> 4;     // k-steps that hold valid items
+          const bool last = c.t == c.nt - 1 && c.h + kGateGroups >= H;      // my last unit of the segment
+          if (leader) {
 #pragma unroll 4
-              for (int ks = 0; ks < ks2; ++ks) mma_ts(dO, aP + ks * 8, vd + ks * v_step, id2, (t | ks) != 0);
-              tc_commit(&bars.sp_free[gb]);
-              if (++gb == kGateGroups) { gb = 0; p_par ^= 1; }
-            }
-            tc_commit(&bars.kv_empty[st]);   // the scores of this tile were consumed before its gates were written
-            if (++st == kKvStages) st = 0;
+            for (int ks = 0; ks < ks2; ++ks) mma_ts(dO, tP + ks * 8, vd + ks * v_step, id2, (c.t | ks) != 0);
+            tc_commit(&bars.p_free[wgi]);
+            tc_commit(&bars.kv_empty[c.st]);              // this unit's scores were consumed before its gates existed
+            if (last) tc_commit(&bars.o_full[ob]);
           }
-          tc_commit(&bars.o_full[ob]);
-          if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
+          __syncwarp();
+          if (last && (int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
+        };
+
+        Cursor cur;
+        cur.w.init(P, unit_lo);
+        cur.it = 0; cur.t = 0; cur.h = wgi; cur.nt = cur.w.ntiles(P); cur.st = 0; cur.kv_par = 0;
+        issue_scores(cur);
+        while (ok) {
+          Cursor nxt = cur;
+          const bool more = advance(nxt);
+          if (more) {                                     // next scores as soon as the warpgroup has read the current ones
+            ok = wait_all(&bars.s_free[wgi], sf_par);
+            if (!ok) break;
+            sf_par ^= 1;
+            issue_scores(nxt);
+            if (!ok) break;
+          }
+          issue_values(cur);
+          if (!more) break;
+          cur = nxt;
         }
-        tc_commit(&bars.done[1]);
-        mbar_wait(&bars.done[1], 0, abortp);
+        // every MMA issued by the leader has completed once `done` flips
+        if (leader) tc_commit(&bars.done[wgi]);
+        __syncwarp();
+        wait_all(&bars.done[wgi], 0);
       }
-    } else if (warp >= 8) {
-      // ------------------------------------------------------------------ gate warps: P' = tanh(scores), in place
-      const int wg = (warp - 8) >> 2;                       // warpgroup wg owns buffer wg
+    } else if (warp >= 8 && warp < kProducerWarp) {
+      // ------------------------------------------------------------------ gate warps: P' = tanh(scores)
+      const int wg = (warp - 8) >> 2;                       // warpgroup wg owns buffers wg and heads wg, wg + 4, ...
       const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-      const uint32_t tS = tmem + lane_base + colSP + wg * IT;
+      const uint32_t tS = tmem + lane_base + kColS + wg * kItMax;
+      const uint32_t tP = tmem + lane_base + kColP + wg * (kItMax / 2);
       UnitWalker w;
       w.init(P, unit_lo);
-      uint32_t g = 0, par = 0;
-      bool ok = true;
+      uint32_t s_par = 0, pf_par = 1;
+      int my_heads = 0;
+      for (int h = wg; h < H; h += kGateGroups) ++my_heads;
+      bool ok = wg < n_groups;
+      auto release_scores = [&]() {                         // every score column of the unit is in registers
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.s_free[wg]);
+      };
       for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
-        const int n_sub = w.ntiles(P) * H;
-        for (int s = 0; s < n_sub && ok; ++s, ++g) {
-          if ((int)(g % kGateGroups) != wg) continue;
-          ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], par, abortp));
-          if (!ok) break;
-          par ^= 1;
-          tc_fence_after();
-          // columns [c, c+32) of the scores become columns [c/2, c/2+16) of the gates: always inside the part of the
-          // buffer that has already been read
-          int c = 0;
-          for (; c + 32 <= IT; c += 32) {
-            uint32_t v[32], o[16];
-            tmem_ld32(tS + c, v);
-            tc_wait_ld();
+        const int nt = w.ntiles(P);
+        for (int t = 0; t < nt && ok; ++t) {
+          const int cols = w.tile_cols(P, t);               // columns past this hold zero K rows: their gates are 0
+          for (int hh = 0; hh < my_heads && ok; ++hh) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], s_par, abortp));
+            if (!ok) break;
+            s_par ^= 1;
+            tc_fence_after();
+            bool first = true;
+            int c = 0;
+            for (; c + 32 <= cols; c += 32) {
+              uint32_t v[32], o[16];
+              tmem_ld32(tS + c, v);
+              tc_wait_ld();
+              if (c + 32 >= cols) release_scores();
 #pragma unroll
-            for (int e = 0; e < 16; ++e)
-              o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
-            tmem_st16(tS + (c >> 1), o);
-          }
-          if (c < IT) {   // 16-column tail
-            uint32_t v[16], o[8];
-            tmem_ld16(tS + c, v);
-            tc_wait_ld();
+              for (int e = 0; e < 16; ++e)
+                o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+              if (first) {                                  // the previous unit's gates have been multiplied
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
+                pf_par ^= 1;
+                first = false;
+                tc_fence_after();
+              }
+              tmem_st16(tP + (c >> 1), o);
+            }
+            if (c < cols) {   // 16-column tail
+              uint32_t v[16], o[8];
+              tmem_ld16(tS + c, v);
+              tc_wait_ld();
+              release_scores();
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
-            tmem_st8(tS + (c >> 1), o);
+              for (int e = 0; e < 8; ++e)
+                o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+              if (first) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
+                pf_par ^= 1;
+                first = false;
+                tc_fence_after();
+              }
+              tmem_st8(tP + (c >> 1), o);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.p_full[wg]);
           }
-          tc_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars.p_full[wg]);
         }
       }
     } else if (warp >= 4) {
@@ -664,44 +723,50 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         UnitWalker wn = w;
         wn.next(P);
         if (it + 1 < my_units) fetch_sv(wn);
+        uint8_t* row = Os + ((size_t)(it & 1) * kCandTile + m) * out_row;
+        bulk_wait_read<1>();                               // my store from this staging buffer (two units ago) has left it
         __syncwarp();
         ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], o_par, abortp));
         if (!ok) break;
         tc_fence_after();
-        const int ci = w.j * kCandTile + m;
-        const bool valid = ci < w.nc;
-        bf16* out = P.Hp + ((size_t)(w.c0 + (valid ? ci : 0)) * P.Lp + w.seg) * d;
-        const uint32_t tO = tmem + lane_base + colO + ob * d;
+        const uint32_t tO = tmem + lane_base + kColO + ob * d;
         for (int c = 0; c < d; c += 16) {
           uint32_t v[16];
           tmem_ld16(tO + c, v);
           tc_wait_ld();
-          if (valid) {
+          if (c + 16 >= d) {                               // the accumulator is in registers: hand it back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
+          }
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const float4 s0 = *reinterpret_cast<const float4*>(svb + c + half * 8);
-              const float4 s1 = *reinterpret_cast<const float4*>(svb + c + half * 8 + 4);
-              uint4 o;
-              o.x = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 0]) + s0.x), 0.5f * (__uint_as_float(v[half * 8 + 1]) + s0.y));
-              o.y = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 2]) + s0.z), 0.5f * (__uint_as_float(v[half * 8 + 3]) + s0.w));
-              o.z = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 4]) + s1.x), 0.5f * (__uint_as_float(v[half * 8 + 5]) + s1.y));
-              o.w = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 6]) + s1.z), 0.5f * (__uint_as_float(v[half * 8 + 7]) + s1.w));
-              *reinterpret_cast<uint4*>(out + c + half * 8) = o;
-            }
+          for (int half = 0; half < 2; ++half) {
+            const float4 s0 = *reinterpret_cast<const float4*>(svb + c + half * 8);
+            const float4 s1 = *reinterpret_cast<const float4*>(svb + c + half * 8 + 4);
+            uint4 o;
+            o.x = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 0]) + s0.x), 0.5f * (__uint_as_float(v[half * 8 + 1]) + s0.y));
+            o.y = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 2]) + s0.z), 0.5f * (__uint_as_float(v[half * 8 + 3]) + s0.w));
+            o.z = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 4]) + s1.x), 0.5f * (__uint_as_float(v[half * 8 + 5]) + s1.y));
+            o.w = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 6]) + s1.z), 0.5f * (__uint_as_float(v[half * 8 + 7]) + s1.w));
+            *reinterpret_cast<uint4*>(row + (c + half * 8) * 2) = o;
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
+        const int ci = w.j * kCandTile + m;
+        if (ci < w.nc) {                                   // my candidate's row of this segment: one contiguous store
+          fence_proxy_async_smem();
+          bulk_s2g(P.Hp + ((size_t)(w.c0 + ci) * P.Lp + w.seg) * d, row, d * 2);
+        }
+        bulk_commit();
         if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
         w = wn;
       }
+      bulk_wait<0>();
     }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 2) tmem_dealloc(tmem, kStaTmemCols);
+  if (warp == kProducerWarp) tmem_dealloc(tmem, kStaTmemCols);
   if (tid == 0 && s_abort) report_status(P.status, LASER_ERR_TIMEOUT);
 }
 
@@ -721,7 +786,7 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.dqh = p.dqh; P.dvh = p.dvh; P.maxC = p.maxC;
   P.IT = p.tg.IT; P.NT = p.tg.NT; P.n_tiles = p.tg.n_tiles; P.cand_tiles_max = p.tg.cand_tiles_max;
-  P.n_obuf = 2 * p.d + kGateGroups * P.IT <= kStaTmemCols ? 2 : 1;
+  P.n_obuf = (int)kColO + 2 * p.d <= kStaTmemCols ? 2 : 1;
   P.NTG = P.IT <= 64 ? (128 / P.IT < P.NT ? 128 / P.IT : P.NT) : 1;
   P.NG = (P.NT + P.NTG - 1) / P.NTG;
   P.q_scale = 0.5f * p.inv_gamma;
@@ -756,8 +821,7 @@ bool tensor_supported(const Plan& p) {
 }
 
 void tensor_geometry(const Plan& p, TensorGeom* g) {
-  // TMEM: one or two output accumulators (d columns each) + kGateGroups score / gate buffers (IT columns each) <= 512
-  const int it_max = ((512 - p.d) / kGateGroups) / 16 * 16 > 128 ? 128 : ((512 - p.d) / kGateGroups) / 16 * 16;
+  const int it_max = 64;   // one 64-column fp32 score buffer per gate warpgroup in TMEM
   g->NT = (p.S + it_max - 1) / it_max;
   const int per = (p.S + g->NT - 1) / g->NT;
   g->IT = (per + 15) / 16 * 16;
@@ -788,8 +852,9 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     tc_zero_empty_kernel<<<dim3(p.Lp, p.U), 256, 0, st>>>(P);
   }
   {
-    const size_t smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * P.IT * (p.dqk + p.d) * 2;
-    if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * P.IT * (p.dqk + p.d) * 2 +
+                        (size_t)2 * kCandTile * (p.d * 2 + 16);
+    if (smem > 220 * 1024) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_sta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("sta_tc", st);
     tc_sta_kernel<<<sms, kStaThreads, smem, st>>>(P);
