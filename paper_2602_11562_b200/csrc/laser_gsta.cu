@@ -5,7 +5,7 @@
 //   A   Q   = T W_q^l                              [16 x d]    batched over the 16 candidates
 //   B   Qt_h = Q[:, head h] W_k^l[:, head h]^T / tau  [16 x d] per head: (s_j W_k)_h . q_h = s_j . Qt_h
 //   C   per candidate: scores e_{h,j} = Qt_h . s_j over its non-empty segments j, softmax over j, m_h = sum_j a_{h,j} s_j.
-//       The candidate's segment vectors are staged in shared memory (cp.async, two buffers per warp, 32 vectors per
+//       The candidate's segment vectors are staged in shared memory (cp.async, two buffers per warp, 16 vectors per
 //       chunk); every vector is read from global memory once per layer and used for both contractions, with an online
 //       softmax across chunks.
 //   D   o[:, head h] = m_h W_v^l[:, head h];  T += o
@@ -25,9 +25,9 @@ using bf16 = __nv_bfloat16;
 using namespace mma;
 
 constexpr int kGT = 16;        // candidates per block
-constexpr int kGW = 4;         // warps per block
+constexpr int kGW = 8;         // warps per block: two candidates per warp
 constexpr int kGThreads = kGW * 32;
-constexpr int kChunk = 32;     // segment vectors per staged chunk
+constexpr int kChunk = 16;     // segment vectors per staged chunk (one MMA k-step)
 
 struct GstaParams {
   int N, U, L, S, Lp, H, M, d;
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
 }
 
 template <int D16>
-__global__ void __launch_bounds__(kGThreads) gsta_mma_kernel(GstaParams P) {
+__global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   constexpr int d = D16 * 16;
   constexpr int RS = 2 * d + 16;            // bytes per staged bf16 row (16 bytes of padding: conflict-free ldmatrix)
   constexpr int TS = d + 8;                 // floats per row of the running target
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(kGThreads) gsta_mma_kernel(GstaParams P) {
   for (int i = tid; i < RS / 4; i += kGThreads) reinterpret_cast<uint32_t*>(zrow)[i] = 0u;
   __syncthreads();
 
-  // ---- chunk pipeline of this warp: (layer, candidate slot ci -> candidate warp + 4 ci, chunk) in processing order
+  // ---- chunk pipeline of this warp: (layer, candidate slot ci -> candidate warp + kGW ci, chunk) in processing order
   uint8_t* my_stage = stage + (size_t)warp * 2 * kChunk * RS;
   int f_layer = 0, f_ci = 0, f_ch = 0;
   bool f_valid = false;
@@ -129,8 +129,9 @@ __global__ void __launch_bounds__(kGThreads) gsta_mma_kernel(GstaParams P) {
     const bf16* src = P.Hp + ((size_t)(c_base + c) * P.Lp + f_ch * kChunk) * d;
     const uint32_t dst = smem_addr(my_stage + (size_t)buf * kChunk * RS);
     const int rows = min(kChunk, nv - f_ch * kChunk);
+    static_assert((kChunk * 2 * D16) % 32 == 0, "a chunk is a whole number of 16-byte pieces per lane");
 #pragma unroll
-    for (int i = 0; i < 2 * D16; ++i) {
+    for (int i = 0; i < kChunk * 2 * D16 / 32; ++i) {      // kChunk rows of 2 D16 16-byte pieces
       const int piece = i * 32 + lane;
       const int r = piece / (2 * D16), q = piece - r * (2 * D16);
       const bool ok = r < rows;
@@ -251,28 +252,34 @@ __global__ void __launch_bounds__(kGThreads) gsta_mma_kernel(GstaParams P) {
         const uint32_t sb = smem_addr(my_stage + (size_t)buf * kChunk * RS);
         const int rows = min(kChunk, nv - ch * kChunk);
 
-        // scores e[h][j] for the chunk's (up to) 32 segments: 4 column tiles of 8 segments
-        float e[4][4];
+        // scores e[h][j] for the chunk's (up to) 16 segments: 2 column tiles of 8 segments; even and odd k-tiles
+        // accumulate separately so that four MMA chains are in flight
+        float e[2][4], e2[2][4];
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) e[nt][0] = e[nt][1] = e[nt][2] = e[nt][3] = 0.f;
+        for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-        for (int np = 0; np < 2; ++np) {
-          if (np * 16 < rows) {
-            const uint32_t a = sb + (np * 16 + (lane & 7) + ((lane >> 4) & 1) * 8) * RS + ((lane >> 3) & 1) * 16;
+          for (int q = 0; q < 4; ++q) e[nt][q] = e2[nt][q] = 0.f;
+        {
+          const uint32_t a = sb + ((lane & 7) + ((lane >> 4) & 1) * 8) * RS + ((lane >> 3) & 1) * 16;
 #pragma unroll
-            for (int kt = 0; kt < D16; ++kt) {
-              uint32_t b[4];
-              ldsm_x4(b, a + kt * 32);
-              mma16816(e[2 * np], qa[kt][0], 0u, qa[kt][1], 0u, b[0], b[1]);
-              mma16816(e[2 * np + 1], qa[kt][0], 0u, qa[kt][1], 0u, b[2], b[3]);
+          for (int kt = 0; kt < D16; ++kt) {
+            uint32_t b[4];
+            ldsm_x4(b, a + kt * 32);
+            if (kt & 1) {
+              mma16816(e2[0], qa[kt][0], 0u, qa[kt][1], 0u, b[0], b[1]);
+              mma16816(e2[1], qa[kt][0], 0u, qa[kt][1], 0u, b[2], b[3]);
+            } else {
+              mma16816(e[0], qa[kt][0], 0u, qa[kt][1], 0u, b[0], b[1]);
+              mma16816(e[1], qa[kt][0], 0u, qa[kt][1], 0u, b[2], b[3]);
             }
           }
         }
         float mx = -INFINITY;
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
+        for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
+            e[nt][q] += e2[nt][q];
             if (nt * 8 + 2 * t + q >= rows) e[nt][q] = -INFINITY;
             mx = fmaxf(mx, e[nt][q]);
           }
@@ -281,31 +288,26 @@ __global__ void __launch_bounds__(kGThreads) gsta_mma_kernel(GstaParams P) {
         const float scale = __expf(run_max - new_max);
         run_max = new_max;
         float psum = 0.f;
-        uint32_t pa[2][2];
+        uint32_t pa[2];
 #pragma unroll
-        for (int kk = 0; kk < 2; ++kk)
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            const float p0 = __expf(e[2 * kk + q][0] - new_max), p1 = __expf(e[2 * kk + q][1] - new_max);
-            pa[kk][q] = pack2(p0, p1);
-            psum += bf16_lo(pa[kk][q]) + bf16_hi(pa[kk][q]);   // normalise by exactly the weights the MMA uses
-          }
+        for (int q = 0; q < 2; ++q) {
+          const float p0 = __expf(e[q][0] - new_max), p1 = __expf(e[q][1] - new_max);
+          pa[q] = pack2(p0, p1);
+          psum += bf16_lo(pa[q]) + bf16_hi(pa[q]);   // normalise by exactly the weights the MMA uses
+        }
         run_sum = run_sum * scale + psum;
 #pragma unroll
         for (int j = 0; j < 2 * D16; ++j) { macc[j][0] *= scale; macc[j][1] *= scale; }
 
         // m += P S   (rows = heads, k = the chunk's segments, columns = d)
+        {
+          const uint32_t a = sb + ((lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16;
 #pragma unroll
-        for (int kk = 0; kk < 2; ++kk) {
-          if (kk * 16 < rows) {
-            const uint32_t a = sb + (kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16;
-#pragma unroll
-            for (int jp = 0; jp < D16; ++jp) {
-              uint32_t b[4];
-              ldsm_x4_t(b, a + jp * 32);
-              mma16816(macc[2 * jp], pa[kk][0], 0u, pa[kk][1], 0u, b[0], b[1]);
-              mma16816(macc[2 * jp + 1], pa[kk][0], 0u, pa[kk][1], 0u, b[2], b[3]);
-            }
+          for (int jp = 0; jp < D16; ++jp) {
+            uint32_t b[4];
+            ldsm_x4_t(b, a + jp * 32);
+            mma16816(macc[2 * jp], pa[0], 0u, pa[1], 0u, b[0], b[1]);
+            mma16816(macc[2 * jp + 1], pa[0], 0u, pa[1], 0u, b[2], b[3]);
           }
         }
         __syncwarp();   // every lane is done with this buffer before the next iteration refills it
