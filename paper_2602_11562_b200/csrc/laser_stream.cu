@@ -118,8 +118,12 @@ __global__ void __launch_bounds__(128) stream_pre_kernel(StreamParams P, int use
 }
 
 __device__ __forceinline__ float sigmoid_fast(float x) {
-  // 1 / (1 + e^-x); e^-x overflowing to +inf gives exactly 0
-  return __frcp_rn(1.f + __expf(-x));
+  // 1 / (1 + 2^(-x log2 e)) with the approximate ex2 and rcp units (relative error ~1e-7 each);
+  // the exponential overflowing to +inf gives exactly 0
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.f + e));
+  return r;
 }
 
 template <int D16>
@@ -159,21 +163,31 @@ __global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
     }
     const bf16* xu = P.items + (size_t)u * P.L * d;
 
-    // fetch cursor over this warp's (segment, 16-row group) sequence
+    // fetch cursor over this warp's (segment, 16-row group) sequence.  A stage is kSRows rows of 2 D16 16-byte
+    // pieces; lane l copies pieces l, l + 32, ...: their row, source offset and destination offset never change.
     int f_seg = warp, f_grp = 0;
     bool f_valid = warp < nv;
+    int p_row[D16], p_src[D16];
+    uint32_t p_dst[D16];
+#pragma unroll
+    for (int i = 0; i < D16; ++i) {
+      const int piece = i * 32 + lane;
+      p_row[i] = piece / (2 * D16);
+      const int q = piece - p_row[i] * (2 * D16);
+      p_src[i] = p_row[i] * d + q * 8;
+      p_dst[i] = p_row[i] * RS + q * 16;
+    }
+    const uint32_t ring_addr = smem_addr(ring);
     auto groups_of = [&](int seg) { return (min(P.S, len - seg * P.S) + kSRows - 1) / kSRows; };
     auto issue = [&](int stage) {
-      const int seg_end = min((f_seg + 1) * P.S, len);
       const int n0 = f_seg * P.S + f_grp * kSRows;
-      const uint32_t dst = smem_addr(ring + (size_t)stage * kSRows * RS);
+      const int rows = min((f_seg + 1) * P.S, len) - n0;   // rows past the segment (or the valid prefix) become zeros
+      const bf16* src = xu + (size_t)n0 * d;
+      const uint32_t dst = ring_addr + stage * (kSRows * RS);
 #pragma unroll
       for (int i = 0; i < D16; ++i) {
-        const int piece = i * 32 + lane;
-        const int r = piece / (2 * D16), q = piece - r * (2 * D16);
-        const bool ok = n0 + r < seg_end;        // rows past the segment (or the valid prefix) are staged as zeros
-        cp16(dst + r * RS + q * 16, ok ? (const void*)(xu + (size_t)(n0 + r) * d + q * 8) : (const void*)P.items,
-             ok ? 16u : 0u);
+        const bool ok = p_row[i] < rows;
+        cp16(dst + p_dst[i], ok ? (const void*)(src + p_src[i]) : (const void*)P.items, ok ? 16u : 0u);
       }
       if (++f_grp >= groups_of(f_seg)) {
         f_grp = 0;
@@ -200,7 +214,7 @@ __global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
         __syncwarp();
         if (f_valid) issue((stage + kSStages - 1) % kSStages);
         cp_commit();
-        const uint32_t sb = smem_addr(ring + (size_t)stage * kSRows * RS);
+        const uint32_t sb = ring_addr + stage * (kSRows * RS);
         // scores (Eq. 10 before the sigmoid): rows = heads (high / low parts), columns = the 16 items
         float sc[2][4] = {};
 #pragma unroll
