@@ -31,7 +31,7 @@ constexpr int kSW = 4;            // warps per block
 constexpr int kSThreads = kSW * 32;
 constexpr int kSRows = 16;        // item rows per stage (one MMA k / n step)
 constexpr int kSStages = 4;       // ring depth per warp
-constexpr int kPreUsers = 8;      // users per block of the pre kernel
+constexpr int kPreUsers = 16;     // users per block of the pre kernel
 
 struct StreamParams {
   int U, L, d, dqk, H, S, Lp, N;
@@ -56,7 +56,7 @@ __device__ __forceinline__ int user_candidate(const StreamParams& P, int u, int*
   return c1 > c0 ? c0 : -1;
 }
 
-__global__ void __launch_bounds__(128) stream_pre_kernel(StreamParams P, int user_blocks) {
+__global__ void __launch_bounds__(256) stream_pre_kernel(StreamParams P, int user_blocks) {
   const int tid = threadIdx.x;
   const int d = P.d, dqk = P.dqk, H = P.H, dqh = dqk / H;
   if ((int)blockIdx.x >= user_blocks) {
@@ -76,14 +76,23 @@ __global__ void __launch_bounds__(128) stream_pre_kernel(StreamParams P, int use
     }
     return;
   }
+  // shared: W_q [d][dqk+1], W_k [d][dqk+1] (fp32, padded rows), t [kPreUsers][d], q [kPreUsers][dqk]
   extern __shared__ float sm[];
-  float* ts = sm;                      // [kPreUsers][d]
-  float* qs = ts + kPreUsers * d;      // [kPreUsers][dqk]
+  const int wld = dqk + 1;
+  float* wq = sm;
+  float* wk = wq + d * wld;
+  float* ts = wk + d * wld;
+  float* qs = ts + kPreUsers * d;
   __shared__ int cand_s[kPreUsers];
   const int u0 = blockIdx.x * kPreUsers;
   if (tid < kPreUsers) {
     int len = 0;
     cand_s[tid] = u0 + tid < P.U ? user_candidate(P, u0 + tid, &len) : -1;
+  }
+  for (int i = tid; i < d * dqk; i += blockDim.x) {
+    const int r = i / dqk, c = i - r * dqk;
+    wq[r * wld + c] = __bfloat162float(P.Wq[i]);
+    wk[r * wld + c] = __bfloat162float(P.Wk[i]);
   }
   __syncthreads();
   for (int i = tid; i < kPreUsers * d; i += blockDim.x) {
@@ -91,29 +100,18 @@ __global__ void __launch_bounds__(128) stream_pre_kernel(StreamParams P, int use
     ts[i] = c >= 0 ? __bfloat162float(P.cands[(size_t)c * d + (i - uu * d)]) : 0.f;
   }
   __syncthreads();
-  for (int a = tid; a < dqk; a += blockDim.x) {        // q = t W_q / gamma   (Eq. 4 / Eq. 8)
-    float acc[kPreUsers] = {};
-    for (int i = 0; i < d; ++i) {
-      const float w = __bfloat162float(P.Wq[(size_t)i * dqk + a]);
-#pragma unroll
-      for (int uu = 0; uu < kPreUsers; ++uu) acc[uu] = fmaf(ts[uu * d + i], w, acc[uu]);
-    }
-#pragma unroll
-    for (int uu = 0; uu < kPreUsers; ++uu) qs[uu * dqk + a] = acc[uu] * P.inv_gamma;
+  for (int o = tid; o < kPreUsers * dqk; o += blockDim.x) {      // q = t W_q / gamma   (Eq. 4 / Eq. 8)
+    const int uu = o / dqk, a = o - uu * dqk;
+    float acc = 0.f;
+    for (int i = 0; i < d; ++i) acc = fmaf(ts[uu * d + i], wq[i * wld + a], acc);
+    qs[o] = acc * P.inv_gamma;
   }
   __syncthreads();
-  for (int i = tid; i < d; i += blockDim.x) {          // u_h[i] = sum_{a in head h} W_k[i][a] q[a]
-    for (int h = 0; h < H; ++h) {
-      float acc[kPreUsers] = {};
-      for (int a = h * dqh; a < (h + 1) * dqh; ++a) {
-        const float w = __bfloat162float(P.Wk[(size_t)i * dqk + a]);
-#pragma unroll
-        for (int uu = 0; uu < kPreUsers; ++uu) acc[uu] = fmaf(w, qs[uu * dqk + a], acc[uu]);
-      }
-#pragma unroll
-      for (int uu = 0; uu < kPreUsers; ++uu)
-        if (u0 + uu < P.U) P.u[((size_t)(u0 + uu) * H + h) * d + i] = acc[uu];
-    }
+  for (int o = tid; o < kPreUsers * H * d; o += blockDim.x) {    // u_h[i] = sum_{a in head h} W_k[i][a] q[a]
+    const int uu = o / (H * d), h = (o / d) % H, i = o % d;
+    float acc = 0.f;
+    for (int a = h * dqh; a < (h + 1) * dqh; ++a) acc = fmaf(wk[i * wld + a], qs[uu * dqk + a], acc);
+    if (u0 + uu < P.U) P.u[(size_t)(u0 + uu) * H * d + (o - uu * H * d)] = acc;
   }
 }
 
@@ -352,9 +350,11 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   P.status = reinterpret_cast<int*>(ws + p.off_status);
   {
     const int user_blocks = (p.U + kPreUsers - 1) / kPreUsers;
-    const size_t smem = (size_t)kPreUsers * (p.d + p.dqk) * sizeof(float);
+    const size_t smem = ((size_t)2 * p.d * (p.dqk + 1) + (size_t)kPreUsers * (p.d + p.dqk)) * sizeof(float);
+    if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+    LASER_CUDA_OK(cudaFuncSetAttribute(stream_pre_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("stream_pre", st);
-    stream_pre_kernel<<<user_blocks + 4, 128, smem, st>>>(P, user_blocks);
+    stream_pre_kernel<<<user_blocks + 4, 256, smem, st>>>(P, user_blocks);
   }
   int rc;
   switch (p.d / 16) {

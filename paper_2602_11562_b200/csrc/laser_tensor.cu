@@ -21,7 +21,7 @@ using bf16 = __nv_bfloat16;
 using namespace ptx;
 
 constexpr int kCandTile = 128;        // candidates per tile = MMA M = TMEM lanes
-constexpr int kProjThreads = 128;
+constexpr int kProjThreads = 256;     // two warps per TMEM lane quadrant: they split the accumulator columns
 constexpr int kProjTmemCols = 256;    // K / Q accumulator at column 0, V^T accumulator at column 128
 constexpr int kGateGroups = 4;        // gate warpgroups; each owns one score / gate buffer in TMEM
 constexpr int kStaThreads = (9 + 4 * kGateGroups) * 32;
@@ -144,19 +144,21 @@ __global__ void __launch_bounds__(256) tc_zero_empty_kernel(TcParams P) {
 }
 
 // ------------------------------------------------------------------------------------------------------- projection
-struct ProjSmem {
-  bf16 *imgK, *imgQ, *imgV, *X;
-};
-
+// One unit = up to 128 item rows of one segment (K rows and V^T columns of whole item tiles), or one 128-candidate
+// tile (Q rows).  Per unit: stage the rows into the canonical K-major layout (cp.async), two MMA groups into TMEM
+// (rows x d_qk for K or Q; d x rows for V^T), then the eight warps drain the accumulators: warp w reads TMEM lanes
+// 32 (w mod 4) .. +31 and the first or second half of the columns.
 __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ uint64_t bar_img, bar_mma;
   __shared__ uint32_t s_tmem;
   __shared__ int s_ticket;
   __shared__ int s_abort;
+  __shared__ int s_kcol[16];            // per 8-column group of K / Q: (head << 8) | (8-column chunk within the head)
 
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int d = P.d, dqk = P.dqk;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int quad = warp & 3, half = warp >> 2;
+  const int d = P.d, dqk = P.dqk, IT = P.IT;
   bf16* imgK = reinterpret_cast<bf16*>(smem_raw);
   bf16* imgQ = imgK + dqk * d;
   bf16* imgV = imgQ + dqk * d;
@@ -167,6 +169,10 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     mbar_init(&bar_mma, 1);
     s_abort = 0;
     fence_mbar_init();
+  }
+  if (tid < (dqk >> 3)) {
+    const int col = tid * 8, h = col / P.dqh;
+    s_kcol[tid] = (h << 8) | ((col - h * P.dqh) >> 3);
   }
   if (warp == 0) {
     tmem_alloc(&s_tmem, kProjTmemCols);
@@ -191,8 +197,23 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const int total_units = n_item_units + P.cand_tiles_max;
   const int n_ctiles = P.counters[1];
   const uint32_t sbo = (d >> 3) * 128, lbo = 128;
-  const uint32_t tmem_lane = tmem + ((uint32_t)(warp * 32) << 16);
+  const uint32_t tmem_lane = tmem + ((uint32_t)(quad * 32) << 16);
   uint32_t mma_phase = 0;
+
+  // staging: a 16-byte piece is (8-row group, 8-column chunk, row in group); this thread copies pieces
+  // (tid >> 3) + 32 i of row (tid & 7) in their group, i.e. it walks (group, chunk) with a fixed stride
+  const int cpr = d >> 3;                              // 8-column chunks per row
+  const int step_g = 32 / cpr, step_c = 32 % cpr;
+  const int g0 = (tid >> 3) / cpr, c0 = (tid >> 3) % cpr;
+  // K / Q epilogue: this thread owns row r0 of the unit
+  const int r0 = quad * 32 + lane;
+  const int r0_tile = r0 / IT, r0_in = r0 - r0_tile * IT;
+  const int cpr_k = P.dqh >> 3;                        // 8-element chunks per head row
+  const int n16k = dqk >> 4, k_lo = half ? (n16k + 1) >> 1 : 0, k_hi = half ? n16k : (n16k + 1) >> 1;
+  // V^T epilogue: this thread owns value feature j
+  const int j = quad * 32 + lane;
+  const int jh = j / P.dvh, jj = j - jh * P.dvh;
+  const int npr = P.dvh >> 3;                          // 8-row groups per head
 
   while (ok) {
     __syncthreads();                       // previous unit fully drained (TMEM read, X consumed, s_ticket read)
@@ -202,8 +223,8 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     if (t >= total_units) break;
 
     // ---- decode the unit
-    bool is_item = t < n_item_units;
-    int u = 0, seg = 0, t0 = 0, rows = 0, jt = 0;
+    const bool is_item = t < n_item_units;
+    int u = 0, seg = 0, t0 = 0, rows = 0, jt = 0, seg_items = 0;
     UserShape us;
     if (is_item) {
       u = t / (P.Lp * P.NG);
@@ -212,10 +233,10 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
       t0 = (rem - seg * P.NG) * P.NTG;
       us = user_shape(P, u);
       if (seg >= us.nseg) continue;
-      const int seg_items = min(P.S, us.len - seg * P.S);
-      if (t0 * P.IT >= seg_items) continue;                 // a tile group beyond the segment's valid items
+      seg_items = min(P.S, us.len - seg * P.S);
+      if (t0 * IT >= seg_items) continue;                   // a tile group beyond the segment's valid items
       const int t1 = min(P.NT, t0 + P.NTG);
-      rows = (t1 - t0) * P.IT;
+      rows = (t1 - t0) * IT;
     } else {
       const int ct = t - n_item_units;
       if (ct >= n_ctiles) continue;
@@ -230,26 +251,27 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
       rows = kCandTile;
     }
 
-    // ---- stage the rows into the canonical K-major layout (16-byte chunks; 8 lanes cover one core matrix)
+    // ---- stage the rows
     {
-      const int chunks_per_row = d >> 3;
-      const int total = rows * chunks_per_row;
-      for (int q = tid; q < total; q += kProjThreads) {
-        const int r = ((q / (8 * chunks_per_row)) << 3) + (q & 7);
-        const int c = (q >> 3) % chunks_per_row;
-        const bf16* src;
-        uint32_t nbytes = 16;
-        if (is_item) {
-          const int tt = t0 + r / P.IT, rr = r % P.IT;
-          const int n = seg * P.S + tt * P.IT + rr;
-          if (n < P.L) src = P.items + ((size_t)u * P.L + n) * d + c * 8;
-          else { src = P.items; nbytes = 0; }
-        } else {
-          const int ci = jt * kCandTile + r;
-          if (ci < us.nc) src = P.cands + (size_t)(us.c0 + ci) * d + c * 8;
-          else { src = P.cands; nbytes = 0; }
-        }
-        cp_async16(X + ((r >> 3) * chunks_per_row + c) * 64 + (r & 7) * 8, src, nbytes);
+      const int n_groups = rows >> 3;
+      const bf16* base;
+      int row_limit;                                         // rows at or past it are staged as zeros
+      if (is_item) {
+        const int n0 = seg * P.S + t0 * IT;                  // unit row r is item n0 + r
+        base = P.items + ((size_t)u * P.L + n0) * d;
+        row_limit = P.L - n0;
+      } else {
+        base = P.cands + (size_t)(us.c0 + jt * kCandTile) * d;
+        row_limit = us.nc - jt * kCandTile;
+      }
+      int gq = g0, c = c0;
+      while (gq < n_groups) {
+        const int r = (gq << 3) + (tid & 7);
+        const bool in = r < row_limit;
+        cp_async16(X + (gq * cpr + c) * 64 + (tid & 7) * 8, in ? base + (size_t)r * d + c * 8 : base, in ? 16u : 0u);
+        gq += step_g;
+        c += step_c;
+        if (c >= cpr) { c -= cpr; ++gq; }
       }
       cp_async_wait_all();
       fence_proxy_async_smem();
@@ -278,83 +300,77 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     if (!ok) break;
     tc_fence_after();
 
-    // ---- epilogue 1: K (or Q) rows.  TMEM lane = row of the unit; 16 columns per load.
-    if (warp * 32 < rows) {
-      const int r = tid;
+    // ---- epilogue 1: K (or Q) rows.  TMEM lane = row of the unit; this warp's half of the columns, 16 per load.
+    if (quad * 32 < rows) {
       const float scale = is_item ? 1.f : P.q_scale;
       bool valid;
-      bf16* dst_tile;
-      int rr, tile_rows;
+      bf16* dst_row;                                       // start of row r0 inside head 0's block of its tile
+      size_t head_stride;
       if (is_item) {
-        const int tt = t0 + r / P.IT;
-        rr = r % P.IT;
-        const int pos = tt * P.IT + rr;
-        valid = r < rows && pos < P.S && seg * P.S + pos < us.len;
-        dst_tile = P.Kblk + ((size_t)u * P.n_tiles + seg * P.NT + tt) * ((size_t)P.IT * dqk);
-        tile_rows = P.IT;
+        const int pos = (t0 + r0_tile) * IT + r0_in;
+        valid = r0 < rows && pos < seg_items;
+        dst_row = P.Kblk + ((size_t)u * P.n_tiles + seg * P.NT + t0 + r0_tile) * ((size_t)IT * dqk) +
+                  (r0_in >> 3) * (cpr_k * 64) + (r0_in & 7) * 8;
+        head_stride = (size_t)IT * P.dqh;
       } else {
-        rr = r;
-        valid = jt * kCandTile + r < us.nc;
-        dst_tile = P.Qblk + (size_t)(P.tile_off[u] + jt) * (kCandTile * dqk);
-        tile_rows = kCandTile;
+        valid = jt * kCandTile + r0 < us.nc;
+        dst_row = P.Qblk + (size_t)(P.tile_off[u] + jt) * (kCandTile * dqk) + (r0 >> 3) * (cpr_k * 64) + (r0 & 7) * 8;
+        head_stride = (size_t)kCandTile * P.dqh;
       }
-      const int cpr = P.dqh >> 3;   // 8-element chunks per head row
-      for (int c16 = 0; c16 < dqk; c16 += 16) {
+      for (int c16 = k_lo; c16 < k_hi; ++c16) {
         uint32_t v[16];
-        tmem_ld16(tmem_lane + c16, v);
+        tmem_ld16(tmem_lane + c16 * 16, v);
         tc_wait_ld();
-        if (r < rows) {
+        if (r0 < rows) {
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int col = c16 + half * 8;
-            const int h = col / P.dqh, c = (col - h * P.dqh) >> 3;
-            uint4 o;
+          for (int hf = 0; hf < 2; ++hf) {
+            const int info = s_kcol[c16 * 2 + hf];
+            uint4 o = make_uint4(0, 0, 0, 0);
             if (valid) {
-              o.x = pack_bf16x2(__uint_as_float(v[half * 8 + 0]) * scale, __uint_as_float(v[half * 8 + 1]) * scale);
-              o.y = pack_bf16x2(__uint_as_float(v[half * 8 + 2]) * scale, __uint_as_float(v[half * 8 + 3]) * scale);
-              o.z = pack_bf16x2(__uint_as_float(v[half * 8 + 4]) * scale, __uint_as_float(v[half * 8 + 5]) * scale);
-              o.w = pack_bf16x2(__uint_as_float(v[half * 8 + 6]) * scale, __uint_as_float(v[half * 8 + 7]) * scale);
-            } else {
-              o = make_uint4(0, 0, 0, 0);
+              o.x = pack_bf16x2(__uint_as_float(v[hf * 8 + 0]) * scale, __uint_as_float(v[hf * 8 + 1]) * scale);
+              o.y = pack_bf16x2(__uint_as_float(v[hf * 8 + 2]) * scale, __uint_as_float(v[hf * 8 + 3]) * scale);
+              o.z = pack_bf16x2(__uint_as_float(v[hf * 8 + 4]) * scale, __uint_as_float(v[hf * 8 + 5]) * scale);
+              o.w = pack_bf16x2(__uint_as_float(v[hf * 8 + 6]) * scale, __uint_as_float(v[hf * 8 + 7]) * scale);
             }
-            bf16* dst = dst_tile + (size_t)h * tile_rows * P.dqh + ((rr >> 3) * cpr + c) * 64 + (rr & 7) * 8;
-            *reinterpret_cast<uint4*>(dst) = o;
+            *reinterpret_cast<uint4*>(dst_row + (info >> 8) * head_stride + (info & 255) * 64) = o;
           }
         }
       }
     }
-    // ---- epilogue 2: V^T.  TMEM lane = value feature j; columns = rows of the unit.
-    if (is_item && warp * 32 < d) {
-      const int j = tid;
-      const int h = j / P.dvh, jj = j - h * P.dvh;
-      const int npr = P.dvh >> 3;   // 8-row groups per head
+    // ---- epilogue 2: V^T.  TMEM lane = value feature j; columns = rows of the unit, this warp's half of them.
+    if (is_item && quad * 32 < d) {
+      const int n16 = rows >> 4;
+      const int lo16 = half ? (n16 + 1) >> 1 : 0, hi16 = half ? n16 : (n16 + 1) >> 1;
       float sv = 0.f;
-      for (int c16 = 0; c16 < rows; c16 += 16) {
+      for (int c16 = lo16; c16 < hi16; ++c16) {
         uint32_t v[16];
-        tmem_ld16(tmem_lane + 128 + c16, v);
+        tmem_ld16(tmem_lane + 128 + c16 * 16, v);
         tc_wait_ld();
         if (j < d) {
+          const int rr = c16 * 16;                          // unit row of the first of these 16 columns
+          const int tt = rr / IT, in_tile = rr - tt * IT;   // IT is a multiple of 16: the 16 columns share a tile
+          const int n_valid = seg_items - ((t0 + tt) * IT + in_tile);   // valid items among them (may be <= 0 or >= 16)
+          bf16* dst = P.Vtblk + ((size_t)u * P.n_tiles + seg * P.NT + t0 + tt) * ((size_t)IT * d) +
+                      (size_t)jh * IT * P.dvh + ((in_tile >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int r0 = c16 + half * 8;
-            const int tt = t0 + r0 / P.IT, rr0 = r0 % P.IT;
+          for (int hf = 0; hf < 2; ++hf) {
+            const int cnt = n_valid - hf * 8;
             uint32_t pk[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              float a = __uint_as_float(v[half * 8 + 2 * e]), b = __uint_as_float(v[half * 8 + 2 * e + 1]);
-              const int pa = tt * P.IT + rr0 + 2 * e, pb = pa + 1;
-              if (!(pa < P.S && seg * P.S + pa < us.len)) a = 0.f;
-              if (!(pb < P.S && seg * P.S + pb < us.len)) b = 0.f;
+              float a = __uint_as_float(v[hf * 8 + 2 * e]), b = __uint_as_float(v[hf * 8 + 2 * e + 1]);
+              if (cnt < 8) {                                // ragged end of the segment: masked items are exact zeros
+                if (2 * e >= cnt) a = 0.f;
+                if (2 * e + 1 >= cnt) b = 0.f;
+              }
               pk[e] = pack_bf16x2(a, b);
               sv += __uint_as_float(pk[e] << 16) + __uint_as_float(pk[e] & 0xFFFF0000u);
             }
-            bf16* dst = P.Vtblk + ((size_t)u * P.n_tiles + seg * P.NT + tt) * ((size_t)P.IT * d) +
-                        (size_t)h * P.IT * P.dvh + ((rr0 >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
-            *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(dst + hf * npr * 64) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
-      if (j < d) atomicAdd(&P.SV[((size_t)u * P.Lp + seg) * d + j], sv);
+      if (j < d && hi16 > lo16) atomicAdd(&P.SV[((size_t)u * P.Lp + seg) * d + j], sv);
     }
     tc_fence_before();
   }
