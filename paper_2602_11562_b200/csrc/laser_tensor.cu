@@ -39,7 +39,8 @@ struct TcParams {
   bf16 *Qblk, *Kblk, *Vtblk;
   float* SV;                          // [U, Lp, d] sum of the valid (bf16-rounded) V rows of each segment
   int *unit_start, *tile_off;         // [U+1] prefix of attention units / candidate tiles per user
-  int* counters;                      // [0] attention units, [1] candidate tiles, [2] projection ticket
+  int* proj_start;                    // [U+1] prefix of projection units (groups of item tiles that hold valid items)
+  int* counters;                      // [0] attention units, [1] candidate tiles, [2] projection units
   bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
   int* status;
   bf16* Hp;
@@ -61,6 +62,15 @@ __device__ __forceinline__ UserShape user_shape(const TcParams& P, int u) {
   return s;
 }
 
+// Projection units of a user: every segment with valid items is cut into groups of NTG item tiles (<= 128 rows);
+// only groups that hold at least one valid item count.
+__device__ __forceinline__ int proj_units_of(const TcParams& P, const UserShape& s) {
+  if (s.nseg == 0) return 0;
+  const int last_items = s.len - (s.nseg - 1) * P.S;
+  const int last_tiles = min(P.NT, (last_items + P.IT - 1) / P.IT);
+  return (s.nseg - 1) * P.NG + (last_tiles + P.NTG - 1) / P.NTG;
+}
+
 // Canonical K-major (no swizzle) element offset of (row, k) in a [rows x kdim] operand: 8x8-element core matrices of
 // 64 contiguous elements, core matrices of one 8-row group adjacent along k.
 __device__ __forceinline__ int canon_off(int row, int k, int kdim) {
@@ -71,10 +81,10 @@ __device__ __forceinline__ int canon_off(int row, int k, int kdim) {
 __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
   const int tid = threadIdx.x;
   if (blockIdx.x == 0) {
-    __shared__ int sa[1024], sb[1024];
+    __shared__ int sa[1024], sb[1024], sc[1024];
     const int per = (P.U + 1023) / 1024;
     const int u0 = min(tid * per, P.U), u1 = min(u0 + per, P.U);
-    int a = 0, b = 0;
+    int a = 0, b = 0, c = 0;
     bool bad = false;
     for (int u = u0; u < u1; ++u) {
       const int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
@@ -82,33 +92,39 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
       const UserShape s = user_shape(P, u);
       a += s.ctiles;
       b += s.ctiles * s.nseg;
+      c += proj_units_of(P, s);
     }
     if (bad) report_status(P.status, LASER_ERR_BAD_INPUT);
     sa[tid] = a;
     sb[tid] = b;
+    sc[tid] = c;
     __syncthreads();
     for (int off = 1; off < 1024; off <<= 1) {
-      int va = 0, vb = 0;
-      if (tid >= off) { va = sa[tid - off]; vb = sb[tid - off]; }
+      int va = 0, vb = 0, vc = 0;
+      if (tid >= off) { va = sa[tid - off]; vb = sb[tid - off]; vc = sc[tid - off]; }
       __syncthreads();
       sa[tid] += va;
       sb[tid] += vb;
+      sc[tid] += vc;
       __syncthreads();
     }
-    int pa = sa[tid] - a, pb = sb[tid] - b;   // exclusive prefixes
+    int pa = sa[tid] - a, pb = sb[tid] - b, pc = sc[tid] - c;   // exclusive prefixes
     for (int u = u0; u < u1; ++u) {
       const UserShape s = user_shape(P, u);
       P.tile_off[u] = pa;
       P.unit_start[u] = pb;
+      P.proj_start[u] = pc;
       pa += s.ctiles;
       pb += s.ctiles * s.nseg;
+      pc += proj_units_of(P, s);
     }
     if (tid == 1023) {
       P.tile_off[P.U] = sa[1023];
       P.unit_start[P.U] = sb[1023];
+      P.proj_start[P.U] = sc[1023];
       P.counters[0] = sb[1023];
       P.counters[1] = sa[1023];
-      P.counters[2] = 0;
+      P.counters[2] = sc[1023];
     }
     return;
   }
@@ -145,24 +161,29 @@ __global__ void __launch_bounds__(256) tc_zero_empty_kernel(TcParams P) {
 
 // ------------------------------------------------------------------------------------------------------- projection
 // One unit = up to 128 item rows of one segment (K rows and V^T columns of whole item tiles), or one 128-candidate
-// tile (Q rows).  Per unit: stage the rows into the canonical K-major layout (cp.async), two MMA groups into TMEM
-// (rows x d_qk for K or Q; d x rows for V^T), then the eight warps drain the accumulators: warp w reads TMEM lanes
-// 32 (w mod 4) .. +31 and the first or second half of the columns.
+// tile (Q rows).  Every block takes a contiguous range of the item units (no empty ones: tc_prep_kernel counted them)
+// and runs them through a two-deep pipeline: while unit n is multiplied (two MMA groups into TMEM: rows x d_qk for K,
+// d x rows for V^T) and drained by the eight warps (warp w reads TMEM lanes 32 (w mod 4) .. +31 and one half of the
+// columns), the rows of unit n + 1 are already on their way into the other staging buffer (cp.async, canonical K-major
+// layout).  Afterwards the blocks share out the candidate tiles (Q = T W_q / 2 gamma) the same way.
+struct ProjUnit {
+  int u, seg, t0, rows, seg_items;      // item unit: tiles t0.. of segment seg; rows = staged rows; valid items of seg
+  int jt, c0, nc;                       // candidate unit: tile jt of user u, whose candidates are [c0, c0 + nc)
+};
+
 __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ uint64_t bar_img, bar_mma;
   __shared__ uint32_t s_tmem;
-  __shared__ int s_ticket;
   __shared__ int s_abort;
   __shared__ int s_kcol[16];            // per 8-column group of K / Q: (head << 8) | (8-column chunk within the head)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int quad = warp & 3, half = warp >> 2;
   const int d = P.d, dqk = P.dqk, IT = P.IT;
-  bf16* imgK = reinterpret_cast<bf16*>(smem_raw);
-  bf16* imgQ = imgK + dqk * d;
-  bf16* imgV = imgQ + dqk * d;
-  bf16* X = imgV + kCandTile * d;
+  bf16* imgK = reinterpret_cast<bf16*>(smem_raw);          // W_k^T, later W_q^T
+  bf16* imgV = imgK + dqk * d;
+  bf16* Xbuf = imgV + kCandTile * d;                       // [2][128 x d]
 
   if (tid == 0) {
     mbar_init(&bar_img, 1);
@@ -183,19 +204,14 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
+  const uint32_t bK = dqk * d * 2, bV = kCandTile * d * 2;
 
   if (tid == 0) {
-    const uint32_t bK = dqk * d * 2, bV = kCandTile * d * 2;
-    mbar_arrive_expect_tx(&bar_img, 2 * bK + bV);
+    mbar_arrive_expect_tx(&bar_img, bK + bV);
     bulk_g2s(imgK, P.imgK, bK, &bar_img);
-    bulk_g2s(imgQ, P.imgQ, bK, &bar_img);
     bulk_g2s(imgV, P.imgV, bV, &bar_img);
   }
-  bool ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
 
-  const int n_item_units = P.U * P.Lp * P.NG;
-  const int total_units = n_item_units + P.cand_tiles_max;
-  const int n_ctiles = P.counters[1];
   const uint32_t sbo = (d >> 3) * 128, lbo = 128;
   const uint32_t tmem_lane = tmem + ((uint32_t)(quad * 32) << 16);
   uint32_t mma_phase = 0;
@@ -205,6 +221,28 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const int cpr = d >> 3;                              // 8-column chunks per row
   const int step_g = 32 / cpr, step_c = 32 % cpr;
   const int g0 = (tid >> 3) / cpr, c0 = (tid >> 3) % cpr;
+  auto stage = [&](const ProjUnit& pu, bool is_item, bf16* X) {
+    const int n_groups = pu.rows >> 3;
+    const bf16* base;
+    int row_limit;                                         // rows at or past it are staged as zeros
+    if (is_item) {
+      const int n0 = pu.seg * P.S + pu.t0 * IT;            // unit row r is item n0 + r
+      base = P.items + ((size_t)pu.u * P.L + n0) * d;
+      row_limit = P.L - n0;
+    } else {
+      base = P.cands + (size_t)(pu.c0 + pu.jt * kCandTile) * d;
+      row_limit = pu.nc - pu.jt * kCandTile;
+    }
+    int gq = g0, c = c0;
+    while (gq < n_groups) {
+      const int r = (gq << 3) + (tid & 7);
+      const bool in = r < row_limit;
+      cp_async16(X + (gq * cpr + c) * 64 + (tid & 7) * 8, in ? base + (size_t)r * d + c * 8 : base, in ? 16u : 0u);
+      gq += step_g;
+      c += step_c;
+      if (c >= cpr) { c -= cpr; ++gq; }
+    }
+  };
   // K / Q epilogue: this thread owns row r0 of the unit
   const int r0 = quad * 32 + lane;
   const int r0_tile = r0 / IT, r0_in = r0 - r0_tile * IT;
@@ -215,106 +253,45 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const int jh = j / P.dvh, jj = j - jh * P.dvh;
   const int npr = P.dvh >> 3;                          // 8-row groups per head
 
-  while (ok) {
-    __syncthreads();                       // previous unit fully drained (TMEM read, X consumed, s_ticket read)
-    if (tid == 0) s_ticket = atomicAdd(&P.counters[2], 1);
-    __syncthreads();
-    const int t = s_ticket;
-    if (t >= total_units) break;
-
-    // ---- decode the unit
-    const bool is_item = t < n_item_units;
-    int u = 0, seg = 0, t0 = 0, rows = 0, jt = 0, seg_items = 0;
-    UserShape us;
-    if (is_item) {
-      u = t / (P.Lp * P.NG);
-      const int rem = t - u * (P.Lp * P.NG);
-      seg = rem / P.NG;
-      t0 = (rem - seg * P.NG) * P.NTG;
-      us = user_shape(P, u);
-      if (seg >= us.nseg) continue;
-      seg_items = min(P.S, us.len - seg * P.S);
-      if (t0 * IT >= seg_items) continue;                   // a tile group beyond the segment's valid items
-      const int t1 = min(P.NT, t0 + P.NTG);
-      rows = (t1 - t0) * IT;
-    } else {
-      const int ct = t - n_item_units;
-      if (ct >= n_ctiles) continue;
-      int lo = 0, hi = P.U;                                  // tile_off[lo] <= ct < tile_off[hi]
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (P.tile_off[mid] <= ct) lo = mid; else hi = mid;
-      }
-      u = lo;
-      us = user_shape(P, u);
-      jt = ct - P.tile_off[u];
-      rows = kCandTile;
-    }
-
-    // ---- stage the rows
-    {
-      const int n_groups = rows >> 3;
-      const bf16* base;
-      int row_limit;                                         // rows at or past it are staged as zeros
-      if (is_item) {
-        const int n0 = seg * P.S + t0 * IT;                  // unit row r is item n0 + r
-        base = P.items + ((size_t)u * P.L + n0) * d;
-        row_limit = P.L - n0;
-      } else {
-        base = P.cands + (size_t)(us.c0 + jt * kCandTile) * d;
-        row_limit = us.nc - jt * kCandTile;
-      }
-      int gq = g0, c = c0;
-      while (gq < n_groups) {
-        const int r = (gq << 3) + (tid & 7);
-        const bool in = r < row_limit;
-        cp_async16(X + (gq * cpr + c) * 64 + (tid & 7) * 8, in ? base + (size_t)r * d + c * 8 : base, in ? 16u : 0u);
-        gq += step_g;
-        c += step_c;
-        if (c >= cpr) { c -= cpr; ++gq; }
-      }
-      cp_async_wait_all();
-      fence_proxy_async_smem();
-    }
-    __syncthreads();
-
-    // ---- MMAs (one thread issues)
+  // multiply the staged unit and drain the accumulators
+  auto run_unit = [&](const ProjUnit& pu, bool is_item, bf16* X) -> bool {
     if (tid == 0) {
       tc_fence_after();
       const uint32_t xa = smem_u32(X);
       const int ksteps = d >> 4;
-      const uint32_t wa = smem_u32(is_item ? imgK : imgQ);
+      const uint32_t wa = smem_u32(imgK);
       const uint32_t id1 = idesc_bf16(128, dqk);
       for (int ks = 0; ks < ksteps; ++ks)
         mma_ss(tmem, smem_desc(xa + ks * 256, lbo, sbo), smem_desc(wa + ks * 256, lbo, sbo), id1, ks > 0);
       if (is_item) {
         const uint32_t va = smem_u32(imgV);
-        const uint32_t id2 = idesc_bf16(128, rows);
+        const uint32_t id2 = idesc_bf16(128, pu.rows);
         for (int ks = 0; ks < ksteps; ++ks)
           mma_ss(tmem + 128, smem_desc(va + ks * 256, lbo, sbo), smem_desc(xa + ks * 256, lbo, sbo), id2, ks > 0);
       }
       tc_commit(&bar_mma);
     }
-    ok = __syncthreads_and(mbar_wait(&bar_mma, mma_phase, abortp));
+    const bool ok = __syncthreads_and(mbar_wait(&bar_mma, mma_phase, abortp));
     mma_phase ^= 1;
-    if (!ok) break;
+    if (!ok) return false;
     tc_fence_after();
+    const int rows = pu.rows;
 
-    // ---- epilogue 1: K (or Q) rows.  TMEM lane = row of the unit; this warp's half of the columns, 16 per load.
+    // ---- K (or Q) rows.  TMEM lane = row of the unit; this warp's half of the columns, 16 per load.
     if (quad * 32 < rows) {
       const float scale = is_item ? 1.f : P.q_scale;
       bool valid;
       bf16* dst_row;                                       // start of row r0 inside head 0's block of its tile
       size_t head_stride;
       if (is_item) {
-        const int pos = (t0 + r0_tile) * IT + r0_in;
-        valid = r0 < rows && pos < seg_items;
-        dst_row = P.Kblk + ((size_t)u * P.n_tiles + seg * P.NT + t0 + r0_tile) * ((size_t)IT * dqk) +
+        const int pos = (pu.t0 + r0_tile) * IT + r0_in;
+        valid = r0 < rows && pos < pu.seg_items;
+        dst_row = P.Kblk + ((size_t)pu.u * P.n_tiles + pu.seg * P.NT + pu.t0 + r0_tile) * ((size_t)IT * dqk) +
                   (r0_in >> 3) * (cpr_k * 64) + (r0_in & 7) * 8;
         head_stride = (size_t)IT * P.dqh;
       } else {
-        valid = jt * kCandTile + r0 < us.nc;
-        dst_row = P.Qblk + (size_t)(P.tile_off[u] + jt) * (kCandTile * dqk) + (r0 >> 3) * (cpr_k * 64) + (r0 & 7) * 8;
+        valid = pu.jt * kCandTile + r0 < pu.nc;
+        dst_row = P.Qblk + (size_t)(P.tile_off[pu.u] + pu.jt) * (kCandTile * dqk) + (r0 >> 3) * (cpr_k * 64) + (r0 & 7) * 8;
         head_stride = (size_t)kCandTile * P.dqh;
       }
       for (int c16 = k_lo; c16 < k_hi; ++c16) {
@@ -337,7 +314,7 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
         }
       }
     }
-    // ---- epilogue 2: V^T.  TMEM lane = value feature j; columns = rows of the unit, this warp's half of them.
+    // ---- V^T.  TMEM lane = value feature j; columns = rows of the unit, this warp's half of them.
     if (is_item && quad * 32 < d) {
       const int n16 = rows >> 4;
       const int lo16 = half ? (n16 + 1) >> 1 : 0, hi16 = half ? n16 : (n16 + 1) >> 1;
@@ -349,8 +326,8 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
         if (j < d) {
           const int rr = c16 * 16;                          // unit row of the first of these 16 columns
           const int tt = rr / IT, in_tile = rr - tt * IT;   // IT is a multiple of 16: the 16 columns share a tile
-          const int n_valid = seg_items - ((t0 + tt) * IT + in_tile);   // valid items among them (may be <= 0 or >= 16)
-          bf16* dst = P.Vtblk + ((size_t)u * P.n_tiles + seg * P.NT + t0 + tt) * ((size_t)IT * d) +
+          const int n_valid = pu.seg_items - ((pu.t0 + tt) * IT + in_tile);   // valid items among them (<= 0 .. >= 16)
+          bf16* dst = P.Vtblk + ((size_t)pu.u * P.n_tiles + pu.seg * P.NT + pu.t0 + tt) * ((size_t)IT * d) +
                       (size_t)jh * IT * P.dvh + ((in_tile >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
 #pragma unroll
           for (int hf = 0; hf < 2; ++hf) {
@@ -370,9 +347,108 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
           }
         }
       }
-      if (j < d && hi16 > lo16) atomicAdd(&P.SV[((size_t)u * P.Lp + seg) * d + j], sv);
+      if (j < d && hi16 > lo16) atomicAdd(&P.SV[((size_t)pu.u * P.Lp + pu.seg) * d + j], sv);
     }
     tc_fence_before();
+    return true;
+  };
+
+  bool ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
+
+  // ---- item units: this block's contiguous range, two-deep pipeline
+  const int n_proj = P.counters[2];
+  const int G = gridDim.x, bidx = blockIdx.x;
+  const int lo = (int)(((long long)n_proj * bidx) / G), hi = (int)(((long long)n_proj * (bidx + 1)) / G);
+  if (ok && hi > lo) {
+    // cursor over (user, segment, tile group)
+    int cu, cseg, cgrp, c_nseg, c_len, c_last_groups;
+    auto load_user = [&]() {
+      const UserShape s = user_shape(P, cu);
+      c_nseg = s.nseg; c_len = s.len;
+      const int last_items = s.nseg > 0 ? s.len - (s.nseg - 1) * P.S : 0;
+      c_last_groups = (min(P.NT, (last_items + IT - 1) / IT) + P.NTG - 1) / P.NTG;
+    };
+    {
+      int a = 0, b = P.U;   // proj_start[a] <= lo < proj_start[b]
+      while (b - a > 1) {
+        const int mid = (a + b) >> 1;
+        if (P.proj_start[mid] <= lo) a = mid; else b = mid;
+      }
+      cu = a;
+      load_user();
+      const int local = lo - P.proj_start[cu];
+      cseg = local / P.NG;                                   // only the last segment can have fewer than NG groups
+      cgrp = local - cseg * P.NG;
+    }
+    auto make_unit = [&]() {
+      ProjUnit pu;
+      pu.u = cu; pu.seg = cseg; pu.t0 = cgrp * P.NTG;
+      pu.seg_items = min(P.S, c_len - cseg * P.S);
+      const int t1 = min(min(P.NT, pu.t0 + P.NTG), (pu.seg_items + IT - 1) / IT);   // tiles with valid items only
+      pu.rows = (t1 - pu.t0) * IT;
+      pu.jt = 0; pu.c0 = 0; pu.nc = 0;
+      return pu;
+    };
+    auto step = [&]() {
+      const int groups = cseg == c_nseg - 1 ? c_last_groups : P.NG;
+      if (++cgrp < groups) return;
+      cgrp = 0;
+      if (++cseg < c_nseg) return;
+      cseg = 0;
+      do {
+        ++cu;
+        if (cu >= P.U) return;
+        load_user();
+      } while (c_nseg == 0);
+    };
+
+    ProjUnit cur = make_unit();
+    int buf = 0;
+    stage(cur, true, Xbuf);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int n = lo; n < hi && ok; ++n) {
+      ProjUnit nxt = cur;
+      if (n + 1 < hi) {
+        step();
+        nxt = make_unit();
+        stage(nxt, true, Xbuf + (size_t)(buf ^ 1) * kCandTile * d);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+      fence_proxy_async_smem();
+      __syncthreads();                    // unit n staged by every thread; TMEM of unit n - 1 drained
+      ok = run_unit(cur, true, Xbuf + (size_t)buf * kCandTile * d);
+      cur = nxt;
+      buf ^= 1;
+    }
+  }
+
+  // ---- candidate tiles, dealt round-robin over the blocks (W_q^T replaces W_k^T in shared memory)
+  const int n_ctiles = P.counters[1];
+  if (ok && bidx < n_ctiles) {
+    __syncthreads();                      // every MMA that read W_k^T has completed (its accumulators were drained)
+    if (tid == 0) {
+      mbar_arrive_expect_tx(&bar_img, bK);
+      bulk_g2s(imgK, P.imgQ, bK, &bar_img);
+    }
+    ok = __syncthreads_and(mbar_wait(&bar_img, 1, abortp));
+    for (int ct = bidx; ct < n_ctiles && ok; ct += G) {
+      int a = 0, b = P.U;                 // tile_off[a] <= ct < tile_off[b]
+      while (b - a > 1) {
+        const int mid = (a + b) >> 1;
+        if (P.tile_off[mid] <= ct) a = mid; else b = mid;
+      }
+      const UserShape us = user_shape(P, a);
+      ProjUnit pu;
+      pu.u = a; pu.seg = 0; pu.t0 = 0; pu.rows = kCandTile; pu.seg_items = 0;
+      pu.jt = ct - P.tile_off[a]; pu.c0 = us.c0; pu.nc = us.nc;
+      __syncthreads();                    // staging buffer and TMEM of the previous unit are free
+      stage(pu, false, Xbuf);
+      cp_async_wait_all();
+      fence_proxy_async_smem();
+      __syncthreads();
+      ok = run_unit(pu, false, Xbuf);
+    }
   }
 
   tc_fence_before();
@@ -813,6 +889,7 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.SV = (float*)(ws + p.off_tsv);
   P.unit_start = (int*)(ws + p.off_twork);
   P.tile_off = P.unit_start + (p.U + 1);
+  P.proj_start = P.tile_off + (p.U + 1);
   P.counters = (int*)(ws + p.off_tcount);
   P.imgK = (bf16*)(ws + p.off_timg);
   P.imgQ = P.imgK + (size_t)p.dqk * p.d;
@@ -858,7 +935,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     tc_prep_kernel<<<1 + 32, 1024, 0, st>>>(P);
   }
   {
-    const size_t smem = ((size_t)2 * p.dqk * p.d + 2 * (size_t)kCandTile * p.d) * 2;
+    const size_t smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;   // W_k^T | W_q^T, W_v^T, two staging buffers
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("tc_proj", st);
     tc_proj_kernel<<<2 * sms, kProjThreads, smem, st>>>(P);
