@@ -84,9 +84,8 @@ int make_plan(const laser_config* c, Plan* p) {
     p->off_tq = off; off = align_up(off + q_tiles * 128 * p->dqk * 2);
     p->off_tk = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->dqk * 2);
     p->off_tv = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->d * 2);
-    p->off_tsv = off; off = align_up(off + (size_t)p->U * p->Lp * p->d * sizeof(float));
     p->off_twork = off; off = align_up(off + ((size_t)p->U + 1) * 3 * sizeof(int));
-    p->off_tcount = off; off = align_up(off + 64 * sizeof(int));
+    p->off_tcount = off; off = align_up(off + 64 * sizeof(int) + 2 * 1024 * 4 * sizeof(int));   // counters + per-block start tables
     p->off_timg = off; off = align_up(off + ((size_t)2 * p->dqk * p->d + (size_t)128 * p->d) * 2);
     if (gsta_mma_supported(*p)) { p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p)); }
   } else if (path == LASER_PATH_STREAM) {

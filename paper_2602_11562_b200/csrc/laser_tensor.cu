@@ -5,12 +5,12 @@
 //                    value sums, and writes the transposed weight images in UMMA canonical layout.
 //   tc_proj_kernel   Eq. 8-9: K = X W_k, V = X W_v (and Q = T W_q / (2 gamma)) on the tensor cores.  Outputs are written
 //                    tile by tile in exactly the shared-memory layout the attention kernel's MMAs consume, so that
-//                    kernel stages them with plain bulk copies.  Also accumulates SV = sum of valid V rows per segment.
+//                    kernel stages them with plain bulk copies.
 //   tc_sta_kernel    Eq. 10-12 fused: per (user, 128-candidate tile, segment) and head,
-//                      scores = Q_h K_h^T (MMA, TMEM)  ->  P' = tanh(scores) (registers)  ->  O_h += P' V_h (MMA, TMEM)
-//                    and H' = (SV + O) / 2.  Uses Sigmoid(x) = 1/2 + 1/2 tanh(x/2): the 1/2 term is the candidate-
-//                    independent sum SV, the tanh term needs one transcendental and nothing else per gate.  Masked
-//                    items have zero K and V rows, so they contribute exactly nothing.  No score ever leaves the SM.
+//                      scores = Q_h K_h^T (MMA, TMEM)  ->  P = 1 + tanh(scores) (registers)  ->  O_h += P V_h (MMA, TMEM)
+//                    and H' = O / 2.  Uses Sigmoid(x) = (1 + tanh(x/2)) / 2 with 1 / (2 gamma) folded into Q: one
+//                    transcendental and one add per gate.  Masked items have zero K and V rows, so they contribute
+//                    exactly nothing.  No score ever leaves the SM.
 #include "laser_common.cuh"
 #include "laser_ptx.cuh"
 
@@ -37,10 +37,12 @@ struct TcParams {
   const bf16 *items, *cands, *Wq, *Wk, *Wv;
   const int *lengths, *cand_offsets;
   bf16 *Qblk, *Kblk, *Vtblk;
-  float* SV;                          // [U, Lp, d] sum of the valid (bf16-rounded) V rows of each segment
   int *unit_start, *tile_off;         // [U+1] prefix of attention units / candidate tiles per user
   int* proj_start;                    // [U+1] prefix of projection units (groups of item tiles that hold valid items)
   int* counters;                      // [0] attention units, [1] candidate tiles, [2] projection units
+  int4* sta_begin;                    // [sta_grid]  first attention unit of every block: (user, candidate tile, segment, -)
+  int4* proj_begin;                   // [proj_grid] first projection unit of every block: (user, segment, tile group, -)
+  int sta_grid, proj_grid;
   bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
   int* status;
   bf16* Hp;
@@ -126,9 +128,39 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
       P.counters[1] = sa[1023];
       P.counters[2] = sc[1023];
     }
+    // First unit of every block of the two main kernels (block b of G owns units [n b / G, n (b + 1) / G)): find the
+    // scan chunk in shared memory, then the user inside the chunk.
+    const int n_att = sb[1023], n_proj = sc[1023];
+    for (int b = tid; b < P.sta_grid + P.proj_grid; b += 1024) {
+      const bool att = b < P.sta_grid;
+      const int* incl = att ? sb : sc;
+      const int n = att ? n_att : n_proj, G = att ? P.sta_grid : P.proj_grid, bb = att ? b : b - P.sta_grid;
+      const int id = (int)(((long long)n * bb) / G);
+      int4 out = make_int4(-1, 0, 0, 0);
+      if (id < n) {
+        int lo = 0, hi = 1023;                     // smallest chunk k with incl[k] > id
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (incl[mid] > id) hi = mid; else lo = mid + 1;
+        }
+        int base = lo > 0 ? incl[lo - 1] : 0;      // units before the chunk
+        int u = min(lo * per, P.U);
+        UserShape s = user_shape(P, u);
+        for (;;) {
+          const int cnt = att ? s.ctiles * s.nseg : proj_units_of(P, s);
+          if (id < base + cnt) break;
+          base += cnt;
+          s = user_shape(P, ++u);
+        }
+        const int local = id - base;
+        if (att) out = make_int4(u, local / s.nseg, local % s.nseg, 0);
+        else out = make_int4(u, local / P.NG, local % P.NG, 0);
+      }
+      if (att) P.sta_begin[bb] = out; else P.proj_begin[bb] = out;
+    }
     return;
   }
-  // remaining blocks: weight images and SV zero fill, grid-stride
+  // remaining blocks: weight images, grid-stride
   const int nthreads = (gridDim.x - 1) * blockDim.x;
   const int g = (blockIdx.x - 1) * blockDim.x + tid;
   const int nK = P.dqk * P.d;
@@ -143,8 +175,6 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     const int k = i / kCandTile, j = i - k * kCandTile;
     P.imgV[canon_off(j, k, P.d)] = j < P.d ? P.Wv[(size_t)k * P.d + j] : __float2bfloat16_rn(0.f);
   }
-  const size_t nS = (size_t)P.U * P.Lp * P.d;
-  for (size_t i = g; i < nS; i += nthreads) P.SV[i] = 0.f;
 }
 
 // H' rows of segments without valid items are zero rows (only needed when the caller wants H').
@@ -255,21 +285,19 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
 
   // multiply the staged unit and drain the accumulators
   auto run_unit = [&](const ProjUnit& pu, bool is_item, bf16* X) -> bool {
-    if (tid == 0) {
+    if (warp == 0) {                                         // warp-uniform loop, one elected lane issues
       tc_fence_after();
-      const uint32_t xa = smem_u32(X);
+      const uint64_t xd = smem_desc(smem_u32(X), lbo, sbo), wd = smem_desc(smem_u32(imgK), lbo, sbo);
+      const uint64_t vd = smem_desc(smem_u32(imgV), lbo, sbo);
       const int ksteps = d >> 4;
-      const uint32_t wa = smem_u32(imgK);
-      const uint32_t id1 = idesc_bf16(128, dqk);
-      for (int ks = 0; ks < ksteps; ++ks)
-        mma_ss(tmem, smem_desc(xa + ks * 256, lbo, sbo), smem_desc(wa + ks * 256, lbo, sbo), id1, ks > 0);
-      if (is_item) {
-        const uint32_t va = smem_u32(imgV);
-        const uint32_t id2 = idesc_bf16(128, pu.rows);
-        for (int ks = 0; ks < ksteps; ++ks)
-          mma_ss(tmem + 128, smem_desc(va + ks * 256, lbo, sbo), smem_desc(xa + ks * 256, lbo, sbo), id2, ks > 0);
+      const uint32_t id1 = idesc_bf16(128, dqk), id2 = idesc_bf16(128, pu.rows);
+      if (elect_one()) {
+        for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem, xd + ks * 16, wd + ks * 16, id1, ks > 0);
+        if (is_item)
+          for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem + 128, vd + ks * 16, xd + ks * 16, id2, ks > 0);
+        tc_commit(&bar_mma);
       }
-      tc_commit(&bar_mma);
+      __syncwarp();
     }
     const bool ok = __syncthreads_and(mbar_wait(&bar_mma, mma_phase, abortp));
     mma_phase ^= 1;
@@ -318,7 +346,6 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     if (is_item && quad * 32 < d) {
       const int n16 = rows >> 4;
       const int lo16 = half ? (n16 + 1) >> 1 : 0, hi16 = half ? n16 : (n16 + 1) >> 1;
-      float sv = 0.f;
       for (int c16 = lo16; c16 < hi16; ++c16) {
         uint32_t v[16];
         tmem_ld16(tmem_lane + 128 + c16 * 16, v);
@@ -341,13 +368,11 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
                 if (2 * e + 1 >= cnt) b = 0.f;
               }
               pk[e] = pack_bf16x2(a, b);
-              sv += __uint_as_float(pk[e] << 16) + __uint_as_float(pk[e] & 0xFFFF0000u);
             }
             *reinterpret_cast<uint4*>(dst + hf * npr * 64) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
-      if (j < d && hi16 > lo16) atomicAdd(&P.SV[((size_t)pu.u * P.Lp + pu.seg) * d + j], sv);
     }
     tc_fence_before();
     return true;
@@ -369,16 +394,9 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
       c_last_groups = (min(P.NT, (last_items + IT - 1) / IT) + P.NTG - 1) / P.NTG;
     };
     {
-      int a = 0, b = P.U;   // proj_start[a] <= lo < proj_start[b]
-      while (b - a > 1) {
-        const int mid = (a + b) >> 1;
-        if (P.proj_start[mid] <= lo) a = mid; else b = mid;
-      }
-      cu = a;
+      const int4 b = P.proj_begin[bidx];                     // this block's first unit, as found by tc_prep_kernel
+      cu = b.x; cseg = b.y; cgrp = b.z;
       load_user();
-      const int local = lo - P.proj_start[cu];
-      cseg = local / P.NG;                                   // only the last segment can have fewer than NG groups
-      cgrp = local - cseg * P.NG;
     }
     auto make_unit = [&]() {
       ProjUnit pu;
@@ -469,17 +487,10 @@ struct UnitWalker {
     last_items = s.nseg > 0 ? s.len - (s.nseg - 1) * P.S : 0;       // items of the last non-empty segment
     last_tiles = min(P.NT, (last_items + P.IT - 1) / P.IT);
   }
-  __device__ void init(const TcParams& P, int id) {
-    int lo = 0, hi = P.U;   // unit_start[lo] <= id < unit_start[hi]
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (P.unit_start[mid] <= id) lo = mid; else hi = mid;
-    }
-    u = lo;
+  __device__ void init(const TcParams& P) {       // this block's first unit, as found by tc_prep_kernel
+    const int4 b = P.sta_begin[blockIdx.x];
+    u = b.x; j = b.y; seg = b.z;
     load_user(P);
-    const int local = id - P.unit_start[u];
-    j = local / nseg;
-    seg = local - j * nseg;
   }
   __device__ void next(const TcParams& P) {
     if (++seg < nseg) return;
@@ -517,20 +528,19 @@ constexpr uint32_t kColO = kColP + kGateGroups * (kItMax / 2);   // outputs [n_o
 
 // Roles of the 25 warps of a block (one block per SM):
 //   warps 0-3   MMA issuers, one per gate warpgroup (the warp runs the loop, one elected lane issues)
-//   warps 4-7   epilogue: H' = (SV + O) / 2 per finished segment, staged in shared memory, written by bulk stores
-//   warps 8-23  four gate warpgroups: P' = tanh(S)
+//   warps 4-7   epilogue: H' = O / 2 per finished segment, staged in shared memory, written by bulk stores
+//   warps 8-23  four gate warpgroups: P = 1 + tanh(S)
 //   warp 24     bulk-copy producer (Q tile per (user, candidate tile), K / V^T tile per item tile, mbarrier rings) and
 //               TMEM allocation
 // A gate-unit is one (item tile, head).  Head h always belongs to warpgroup / issuer h % 4, which owns one score buffer
 // and one gate buffer in TMEM.  Per unit: the issuer writes S = Q_h K_h^T; the warpgroup reads it (releasing the score
-// buffer for the issuer's next unit as soon as the last column is in registers), writes P' = tanh(S) as packed bf16; the
-// issuer accumulates O_h += P' V_h.  All MMAs into a head's accumulator come from one thread, in order.
+// buffer for the issuer's next unit as soon as the last column is in registers), writes P = 1 + tanh(S) as packed bf16;
+// the issuer accumulates O_h += P V_h.  All MMAs into a head's accumulator come from one thread, in order.
 __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ StaBars bars;
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
-  __shared__ __align__(16) float sv_s[4][2][128];   // per epilogue warp, double-buffered: SV row of the segment
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d = P.d, dqk = P.dqk, IT = P.IT, H = P.H;
@@ -586,7 +596,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
       // ------------------------------------------------------------------ bulk-copy producer
       if (lane == 0) {
         UnitWalker w;
-        w.init(P, unit_lo);
+        w.init(P);
         int pu = -1, pj = -1;
         uint32_t qcount = 0, st = 0, kv_par = 1;      // kv_par: parity that means "stage st is free"
         bool ok = true;
@@ -702,7 +712,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         };
 
         Cursor cur;
-        cur.w.init(P, unit_lo);
+        cur.w.init(P);
         cur.it = 0; cur.t = 0; cur.h = wgi; cur.nt = cur.w.ntiles(P); cur.st = 0; cur.kv_par = 0;
         issue_scores(cur);
         while (ok) {
@@ -725,13 +735,13 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         wait_all(&bars.done[wgi], 0);
       }
     } else if (warp >= 8 && warp < kProducerWarp) {
-      // ------------------------------------------------------------------ gate warps: P' = tanh(scores)
+      // ------------------------------------------------------------------ gate warps: P = 1 + tanh(scores)
       const int wg = (warp - 8) >> 2;                       // warpgroup wg owns buffers wg and heads wg, wg + 4, ...
       const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
       const uint32_t tS = tmem + lane_base + kColS + wg * kItMax;
       const uint32_t tP = tmem + lane_base + kColP + wg * (kItMax / 2);
       UnitWalker w;
-      w.init(P, unit_lo);
+      w.init(P);
       uint32_t s_par = 0, pf_par = 1;
       int my_heads = 0;
       for (int h = wg; h < H; h += kGateGroups) ++my_heads;
@@ -759,7 +769,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
               if (c + 32 >= cols) release_scores();
 #pragma unroll
               for (int e = 0; e < 16; ++e)
-                o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+                o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
               if (first) {                                  // the previous unit's gates have been multiplied
                 ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
                 pf_par ^= 1;
@@ -775,7 +785,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
               release_scores();
 #pragma unroll
               for (int e = 0; e < 8; ++e)
-                o[e] = pack_bf16x2(tanh_approx(__uint_as_float(v[2 * e])), tanh_approx(__uint_as_float(v[2 * e + 1])));
+                o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
               if (first) {
                 ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
                 pf_par ^= 1;
@@ -792,29 +802,15 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         }
       }
     } else if (warp >= 4) {
-      // ------------------------------------------------------------------ epilogue: H' = (SV + O) / 2
+      // ------------------------------------------------------------------ epilogue: H' = O / 2
       const int q = warp - 4;
       const uint32_t lane_base = (uint32_t)(q * 32) << 16;
       const int m = q * 32 + lane;
       UnitWalker w;
-      w.init(P, unit_lo);
+      w.init(P);
       uint32_t ob = 0, o_par = 0;
       bool ok = true;
-      // the SV row of the next segment is fetched into registers one unit ahead and handed over through shared memory
-      float sv_reg[4];
-      auto fetch_sv = [&](const UnitWalker& ww) {
-        const float* sv = P.SV + ((size_t)ww.u * P.Lp + ww.seg) * d;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) sv_reg[i] = lane + 32 * i < d ? __ldg(sv + lane + 32 * i) : 0.f;
-      };
-      fetch_sv(w);
-      for (int it = 0; it < my_units && ok; ++it) {
-        float* svb = sv_s[q][it & 1];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) svb[lane + 32 * i] = sv_reg[i];
-        UnitWalker wn = w;
-        wn.next(P);
-        if (it + 1 < my_units) fetch_sv(wn);
+      for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
         uint8_t* row = Os + ((size_t)(it & 1) * kCandTile + m) * out_row;
         bulk_wait_read<1>();                               // my store from this staging buffer (two units ago) has left it
         __syncwarp();
@@ -833,13 +829,11 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           }
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            const float4 s0 = *reinterpret_cast<const float4*>(svb + c + half * 8);
-            const float4 s1 = *reinterpret_cast<const float4*>(svb + c + half * 8 + 4);
             uint4 o;
-            o.x = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 0]) + s0.x), 0.5f * (__uint_as_float(v[half * 8 + 1]) + s0.y));
-            o.y = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 2]) + s0.z), 0.5f * (__uint_as_float(v[half * 8 + 3]) + s0.w));
-            o.z = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 4]) + s1.x), 0.5f * (__uint_as_float(v[half * 8 + 5]) + s1.y));
-            o.w = pack_bf16x2(0.5f * (__uint_as_float(v[half * 8 + 6]) + s1.z), 0.5f * (__uint_as_float(v[half * 8 + 7]) + s1.w));
+            o.x = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 0]), 0.5f * __uint_as_float(v[half * 8 + 1]));
+            o.y = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 2]), 0.5f * __uint_as_float(v[half * 8 + 3]));
+            o.z = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 4]), 0.5f * __uint_as_float(v[half * 8 + 5]));
+            o.w = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 6]), 0.5f * __uint_as_float(v[half * 8 + 7]));
             *reinterpret_cast<uint4*>(row + (c + half * 8) * 2) = o;
           }
         }
@@ -850,7 +844,6 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         }
         bulk_commit();
         if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
-        w = wn;
       }
       bulk_wait<0>();
     }
@@ -886,11 +879,14 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.Wq = (const bf16*)Wq; P.Wk = (const bf16*)Wk; P.Wv = (const bf16*)Wv;
   P.lengths = lengths; P.cand_offsets = cand_offsets;
   P.Qblk = (bf16*)(ws + p.off_tq); P.Kblk = (bf16*)(ws + p.off_tk); P.Vtblk = (bf16*)(ws + p.off_tv);
-  P.SV = (float*)(ws + p.off_tsv);
   P.unit_start = (int*)(ws + p.off_twork);
   P.tile_off = P.unit_start + (p.U + 1);
   P.proj_start = P.tile_off + (p.U + 1);
   P.counters = (int*)(ws + p.off_tcount);
+  P.sta_begin = reinterpret_cast<int4*>(ws + p.off_tcount + 64 * sizeof(int));
+  P.proj_begin = P.sta_begin + 1024;
+  P.sta_grid = sm_count() < 1024 ? sm_count() : 1024;
+  P.proj_grid = 2 * sm_count() < 1024 ? 2 * sm_count() : 1024;
   P.imgK = (bf16*)(ws + p.off_timg);
   P.imgQ = P.imgK + (size_t)p.dqk * p.d;
   P.imgV = P.imgQ + (size_t)p.dqk * p.d;
@@ -938,7 +934,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     const size_t smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;   // W_k^T | W_q^T, W_v^T, two staging buffers
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("tc_proj", st);
-    tc_proj_kernel<<<2 * sms, kProjThreads, smem, st>>>(P);
+    tc_proj_kernel<<<P.proj_grid, kProjThreads, smem, st>>>(P);
   }
   if (user_wants_hp) {
     LaunchScope ls("tc_zero_empty", st);
@@ -950,7 +946,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     if (smem > 220 * 1024) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_sta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("sta_tc", st);
-    tc_sta_kernel<<<sms, kStaThreads, smem, st>>>(P);
+    tc_sta_kernel<<<P.sta_grid, kStaThreads, smem, st>>>(P);
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
