@@ -4,10 +4,11 @@
 //
 //   A   Q   = T W_q^l                              [16 x d]    batched over the 16 candidates
 //   B   Qt_h = Q[:, head h] W_k^l[:, head h]^T / tau  [16 x d] per head: (s_j W_k)_h . q_h = s_j . Qt_h
-//   C   per candidate: scores e_{h,j} = Qt_h . s_j over its non-empty segments j, softmax over j, m_h = sum_j a_{h,j} s_j.
-//       The candidate's segment vectors are staged in shared memory (cp.async, two buffers per warp, 16 vectors per
-//       chunk); every vector is read from global memory once per layer and used for both contractions, with an online
-//       softmax across chunks.
+//   C   per candidate: scores e_{j,h} = s_j . Qt_h over its non-empty segments j, softmax over j, m_h = sum_j a_{j,h} s_j.
+//       A candidate's segment vectors are staged in shared memory 16 at a time (cp.async, two buffers per warp, padded
+//       rows); every vector is read from global memory once per layer and feeds both contractions as the 16-row MMA
+//       operand: scores = S Qt^T (rows = segments, columns =
+//       heads) and m^T = S^T P (rows = features), with an online softmax across chunks.
 //   D   o[:, head h] = m_h W_v^l[:, head h];  T += o
 //
 // This is Eq. 7 re-associated (exact in real arithmetic): the key / value projections are applied to the query and to
@@ -113,35 +114,45 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   for (int i = tid; i < RS / 4; i += kGThreads) reinterpret_cast<uint32_t*>(zrow)[i] = 0u;
   __syncthreads();
 
-  // ---- chunk pipeline of this warp: (layer, candidate slot ci -> candidate warp + kGW ci, chunk) in processing order
+  // ---- this warp's two candidates (slots): candidate warp + kGW s; two staging buffers of kChunk rows.
+  // A chunk is kChunk rows of 2 D16 16-byte pieces; lane l copies pieces l, l + 32, ...
+  static_assert(kGT == 2 * kGW, "two candidates per warp");
+  static_assert((kChunk * 2 * D16) % 32 == 0, "a chunk is a whole number of 16-byte pieces per lane");
+  constexpr int kPieces = kChunk * 2 * D16 / 32;
   uint8_t* my_stage = stage + (size_t)warp * 2 * kChunk * RS;
-  int f_layer = 0, f_ci = 0, f_ch = 0;
-  bool f_valid = false;
-  int first_ci = -1;
+  const uint32_t stage_addr = smem_addr(my_stage);
+  int p_row[kPieces], p_src[kPieces];
+  uint32_t p_dst[kPieces];
 #pragma unroll
-  for (int ci = kGT / kGW - 1; ci >= 0; --ci)
-    if (nv_s[warp + kGW * ci] > 0) first_ci = ci;
-  if (first_ci >= 0 && P.M > 0) { f_valid = true; f_ci = first_ci; }
-
-  auto issue = [&](int buf) {   // stage chunk (f_ci, f_ch) into buffer `buf`, then step the fetch cursor
-    const int c = warp + kGW * f_ci;
-    const int nv = nv_s[c];
-    const bf16* src = P.Hp + ((size_t)(c_base + c) * P.Lp + f_ch * kChunk) * d;
-    const uint32_t dst = smem_addr(my_stage + (size_t)buf * kChunk * RS);
-    const int rows = min(kChunk, nv - f_ch * kChunk);
-    static_assert((kChunk * 2 * D16) % 32 == 0, "a chunk is a whole number of 16-byte pieces per lane");
+  for (int i = 0; i < kPieces; ++i) {
+    const int piece = i * 32 + lane;
+    p_row[i] = piece / (2 * D16);
+    const int q = piece - p_row[i] * (2 * D16);
+    p_src[i] = p_row[i] * d + q * 8;
+    p_dst[i] = p_row[i] * RS + q * 16;
+  }
+  // fetch cursor over (layer, slot, chunk) in processing order; the two buffers alternate
+  int nv2[2];
 #pragma unroll
-    for (int i = 0; i < kChunk * 2 * D16 / 32; ++i) {      // kChunk rows of 2 D16 16-byte pieces
-      const int piece = i * 32 + lane;
-      const int r = piece / (2 * D16), q = piece - r * (2 * D16);
-      const bool ok = r < rows;
-      cp16(dst + r * RS + q * 16, ok ? (const void*)(src + (size_t)r * d + q * 8) : (const void*)P.Hp, ok ? 16u : 0u);
+  for (int sl = 0; sl < 2; ++sl) nv2[sl] = nv_s[warp + kGW * sl];
+  const int first_sl = nv2[0] > 0 ? 0 : (nv2[1] > 0 ? 1 : -1);
+  int f_layer = 0, f_sl = first_sl, f_ch = 0;
+  bool f_valid = first_sl >= 0 && P.M > 0;
+  auto issue = [&](int buf) {   // stage chunk (f_sl, f_ch) into buffer `buf`, then step the cursor
+    const int nv = f_sl ? nv2[1] : nv2[0];
+    const bf16* src = P.Hp + ((size_t)(c_base + warp + kGW * f_sl) * P.Lp + f_ch * kChunk) * d;
+    const uint32_t dst = stage_addr + buf * (kChunk * RS);
+    const int rows = nv - f_ch * kChunk;               // rows past the candidate's segments become zeros
+#pragma unroll
+    for (int i = 0; i < kPieces; ++i) {
+      const bool ok = p_row[i] < rows;
+      cp16(dst + p_dst[i], ok ? (const void*)(src + p_src[i]) : (const void*)P.Hp, ok ? 16u : 0u);
     }
     if (++f_ch * kChunk >= nv) {
       f_ch = 0;
-      do { ++f_ci; } while (f_ci < kGT / kGW && nv_s[warp + kGW * f_ci] == 0);
-      if (f_ci >= kGT / kGW) {
-        f_ci = first_ci;
+      if (f_sl == 0 && nv2[1] > 0) f_sl = 1;
+      else {
+        f_sl = first_sl;
         if (++f_layer >= P.M) f_valid = false;
       }
     }
@@ -220,104 +231,79 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
     __syncthreads();
 
     // ---------------------------------------------------------------- C: per candidate, online softmax over chunks
-    for (int ci = 0; ci < kGT / kGW; ++ci) {
-      const int c = warp + kGW * ci;
-      const int nv = nv_s[c];
-      if (nv == 0) {   // no segment to attend to: m = 0 (o_l = 0)
-        for (int i = lane; i < H * (d / 2); i += 32) {
-          const int h = i / (d / 2), q = i - h * (d / 2);
-          *reinterpret_cast<uint32_t*>(Qt + (c * H + h) * RS + q * 4) = 0u;
-        }
-        continue;
-      }
-      // A fragments of Qt_c: rows = heads (rows >= H read the zero row), only rows 0-7 are non-zero
-      uint32_t qa[D16][2];
-      {
-        const int h = lane & 7;
-        const uint8_t* rowp = h < H ? Qt + (c * H + h) * RS : zrow;
+    {
+      const uint32_t a_off = ((lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16;     // S as [segment][k]
+      const uint32_t t_off = ((lane & 7) + (lane >> 4) * 8) * RS + ((lane >> 3) & 1) * 16;     // S^T: [feature][segment]
+#pragma unroll 1
+      for (int sl = 0; sl < 2; ++sl) {
+        const int c = warp + kGW * sl;
+        const int nv = sl ? nv2[1] : nv2[0];
+        float macc[D16][4];           // m^T tiles: (feature 16 jt + g | + 8, heads 2t, 2t+1)
 #pragma unroll
-        for (int kt = 0; kt < D16; ++kt) ldsm_x2(qa[kt], smem_addr(rowp + (kt * 2 + ((lane >> 3) & 1)) * 16));
-      }
-      float macc[2 * D16][4];
-#pragma unroll
-      for (int j = 0; j < 2 * D16; ++j) macc[j][0] = macc[j][1] = macc[j][2] = macc[j][3] = 0.f;
-      float run_max = -INFINITY, run_sum = 0.f;
-
-      const int nch = (nv + kChunk - 1) / kChunk;
-      for (int ch = 0; ch < nch; ++ch) {
-        if (f_valid) issue(buf ^ 1);
-        cp_commit();
-        cp_wait<1>();
-        __syncwarp();
-        const uint32_t sb = smem_addr(my_stage + (size_t)buf * kChunk * RS);
-        const int rows = min(kChunk, nv - ch * kChunk);
-
-        // scores e[h][j] for the chunk's (up to) 16 segments: 2 column tiles of 8 segments; even and odd k-tiles
-        // accumulate separately so that four MMA chains are in flight
-        float e[2][4], e2[2][4];
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int q = 0; q < 4; ++q) e[nt][q] = e2[nt][q] = 0.f;
+        for (int jt = 0; jt < D16; ++jt) macc[jt][0] = macc[jt][1] = macc[jt][2] = macc[jt][3] = 0.f;
+        float rm0 = -INFINITY, rm1 = -INFINITY, rs0 = 0.f, rs1 = 0.f;
+        // B fragments of Qt^T: rows = heads of the candidate's Qt block (rows >= H read the zero row)
+        uint32_t qb[D16][2];
         {
-          const uint32_t a = sb + ((lane & 7) + ((lane >> 4) & 1) * 8) * RS + ((lane >> 3) & 1) * 16;
+          const int h = lane & 7;
+          const uint8_t* qrow = (h < H ? Qt + (c * H + h) * RS : zrow) + ((lane >> 3) & 1) * 16;
+#pragma unroll
+          for (int kt = 0; kt < D16; ++kt) ldsm_x2(qb[kt], smem_addr(qrow + kt * 32));
+        }
+        const int nch = (nv + kChunk - 1) / kChunk;
+        for (int ch = 0; ch < nch; ++ch) {
+          if (f_valid) issue(buf ^ 1);
+          cp_commit();
+          cp_wait<1>();
+          __syncwarp();
+          const uint32_t sb = stage_addr + buf * (kChunk * RS);
+          const int rows = nv - ch * kChunk;
+          float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};   // even / odd k-tiles: two MMA chains
 #pragma unroll
           for (int kt = 0; kt < D16; ++kt) {
-            uint32_t b[4];
-            ldsm_x4(b, a + kt * 32);
-            if (kt & 1) {
-              mma16816(e2[0], qa[kt][0], 0u, qa[kt][1], 0u, b[0], b[1]);
-              mma16816(e2[1], qa[kt][0], 0u, qa[kt][1], 0u, b[2], b[3]);
-            } else {
-              mma16816(e[0], qa[kt][0], 0u, qa[kt][1], 0u, b[0], b[1]);
-              mma16816(e[1], qa[kt][0], 0u, qa[kt][1], 0u, b[2], b[3]);
-            }
+            uint32_t a[4];
+            ldsm_x4(a, sb + a_off + kt * 32);
+            if (kt & 1) mma16816(e1, a[0], a[1], a[2], a[3], qb[kt][0], qb[kt][1]);
+            else mma16816(e0, a[0], a[1], a[2], a[3], qb[kt][0], qb[kt][1]);
+          }
+          float c0 = e0[0] + e1[0], c1 = e0[1] + e1[1], c2 = e0[2] + e1[2], c3 = e0[3] + e1[3];
+          if (g >= rows) c0 = c1 = -INFINITY;
+          if (g + 8 >= rows) c2 = c3 = -INFINITY;
+          // the chunk holds at least one valid segment, so both maxima are finite
+          const float nm0 = fmaxf(rm0, group_max(fmaxf(c0, c2))), nm1 = fmaxf(rm1, group_max(fmaxf(c1, c3)));
+          const float sc0 = __expf(rm0 - nm0), sc1 = __expf(rm1 - nm1);
+          rm0 = nm0;
+          rm1 = nm1;
+          const uint32_t plo = pack2(__expf(c0 - nm0), __expf(c1 - nm1));
+          const uint32_t phi = pack2(__expf(c2 - nm0), __expf(c3 - nm1));
+          // normalise by exactly the weights the MMA uses (this lane's share; summed over the lane groups at the end)
+          rs0 = rs0 * sc0 + bf16_lo(plo) + bf16_lo(phi);
+          rs1 = rs1 * sc1 + bf16_hi(plo) + bf16_hi(phi);
+          const uint32_t pb0 = movmatrix_t(plo), pb1 = movmatrix_t(phi);   // (segments 2t, 2t+1 | + 8, head g)
+#pragma unroll
+          for (int jt = 0; jt < D16; ++jt) {
+            uint32_t a[4];
+            ldsm_x4_t(a, sb + t_off + jt * 32);
+            macc[jt][0] *= sc0; macc[jt][1] *= sc1;
+            macc[jt][2] *= sc0; macc[jt][3] *= sc1;
+            mma16816(macc[jt], a[0], a[1], a[2], a[3], pb0, pb1);
+          }
+          __syncwarp();               // every lane is done with this buffer before the next iteration refills it
+          buf ^= 1;
+        }
+        // m_h = (sum_j p_j s_j) / (sum_j p_j), stored as rows [head][feature] of the candidate's block
+        const float s0 = group_sum(rs0), s1 = group_sum(rs1);
+        const float i0 = s0 > 0.f ? 1.f / s0 : 0.f, i1 = s1 > 0.f ? 1.f / s1 : 0.f;   // no segment: m = 0 (o_l = 0)
+        uint8_t* dst = Qt + (c * H + g) * RS + 4 * t;
+#pragma unroll
+        for (int jt = 0; jt < D16; ++jt) {
+          const uint32_t lo = movmatrix_t(pack2(macc[jt][0] * i0, macc[jt][1] * i1));   // (head g, features 16 jt + 2t..)
+          const uint32_t hi = movmatrix_t(pack2(macc[jt][2] * i0, macc[jt][3] * i1));   // (head g, features 16 jt + 8 + 2t..)
+          if (g < H) {
+            *reinterpret_cast<uint32_t*>(dst + jt * 32) = lo;
+            *reinterpret_cast<uint32_t*>(dst + jt * 32 + 16) = hi;
           }
         }
-        float mx = -INFINITY;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int q = 0; q < 2; ++q) {
-            e[nt][q] += e2[nt][q];
-            if (nt * 8 + 2 * t + q >= rows) e[nt][q] = -INFINITY;
-            mx = fmaxf(mx, e[nt][q]);
-          }
-        mx = quad_max(mx);                       // the chunk holds at least one valid segment, so mx is finite
-        const float new_max = fmaxf(run_max, mx);
-        const float scale = __expf(run_max - new_max);
-        run_max = new_max;
-        float psum = 0.f;
-        uint32_t pa[2];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          const float p0 = __expf(e[q][0] - new_max), p1 = __expf(e[q][1] - new_max);
-          pa[q] = pack2(p0, p1);
-          psum += bf16_lo(pa[q]) + bf16_hi(pa[q]);   // normalise by exactly the weights the MMA uses
-        }
-        run_sum = run_sum * scale + psum;
-#pragma unroll
-        for (int j = 0; j < 2 * D16; ++j) { macc[j][0] *= scale; macc[j][1] *= scale; }
-
-        // m += P S   (rows = heads, k = the chunk's segments, columns = d)
-        {
-          const uint32_t a = sb + ((lane & 7) + ((lane >> 3) & 1) * 8) * RS + (lane >> 4) * 16;
-#pragma unroll
-          for (int jp = 0; jp < D16; ++jp) {
-            uint32_t b[4];
-            ldsm_x4_t(b, a + jp * 32);
-            mma16816(macc[2 * jp], pa[0], 0u, pa[1], 0u, b[0], b[1]);
-            mma16816(macc[2 * jp + 1], pa[0], 0u, pa[1], 0u, b[2], b[3]);
-          }
-        }
-        __syncwarp();   // every lane is done with this buffer before the next iteration refills it
-        buf ^= 1;
-      }
-      const float inv = 1.f / quad_sum(run_sum);
-      if (g < H) {
-#pragma unroll
-        for (int j = 0; j < 2 * D16; ++j)
-          *reinterpret_cast<uint32_t*>(Qt + (c * H + g) * RS + (j * 8 + 2 * t) * 2) = pack2(macc[j][0] * inv, macc[j][1] * inv);
       }
     }
     __syncthreads();
