@@ -118,23 +118,24 @@ static int clear_status(const Plan& p, char* ws, cudaStream_t st) {
   return LASER_OK;
 }
 
+// Wg_images: GSTA weights whose images the STA set-up may build on the side (null when GSTA does not follow).
 static int run_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
                    const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hp, char* ws,
-                   cudaStream_t st) {
+                   cudaStream_t st, const void* Wg_images) {
   switch (p.path) {
     case LASER_PATH_SIMT: return simt_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
-    case LASER_PATH_TENSOR: return tensor_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
-    case LASER_PATH_STREAM: return stream_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+    case LASER_PATH_TENSOR: return tensor_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st, Wg_images);
+    case LASER_PATH_STREAM: return stream_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st, Wg_images);
     default: return LASER_ERR_UNSUPPORTED;
   }
 }
 
 static int run_gsta(const Plan& p, const void* Hp, const int32_t* lengths, const int32_t* cand_offsets,
-                    const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st) {
+                    const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready) {
   switch (p.path) {
     case LASER_PATH_SIMT: return simt_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
-    case LASER_PATH_TENSOR: return tensor_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
-    case LASER_PATH_STREAM: return gsta_mma(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+    case LASER_PATH_TENSOR: return tensor_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st, images_ready);
+    case LASER_PATH_STREAM: return gsta_mma(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st, images_ready);
     default: return LASER_ERR_UNSUPPORTED;
   }
 }
@@ -146,9 +147,10 @@ static int forward_impl(const Plan& p, const void* items, const int32_t* lengths
   if (rc != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
   void* Hp = Hprime ? Hprime : (void*)(ws + p.off_hp);
-  rc = run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st);
+  const bool side_images = p.M > 0 && p.path != LASER_PATH_SIMT && gsta_mma_supported(p);
+  rc = run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st, side_images ? Wg : nullptr);
   if (rc != LASER_OK) return rc;
-  return run_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st);
+  return run_gsta(p, Hp, lengths, cand_offsets, cands, Wg, z, ws, st, side_images);
 }
 
 }  // namespace laser
@@ -177,7 +179,7 @@ int laser_sta_forward(const laser_config* cfg, const void* items, const int32_t*
   char* ws = static_cast<char*>(workspace);
   if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
-  return run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
+  return run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st, nullptr);
 }
 
 int laser_gsta_forward(const laser_config* cfg, const void* Hprime, const int32_t* lengths,
@@ -195,7 +197,7 @@ int laser_gsta_forward(const laser_config* cfg, const void* Hprime, const int32_
   char* ws = static_cast<char*>(workspace);
   if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
-  return run_gsta(p, Hprime, lengths, cand_offsets, cands, Wgsta, z, ws, st);
+  return run_gsta(p, Hprime, lengths, cand_offsets, cands, Wgsta, z, ws, st, false);
 }
 
 int laser_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,

@@ -64,22 +64,26 @@ int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const i
 
 bool tensor_supported(const Plan& p);
 void tensor_geometry(const Plan& p, TensorGeom* g);
+// Wg_images: when non-null (and the fused GSTA kernel will follow), the set-up kernel also builds the GSTA weight images.
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
-               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
+               const void* Wg_images);
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
-                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st);
+                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready);
 
 // Fused warp-MMA GSTA kernel for bf16 (laser_gsta.cu); needs gsta_mma_image_bytes(p) of scratch at off_gimg.
 bool gsta_mma_supported(const Plan& p);
 size_t gsta_mma_image_bytes(const Plan& p);
+// images_ready: the weight images at off_gimg were already built for these weights earlier on the same stream.
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
-             const void* Wg, void* z, char* ws, cudaStream_t st);
+             const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready);
 
 // One-candidate-per-user STA (laser_stream.cu); needs stream_scratch_bytes(p) of scratch at off_su.  Its GSTA is gsta_mma.
 bool stream_supported(const Plan& p);
 size_t stream_scratch_bytes(const Plan& p);
 int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
-               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
+               const void* Wg_images);
 
 // --- device helpers ---------------------------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -17,6 +17,7 @@
 // The weights reach the MMAs as B fragments straight from a fragment-ordered image in global memory (built once per
 // call by gsta_prep_kernel), so they need no shared memory.
 #include "laser_common.cuh"
+#include "laser_gsta_img.cuh"
 #include "laser_mma.cuh"
 
 namespace laser {
@@ -40,34 +41,8 @@ struct GstaParams {
   int* status;
 };
 
-// Fragment-ordered weight images.  Entry (layer, matrix, kt, p, lane) holds the B fragments of k-tile kt for the two
-// 8-column tiles 2p and 2p+1: {b0, b1 of tile 2p, b0, b1 of tile 2p+1}.  For W_q and W_v the MMA's B is W itself
-// (B[k][n] = W[k][n]); for W_k it is the transpose (B[k][n] = W_k[n][k]).
 __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
-  const int D16 = P.d >> 4;
-  const int per_mat = D16 * D16 * 32;
-  const int total = P.M * 3 * per_mat;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-    const int lane = i & 31;
-    int r = i >> 5;
-    const int p = r % D16; r /= D16;
-    const int kt = r % D16; r /= D16;
-    const int m = r % 3;
-    const int l = r / 3;
-    const uint16_t* W = reinterpret_cast<const uint16_t*>(P.Wg) + (size_t)(l * 3 + m) * P.d * P.d;
-    const int g = lane >> 2, t = lane & 3;
-    uint32_t v[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int n = (2 * p + (q >> 1)) * 8 + g;
-      const int k = kt * 16 + 2 * t + (q & 1) * 8;
-      uint32_t lo, hi;
-      if (m == 1) { lo = W[(size_t)n * P.d + k]; hi = W[(size_t)n * P.d + k + 1]; }
-      else { lo = W[(size_t)k * P.d + n]; hi = W[(size_t)(k + 1) * P.d + n]; }
-      v[q] = lo | (hi << 16);
-    }
-    P.img[i] = make_uint4(v[0], v[1], v[2], v[3]);
-  }
+  gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
 }
 
 template <int D16>
@@ -368,7 +343,7 @@ bool gsta_mma_supported(const Plan& p) {
 size_t gsta_mma_image_bytes(const Plan& p) { return (size_t)p.M * 3 * p.d * p.d * 2; }
 
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
-             const void* Wg, void* z, char* ws, cudaStream_t st) {
+             const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready) {
   if (p.N == 0) return LASER_OK;
   GstaParams P;
   P.N = p.N; P.U = p.U; P.L = p.L; P.S = p.S; P.Lp = p.Lp; P.H = p.H; P.M = p.M; P.d = p.d;
@@ -378,7 +353,7 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   P.img = reinterpret_cast<uint4*>(ws + p.off_gimg);
   P.z = (bf16*)z;
   P.status = reinterpret_cast<int*>(ws + p.off_status);
-  if (p.M > 0) {
+  if (p.M > 0 && !images_ready) {
     const int total = p.M * 3 * (p.d / 16) * (p.d / 16) * 32;
     LaunchScope ls("gsta_prep", st);
     gsta_prep_kernel<<<(total + 255) / 256, 256, 0, st>>>(P);

@@ -19,6 +19,7 @@
 //                        its segment sums by W_v (MMA, rows = segments) and writes H'.
 //   GSTA                 the shared fused GSTA kernel (laser_gsta.cu) on that H'.
 #include "laser_common.cuh"
+#include "laser_gsta_img.cuh"
 #include "laser_mma.cuh"
 
 namespace laser {
@@ -42,6 +43,9 @@ struct StreamParams {
   uint4* imgv;                    // W_v as MMA B fragments: [d/16 k-tiles][d/16 column pairs][32 lanes]
   bf16* Hp;                       // [N, Lp, d]
   int zero_empty;                 // write zero rows for segments without valid items
+  const bf16* Wg;                 // GSTA weights whose images the pre kernel also builds (null: none)
+  uint4* gimg;
+  int M;
   int* status;
 };
 
@@ -74,6 +78,9 @@ __global__ void __launch_bounds__(256) stream_pre_kernel(StreamParams P, int use
       }
       P.imgv[i] = make_uint4(v[0], v[1], v[2], v[3]);
     }
+    if (P.Wg)
+      gsta_build_images(P.Wg, P.gimg, d, P.M, (blockIdx.x - user_blocks) * blockDim.x + tid,
+                        (gridDim.x - user_blocks) * blockDim.x);
     return;
   }
   // shared: W_q [d][dqk+1], W_k [d][dqk+1] (fp32, padded rows), t [kPreUsers][d], q [kPreUsers][dqk]
@@ -335,9 +342,13 @@ size_t stream_scratch_bytes(const Plan& p) {
 }
 
 int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
-               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
+               const void* Wg_images) {
   if (p.N == 0 || p.U == 0) return LASER_OK;
   StreamParams P;
+  P.Wg = (const bf16*)Wg_images;
+  P.gimg = reinterpret_cast<uint4*>(ws + p.off_gimg);
+  P.M = p.M;
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.inv_gamma = p.inv_gamma;
   P.items = (const bf16*)items; P.cands = (const bf16*)cands;
@@ -354,7 +365,7 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(stream_pre_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("stream_pre", st);
-    stream_pre_kernel<<<user_blocks + 4, 256, smem, st>>>(P, user_blocks);
+    stream_pre_kernel<<<user_blocks + 8, 256, smem, st>>>(P, user_blocks);
   }
   int rc;
   switch (p.d / 16) {

@@ -12,6 +12,7 @@
 //                    transcendental and one add per gate.  Masked items have zero K and V rows, so they contribute
 //                    exactly nothing.  No score ever leaves the SM.
 #include "laser_common.cuh"
+#include "laser_gsta_img.cuh"
 #include "laser_ptx.cuh"
 
 namespace laser {
@@ -43,6 +44,9 @@ struct TcParams {
   int4* sta_begin;                    // [sta_grid]  first attention unit of every block: (user, candidate tile, segment, -)
   int4* proj_begin;                   // [proj_grid] first projection unit of every block: (user, segment, tile group, -)
   int sta_grid, proj_grid;
+  const bf16* Wg;                     // GSTA weights whose images this set-up also builds (null: none)
+  uint4* gimg;
+  int M;
   bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
   int* status;
   bf16* Hp;
@@ -175,6 +179,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     const int k = i / kCandTile, j = i - k * kCandTile;
     P.imgV[canon_off(j, k, P.d)] = j < P.d ? P.Wv[(size_t)k * P.d + j] : __float2bfloat16_rn(0.f);
   }
+  if (P.Wg) gsta_build_images(P.Wg, P.gimg, P.d, P.M, g, nthreads);
 }
 
 // H' rows of segments without valid items are zero rows (only needed when the caller wants H').
@@ -921,10 +926,14 @@ void tensor_geometry(const Plan& p, TensorGeom* g) {
 }
 
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
-               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+               const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
+               const void* Wg_images) {
   if (p.N == 0 || p.U == 0) return LASER_OK;
   const bool user_wants_hp = Hprime != (void*)(ws + p.off_hp);
   TcParams P = make_params(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws);
+  P.Wg = (const bf16*)Wg_images;
+  P.gimg = reinterpret_cast<uint4*>(ws + p.off_gimg);
+  P.M = p.M;
   const int sms = sm_count();
   {
     LaunchScope ls("tc_prep", st);
@@ -953,8 +962,8 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
 }
 
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
-                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st) {
-  if (gsta_mma_supported(p)) return gsta_mma(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st);
+                const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready) {
+  if (gsta_mma_supported(p)) return gsta_mma(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st, images_ready);
   return simt_gsta(p, Hprime, lengths, cand_offsets, cands, Wg, z, ws, st);
 }
 
