@@ -1,0 +1,42 @@
+// Fragment-ordered images of the GSTA weights, shared by the kernels that can build them on the side (the GSTA
+// kernel's own set-up launch, or spare blocks of the STA paths' set-up kernels when STA and GSTA run back to back).
+//
+// Entry (layer, matrix, kt, p, lane) holds the mma.sync B fragments of k-tile kt for the two 8-column tiles 2p and
+// 2p+1: {b0, b1 of tile 2p, b0, b1 of tile 2p+1}.  For W_q and W_v the MMA's B is W itself (B[k][n] = W[k][n]); for
+// W_k it is the transpose (B[k][n] = W_k[n][k]).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace laser {
+
+// Called by `n_workers` threads with ranks worker = 0 .. n_workers - 1; img has M * 3 * (d/16)^2 * 32 entries.
+__device__ __forceinline__ void gsta_build_images(const __nv_bfloat16* Wg, uint4* img, int d, int M, int worker,
+                                                  int n_workers) {
+  const int D16 = d >> 4;
+  const int total = M * 3 * D16 * D16 * 32;
+  for (int i = worker; i < total; i += n_workers) {
+    const int lane = i & 31;
+    int r = i >> 5;
+    const int p = r % D16; r /= D16;
+    const int kt = r % D16; r /= D16;
+    const int m = r % 3;
+    const int l = r / 3;
+    const uint16_t* W = reinterpret_cast<const uint16_t*>(Wg) + (size_t)(l * 3 + m) * d * d;
+    const int g = lane >> 2, t = lane & 3;
+    uint32_t v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int n = (2 * p + (q >> 1)) * 8 + g;
+      const int k = kt * 16 + 2 * t + (q & 1) * 8;
+      uint32_t lo, hi;
+      if (m == 1) { lo = W[(size_t)n * d + k]; hi = W[(size_t)n * d + k + 1]; }
+      else { lo = W[(size_t)k * d + n]; hi = W[(size_t)(k + 1) * d + n]; }
+      v[q] = lo | (hi << 16);
+    }
+    img[i] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+}  // namespace laser
