@@ -96,6 +96,29 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 
 __device__ __forceinline__ void report_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// Programmatic dependent launch.  Kernels launched with launch_chained may start (block scheduling, shared-memory and
+// barrier set-up) while the previous kernel of the stream is still running; chain_wait() blocks until that kernel
+// has completed and its writes are visible, and must precede every access to global memory.  chain_release() lets the
+// next chained kernel of the stream start launching once every block of this grid has called it (or exited).
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args... args) {
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 #define LASER_CUDA_OK(expr)                          \
   do {                                               \
     cudaError_t _e = (expr);                         \

@@ -42,6 +42,8 @@ struct GstaParams {
 };
 
 __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
+  chain_wait();
+  chain_release();
   gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
 }
 
@@ -61,6 +63,8 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int c_base = blockIdx.x * kGT;
+  chain_wait();
+  chain_release();
 
   // ---- set-up: candidate -> user -> number of non-empty segments; T = candidates; zero row
   if (tid < kGT) {
@@ -327,7 +331,7 @@ int launch_gsta(const GstaParams& P, cudaStream_t st) {
                       (size_t)kGW * 2 * kChunk * RS;
   LASER_CUDA_OK(cudaFuncSetAttribute(gsta_mma_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   LaunchScope ls("gsta_mma", st);
-  gsta_mma_kernel<D16><<<(P.N + kGT - 1) / kGT, kGThreads, smem, st>>>(P);
+  LASER_CUDA_OK(launch_chained(gsta_mma_kernel<D16>, dim3((P.N + kGT - 1) / kGT), dim3(kGThreads), smem, st, P));
   return LASER_OK;
 }
 
@@ -356,7 +360,7 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   if (p.M > 0 && !images_ready) {
     const int total = p.M * 3 * (p.d / 16) * (p.d / 16) * 32;
     LaunchScope ls("gsta_prep", st);
-    gsta_prep_kernel<<<(total + 255) / 256, 256, 0, st>>>(P);
+    LASER_CUDA_OK(launch_chained(gsta_prep_kernel, dim3((total + 255) / 256), dim3(256), 0, st, P));
   }
   int rc;
   switch (p.d / 16) {

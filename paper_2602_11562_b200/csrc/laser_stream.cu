@@ -63,6 +63,8 @@ __device__ __forceinline__ int user_candidate(const StreamParams& P, int u, int*
 __global__ void __launch_bounds__(256) stream_pre_kernel(StreamParams P, int user_blocks) {
   const int tid = threadIdx.x;
   const int d = P.d, dqk = P.dqk, H = P.H, dqh = dqk / H;
+  chain_wait();
+  chain_release();
   if ((int)blockIdx.x >= user_blocks) {
     // W_v image: entry (kt, p, lane) = {b0, b1 of column tile 2p, b0, b1 of column tile 2p+1}, B[k][n] = W_v[k][n]
     const int D16 = d >> 4, total = D16 * D16 * 32;
@@ -139,6 +141,8 @@ __global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
   const int H = P.H, dvh = d / H;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int u = blockIdx.x;
+  chain_wait();
+  chain_release();
   int len = 0;
   const int cand = user_candidate(P, u, &len);
   if (cand < 0) return;
@@ -323,7 +327,7 @@ int launch_stream(const StreamParams& P, cudaStream_t st) {
   const size_t smem = stream_smem_bytes(P.d, P.H, P.Lp);
   LASER_CUDA_OK(cudaFuncSetAttribute(stream_sta_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   LaunchScope ls("stream_sta", st);
-  stream_sta_kernel<D16><<<P.U, kSThreads, smem, st>>>(P);
+  LASER_CUDA_OK(launch_chained(stream_sta_kernel<D16>, dim3(P.U), dim3(kSThreads), smem, st, P));
   return LASER_OK;
 }
 
@@ -365,7 +369,7 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(stream_pre_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("stream_pre", st);
-    stream_pre_kernel<<<user_blocks + 8, 256, smem, st>>>(P, user_blocks);
+    LASER_CUDA_OK(launch_chained(stream_pre_kernel, dim3(user_blocks + 8), dim3(256), smem, st, P, user_blocks));
   }
   int rc;
   switch (p.d / 16) {

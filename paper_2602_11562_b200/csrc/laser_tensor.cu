@@ -86,6 +86,8 @@ __device__ __forceinline__ int canon_off(int row, int k, int kdim) {
 // ------------------------------------------------------------------------------------------------------- prep
 __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
   const int tid = threadIdx.x;
+  chain_wait();
+  chain_release();
   if (blockIdx.x == 0) {
     __shared__ int sa[1024], sb[1024], sc[1024];
     const int per = (P.U + 1023) / 1024;
@@ -185,6 +187,8 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
 // H' rows of segments without valid items are zero rows (only needed when the caller wants H').
 __global__ void __launch_bounds__(256) tc_zero_empty_kernel(TcParams P) {
   const int u = blockIdx.y, seg = blockIdx.x;
+  chain_wait();
+  chain_release();
   const UserShape s = user_shape(P, u);
   if (seg < s.nseg || s.nc == 0) return;
   const int vec = P.d / 8;   // 16-byte chunks per row
@@ -240,6 +244,8 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
   const uint32_t bK = dqk * d * 2, bV = kCandTile * d * 2;
+  chain_wait();                         // the set-up kernel's images, prefixes and start cursors are complete
+  chain_release();
 
   if (tid == 0) {
     mbar_arrive_expect_tx(&bar_img, bK + bV);
@@ -588,6 +594,8 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
   const int n_obuf = P.n_obuf;
+  chain_wait();                         // K, V^T and Q tiles are complete
+  chain_release();
 
   // this block's contiguous range of units
   const int n_units = P.counters[0];
@@ -937,17 +945,17 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   const int sms = sm_count();
   {
     LaunchScope ls("tc_prep", st);
-    tc_prep_kernel<<<1 + 32, 1024, 0, st>>>(P);
+    LASER_CUDA_OK(launch_chained(tc_prep_kernel, dim3(1 + 32), dim3(1024), 0, st, P));
   }
   {
     const size_t smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;   // W_k^T | W_q^T, W_v^T, two staging buffers
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("tc_proj", st);
-    tc_proj_kernel<<<P.proj_grid, kProjThreads, smem, st>>>(P);
+    LASER_CUDA_OK(launch_chained(tc_proj_kernel, dim3(P.proj_grid), dim3(kProjThreads), smem, st, P));
   }
   if (user_wants_hp) {
     LaunchScope ls("tc_zero_empty", st);
-    tc_zero_empty_kernel<<<dim3(p.Lp, p.U), 256, 0, st>>>(P);
+    LASER_CUDA_OK(launch_chained(tc_zero_empty_kernel, dim3(p.Lp, p.U), dim3(256), 0, st, P));
   }
   {
     const size_t smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * P.IT * (p.dqk + p.d) * 2 +
@@ -955,7 +963,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     if (smem > 220 * 1024) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_sta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("sta_tc", st);
-    tc_sta_kernel<<<P.sta_grid, kStaThreads, smem, st>>>(P);
+    LASER_CUDA_OK(launch_chained(tc_sta_kernel, dim3(P.sta_grid), dim3(kStaThreads), smem, st, P));
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
