@@ -191,6 +191,10 @@ def run_reference(args, rank, world):
 # captures summarised under profiles/, keyed by (kernel, workload).  Each entry names the source file of the kernel and
 # the first 12 hex digits of its SHA-256 at capture time: once that file changes, the figure is reported as null.
 NCU_TRAFFIC = {
+    ("sta_tc", "cfg3_batched_bf16"): (111019264, "401bf09fded9"),
+    ("tc_proj", "cfg3_batched_bf16"): (55929600, "401bf09fded9"),
+    ("gsta_mma", "cfg3_batched_bf16"): (88523520, "b4a80c699bc8"),
+    ("stream_sta", "cfg5_onecand_bf16"): (622504192, "25f6657e89fc"),
 }
 KERNEL_SOURCE = {"sta_tc": "laser_tensor.cu", "tc_proj": "laser_tensor.cu", "gsta_mma": "laser_gsta.cu",
                  "stream_sta": "laser_stream.cu"}

@@ -917,6 +917,11 @@ bool tensor_supported(const Plan& p) {
   if (p.dvh % 16) return false;
   TensorGeom g;
   tensor_geometry(p, &g);
+  // shared memory of the attention kernel (Q double buffer, K / V^T ring, staged output) and of the projection kernel
+  const size_t sta_smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * g.IT * (p.dqk + p.d) * 2 +
+                          (size_t)2 * kCandTile * (p.d * 2 + 16);
+  const size_t proj_smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;
+  if (sta_smem > 220 * 1024 || proj_smem > 220 * 1024) return false;
   if ((long long)p.U * g.n_tiles >= (1ll << 30)) return false;
   if ((long long)p.U * p.Lp * 4 >= (1ll << 30)) return false;
   return true;

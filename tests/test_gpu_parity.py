@@ -70,6 +70,7 @@ TENSOR = [
     dict(U=5, C=1, L=300, d=32, H=2, S=10, M=1, d_qh=16, lengths=[300, 9, 10, 11, 0]),   # S = 10, one candidate
     dict(U=2, C=40, L=520, d=64, H=2, S=260, M=1, d_qh=32, lengths=[520, 300]),          # S > 128, d_qh = 32
     dict(U=1, C=16, L=48, d=16, H=1, S=48, M=1, d_qh=16, lengths=[40]),                  # smallest widths, S = L
+    dict(U=2, C=70, L=160, d=96, H=3, S=40, M=1, d_qh=16, lengths=[160, 41]),            # three heads of width 32
 ]
 
 
@@ -77,6 +78,28 @@ TENSOR = [
 def test_small_shapes_tensor_path(case):
     w = make_custom(dtype="bf16", seed=200 + case, **TENSOR[case])
     check_against_oracle(w, "tensor")
+
+
+def test_tensor_path_many_users_few_candidates():
+    """More users than the set-up kernel has threads (several users per scan chunk), uneven candidate counts."""
+    U = 2500
+    w = make_custom(U=U, C=2, L=48, d=32, H=2, S=16, M=1, dtype="bf16", seed=77)
+    rng = np.random.default_rng(5)
+    counts = rng.integers(0, 4, size=U)                     # 0..3 candidates per user
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    w.cand_offsets = offs
+    w.cands = np.ascontiguousarray(np.resize(w.cands, (int(offs[-1]), 32)))
+    check_against_oracle(w, "tensor")
+
+
+def test_auto_path_falls_back_when_the_tensor_kernels_do_not_fit():
+    """d = 128 with d_qk = 128 needs more shared memory than the attention kernel has: AUTO must pick another path."""
+    w = make_custom(U=1, C=20, L=64, d=128, H=8, S=32, M=1, dtype="bf16", seed=78, d_qh=16, lengths=[50])
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
+    if P.laser_workspace_bytes(b.cfg) == 0:                 # explicit TENSOR request is refused at plan time
+        check_against_oracle(w, "auto")
+    else:
+        check_against_oracle(w, "tensor")
 
 
 def test_tensor_path_padding_rows_and_determinism():
