@@ -10,7 +10,9 @@
 // so the item loop only needs the 2 H dot products x_n . u_h and the 2 H d multiply-adds of r += g x per row
 // (Eq. 10-12), and W_v is applied once per segment afterwards.
 //
-//   stream_pre_kernel    u [U, H, d] (fp32) for every user, and the fragment-ordered image of W_v
+//   stream_pre_kernel    u [U, H, d] (fp32) for every user (one warp per 16 users, two small warp-level MMA products
+//                        with the intermediate query split into bf16 high and low parts), and the fragment-ordered
+//                        image of W_v (spare warps)
 //   stream_sta_kernel    one block per user; every warp owns whole segments, streams their rows through a private
 //                        cp.async ring (16 rows per stage, 128-bit copies, padded rows) and feeds them twice to
 //                        warp-level MMAs: scores = U X^T (rows = heads), then R += G X.  u, the gates and r are
@@ -32,7 +34,7 @@ constexpr int kSW = 4;            // warps per block
 constexpr int kSThreads = kSW * 32;
 constexpr int kSRows = 16;        // item rows per stage (one MMA k / n step)
 constexpr int kSStages = 4;       // ring depth per warp
-constexpr int kPreUsers = 16;     // users per block of the pre kernel
+constexpr int kPreWarps = 4;      // warps per block of the pre kernel; a warp folds 16 users
 
 struct StreamParams {
   int U, L, d, dqk, H, S, Lp, N;
@@ -60,67 +62,88 @@ __device__ __forceinline__ int user_candidate(const StreamParams& P, int u, int*
   return c1 > c0 ? c0 : -1;
 }
 
-__global__ void __launch_bounds__(256) stream_pre_kernel(StreamParams P, int user_blocks) {
-  const int tid = threadIdx.x;
-  const int d = P.d, dqk = P.dqk, H = P.H, dqh = dqk / H;
+template <int D16>
+__global__ void __launch_bounds__(kPreWarps * 32) stream_pre_kernel(StreamParams P, int user_warps) {
+  constexpr int d = D16 * 16;
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int wg = blockIdx.x * kPreWarps + (threadIdx.x >> 5);
+  const int dqk = P.dqk, H = P.H, dqh = dqk / H;
   chain_wait();
   chain_release();
-  if ((int)blockIdx.x >= user_blocks) {
-    // W_v image: entry (kt, p, lane) = {b0, b1 of column tile 2p, b0, b1 of column tile 2p+1}, B[k][n] = W_v[k][n]
-    const int D16 = d >> 4, total = D16 * D16 * 32;
+  if (wg >= user_warps) {
+    // spare warps: W_v image, entry (kt, p, lane) = {b0, b1 of column tile 2p, b0, b1 of column tile 2p+1},
+    // B[k][n] = W_v[k][n]; and the GSTA weight images when GSTA follows
+    const int worker = (wg - user_warps) * 32 + lane, n_workers = (gridDim.x * kPreWarps - user_warps) * 32;
+    const int total = D16 * D16 * 32;
     const uint16_t* W = reinterpret_cast<const uint16_t*>(P.Wv);
-    for (int i = (blockIdx.x - user_blocks) * blockDim.x + tid; i < total; i += (gridDim.x - user_blocks) * blockDim.x) {
-      const int lane = i & 31, p = (i >> 5) % D16, kt = (i >> 5) / D16;
-      const int g = lane >> 2, t = lane & 3;
+    for (int i = worker; i < total; i += n_workers) {
+      const int ln = i & 31, p = (i >> 5) % D16, kt = (i >> 5) / D16;
+      const int gg = ln >> 2, tt = ln & 3;
       uint32_t v[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int n = (2 * p + (q >> 1)) * 8 + g, k = kt * 16 + 2 * t + (q & 1) * 8;
+        const int n = (2 * p + (q >> 1)) * 8 + gg, k = kt * 16 + 2 * tt + (q & 1) * 8;
         v[q] = (uint32_t)W[(size_t)k * d + n] | ((uint32_t)W[(size_t)(k + 1) * d + n] << 16);
       }
       P.imgv[i] = make_uint4(v[0], v[1], v[2], v[3]);
     }
-    if (P.Wg)
-      gsta_build_images(P.Wg, P.gimg, d, P.M, (blockIdx.x - user_blocks) * blockDim.x + tid,
-                        (gridDim.x - user_blocks) * blockDim.x);
+    if (P.Wg) gsta_build_images(P.Wg, P.gimg, d, P.M, worker, n_workers);
     return;
   }
-  // shared: W_q [d][dqk+1], W_k [d][dqk+1] (fp32, padded rows), t [kPreUsers][d], q [kPreUsers][dqk]
-  extern __shared__ float sm[];
-  const int wld = dqk + 1;
-  float* wq = sm;
-  float* wk = wq + d * wld;
-  float* ts = wk + d * wld;
-  float* qs = ts + kPreUsers * d;
-  __shared__ int cand_s[kPreUsers];
-  const int u0 = blockIdx.x * kPreUsers;
-  if (tid < kPreUsers) {
-    int len = 0;
-    cand_s[tid] = u0 + tid < P.U ? user_candidate(P, u0 + tid, &len) : -1;
+  // users 16 wg + g (MMA rows g) and 16 wg + g + 8 (rows g + 8); a user without a candidate is a zero row
+  const int uA = wg * 16 + g, uB = uA + 8;
+  int len = 0;
+  const int cA = uA < P.U ? user_candidate(P, uA, &len) : -1;
+  const int cB = uB < P.U ? user_candidate(P, uB, &len) : -1;
+  uint32_t ta[D16][4];                                   // A fragments of T (bf16, exact)
+#pragma unroll
+  for (int kt = 0; kt < D16; ++kt) {
+    const int k = kt * 16 + 2 * t;
+    ta[kt][0] = cA >= 0 ? *reinterpret_cast<const uint32_t*>(P.cands + (size_t)cA * d + k) : 0u;
+    ta[kt][1] = cB >= 0 ? *reinterpret_cast<const uint32_t*>(P.cands + (size_t)cB * d + k) : 0u;
+    ta[kt][2] = cA >= 0 ? *reinterpret_cast<const uint32_t*>(P.cands + (size_t)cA * d + k + 8) : 0u;
+    ta[kt][3] = cB >= 0 ? *reinterpret_cast<const uint32_t*>(P.cands + (size_t)cB * d + k + 8) : 0u;
   }
-  for (int i = tid; i < d * dqk; i += blockDim.x) {
-    const int r = i / dqk, c = i - r * dqk;
-    wq[r * wld + c] = __bfloat162float(P.Wq[i]);
-    wk[r * wld + c] = __bfloat162float(P.Wk[i]);
-  }
-  __syncthreads();
-  for (int i = tid; i < kPreUsers * d; i += blockDim.x) {
-    const int uu = i / d, c = cand_s[uu];
-    ts[i] = c >= 0 ? __bfloat162float(P.cands[(size_t)c * d + (i - uu * d)]) : 0.f;
-  }
-  __syncthreads();
-  for (int o = tid; o < kPreUsers * dqk; o += blockDim.x) {      // q = t W_q / gamma   (Eq. 4 / Eq. 8)
-    const int uu = o / dqk, a = o - uu * dqk;
-    float acc = 0.f;
-    for (int i = 0; i < d; ++i) acc = fmaf(ts[uu * d + i], wq[i * wld + a], acc);
-    qs[o] = acc * P.inv_gamma;
-  }
-  __syncthreads();
-  for (int o = tid; o < kPreUsers * H * d; o += blockDim.x) {    // u_h[i] = sum_{a in head h} W_k[i][a] q[a]
-    const int uu = o / (H * d), h = (o / d) % H, i = o % d;
-    float acc = 0.f;
-    for (int a = h * dqh; a < (h + 1) * dqh; ++a) acc = fmaf(wk[i * wld + a], qs[uu * dqk + a], acc);
-    if (u0 + uu < P.U) P.u[(size_t)(u0 + uu) * H * d + (o - uu * H * d)] = acc;
+  const uint16_t* Wq = reinterpret_cast<const uint16_t*>(P.Wq);
+  for (int h = 0; h < H; ++h) {
+    float uacc[2 * D16][4];                              // u_h of the 16 users: (user g | g + 8, features 8 nt + 2t..)
+#pragma unroll
+    for (int nt = 0; nt < 2 * D16; ++nt) uacc[nt][0] = uacc[nt][1] = uacc[nt][2] = uacc[nt][3] = 0.f;
+    for (int a0 = h * dqh; a0 < (h + 1) * dqh; a0 += 16) {
+      // 16 columns of q = t W_q / gamma   (Eq. 4 / Eq. 8)
+      float qc[2][4] = {};
+#pragma unroll
+      for (int kt = 0; kt < D16; ++kt) {
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          const uint16_t* w = Wq + (size_t)(kt * 16 + 2 * t) * dqk + a0 + nt * 8 + g;
+          const uint32_t b0 = (uint32_t)w[0] | ((uint32_t)w[dqk] << 16);
+          const uint32_t b1 = (uint32_t)w[8 * dqk] | ((uint32_t)w[9 * dqk] << 16);
+          mma16816(qc[nt], ta[kt][0], ta[kt][1], ta[kt][2], ta[kt][3], b0, b1);
+        }
+      }
+      // the accumulator layout of two 8-column tiles is the A layout of one 16-wide k-tile; high and low bf16 parts
+      uint32_t qh[4], ql[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const float x0 = qc[r >> 1][(r & 1) * 2] * P.inv_gamma, x1 = qc[r >> 1][(r & 1) * 2 + 1] * P.inv_gamma;
+        qh[r] = pack2(x0, x1);
+        ql[r] = pack2(x0 - bf16_lo(qh[r]), x1 - bf16_hi(qh[r]));
+      }
+      // u_h[i] += sum_{a in this chunk} W_k[i][a] q[a]: B[k = a][n = i] = W_k[i][a0 + k]
+#pragma unroll
+      for (int nt = 0; nt < 2 * D16; ++nt) {
+        const bf16* w = P.Wk + (size_t)(nt * 8 + g) * dqk + a0 + 2 * t;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(w), b1 = *reinterpret_cast<const uint32_t*>(w + 8);
+        mma16816(uacc[nt], qh[0], qh[1], qh[2], qh[3], b0, b1);
+        mma16816(uacc[nt], ql[0], ql[1], ql[2], ql[3], b0, b1);
+      }
+    }
+#pragma unroll
+    for (int nt = 0; nt < 2 * D16; ++nt) {
+      if (uA < P.U) *reinterpret_cast<float2*>(P.u + ((size_t)uA * H + h) * d + nt * 8 + 2 * t) = make_float2(uacc[nt][0], uacc[nt][1]);
+      if (uB < P.U) *reinterpret_cast<float2*>(P.u + ((size_t)uB * H + h) * d + nt * 8 + 2 * t) = make_float2(uacc[nt][2], uacc[nt][3]);
+    }
   }
 }
 
@@ -337,6 +360,7 @@ bool stream_supported(const Plan& p) {
   if (p.dtype != LASER_BF16 || p.maxC > 1) return false;
   if (p.d % 16 || p.d < 16 || p.d > 128) return false;
   if (p.H > 8 || p.dvh % 16) return false;
+  if (p.dqh % 16) return false;                    // the query fold works on 16-column chunks of a head
   if (!gsta_mma_supported(p)) return false;
   return stream_smem_bytes(p.d, p.H, p.Lp) <= 200 * 1024;
 }
@@ -364,12 +388,22 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   P.zero_empty = Hprime != (void*)(ws + p.off_hp);
   P.status = reinterpret_cast<int*>(ws + p.off_status);
   {
-    const int user_blocks = (p.U + kPreUsers - 1) / kPreUsers;
-    const size_t smem = ((size_t)2 * p.d * (p.dqk + 1) + (size_t)kPreUsers * (p.d + p.dqk)) * sizeof(float);
-    if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
-    LASER_CUDA_OK(cudaFuncSetAttribute(stream_pre_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int user_warps = (p.U + 15) / 16;
+    const dim3 grid((user_warps + kPreWarps - 1) / kPreWarps + 2), block(kPreWarps * 32);
     LaunchScope ls("stream_pre", st);
-    LASER_CUDA_OK(launch_chained(stream_pre_kernel, dim3(user_blocks + 8), dim3(256), smem, st, P, user_blocks));
+    cudaError_t e;
+    switch (p.d / 16) {
+      case 1: e = launch_chained(stream_pre_kernel<1>, grid, block, 0, st, P, user_warps); break;
+      case 2: e = launch_chained(stream_pre_kernel<2>, grid, block, 0, st, P, user_warps); break;
+      case 3: e = launch_chained(stream_pre_kernel<3>, grid, block, 0, st, P, user_warps); break;
+      case 4: e = launch_chained(stream_pre_kernel<4>, grid, block, 0, st, P, user_warps); break;
+      case 5: e = launch_chained(stream_pre_kernel<5>, grid, block, 0, st, P, user_warps); break;
+      case 6: e = launch_chained(stream_pre_kernel<6>, grid, block, 0, st, P, user_warps); break;
+      case 7: e = launch_chained(stream_pre_kernel<7>, grid, block, 0, st, P, user_warps); break;
+      case 8: e = launch_chained(stream_pre_kernel<8>, grid, block, 0, st, P, user_warps); break;
+      default: return LASER_ERR_UNSUPPORTED;
+    }
+    LASER_CUDA_OK(e);
   }
   int rc;
   switch (p.d / 16) {
