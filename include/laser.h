@@ -125,6 +125,21 @@ LASER_API int laser_forward(const laser_config* cfg, const void* items, const in
                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
                   void* Hprime, void* z, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Multi-resolution feature fusion (section "Multi-resolution Feature Fusion"): per candidate the concatenation
+ *   fused = [ z | max over the non-empty segments j of s_j (element-wise) | s_0 | ... | s_{r-1} ]     in R^{(2 + r) d}
+ * of the GSTA output, the max-pooled compact sequence and the r most recent segment vectors.  Segment 0 holds the most
+ * recent items; empty segments take no part in the max (a user without segments gets zeros there), and a recent slot
+ * j beyond the user's non-empty segments (or beyond L') is a zero vector.
+ *   Hprime      [N, L', d]        segment vectors (rows of empty segments are not read)
+ *   z           [N, d]            GSTA output
+ *   num_recent  r >= 0
+ *   fused       [N, (2 + r) * d]  OUT
+ *   workspace   at least 256 bytes, 256-byte aligned: only the status word at its start is used
+ * Works for either dtype and any path; d * sizeof(element) must be a multiple of 16. */
+LASER_API int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void* z, const int32_t* lengths,
+                                   const int32_t* cand_offsets, int32_t num_recent, void* fused, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream);
+
 /* STA without any workspace argument, for callers that cannot allocate device memory (no counterpart in the
  * paper: this is a deployment convenience of this library).  Think of a plug-in inside a serving process
  * whose GPU memory belongs entirely to the host framework's pool, or of a request thread that must never hit

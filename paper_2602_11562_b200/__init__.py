@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     laser_sta_forward,
     laser_sta_forward_static,
     laser_gsta_forward,
+    laser_fusion_forward,
     laser_forward,
     laser_forward_host,
     laser_check_status,

@@ -71,6 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.laser_forward_host.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.c_int]
     lib.laser_sta_forward_static.restype = ctypes.c_int
     lib.laser_sta_forward_static.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp]
+    lib.laser_fusion_forward.restype = ctypes.c_int
+    lib.laser_fusion_forward.argtypes = [cfgp, vp, vp, i32p, i32p, ctypes.c_int32, vp, vp, sz, vp]
     lib.laser_check_status.restype = ctypes.c_int
     lib.laser_check_status.argtypes = [vp, vp]
     lib.laser_last_launch_count.restype = ctypes.c_int
@@ -208,6 +210,21 @@ def laser_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, H
                            ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     _check(rc, "laser_forward")
     return (Hprime, z) if Hprime is not None else z
+
+
+def laser_fusion_forward(cfg, Hprime, z, lengths, cand_offsets, num_recent, fused=None, workspace=None, stream=None):
+    """Multi-resolution fusion: returns fused [N, (2 + num_recent) * d] = [z | max-pooled H' | most recent segments]."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=Hprime.device)
+    if fused is None:
+        fused = torch.empty((cfg.total_cands, (2 + num_recent) * cfg.d_model), dtype=dt, device=Hprime.device)
+    rc = lib.laser_fusion_forward(ctypes.byref(cfg), _dev(Hprime, dt, "Hprime"), _dev(z, dt, "z"),
+                                  _dev(lengths, torch.int32, "lengths"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                                  int(num_recent), _dev(fused, dt, "fused"), workspace.data_ptr(), workspace.numel(),
+                                  _stream_ptr(stream))
+    _check(rc, "laser_fusion_forward")
+    return fused
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> int:

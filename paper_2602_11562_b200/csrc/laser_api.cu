@@ -216,6 +216,24 @@ int laser_forward(const laser_config* cfg, const void* items, const int32_t* len
                       static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
 }
 
+int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void* z, const int32_t* lengths,
+                         const int32_t* cand_offsets, int32_t num_recent, void* fused, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (num_recent < 0) return LASER_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
+  if (workspace_bytes < kAlign) return LASER_ERR_WORKSPACE;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({Hprime, z, fused})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  return fusion_forward(p, Hprime, z, lengths, cand_offsets, num_recent, fused, ws, st);
+}
+
 namespace {
 struct HostStage {
   size_t items, lengths, cands, offs, wq, wk, wv, wg, z, total;

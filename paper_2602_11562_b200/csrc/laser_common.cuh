@@ -85,6 +85,10 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
                const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
                const void* Wg_images);
 
+// Multi-resolution feature fusion (laser_fusion.cu); uses only the status word of the workspace.
+int fusion_forward(const Plan& p, const void* Hprime, const void* z, const int32_t* lengths, const int32_t* cand_offsets,
+                   int num_recent, void* fused, char* ws, cudaStream_t st);
+
 // --- device helpers ---------------------------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
