@@ -7,7 +7,7 @@ synthetic inputs of a named configuration.  Prints ONE JSON line (rank 0).
   value        user x candidate scores per second, whole job, inputs resident in HBM
   e2e          the same metric through laser_forward_host with pinned HOST buffers (H2D + D2H in the timed region)
   roofline     the dominant kernel's algorithmic work / its CUDA-event duration, against the measured peak
-  cpu_baseline the float64 numpy oracle timed on this machine's host cores on a bounded sample of the same workload
+  cpu_baseline the float64 numpy oracle timed on the host cores on a bounded sample of the same workload
 
 --impl reference times the oracle alone (there is no reference implementation to install for this paper).
 With torchrun (N > 1) every rank runs the same configuration on its own batch (seed offset = rank); users are

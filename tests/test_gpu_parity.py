@@ -225,6 +225,17 @@ def test_cfg2_serving_bf16_full_simt():
     check_against_oracle(make_workload("cfg2"), "simt")
 
 
+def test_cfg2_serving_bf16_full_tensor_path():
+    w = make_workload("cfg2")
+    check_against_oracle(w, "auto")
+    b = P.DeviceBatch.from_workload(w)                     # the benchmark's call: no H' output, internal buffer
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    z = P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    _, z_ref = oracle_forward(w)
+    assert err_metric(to_np(z), z_ref) <= TOL["bf16"]
+
+
 def test_uneven_candidate_counts_and_users_without_candidates():
     w = make_custom(U=4, C=4, L=64, d=32, H=2, S=16, M=1, dtype="f32", seed=3, lengths=[64, 10, 0, 33])
     offs = np.array([0, 7, 7, 8, 16], dtype=np.int32)       # 7, 0, 1, 8 candidates
@@ -293,3 +304,10 @@ def test_full_size_configs_sampled_users(name, n_users):
     order = np.argsort(w.lengths)
     users = sorted({int(order[0]), int(order[-1]), *rng.choice(w.spec.U, size=n_users, replace=False).tolist()})
     check_against_oracle(w, "auto", users=users)
+    # the benchmark's call (no H' output: internal buffer, no zero fill of empty segments) must give the same z
+    b = P.DeviceBatch.from_workload(w)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    z = P.laser_forward(b.cfg, *b.args(), b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    _, z_full = run_forward(w, "auto")
+    assert torch.equal(z, z_full)
