@@ -12,6 +12,7 @@ from .configs import (  # noqa: F401
     WorkloadSpec,
     make_workload,
     make_custom,
+    make_ffn_weights,
     round_to_dtype,
     shard_users,
 )

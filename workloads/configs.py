@@ -222,3 +222,19 @@ def shard_users(num_users: int, rank: int, world_size: int) -> range:
     lo = rank * base + min(rank, rem)
     hi = lo + base + (1 if rank < rem else 0)
     return range(lo, hi)
+
+
+def make_ffn_weights(d: int, r: int = 4, dtype: str = "bf16", seed: int = 0) -> dict:
+    """Seeded weights of the feed-forward refinement (Eq. 6): W1 [d, r d], b1 [r d], W2 [r d, d], b2 [d] and the
+    layer norm's gain / shift [d], all rounded to `dtype` and returned as float32 arrays."""
+    rng = np.random.Generator(np.random.PCG64(77_000 + seed))
+    hid = r * d
+    w = {
+        "W1": _xavier_uniform(rng, d, hid, (d, hid)),
+        "b1": (0.05 * rng.standard_normal(hid)).astype(np.float32),
+        "W2": _xavier_uniform(rng, hid, d, (hid, d)),
+        "b2": (0.05 * rng.standard_normal(d)).astype(np.float32),
+        "ln_g": (1.0 + 0.1 * rng.standard_normal(d)).astype(np.float32),
+        "ln_b": (0.1 * rng.standard_normal(d)).astype(np.float32),
+    }
+    return {k: round_to_dtype(v, dtype) for k, v in w.items()}
