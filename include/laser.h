@@ -17,8 +17,8 @@
  * the GSTA weights ([d, d]) into H contiguous slices, head outputs are concatenated, there is no output
  * projection and no bias; an item at or beyond a user's length contributes exactly nothing (whatever the
  * padded rows contain, as long as it is finite); a segment without valid items yields a zero row of H' and
- * takes no part in the GSTA softmax; a user of length 0 yields H' = 0 and z = t.  No FFN / LayerNorm
- * (Eq. 6) sits between the two stages.
+ * takes no part in the GSTA softmax; a user of length 0 yields H' = 0 and z = t.  laser_forward runs the two
+ * stages back to back; laser_forward_ffn puts the FFN / LayerNorm of Eq. 6 between them.
  *
  * General rules for every entry point
  *   - Unless stated otherwise every pointer is a DEVICE pointer to memory owned by the caller; the library
@@ -139,6 +139,44 @@ LASER_API int laser_forward(const laser_config* cfg, const void* items, const in
 LASER_API int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void* z, const int32_t* lengths,
                                    const int32_t* cand_offsets, int32_t num_recent, void* fused, void* workspace,
                                    size_t workspace_bytes, void* cuda_stream);
+
+/* Feed-forward refinement of the segment vectors (Eq. 6):  s_i <- LN(FFN(s_i) + s_i)  for every non-empty segment of
+ * every candidate.  The paper fixes the residual + layer-norm form and the expansion ratio r (d_hidden = r d, r = 4 in
+ * its cost model); this library takes FFN(s) = max(s W1 + b1, 0) W2 + b2 and LN(y) = (y - mean) / sqrt(var + eps) *
+ * gain + shift over the d features (biased variance).  Rows of empty segments are left as they are.
+ * All pointers are DEVICE pointers in the config's dtype, 16-byte aligned, owned by the caller. */
+typedef struct laser_ffn_params {
+  int32_t d_hidden;      /* r * d >= 1 (the tcgen05 kernel needs a multiple of 128; other widths run on the FP32 ALUs) */
+  float ln_eps;          /* <= 0 selects 1e-5                                                                          */
+  const void* W1;        /* [d, d_hidden]                                                                              */
+  const void* b1;        /* [d_hidden]                                                                                 */
+  const void* W2;        /* [d_hidden, d]                                                                              */
+  const void* b2;        /* [d]                                                                                        */
+  const void* ln_gain;   /* [d]                                                                                        */
+  const void* ln_shift;  /* [d]                                                                                        */
+} laser_ffn_params;
+
+/* Bytes of device scratch laser_ffn_forward and laser_forward_ffn need: laser_workspace_bytes(cfg) plus the row
+ * prefix and the weight images of the FFN.  Returns 0 if cfg is NULL / invalid or d_hidden < 1.  Host-only. */
+LASER_API size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hidden);
+
+/* Eq. 6 in place on a caller-supplied H'.
+ *   Hprime  [N, L', d]  IN / OUT: rows of non-empty segments are replaced by LN(FFN(s) + s)
+ *   workspace           at least laser_ffn_workspace_bytes(cfg, ffn->d_hidden) bytes, 256-byte aligned
+ * BF16 with d a multiple of 16 (<= 128) and d_hidden a multiple of 128 runs on the tensor cores (bf16 operands and
+ * hidden activations, fp32 accumulation and normalisation) unless cfg->path is LASER_PATH_SIMT; everything else runs
+ * in fp32 on the ALUs.  LASER_ERR_UNSUPPORTED when neither kernel takes the shape. */
+LASER_API int laser_ffn_forward(const laser_config* cfg, const laser_ffn_params* ffn, void* Hprime,
+                                const int32_t* lengths, const int32_t* cand_offsets, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
+
+/* The paper's full compression stack: STA (Eq. 8-12), then Eq. 6 on every segment vector, then GSTA (Eq. 7).
+ * Arguments as for laser_forward plus `ffn`; Hprime (optional) receives the refined segment vectors.
+ *   workspace  at least laser_ffn_workspace_bytes(cfg, ffn->d_hidden) bytes */
+LASER_API int laser_forward_ffn(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                                const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv,
+                                const void* Wgsta, const laser_ffn_params* ffn, void* Hprime, void* z, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream);
 
 /* STA without any workspace argument, for callers that cannot allocate device memory (no counterpart in the
  * paper: this is a deployment convenience of this library).  Think of a plug-in inside a serving process

@@ -19,6 +19,10 @@ from .binding import (  # noqa: F401
     laser_sta_forward_static,
     laser_gsta_forward,
     laser_fusion_forward,
+    laser_ffn_workspace_bytes,
+    laser_ffn_forward,
+    laser_forward_ffn,
+    LaserFfnParams,
     laser_forward,
     laser_forward_host,
     laser_check_status,

@@ -42,6 +42,15 @@ class LaserConfig(ctypes.Structure):
         return torch.float32 if self.dtype == DTYPE_F32 else torch.bfloat16
 
 
+class LaserFfnParams(ctypes.Structure):
+    """Mirror of `laser_ffn_params` in include/laser.h."""
+    _fields_ = [
+        ("d_hidden", ctypes.c_int32), ("ln_eps", ctypes.c_float),
+        ("W1", ctypes.c_void_p), ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p),
+        ("ln_gain", ctypes.c_void_p), ("ln_shift", ctypes.c_void_p),
+    ]
+
+
 def library_path() -> str:
     return os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblaser.so")
 
@@ -73,6 +82,13 @@ def load_library() -> ctypes.CDLL:
     lib.laser_sta_forward_static.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp]
     lib.laser_fusion_forward.restype = ctypes.c_int
     lib.laser_fusion_forward.argtypes = [cfgp, vp, vp, i32p, i32p, ctypes.c_int32, vp, vp, sz, vp]
+    ffnp = ctypes.POINTER(LaserFfnParams)
+    lib.laser_ffn_workspace_bytes.restype = sz
+    lib.laser_ffn_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
+    lib.laser_ffn_forward.restype = ctypes.c_int
+    lib.laser_ffn_forward.argtypes = [cfgp, ffnp, vp, i32p, i32p, vp, sz, vp]
+    lib.laser_forward_ffn.restype = ctypes.c_int
+    lib.laser_forward_ffn.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, ffnp, vp, vp, vp, sz, vp]
     lib.laser_check_status.restype = ctypes.c_int
     lib.laser_check_status.argtypes = [vp, vp]
     lib.laser_last_launch_count.restype = ctypes.c_int
@@ -225,6 +241,57 @@ def laser_fusion_forward(cfg, Hprime, z, lengths, cand_offsets, num_recent, fuse
                                   _stream_ptr(stream))
     _check(rc, "laser_fusion_forward")
     return fused
+
+
+def laser_ffn_workspace_bytes(cfg: LaserConfig, d_hidden: int) -> int:
+    return int(load_library().laser_ffn_workspace_bytes(ctypes.byref(cfg), int(d_hidden)))
+
+
+def _ffn_params(cfg, ffn: dict, ln_eps: float):
+    """ffn: {"W1" [d, hid], "b1" [hid], "W2" [hid, d], "b2" [d], "ln_g" [d], "ln_b" [d]} device tensors."""
+    dt = cfg.torch_dtype()
+    hid = int(ffn["W1"].shape[1])
+    return LaserFfnParams(hid, float(ln_eps), _dev(ffn["W1"], dt, "W1"), _dev(ffn["b1"], dt, "b1"),
+                          _dev(ffn["W2"], dt, "W2"), _dev(ffn["b2"], dt, "b2"), _dev(ffn["ln_g"], dt, "ln_g"),
+                          _dev(ffn["ln_b"], dt, "ln_b")), hid
+
+
+def _ffn_workspace(cfg, hid, workspace, device):
+    need = laser_ffn_workspace_bytes(cfg, hid)
+    if need == 0:
+        raise LaserError(-1, "laser_ffn_workspace_bytes (invalid or unsupported configuration)")
+    return torch.empty(need, dtype=torch.uint8, device=device) if workspace is None else workspace
+
+
+def laser_ffn_forward(cfg, ffn, Hprime, lengths, cand_offsets, ln_eps=0.0, workspace=None, stream=None):
+    """Eq. 6 in place on H' [N, L', d]: rows of non-empty segments become LN(FFN(s) + s).  Returns Hprime."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    params, hid = _ffn_params(cfg, ffn, ln_eps)
+    ws = _ffn_workspace(cfg, hid, workspace, Hprime.device)
+    rc = lib.laser_ffn_forward(ctypes.byref(cfg), ctypes.byref(params), _dev(Hprime, dt, "Hprime"),
+                               _dev(lengths, torch.int32, "lengths"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                               ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_ffn_forward")
+    return Hprime
+
+
+def laser_forward_ffn(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, ffn, Hprime=None, z=None,
+                      ln_eps=0.0, workspace=None, stream=None, want_hprime=False):
+    """STA, Eq. 6 on every segment vector, GSTA: returns z, or (refined H', z)."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    params, hid = _ffn_params(cfg, ffn, ln_eps)
+    ws = _ffn_workspace(cfg, hid, workspace, items.device)
+    if z is None:
+        z = torch.empty((cfg.total_cands, cfg.d_model), dtype=dt, device=items.device)
+    if Hprime is None and want_hprime:
+        Hprime = torch.empty((cfg.total_cands, cfg.n_seg, cfg.d_model), dtype=dt, device=items.device)
+    rc = lib.laser_forward_ffn(ctypes.byref(cfg), _dev(items, dt, "items"), _dev(lengths, torch.int32, "lengths"),
+                               _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                               _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Wgsta, dt, "Wgsta"),
+                               ctypes.byref(params), None if Hprime is None else _dev(Hprime, dt, "Hprime"),
+                               _dev(z, dt, "z"), ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_forward_ffn")
+    return (Hprime, z) if Hprime is not None else z
 
 
 def _host(t: torch.Tensor, dtype, name: str) -> int:

@@ -234,6 +234,66 @@ int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void
   return fusion_forward(p, Hprime, z, lengths, cand_offsets, num_recent, fused, ws, st);
 }
 
+size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hidden) {
+  Plan p;
+  if (make_plan(cfg, &p) != LASER_OK || d_hidden < 1) return 0;
+  return p.total + ffn_scratch_bytes(p, d_hidden);
+}
+
+static int check_ffn(const Plan& p, const laser_ffn_params* f, const void* workspace, size_t workspace_bytes) {
+  if (!f || f->d_hidden < 1) return LASER_ERR_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
+  if (workspace_bytes < p.total + ffn_scratch_bytes(p, f->d_hidden)) return LASER_ERR_WORKSPACE;
+  if (p.N > 0) {
+    const int rc = check_ptrs({f->W1, f->b1, f->W2, f->b2, f->ln_gain, f->ln_shift});
+    if (rc != LASER_OK) return rc;
+    if (!ffn_supported(p, f->d_hidden)) return LASER_ERR_UNSUPPORTED;
+  }
+  return LASER_OK;
+}
+
+int laser_ffn_forward(const laser_config* cfg, const laser_ffn_params* ffn, void* Hprime, const int32_t* lengths,
+                      const int32_t* cand_offsets, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if ((rc = check_ffn(p, ffn, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({Hprime})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  return ffn_forward(p, ffn, Hprime, lengths, cand_offsets, ws, ws + p.total, st);
+}
+
+int laser_forward_ffn(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                      const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
+                      const laser_ffn_params* ffn, void* Hprime, void* z, void* workspace, size_t workspace_bytes,
+                      void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if ((rc = check_ffn(p, ffn, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({items, cands, Wq, Wk, Wv, z})) != LASER_OK) return rc;
+  if (p.N > 0 && p.M > 0 && (rc = check_ptrs({Wgsta})) != LASER_OK) return rc;
+  if (Hprime && !aligned16(Hprime)) return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  void* Hp = Hprime ? Hprime : (void*)(ws + p.off_hp);
+  const bool side_images = p.M > 0 && p.path != LASER_PATH_SIMT && gsta_mma_supported(p);
+  rc = run_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hp, ws, st, side_images ? Wgsta : nullptr);
+  if (rc != LASER_OK) return rc;
+  rc = ffn_forward(p, ffn, Hp, lengths, cand_offsets, ws, ws + p.total, st);
+  if (rc != LASER_OK) return rc;
+  return run_gsta(p, Hp, lengths, cand_offsets, cands, Wgsta, z, ws, st, side_images);
+}
+
 namespace {
 struct HostStage {
   size_t items, lengths, cands, offs, wq, wk, wv, wg, z, total;

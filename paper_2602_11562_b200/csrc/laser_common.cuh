@@ -89,6 +89,12 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
 int fusion_forward(const Plan& p, const void* Hprime, const void* z, const int32_t* lengths, const int32_t* cand_offsets,
                    int num_recent, void* fused, char* ws, cudaStream_t st);
 
+// Feed-forward refinement of H' (laser_ffn.cu); needs ffn_scratch_bytes(p, d_hidden) of scratch of its own.
+bool ffn_supported(const Plan& p, int hid);
+size_t ffn_scratch_bytes(const Plan& p, int hid);
+int ffn_forward(const Plan& p, const laser_ffn_params* f, void* H, const int32_t* lengths, const int32_t* cand_offsets,
+                char* ws, char* scratch, cudaStream_t st);
+
 // --- device helpers ---------------------------------------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }

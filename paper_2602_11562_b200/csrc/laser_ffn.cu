@@ -1,0 +1,634 @@
+// Feed-forward refinement of the segment vectors (Eq. 6):  s <- LN(max(s W_1 + b_1, 0) W_2 + b_2 + s), applied in place
+// to the rows of H' that belong to non-empty segments.
+//
+//   ffn_prep_kernel   prefix of the valid rows per user (the "compact" row numbering the main kernel tiles over) and the
+//                     weights re-laid as MMA operand images, one 128-hidden-unit chunk after the other.
+//   ffn_tc_kernel     bf16, tcgen05: a persistent block owns pairs of 128-row tiles.  Per pair and per chunk j of 128
+//                     hidden units:   acc1 = X W_1[:, j]  (TMEM)  ->  registers: + b_1, ReLU, bf16  ->  shared memory
+//                     ->  acc2 += hidden_j W_2[j, :]  (TMEM).  The hidden activations never leave the SM; the weights
+//                     stream through a three-slot ring of bulk copies (from L2) and are shared by both tiles of the pair.
+//                     The last step adds b_2 and the residual, normalises each row (one thread owns one row of the
+//                     accumulator) and writes bf16.
+//   ffn_simt_kernel   FP32-ALU version for fp32 data and for shapes outside the tensor kernel's envelope.
+#include "laser_common.cuh"
+#include "laser_ptx.cuh"
+
+namespace laser {
+namespace {
+
+using bf16 = __nv_bfloat16;
+using namespace ptx;
+
+constexpr int kRows = 128;            // rows per tile = MMA M = TMEM lanes
+constexpr int kChunk = 128;           // hidden units per step
+constexpr int kPairRows = 2 * kRows;  // two tiles share every weight chunk
+constexpr int kFfnThreads = 384;      // warp 0 weight producer + TMEM, warp 1 MMA issuer, warps 2-3 row staging,
+                                      // warps 4-7 / 8-11 epilogue warpgroups of tile 0 / tile 1
+constexpr int kWStages = 3;
+constexpr int kFfnTmemCols = 512;     // acc2[t] at 128 t, acc1[t] at 256 + 128 t
+constexpr int kSimtRows = 8;
+
+struct FfnParams {
+  int U, N, L, Lp, S, d, hid, NJ, maxC;
+  float eps;
+  bf16* H;                                    // [N, Lp, d] in / out
+  const bf16 *W1, *b1, *W2, *b2, *g, *beta;
+  const int *lengths, *cand_offsets;
+  int* prefix;                                // [U + 1] valid rows before each user
+  int* counters;                              // [0] total valid rows
+  bf16 *img1, *img2;                          // chunk j of W_1^T / W_2^T at + j * 128 * d
+  int* status;
+};
+
+struct RowUser {
+  int c0, nc, nseg;
+};
+// Sanitised view of one user (an invalid length / offset pair behaves like an empty user).
+template <typename PT>
+__device__ __forceinline__ RowUser row_user(const PT& P, int u) {
+  const int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
+  const bool bad = len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+  RowUser s;
+  s.c0 = bad ? 0 : c0;
+  s.nc = bad ? 0 : c1 - c0;
+  s.nseg = bad ? 0 : (len + P.S - 1) / P.S;
+  return s;
+}
+// Compact row -> row of H' (candidate * Lp + segment); compact rows enumerate, user by user and candidate by candidate,
+// the segments that hold items.  -1 past the end.
+template <typename PT>
+__device__ __forceinline__ int global_row(const PT& P, int crow, int total) {
+  if (crow >= total) return -1;
+  int lo = 0, hi = P.U - 1;                   // largest u with prefix[u] <= crow
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (P.prefix[mid] <= crow) lo = mid; else hi = mid - 1;
+  }
+  const RowUser s = row_user(P, lo);
+  const int local = crow - P.prefix[lo];
+  if (s.nseg <= 0 || local >= s.nc * s.nseg) return -1;
+  const int c = local / s.nseg;
+  return (s.c0 + c) * P.Lp + (local - c * s.nseg);
+}
+
+__device__ __forceinline__ int canon_off(int row, int k, int kdim) {   // K-major 8x8 core matrices, no swizzle
+  return ((row >> 3) * (kdim >> 3) + (k >> 3)) * 64 + (row & 7) * 8 + (k & 7);
+}
+
+// ------------------------------------------------------------------------------------------------------- set-up
+template <typename PT>
+__device__ void scan_rows(const PT& P, int* status) {
+  __shared__ int sa[1024];
+  const int tid = threadIdx.x;
+  const int per = (P.U + 1023) / 1024;
+  const int u0 = min(tid * per, P.U), u1 = min(u0 + per, P.U);
+  int a = 0;
+  bool bad = false;
+  for (int u = u0; u < u1; ++u) {
+    const int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
+    bad |= len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+    const RowUser s = row_user(P, u);
+    a += s.nc * s.nseg;
+  }
+  if (bad) report_status(status, LASER_ERR_BAD_INPUT);
+  sa[tid] = a;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {
+    const int v = tid >= off ? sa[tid - off] : 0;
+    __syncthreads();
+    sa[tid] += v;
+    __syncthreads();
+  }
+  int pa = sa[tid] - a;
+  for (int u = u0; u < u1; ++u) {
+    const RowUser s = row_user(P, u);
+    P.prefix[u] = pa;
+    pa += s.nc * s.nseg;
+  }
+  if (tid == 1023) {
+    P.prefix[P.U] = sa[1023];
+    P.counters[0] = sa[1023];
+  }
+}
+
+__global__ void __launch_bounds__(1024) ffn_prep_kernel(FfnParams P, int build_images) {
+  chain_wait();
+  chain_release();
+  if (blockIdx.x == 0) {
+    scan_rows(P, P.status);
+    return;
+  }
+  if (!build_images) return;
+  const int nthreads = (gridDim.x - 1) * blockDim.x;
+  const int g = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
+  const int n = P.d * P.hid;
+  const int chunk_elems = kChunk * P.d;
+  for (int i = g; i < n; i += nthreads) {          // W_1[k][h]: B operand of step j = h / 128, row h % 128, K index k
+    const int k = i / P.hid, h = i - k * P.hid;
+    P.img1[(h / kChunk) * chunk_elems + canon_off(h % kChunk, k, P.d)] = P.W1[i];
+  }
+  for (int i = g; i < n; i += nthreads) {          // W_2[h][e]: B operand of step j = h / 128, row e, K index h % 128
+    const int h = i / P.d, e = i - h * P.d;
+    P.img2[(h / kChunk) * chunk_elems + canon_off(e, h % kChunk, kChunk)] = P.W2[i];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------- tensor kernel
+// Order of the 2 NJ weight chunks of one tile pair: the first-layer product of chunk j + 1 is issued ahead of the
+// second-layer product of chunk j, so the tensor pipe has work while the epilogue warps turn acc1 into hidden activations.
+__device__ __forceinline__ void ffn_step(int s, int NJ, bool& second, int& j) {
+  if (NJ == 1) { second = s != 0; j = 0; return; }
+  if (s < 2) { second = false; j = s; return; }
+  if (s == 2 * NJ - 1) { second = true; j = NJ - 1; return; }
+  const int q = s - 2;
+  second = !(q & 1);
+  j = second ? q >> 1 : (q >> 1) + 2;
+}
+
+struct FfnBars {
+  uint64_t w_full[kWStages], w_empty[kWStages];
+  uint64_t x_full[2], x_free[2];
+  uint64_t a1_full[2], a1_free[2];
+  uint64_t hs_full[2], hs_free[2];
+  uint64_t a2_full[2], a2_free[2];
+  uint64_t done;
+};
+
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+
+__global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ FfnBars bars;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int d = P.d, NJ = P.NJ;
+  const uint32_t x_bytes = kRows * d * 2, hs_bytes = kRows * kChunk * 2, w_bytes = kChunk * d * 2;
+  uint8_t* Xs = smem_raw;                              // [2][128 x d]       K-major, K = d
+  uint8_t* Hs = Xs + 2 * x_bytes;                      // [2][128 x 128]     K-major, K = 128 hidden units
+  uint8_t* Ws = Hs + 2 * hs_bytes;                     // [kWStages][128 d]  one weight chunk each
+  int* rowmap = reinterpret_cast<int*>(Ws + kWStages * w_bytes);   // [2 tiles][2][128] rows of H' behind the staged tiles
+
+  if (tid == 0) {
+    for (int i = 0; i < kWStages; ++i) { mbar_init(&bars.w_full[i], 1); mbar_init(&bars.w_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars.x_full[i], 1);
+      mbar_init(&bars.x_free[i], 1);
+      mbar_init(&bars.a1_full[i], 1);
+      mbar_init(&bars.a1_free[i], 4);
+      mbar_init(&bars.hs_full[i], 4);
+      mbar_init(&bars.hs_free[i], 1);
+      mbar_init(&bars.a2_full[i], 1);
+      mbar_init(&bars.a2_free[i], 4);
+    }
+    mbar_init(&bars.done, 1);
+    s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&s_tmem, kFfnTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+  chain_wait();                         // H' rows, the row prefix and the weight images are complete
+  chain_release();
+
+  const int total = P.counters[0];
+  const int n_pairs = (total + kPairRows - 1) / kPairRows;
+  const int G = gridDim.x, bidx = blockIdx.x;
+  const int my_pairs = bidx < n_pairs ? (n_pairs - bidx + G - 1) / G : 0;
+  auto wait_all = [&](uint64_t* bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abortp)) != 0;
+  };
+
+  if (my_pairs > 0) {
+    if (warp == 0) {
+      // ------------------------------------------------------------------ weight chunks: L2 -> ring
+      if (lane == 0) {
+        uint32_t use = 0;
+        bool ok = true;
+        for (int it = 0; it < my_pairs && ok; ++it) {
+          for (int s = 0; s < 2 * NJ && ok; ++s, ++use) {
+            bool second;
+            int j;
+            ffn_step(s, NJ, second, j);
+            const uint32_t slot = use % kWStages;
+            ok = mbar_wait(&bars.w_empty[slot], ((use / kWStages) & 1) ^ 1, abortp);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&bars.w_full[slot], w_bytes);
+            bulk_g2s(Ws + slot * w_bytes, (second ? P.img2 : P.img1) + (size_t)j * kChunk * d, w_bytes, &bars.w_full[slot]);
+          }
+        }
+        if (!ok) {                                       // let the copies in flight land before the block goes away
+          const uint32_t first = use > kWStages ? use - kWStages : 0;
+          for (uint32_t k = first; k < use; ++k) {
+            const uint32_t slot = k % kWStages, par = (k / kWStages) & 1;
+            for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&bars.w_full[slot], par); ++i) __nanosleep(64);
+          }
+        }
+      }
+    } else if (warp == 1) {
+      // ------------------------------------------------------------------ MMA issuer (warp-uniform loop, one lane issues)
+      const bool leader = elect_one();
+      const uint32_t x_sbo = (d >> 3) * 128, h_sbo = (kChunk >> 3) * 128;
+      const uint32_t id1 = idesc_bf16(128, kChunk), id2 = idesc_bf16(128, d);
+      const int ks1 = d >> 4, ks2 = kChunk >> 4;
+      uint32_t use = 0;
+      bool ok = true;
+      for (int it = 0; it < my_pairs && ok; ++it) {
+        for (int s = 0; s < 2 * NJ && ok; ++s, ++use) {
+          bool second;
+          int j;
+          ffn_step(s, NJ, second, j);
+          const uint32_t slot = use % kWStages;
+          ok = wait_all(&bars.w_full[slot], (use / kWStages) & 1);
+          if (!ok) break;
+          for (int t = 0; t < 2 && ok; ++t) {
+            if (!second) {
+              if (j == 0) ok = wait_all(&bars.x_full[t], it & 1);
+              const uint32_t k = (uint32_t)it * NJ + j;
+              ok = ok && wait_all(&bars.a1_free[t], (k & 1) ^ 1);
+              if (!ok) break;
+              tc_fence_after();
+              const uint64_t ad = smem_desc(smem_u32(Xs + t * x_bytes), 128, x_sbo);
+              const uint64_t bd = smem_desc(smem_u32(Ws + slot * w_bytes), 128, x_sbo);
+              const uint32_t dcol = tmem + 256 + t * kChunk;
+              if (leader) {
+                for (int ks = 0; ks < ks1; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id1, ks > 0);
+                tc_commit(&bars.a1_full[t]);
+                if (j == NJ - 1) tc_commit(&bars.x_free[t]);
+              }
+            } else {
+              const uint32_t k = (uint32_t)it * NJ + j;
+              ok = wait_all(&bars.hs_full[t], k & 1);
+              if (ok && j == 0) ok = wait_all(&bars.a2_free[t], (it & 1) ^ 1);
+              if (!ok) break;
+              tc_fence_after();
+              const uint64_t ad = smem_desc(smem_u32(Hs + t * hs_bytes), 128, h_sbo);
+              const uint64_t bd = smem_desc(smem_u32(Ws + slot * w_bytes), 128, h_sbo);
+              const uint32_t dcol = tmem + t * 128;
+              if (leader) {
+                for (int ks = 0; ks < ks2; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id2, (j | ks) != 0);
+                tc_commit(&bars.hs_free[t]);
+                if (j == NJ - 1) tc_commit(&bars.a2_full[t]);
+              }
+            }
+            __syncwarp();
+          }
+          if (ok && leader) tc_commit(&bars.w_empty[slot]);
+          __syncwarp();
+        }
+      }
+      if (leader) tc_commit(&bars.done);
+      __syncwarp();
+      wait_all(&bars.done, 0);
+    } else if (warp < 4) {
+      // ------------------------------------------------------------------ row staging: warp 2 + t fills tile t
+      const int t = warp - 2;
+      const int cpr = d >> 3;                              // 16-byte chunks per row
+      const int rin = lane & 7;
+      uint8_t* X = Xs + t * x_bytes;
+      int* maps = rowmap + t * (2 * kRows);                // [2][128] rows of H' behind this warp's tile, two pairs deep
+      auto fill_map = [&](int it) {
+        const int pair = bidx + it * G;
+        int* m = maps + (it & 1) * kRows;
+        for (int r = lane; r < kRows; r += 32)
+          m[r] = it < my_pairs ? global_row(P, pair * kPairRows + t * kRows + r, total) : -1;
+        __syncwarp();
+      };
+      fill_map(0);
+      bool ok = true;
+      for (int it = 0; it < my_pairs && ok; ++it) {
+        const int* m = maps + (it & 1) * kRows;
+        ok = wait_all(&bars.x_free[t], (it & 1) ^ 1);
+        if (!ok) break;
+        for (int idx = lane >> 3; idx < 16 * cpr; idx += 4) {          // idx = (8-row group) * cpr + chunk
+          const int gq = idx / cpr, c = idx - gq * cpr;
+          const int grow = m[gq * 8 + rin];
+          const bf16* src = grow >= 0 ? P.H + (size_t)grow * d + c * 8 : P.H;
+          cp_async16(X + (size_t)idx * 128 + rin * 16, src, grow >= 0 ? 16u : 0u);
+        }
+        cp_async_wait_all();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.x_full[t]);
+        fill_map(it + 1);                                  // the other map: its pair is long staged
+      }
+      cp_async_wait_all();
+    } else {
+      // ------------------------------------------------------------------ epilogue warpgroup of tile t
+      const int t = (warp - 4) >> 2, quad = warp & 3;
+      const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
+      const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+      uint8_t* hs_row = Hs + t * hs_bytes + (r >> 3) * ((kChunk >> 3) * 128) + (r & 7) * 16;
+      const float inv_d = 1.f / (float)d;
+      bool ok = true;
+      for (int it = 0; it < my_pairs && ok; ++it) {
+        const int pair = bidx + it * G;
+        const int grow = global_row(P, pair * kPairRows + t * kRows + r, total);
+        // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> shared memory (A operand of the second layer)
+        for (int j = 0; j < NJ && ok; ++j) {
+          const uint32_t kh = (uint32_t)it * NJ + j;
+          ok = wait_all(&bars.a1_full[t], kh & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tA = tmem + lane_base + 256 + t * kChunk;
+          const uint4* bias = reinterpret_cast<const uint4*>(P.b1 + (size_t)j * kChunk);
+          uint32_t o[kChunk / 2];                          // the whole chunk of my row, packed bf16
+#pragma unroll
+          for (int c = 0; c < kChunk / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tA + c * 32, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 bb = __ldg(bias + c * 4 + q);
+              const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float lo = fmaxf(__uint_as_float(v[q * 8 + 2 * e]) + bf_lo(bw[e]), 0.f);
+                const float hi = fmaxf(__uint_as_float(v[q * 8 + 2 * e + 1]) + bf_hi(bw[e]), 0.f);
+                o[c * 16 + q * 4 + e] = pack_bf16x2(lo, hi);
+              }
+            }
+          }
+          tc_fence_before();                               // the accumulator is in registers: hand it back
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.a1_free[t]);
+          ok = wait_all(&bars.hs_free[t], (kh & 1) ^ 1);   // the previous chunk's second-layer product has read Hs
+          if (!ok) break;
+#pragma unroll
+          for (int k8 = 0; k8 < kChunk / 8; ++k8)
+            *reinterpret_cast<uint4*>(hs_row + k8 * 128) = make_uint4(o[k8 * 4], o[k8 * 4 + 1], o[k8 * 4 + 2], o[k8 * 4 + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.hs_full[t]);
+        }
+        if (!ok) break;
+        // ---- second layer done: y = acc2 + b_2 + s, layer norm over the row, bf16 out
+        ok = wait_all(&bars.a2_full[t], it & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tO = tmem + lane_base + t * 128;
+        const bool live = grow >= 0;
+        bf16* row = P.H + (size_t)(live ? grow : 0) * d;
+        float mean = 0.f, rstd = 0.f;
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+          float acc = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < d; c += 16) {
+            uint32_t v[16];
+            tmem_ld16(tO + c, v);
+            tc_wait_ld();
+            if (pass == 2 && c + 16 >= d) {                // last read of the accumulator
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&bars.a2_free[t]);
+            }
+            if (live) {
+              float y[16];
+#pragma unroll
+              for (int q = 0; q < 2; ++q) {
+                const uint4 xx = *reinterpret_cast<const uint4*>(row + c + q * 8);
+                const uint4 bb = __ldg(reinterpret_cast<const uint4*>(P.b2 + c + q * 8));
+                const uint32_t xw[4] = {xx.x, xx.y, xx.z, xx.w}, bw[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  y[q * 8 + 2 * e] = __uint_as_float(v[q * 8 + 2 * e]) + bf_lo(bw[e]) + bf_lo(xw[e]);
+                  y[q * 8 + 2 * e + 1] = __uint_as_float(v[q * 8 + 2 * e + 1]) + bf_hi(bw[e]) + bf_hi(xw[e]);
+                }
+              }
+              if (pass == 0) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) acc += y[e];
+              } else if (pass == 1) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) acc += (y[e] - mean) * (y[e] - mean);
+              } else {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                  const uint4 gg = __ldg(reinterpret_cast<const uint4*>(P.g + c + q * 8));
+                  const uint4 be = __ldg(reinterpret_cast<const uint4*>(P.beta + c + q * 8));
+                  const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w}, ew[4] = {be.x, be.y, be.z, be.w};
+                  uint32_t o[4];
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float lo = (y[q * 8 + 2 * e] - mean) * rstd * bf_lo(gw[e]) + bf_lo(ew[e]);
+                    const float hi = (y[q * 8 + 2 * e + 1] - mean) * rstd * bf_hi(gw[e]) + bf_hi(ew[e]);
+                    o[e] = pack_bf16x2(lo, hi);
+                  }
+                  *reinterpret_cast<uint4*>(row + c + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+              }
+            }
+          }
+          if (pass == 0) mean = acc * inv_d;
+          if (pass == 1) rstd = rsqrtf(acc * inv_d + P.eps);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, kFfnTmemCols);
+  if (tid == 0 && s_abort) report_status(P.status, LASER_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------------- FP32-ALU kernel
+template <typename T>
+struct FfnSimtParams {
+  int U, N, L, Lp, S, d, hid, maxC;
+  float eps;
+  T* H;
+  const T *W1, *b1, *W2, *b2, *g, *beta;
+  const int *lengths, *cand_offsets;
+  int* prefix;
+  int* counters;
+  int* status;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(1024) ffn_simt_prep_kernel(FfnSimtParams<T> P) {
+  chain_wait();
+  chain_release();
+  scan_rows(P, P.status);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) ffn_simt_kernel(FfnSimtParams<T> P) {
+  extern __shared__ __align__(16) float sm[];
+  const int d = P.d, hid = P.hid, tid = threadIdx.x;
+  float* xs = sm;                      // [8][d]
+  float* ys = xs + kSimtRows * d;      // [8][d]
+  float* hs = ys + kSimtRows * d;      // [8][hid]
+  __shared__ int s_row[kSimtRows];
+  chain_wait();
+  chain_release();
+  const int total = P.counters[0];
+  for (int base = blockIdx.x * kSimtRows; base < total; base += gridDim.x * kSimtRows) {
+    __syncthreads();
+    if (tid < kSimtRows) s_row[tid] = global_row(P, base + tid, total);
+    __syncthreads();
+    for (int i = tid; i < kSimtRows * d; i += blockDim.x) {
+      const int r = i / d, k = i - r * d;
+      xs[i] = s_row[r] >= 0 ? to_f32<T>(P.H[(size_t)s_row[r] * d + k]) : 0.f;
+    }
+    __syncthreads();
+    for (int h = tid; h < hid; h += blockDim.x) {
+      float acc[kSimtRows];
+#pragma unroll
+      for (int r = 0; r < kSimtRows; ++r) acc[r] = 0.f;
+      for (int k = 0; k < d; ++k) {
+        const float w = to_f32<T>(P.W1[(size_t)k * hid + h]);
+#pragma unroll
+        for (int r = 0; r < kSimtRows; ++r) acc[r] = fmaf(xs[r * d + k], w, acc[r]);
+      }
+      const float bb = to_f32<T>(P.b1[h]);
+#pragma unroll
+      for (int r = 0; r < kSimtRows; ++r) hs[r * hid + h] = fmaxf(acc[r] + bb, 0.f);
+    }
+    __syncthreads();
+    for (int e = tid; e < d; e += blockDim.x) {
+      float acc[kSimtRows];
+#pragma unroll
+      for (int r = 0; r < kSimtRows; ++r) acc[r] = 0.f;
+      for (int j = 0; j < hid; ++j) {
+        const float w = to_f32<T>(P.W2[(size_t)j * d + e]);
+#pragma unroll
+        for (int r = 0; r < kSimtRows; ++r) acc[r] = fmaf(hs[r * hid + j], w, acc[r]);
+      }
+      const float bb = to_f32<T>(P.b2[e]);
+#pragma unroll
+      for (int r = 0; r < kSimtRows; ++r) ys[r * d + e] = acc[r] + bb + xs[r * d + e];
+    }
+    __syncthreads();
+    const int w = tid >> 5, lane = tid & 31;            // warp w normalises row w
+    if (w < kSimtRows && s_row[w] >= 0) {
+      float sum = 0.f;
+      for (int e = lane; e < d; e += 32) sum += ys[w * d + e];
+      for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float mean = sum / (float)d;
+      float sq = 0.f;
+      for (int e = lane; e < d; e += 32) sq += (ys[w * d + e] - mean) * (ys[w * d + e] - mean);
+      for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      const float rstd = rsqrtf(sq / (float)d + P.eps);
+      for (int e = lane; e < d; e += 32)
+        P.H[(size_t)s_row[w] * d + e] =
+            from_f32<T>((ys[w * d + e] - mean) * rstd * to_f32<T>(P.g[e]) + to_f32<T>(P.beta[e]));
+    }
+  }
+}
+
+int ffn_sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+size_t ffn_tc_smem(int d) {
+  return (size_t)2 * kRows * d * 2 + (size_t)2 * kRows * kChunk * 2 + (size_t)kWStages * kChunk * d * 2 +
+         (size_t)2 * kPairRows * sizeof(int);
+}
+
+bool ffn_tc_supported(const Plan& p, int hid) {
+  if (p.dtype != LASER_BF16) return false;
+  if (p.d % 16 || p.d < 16 || p.d > 128) return false;
+  if (hid % kChunk || hid < kChunk) return false;
+  return ffn_tc_smem(p.d) + 1024 <= 227 * 1024;   // dynamic + static shared memory of one block
+}
+
+template <typename T>
+int ffn_simt(const Plan& p, const laser_ffn_params* f, void* H, const int32_t* lengths, const int32_t* cand_offsets,
+             char* ws, char* scratch, cudaStream_t st) {
+  FfnSimtParams<T> P;
+  P.U = p.U; P.N = p.N; P.L = p.L; P.Lp = p.Lp; P.S = p.S; P.d = p.d; P.hid = f->d_hidden; P.maxC = p.maxC;
+  P.eps = f->ln_eps > 0.f ? f->ln_eps : 1e-5f;
+  P.H = (T*)H;
+  P.W1 = (const T*)f->W1; P.b1 = (const T*)f->b1; P.W2 = (const T*)f->W2; P.b2 = (const T*)f->b2;
+  P.g = (const T*)f->ln_gain; P.beta = (const T*)f->ln_shift;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.counters = (int*)scratch;
+  P.prefix = (int*)(scratch + kAlign);
+  P.status = (int*)(ws + p.off_status);
+  const size_t smem = ((size_t)2 * kSimtRows * p.d + (size_t)kSimtRows * f->d_hidden) * sizeof(float);
+  if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("ffn_prep", st);
+    LASER_CUDA_OK(launch_chained(ffn_simt_prep_kernel<T>, dim3(1), dim3(1024), 0, st, P));
+  }
+  {
+    LASER_CUDA_OK(cudaFuncSetAttribute(ffn_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const long long blocks_needed = ((long long)p.N * p.Lp + kSimtRows - 1) / kSimtRows;
+    const int grid = (int)(blocks_needed < 8LL * ffn_sm_count() ? (blocks_needed > 0 ? blocks_needed : 1) : 8LL * ffn_sm_count());
+    LaunchScope ls("ffn_simt", st);
+    LASER_CUDA_OK(launch_chained(ffn_simt_kernel<T>, dim3(grid), dim3(256), smem, st, P));
+  }
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+}  // namespace
+
+size_t ffn_scratch_bytes(const Plan& p, int hid) {
+  return kAlign + align_up(((size_t)p.U + 1) * sizeof(int)) + 2 * align_up((size_t)p.d * hid * 2);
+}
+
+bool ffn_supported(const Plan& p, int hid) {
+  if (hid < 1) return false;
+  if ((long long)p.N * p.Lp >= (1ll << 31) - kPairRows) return false;
+  if (ffn_tc_supported(p, hid) && p.path != LASER_PATH_SIMT) return true;
+  if ((p.d * p.esize) % 16) return false;
+  return ((size_t)2 * kSimtRows * p.d + (size_t)kSimtRows * hid) * sizeof(float) <= 200 * 1024;
+}
+
+int ffn_forward(const Plan& p, const laser_ffn_params* f, void* H, const int32_t* lengths, const int32_t* cand_offsets,
+                char* ws, char* scratch, cudaStream_t st) {
+  if (p.N == 0 || p.U == 0) return LASER_OK;
+  const int hid = f->d_hidden;
+  if (!ffn_supported(p, hid)) return LASER_ERR_UNSUPPORTED;
+  if (!(ffn_tc_supported(p, hid) && p.path != LASER_PATH_SIMT)) {
+    if (p.dtype == LASER_F32) return ffn_simt<float>(p, f, H, lengths, cand_offsets, ws, scratch, st);
+    return ffn_simt<bf16>(p, f, H, lengths, cand_offsets, ws, scratch, st);
+  }
+  FfnParams P;
+  P.U = p.U; P.N = p.N; P.L = p.L; P.Lp = p.Lp; P.S = p.S; P.d = p.d; P.hid = hid; P.NJ = hid / kChunk; P.maxC = p.maxC;
+  P.eps = f->ln_eps > 0.f ? f->ln_eps : 1e-5f;
+  P.H = (bf16*)H;
+  P.W1 = (const bf16*)f->W1; P.b1 = (const bf16*)f->b1; P.W2 = (const bf16*)f->W2; P.b2 = (const bf16*)f->b2;
+  P.g = (const bf16*)f->ln_gain; P.beta = (const bf16*)f->ln_shift;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.counters = (int*)scratch;
+  P.prefix = (int*)(scratch + kAlign);
+  P.img1 = (bf16*)(scratch + kAlign + align_up(((size_t)p.U + 1) * sizeof(int)));
+  P.img2 = (bf16*)((char*)P.img1 + align_up((size_t)p.d * hid * 2));
+  P.status = (int*)(ws + p.off_status);
+  {
+    LaunchScope ls("ffn_prep", st);
+    LASER_CUDA_OK(launch_chained(ffn_prep_kernel, dim3(1 + 16), dim3(1024), 0, st, P, 1));
+  }
+  {
+    const size_t smem = ffn_tc_smem(p.d);
+    LASER_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const long long pairs_max = ((long long)p.N * p.Lp + kPairRows - 1) / kPairRows;
+    const int sms = ffn_sm_count();
+    const int grid = (int)(pairs_max < sms ? (pairs_max > 0 ? pairs_max : 1) : sms);
+    LaunchScope ls("ffn_tc", st);
+    LASER_CUDA_OK(launch_chained(ffn_tc_kernel, dim3(grid), dim3(kFfnThreads), smem, st, P));
+  }
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+}  // namespace laser
