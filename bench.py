@@ -254,6 +254,66 @@ def dominant_kernel_roofline(w, prof, peaks):
     return kernel_roofline(w, name, ms, peaks)
 
 
+def ffn_row(P, w, b, Hp, flush, stream, steps, peaks, dev):
+    """Next row of the scope: the feed-forward refinement (Eq. 6, r = 4) of this batch's H', timed on its own (outside
+    the step) after a check of sampled rows against the oracle."""
+    import torch
+    from oracle import ffn_oracle
+    from workloads import make_ffn_weights
+    s = w.spec
+    r = 4
+    hid = r * s.d
+    need = P.laser_ffn_workspace_bytes(b.cfg, hid)
+    if need == 0:
+        return None
+    fw = make_ffn_weights(s.d, r, s.dtype, seed=0)
+    fdev = {k: torch.from_numpy(v).to(b.items.dtype).to(dev) for k, v in fw.items()}
+    fws = torch.empty(need, dtype=torch.uint8, device=dev)
+    nseg = -(-w.lengths.astype(np.int64) // s.S)
+    cpu = np.diff(w.cand_offsets.astype(np.int64))
+    rows = int((nseg * cpu).sum())
+    # parity on sampled rows (the first and last candidate of up to four users)
+    before = {}
+    for u in [u for u in range(s.U) if nseg[u] > 0 and cpu[u] > 0][:4]:
+        for c in {int(w.cand_offsets[u]), int(w.cand_offsets[u + 1]) - 1}:
+            before[c] = (Hp[c, :int(nseg[u])].float().cpu().numpy().astype(np.float64), int(nseg[u]))
+    try:
+        P.laser_ffn_forward(b.cfg, fdev, Hp, b.lengths, b.cand_offsets, workspace=fws, stream=stream)
+    except P.LaserError:
+        return None
+    assert P.laser_check_status(fws) == 0
+    err = 0.0
+    for c, (x, n) in before.items():
+        ref = ffn_oracle.ffn_rows(x, fw["W1"], fw["b1"], fw["W2"], fw["b2"], fw["ln_g"], fw["ln_b"])
+        got = Hp[c, :n].float().cpu().numpy().astype(np.float64)
+        err = max(err, float(np.max(np.abs(got - ref) / np.maximum(1.0, np.abs(ref)))))
+    tol = 1e-4 if s.dtype == "f32" else 2e-2
+    if not (err <= tol):
+        raise SystemExit(f"FFN parity failure before timing: error {err:.3e} > {tol}")
+    P.laser_profile_enable(True)
+    prof = {}
+    tot = 0.0
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        P.laser_ffn_forward(b.cfg, fdev, Hp, b.lengths, b.cand_offsets, workspace=fws, stream=stream)
+        e1.record(stream)
+        for name, ms in P.laser_profile_read():
+            prof[name] = prof.get(name, 0.0) + ms / steps
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1) / steps
+    P.laser_profile_enable(False)
+    main = "ffn_tc" if "ffn_tc" in prof else "ffn_simt"
+    flops = 4.0 * rows * s.d * hid                       # two products of 2 * d * hid flops per row
+    ach = flops / (prof[main] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    return {"kernel": main, "expansion": r, "rows": rows, "ms": tot, "kernels_ms": prof,
+            "bound": "tensor" if main == "ffn_tc" else "alu", "achieved": ach, "peak": peak if main == "ffn_tc" else None,
+            "unit": "TFLOP/s", "frac": ach / peak if main == "ffn_tc" else None, "flops": flops,
+            "parity": {"err": err, "tol": tol, "rows_checked": sum(n for _, n in before.values())}}
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -348,6 +408,7 @@ def run_ours(args, rank, world, local_rank):
 
     # next row of the scope: multi-resolution fusion outputs on the H' and z of this batch (outside the timed step)
     fusion = None
+    ffn = None
     if rank == 0:
         r_recent = 2
         Hp_full = torch.empty((b.cfg.total_cands, b.cfg.n_seg, s.d), dtype=b.items.dtype, device=dev)
@@ -369,7 +430,9 @@ def run_ours(args, rank, world, local_rank):
         fusion = {"kernel": "fusion", "num_recent": r_recent, "ms": f_ms, "bound": "hbm",
                   "achieved": f_bytes / (f_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                   "frac": f_bytes / (f_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-        del Hp_full, fused
+        del fused
+        ffn = ffn_row(P, w, b, Hp_full, flush, stream, args.steps, peaks, dev)
+        del Hp_full
 
     # end to end: pinned host buffers in, z out, through laser_forward_host
     hb = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device="cpu", pin_host=True)
@@ -420,6 +483,7 @@ def run_ours(args, rank, world, local_rank):
                 "roofline": roof,
                 "kernels_ms": prof,
                 "fusion": fusion,
+                "ffn": ffn,
                 "kernel_rooflines": [kernel_roofline(w, k, v, peaks) for k, v in prof.items() if k in KERNEL_SOURCE],
                 "cpu_baseline": cpu_base,
                 "parity": parity,

@@ -22,8 +22,8 @@ using namespace ptx;
 constexpr int kRows = 128;            // rows per tile = MMA M = TMEM lanes
 constexpr int kChunk = 128;           // hidden units per step
 constexpr int kPairRows = 2 * kRows;  // two tiles share every weight chunk
-constexpr int kFfnThreads = 384;      // warp 0 weight producer + TMEM, warp 1 MMA issuer, warps 2-3 row staging,
-                                      // warps 4-7 / 8-11 epilogue warpgroups of tile 0 / tile 1
+constexpr int kFfnThreads = 320;      // warp 0 weight producer + TMEM, warp 1 MMA issuer,
+                                      // warps 2-5 / 6-9 epilogue warpgroups of tile 0 / tile 1
 constexpr int kWStages = 3;
 constexpr int kFfnTmemCols = 512;     // acc2[t] at 128 t, acc1[t] at 256 + 128 t
 constexpr int kSimtRows = 8;
@@ -37,6 +37,7 @@ struct FfnParams {
   int* prefix;                                // [U + 1] valid rows before each user
   int* counters;                              // [0] total valid rows
   bf16 *img1, *img2;                          // chunk j of W_1^T / W_2^T at + j * 128 * d
+  float* lnv;                                 // [3][d] fp32 copies of b_2, the layer norm's gain and its shift
   int* status;
 };
 
@@ -121,6 +122,11 @@ __global__ void __launch_bounds__(1024) ffn_prep_kernel(FfnParams P, int build_i
   if (!build_images) return;
   const int nthreads = (gridDim.x - 1) * blockDim.x;
   const int g = (blockIdx.x - 1) * blockDim.x + threadIdx.x;
+  for (int i = g; i < P.d; i += nthreads) {
+    P.lnv[i] = __bfloat162float(P.b2[i]);
+    P.lnv[P.d + i] = __bfloat162float(P.g[i]);
+    P.lnv[2 * P.d + i] = __bfloat162float(P.beta[i]);
+  }
   const int n = P.d * P.hid;
   const int chunk_elems = kChunk * P.d;
   for (int i = g; i < n; i += nthreads) {          // W_1[k][h]: B operand of step j = h / 128, row h % 128, K index k
@@ -147,7 +153,7 @@ __device__ __forceinline__ void ffn_step(int s, int NJ, bool& second, int& j) {
 
 struct FfnBars {
   uint64_t w_full[kWStages], w_empty[kWStages];
-  uint64_t x_full[2], x_free[2];
+  uint64_t x_full[2];
   uint64_t a1_full[2], a1_free[2];
   uint64_t hs_full[2], hs_free[2];
   uint64_t a2_full[2], a2_free[2];
@@ -156,7 +162,17 @@ struct FfnBars {
 
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+// max(a + b, 0) on two packed bf16 values (one fused multiply-add by 1 with the ReLU modifier)
+__device__ __forceinline__ uint32_t relu_add_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("fma.rn.relu.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(0x3F803F80u), "r"(b));
+  return r;
+}
 
+// Roles: warp 0 streams the weight chunks, warp 1 issues the MMAs, warps 2-5 / 6-9 are the epilogue warpgroups of tile
+// 0 / tile 1.  An epilogue warp owns 32 rows of its tile (TMEM lanes 32 (warp mod 4) .. + 31): it stages them (K-major)
+// for the first layer, turns acc1 into hidden activations, normalises them at the end and writes them back; the shared
+// memory it touches for all of this is its own rows' slice of X and Hs, so the warps never have to meet at a barrier.
 __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ FfnBars bars;
@@ -169,13 +185,11 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
   uint8_t* Xs = smem_raw;                              // [2][128 x d]       K-major, K = d
   uint8_t* Hs = Xs + 2 * x_bytes;                      // [2][128 x 128]     K-major, K = 128 hidden units
   uint8_t* Ws = Hs + 2 * hs_bytes;                     // [kWStages][128 d]  one weight chunk each
-  int* rowmap = reinterpret_cast<int*>(Ws + kWStages * w_bytes);   // [2 tiles][2][128] rows of H' behind the staged tiles
 
   if (tid == 0) {
     for (int i = 0; i < kWStages; ++i) { mbar_init(&bars.w_full[i], 1); mbar_init(&bars.w_empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars.x_full[i], 1);
-      mbar_init(&bars.x_free[i], 1);
+      mbar_init(&bars.x_full[i], 4);
       mbar_init(&bars.a1_full[i], 1);
       mbar_init(&bars.a1_free[i], 4);
       mbar_init(&bars.hs_full[i], 4);
@@ -239,99 +253,87 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       const uint32_t x_sbo = (d >> 3) * 128, h_sbo = (kChunk >> 3) * 128;
       const uint32_t id1 = idesc_bf16(128, kChunk), id2 = idesc_bf16(128, d);
       const int ks1 = d >> 4, ks2 = kChunk >> 4;
-      uint32_t use = 0;
+      const uint64_t xd0 = smem_desc(smem_u32(Xs), 128, x_sbo), hd0 = smem_desc(smem_u32(Hs), 128, h_sbo);
+      const uint64_t w1d0 = smem_desc(smem_u32(Ws), 128, x_sbo), w2d0 = smem_desc(smem_u32(Ws), 128, h_sbo);
+      uint32_t use = 0, slot = 0, w_par = 0;
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
         for (int s = 0; s < 2 * NJ && ok; ++s, ++use) {
           bool second;
           int j;
           ffn_step(s, NJ, second, j);
-          const uint32_t slot = use % kWStages;
-          ok = wait_all(&bars.w_full[slot], (use / kWStages) & 1);
+          ok = wait_all(&bars.w_full[slot], w_par);
           if (!ok) break;
+          const uint32_t k = (uint32_t)it * NJ + j;
           for (int t = 0; t < 2 && ok; ++t) {
             if (!second) {
               if (j == 0) ok = wait_all(&bars.x_full[t], it & 1);
-              const uint32_t k = (uint32_t)it * NJ + j;
               ok = ok && wait_all(&bars.a1_free[t], (k & 1) ^ 1);
               if (!ok) break;
               tc_fence_after();
-              const uint64_t ad = smem_desc(smem_u32(Xs + t * x_bytes), 128, x_sbo);
-              const uint64_t bd = smem_desc(smem_u32(Ws + slot * w_bytes), 128, x_sbo);
+              const uint64_t ad = xd0 + (uint64_t)(t * (x_bytes >> 4)), bd = w1d0 + (uint64_t)(slot * (w_bytes >> 4));
               const uint32_t dcol = tmem + 256 + t * kChunk;
               if (leader) {
                 for (int ks = 0; ks < ks1; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id1, ks > 0);
                 tc_commit(&bars.a1_full[t]);
-                if (j == NJ - 1) tc_commit(&bars.x_free[t]);
               }
             } else {
-              const uint32_t k = (uint32_t)it * NJ + j;
               ok = wait_all(&bars.hs_full[t], k & 1);
               if (ok && j == 0) ok = wait_all(&bars.a2_free[t], (it & 1) ^ 1);
               if (!ok) break;
               tc_fence_after();
-              const uint64_t ad = smem_desc(smem_u32(Hs + t * hs_bytes), 128, h_sbo);
-              const uint64_t bd = smem_desc(smem_u32(Ws + slot * w_bytes), 128, h_sbo);
+              const uint64_t ad = hd0 + (uint64_t)(t * (hs_bytes >> 4)), bd = w2d0 + (uint64_t)(slot * (w_bytes >> 4));
               const uint32_t dcol = tmem + t * 128;
               if (leader) {
-                for (int ks = 0; ks < ks2; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id2, (j | ks) != 0);
-                tc_commit(&bars.hs_free[t]);
-                if (j == NJ - 1) tc_commit(&bars.a2_full[t]);
+#pragma unroll
+                for (int ks = 0; ks < kChunk / 16; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id2, (j | ks) != 0);
+                tc_commit(j == NJ - 1 ? &bars.a2_full[t] : &bars.hs_free[t]);   // a2_full also says "Hs[t] is free"
               }
             }
             __syncwarp();
           }
           if (ok && leader) tc_commit(&bars.w_empty[slot]);
           __syncwarp();
+          if (++slot == kWStages) { slot = 0; w_par ^= 1; }
         }
       }
+      (void)ks2;
       if (leader) tc_commit(&bars.done);
       __syncwarp();
       wait_all(&bars.done, 0);
-    } else if (warp < 4) {
-      // ------------------------------------------------------------------ row staging: warp 2 + t fills tile t
-      const int t = warp - 2;
+    } else {
+      // ------------------------------------------------------------------ epilogue warp: rows 32 quad .. + 31 of tile t
+      const int t = (warp - 2) >> 2, quad = warp & 3;
+      const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
+      const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
       const int cpr = d >> 3;                              // 16-byte chunks per row
-      const int rin = lane & 7;
-      uint8_t* X = Xs + t * x_bytes;
-      int* maps = rowmap + t * (2 * kRows);                // [2][128] rows of H' behind this warp's tile, two pairs deep
-      auto fill_map = [&](int it) {
-        const int pair = bidx + it * G;
-        int* m = maps + (it & 1) * kRows;
-        for (int r = lane; r < kRows; r += 32)
-          m[r] = it < my_pairs ? global_row(P, pair * kPairRows + t * kRows + r, total) : -1;
-        __syncwarp();
-      };
-      fill_map(0);
-      bool ok = true;
-      for (int it = 0; it < my_pairs && ok; ++it) {
-        const int* m = maps + (it & 1) * kRows;
-        ok = wait_all(&bars.x_free[t], (it & 1) ^ 1);
-        if (!ok) break;
-        for (int idx = lane >> 3; idx < 16 * cpr; idx += 4) {          // idx = (8-row group) * cpr + chunk
+      uint8_t* hs_row = Hs + t * hs_bytes + (r >> 3) * ((kChunk >> 3) * 128) + (r & 7) * 16;
+      uint8_t* x_warp = Xs + t * x_bytes + (size_t)(quad * 4) * cpr * 128;    // this warp's four 8-row groups of X[t]
+      uint8_t* o_warp = Hs + t * hs_bytes + quad * (hs_bytes / 4);            // this warp's slice of Hs[t]: output staging
+      const float inv_d = 1.f / (float)d;
+      const bool swz = (cpr & (cpr - 1)) == 0;             // XOR-swizzled staging rows when cpr is a power of two
+      const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
+      // stage my warp's rows of the pair `it`: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
+      auto stage = [&](int grow_mine) {
+        for (int idx = lane >> 3; idx < 4 * cpr; idx += 4) {
           const int gq = idx / cpr, c = idx - gq * cpr;
-          const int grow = m[gq * 8 + rin];
+          const int grow = __shfl_sync(0xffffffffu, grow_mine, gq * 8 + (lane & 7));
           const bf16* src = grow >= 0 ? P.H + (size_t)grow * d + c * 8 : P.H;
-          cp_async16(X + (size_t)idx * 128 + rin * 16, src, grow >= 0 ? 16u : 0u);
+          cp_async16(x_warp + (size_t)idx * 128 + (lane & 7) * 16, src, grow >= 0 ? 16u : 0u);
         }
+      };
+      auto publish_x = [&]() {                             // my copies have landed: tell the issuer
         cp_async_wait_all();
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars.x_full[t]);
-        fill_map(it + 1);                                  // the other map: its pair is long staged
-      }
-      cp_async_wait_all();
-    } else {
-      // ------------------------------------------------------------------ epilogue warpgroup of tile t
-      const int t = (warp - 4) >> 2, quad = warp & 3;
-      const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
-      const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-      uint8_t* hs_row = Hs + t * hs_bytes + (r >> 3) * ((kChunk >> 3) * 128) + (r & 7) * 16;
-      const float inv_d = 1.f / (float)d;
+      };
+      int grow = global_row(P, bidx * kPairRows + t * kRows + r, total);
+      stage(grow);
+      publish_x();
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
-        const int pair = bidx + it * G;
-        const int grow = global_row(P, pair * kPairRows + t * kRows + r, total);
+        const int grow_next = it + 1 < my_pairs ? global_row(P, (bidx + (it + 1) * G) * kPairRows + t * kRows + r, total) : -1;
         // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> shared memory (A operand of the second layer)
         for (int j = 0; j < NJ && ok; ++j) {
           const uint32_t kh = (uint32_t)it * NJ + j;
@@ -351,17 +353,17 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
               const uint4 bb = __ldg(bias + c * 4 + q);
               const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float lo = fmaxf(__uint_as_float(v[q * 8 + 2 * e]) + bf_lo(bw[e]), 0.f);
-                const float hi = fmaxf(__uint_as_float(v[q * 8 + 2 * e + 1]) + bf_hi(bw[e]), 0.f);
-                o[c * 16 + q * 4 + e] = pack_bf16x2(lo, hi);
-              }
+              for (int e = 0; e < 4; ++e)                  // round the pair to bf16, then max(h + b_1, 0) on both halves at once
+                o[c * 16 + q * 4 + e] = relu_add_bf16x2(
+                    pack_bf16x2(__uint_as_float(v[q * 8 + 2 * e]), __uint_as_float(v[q * 8 + 2 * e + 1])), bw[e]);
             }
           }
           tc_fence_before();                               // the accumulator is in registers: hand it back
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.a1_free[t]);
-          ok = wait_all(&bars.hs_free[t], (kh & 1) ^ 1);   // the previous chunk's second-layer product has read Hs
+          // Hs[t] is free once the previous chunk's second-layer product has read it (for the first chunk of a pair
+          // that was the previous pair's last product, which this warp has already waited for through a2_full)
+          if (j > 0) ok = wait_all(&bars.hs_free[t], ((uint32_t)(it * (NJ - 1) + j - 1)) & 1);
           if (!ok) break;
 #pragma unroll
           for (int k8 = 0; k8 < kChunk / 8; ++k8)
@@ -371,68 +373,98 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           if (lane == 0) mbar_arrive(&bars.hs_full[t]);
         }
         if (!ok) break;
-        // ---- second layer done: y = acc2 + b_2 + s, layer norm over the row, bf16 out
+        // ---- the last first-layer product has read X[t] (its a1_full arrived): keep my row of s for the residual and
+        // start fetching the next pair's rows into the same place
+        uint4 xr[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          xr[i] = i < cpr ? *reinterpret_cast<const uint4*>(x_warp + ((size_t)(lane >> 3) * cpr + i) * 128 + (lane & 7) * 16)
+                          : make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        if (it + 1 < my_pairs) stage(grow_next);
+        // ---- second layer: y = acc2 + b_2 + s, layer norm over the row
         ok = wait_all(&bars.a2_full[t], it & 1);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tO = tmem + lane_base + t * 128;
-        const bool live = grow >= 0;
-        bf16* row = P.H + (size_t)(live ? grow : 0) * d;
-        float mean = 0.f, rstd = 0.f;
-#pragma unroll 1
-        for (int pass = 0; pass < 3; ++pass) {
-          float acc = 0.f;
-#pragma unroll 1
-          for (int c = 0; c < d; c += 16) {
+        const float4* vb2 = reinterpret_cast<const float4*>(P.lnv);
+        const float4* vg = reinterpret_cast<const float4*>(P.lnv + d);
+        const float4* vbeta = reinterpret_cast<const float4*>(P.lnv + 2 * d);
+        float sum = 0.f, sq = 0.f;
+#pragma unroll
+        for (int c16 = 0; c16 < 8; ++c16) {
+          if (c16 * 16 < d) {
             uint32_t v[16];
-            tmem_ld16(tO + c, v);
+            tmem_ld16(tO + c16 * 16, v);
             tc_wait_ld();
-            if (pass == 2 && c + 16 >= d) {                // last read of the accumulator
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float4 bb = __ldg(vb2 + c16 * 4 + q);
+              const uint4 xx = xr[c16 * 2 + (q >> 1)];
+              const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+              const float y0 = __uint_as_float(v[q * 4 + 0]) + bb.x + bf_lo(x0);
+              const float y1 = __uint_as_float(v[q * 4 + 1]) + bb.y + bf_hi(x0);
+              const float y2 = __uint_as_float(v[q * 4 + 2]) + bb.z + bf_lo(x1);
+              const float y3 = __uint_as_float(v[q * 4 + 3]) + bb.w + bf_hi(x1);
+              sum += (y0 + y1) + (y2 + y3);
+              sq = fmaf(y0, y0, fmaf(y1, y1, fmaf(y2, y2, fmaf(y3, y3, sq))));
+            }
+          }
+        }
+        if (it + 1 < my_pairs) publish_x();                // the next pair's rows have landed by now
+        const float mean = sum * inv_d;
+        const float rstd = rsqrtf(fmaxf(sq * inv_d - mean * mean, 0.f) + P.eps);
+#pragma unroll
+        for (int c16 = 0; c16 < 8; ++c16) {
+          if (c16 * 16 < d) {
+            uint32_t v[16];
+            tmem_ld16(tO + c16 * 16, v);
+            tc_wait_ld();
+            if ((c16 + 1) * 16 >= d) {                     // last read of the accumulator: hand it back
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(&bars.a2_free[t]);
             }
-            if (live) {
-              float y[16];
+            uint32_t o[8];
 #pragma unroll
-              for (int q = 0; q < 2; ++q) {
-                const uint4 xx = *reinterpret_cast<const uint4*>(row + c + q * 8);
-                const uint4 bb = __ldg(reinterpret_cast<const uint4*>(P.b2 + c + q * 8));
-                const uint32_t xw[4] = {xx.x, xx.y, xx.z, xx.w}, bw[4] = {bb.x, bb.y, bb.z, bb.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  y[q * 8 + 2 * e] = __uint_as_float(v[q * 8 + 2 * e]) + bf_lo(bw[e]) + bf_lo(xw[e]);
-                  y[q * 8 + 2 * e + 1] = __uint_as_float(v[q * 8 + 2 * e + 1]) + bf_hi(bw[e]) + bf_hi(xw[e]);
-                }
-              }
-              if (pass == 0) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) acc += y[e];
-              } else if (pass == 1) {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) acc += (y[e] - mean) * (y[e] - mean);
-              } else {
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                  const uint4 gg = __ldg(reinterpret_cast<const uint4*>(P.g + c + q * 8));
-                  const uint4 be = __ldg(reinterpret_cast<const uint4*>(P.beta + c + q * 8));
-                  const uint32_t gw[4] = {gg.x, gg.y, gg.z, gg.w}, ew[4] = {be.x, be.y, be.z, be.w};
-                  uint32_t o[4];
-#pragma unroll
-                  for (int e = 0; e < 4; ++e) {
-                    const float lo = (y[q * 8 + 2 * e] - mean) * rstd * bf_lo(gw[e]) + bf_lo(ew[e]);
-                    const float hi = (y[q * 8 + 2 * e + 1] - mean) * rstd * bf_hi(gw[e]) + bf_hi(ew[e]);
-                    o[e] = pack_bf16x2(lo, hi);
-                  }
-                  *reinterpret_cast<uint4*>(row + c + q * 8) = make_uint4(o[0], o[1], o[2], o[3]);
-                }
-              }
+            for (int q = 0; q < 4; ++q) {
+              const float4 bb = __ldg(vb2 + c16 * 4 + q), gg = __ldg(vg + c16 * 4 + q), be = __ldg(vbeta + c16 * 4 + q);
+              const uint4 xx = xr[c16 * 2 + (q >> 1)];
+              const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+              const float y0 = __uint_as_float(v[q * 4 + 0]) + bb.x + bf_lo(x0);
+              const float y1 = __uint_as_float(v[q * 4 + 1]) + bb.y + bf_hi(x0);
+              const float y2 = __uint_as_float(v[q * 4 + 2]) + bb.z + bf_lo(x1);
+              const float y3 = __uint_as_float(v[q * 4 + 3]) + bb.w + bf_hi(x1);
+              const float a0 = rstd * gg.x, a1 = rstd * gg.y, a2 = rstd * gg.z, a3 = rstd * gg.w;
+              o[q * 2] = pack_bf16x2(fmaf(y0, a0, fmaf(-mean, a0, be.x)), fmaf(y1, a1, fmaf(-mean, a1, be.y)));
+              o[q * 2 + 1] = pack_bf16x2(fmaf(y2, a2, fmaf(-mean, a2, be.z)), fmaf(y3, a3, fmaf(-mean, a3, be.w)));
+            }
+            // my row of the output, staged in my slice of Hs[t] (free: the last second-layer product is complete)
+            const int c0 = c16 * 2, c1 = c16 * 2 + 1;
+            *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c0 ^ (lane & (cpr - 1)) : c0) << 4)) =
+                make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c1 ^ (lane & (cpr - 1)) : c1) << 4)) =
+                make_uint4(o[4], o[5], o[6], o[7]);
+          }
+        }
+        __syncwarp();
+        // coalesced write-back: cpr consecutive lanes write one row, 32 / cpr rows per instruction
+        {
+          const int rr0 = lane / cpr, cc = lane - rr0 * cpr;
+          for (int base = 0; base < 32; base += rows_per) {
+            const int rr = base + rr0;
+            const int g_row = __shfl_sync(0xffffffffu, grow, rr & 31);
+            if (rr0 < rows_per && rr < 32 && g_row >= 0) {
+              const uint4 val = *reinterpret_cast<const uint4*>(
+                  o_warp + (size_t)rr * (d * 2) + ((swz ? cc ^ (rr & (cpr - 1)) : cc) << 4));
+              *reinterpret_cast<uint4*>(P.H + (size_t)g_row * d + cc * 8) = val;
             }
           }
-          if (pass == 0) mean = acc * inv_d;
-          if (pass == 1) rstd = rsqrtf(acc * inv_d + P.eps);
         }
+        __syncwarp();                                      // the staging slice is read: the next pair's E1 may overwrite it
+        grow = grow_next;
       }
+      cp_async_wait_all();
     }
   }
 
@@ -538,8 +570,7 @@ int ffn_sm_count() {
 }
 
 size_t ffn_tc_smem(int d) {
-  return (size_t)2 * kRows * d * 2 + (size_t)2 * kRows * kChunk * 2 + (size_t)kWStages * kChunk * d * 2 +
-         (size_t)2 * kPairRows * sizeof(int);
+  return (size_t)2 * kRows * d * 2 + (size_t)2 * kRows * kChunk * 2 + (size_t)kWStages * kChunk * d * 2;
 }
 
 bool ffn_tc_supported(const Plan& p, int hid) {
@@ -582,7 +613,8 @@ int ffn_simt(const Plan& p, const laser_ffn_params* f, void* H, const int32_t* l
 }  // namespace
 
 size_t ffn_scratch_bytes(const Plan& p, int hid) {
-  return kAlign + align_up(((size_t)p.U + 1) * sizeof(int)) + 2 * align_up((size_t)p.d * hid * 2);
+  return kAlign + align_up(((size_t)p.U + 1) * sizeof(int)) + 2 * align_up((size_t)p.d * hid * 2) +
+         align_up((size_t)3 * p.d * sizeof(float));
 }
 
 bool ffn_supported(const Plan& p, int hid) {
@@ -613,6 +645,7 @@ int ffn_forward(const Plan& p, const laser_ffn_params* f, void* H, const int32_t
   P.prefix = (int*)(scratch + kAlign);
   P.img1 = (bf16*)(scratch + kAlign + align_up(((size_t)p.U + 1) * sizeof(int)));
   P.img2 = (bf16*)((char*)P.img1 + align_up((size_t)p.d * hid * 2));
+  P.lnv = (float*)((char*)P.img2 + align_up((size_t)p.d * hid * 2));
   P.status = (int*)(ws + p.off_status);
   {
     LaunchScope ls("ffn_prep", st);
