@@ -25,7 +25,7 @@ constexpr int kPairRows = 2 * kRows;  // two tiles share every weight chunk
 constexpr int kFfnThreads = 320;      // warp 0 weight producer + TMEM, warp 1 MMA issuer,
                                       // warps 2-5 / 6-9 epilogue warpgroups of tile 0 / tile 1
 constexpr int kWStages = 3;
-constexpr int kFfnTmemCols = 512;     // acc2[t] at 128 t, acc1[t] at 256 + 128 t
+constexpr int kFfnTmemCols = 512;     // acc2[t] at 128 t; acc1[t], then the hidden activations, at 256 + 128 t
 constexpr int kSimtRows = 8;
 
 struct FfnParams {
@@ -38,6 +38,7 @@ struct FfnParams {
   int* counters;                              // [0] total valid rows
   bf16 *img1, *img2;                          // chunk j of W_1^T / W_2^T at + j * 128 * d
   float* lnv;                                 // [3][d] fp32 copies of b_2, the layer norm's gain and its shift
+  int* rowmap;                                // [N * Lp] compact row -> row of H' (first counters[0] entries valid)
   int* status;
 };
 
@@ -139,24 +140,22 @@ __global__ void __launch_bounds__(1024) ffn_prep_kernel(FfnParams P, int build_i
   }
 }
 
-// ------------------------------------------------------------------------------------------------------- tensor kernel
-// Order of the 2 NJ weight chunks of one tile pair: the first-layer product of chunk j + 1 is issued ahead of the
-// second-layer product of chunk j, so the tensor pipe has work while the epilogue warps turn acc1 into hidden activations.
-__device__ __forceinline__ void ffn_step(int s, int NJ, bool& second, int& j) {
-  if (NJ == 1) { second = s != 0; j = 0; return; }
-  if (s < 2) { second = false; j = s; return; }
-  if (s == 2 * NJ - 1) { second = true; j = NJ - 1; return; }
-  const int q = s - 2;
-  second = !(q & 1);
-  j = second ? q >> 1 : (q >> 1) + 2;
+// Compact row -> row of H', for every valid row (the main kernel reads it with coalesced loads).
+__global__ void __launch_bounds__(256) ffn_map_kernel(FfnParams P) {
+  chain_wait();
+  chain_release();
+  const int total = P.counters[0];
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x)
+    P.rowmap[i] = global_row(P, i, total);
 }
 
+// ------------------------------------------------------------------------------------------------------- tensor kernel
 struct FfnBars {
   uint64_t w_full[kWStages], w_empty[kWStages];
-  uint64_t x_full[2];
-  uint64_t a1_full[2], a1_free[2];
-  uint64_t hs_full[2], hs_free[2];
-  uint64_t a2_full[2], a2_free[2];
+  uint64_t x_full[2];                   // X[t] staged (4 epilogue warps)
+  uint64_t a1_full[2];                  // first-layer product of tile t complete
+  uint64_t hid_full[2];                 // hidden activations of tile t written to TMEM (4 epilogue warps)
+  uint64_t a2_full[2], a2_free[2];      // second-layer accumulator of tile t complete / drained (4 epilogue warps)
   uint64_t done;
 };
 
@@ -169,10 +168,18 @@ __device__ __forceinline__ uint32_t relu_add_bf16x2(uint32_t a, uint32_t b) {
   return r;
 }
 
-// Roles: warp 0 streams the weight chunks, warp 1 issues the MMAs, warps 2-5 / 6-9 are the epilogue warpgroups of tile
-// 0 / tile 1.  An epilogue warp owns 32 rows of its tile (TMEM lanes 32 (warp mod 4) .. + 31): it stages them (K-major)
-// for the first layer, turns acc1 into hidden activations, normalises them at the end and writes them back; the shared
-// memory it touches for all of this is its own rows' slice of X and Hs, so the warps never have to meet at a barrier.
+// Roles: warp 0 streams the weight chunks (W_1 chunk 0, W_2 chunk 0, W_1 chunk 1, ...), warp 1 issues the MMAs, warps
+// 2-5 / 6-9 are the epilogue warpgroups of tile 0 / tile 1.  Per chunk j the issue order is
+//     acc1[0] = X[0] W_1j,  acc1[1] = X[1] W_1j,  acc2[0] += hid[0] W_2j,  acc2[1] += hid[1] W_2j
+// so tile 1's first-layer product runs while tile 0's epilogue warps turn acc1[0] into hidden activations, and so on.
+// The hidden activations (bf16) are written back into the first 64 columns of the accumulator they came from and feed
+// the second-layer product straight from TMEM: the first layer's operand reads already take the whole shared-memory
+// bandwidth, the second layer then leaves it to the weight copies, the row staging and the output staging.
+// The tensor pipe executes a block's MMAs in issue order, so the next first-layer product cannot overwrite hidden
+// activations that the second-layer product before it still reads.
+// An epilogue warp owns 32 rows of its tile (TMEM lanes 32 (warp mod 4) .. + 31): it stages them (K-major) for the
+// first layer, produces their hidden activations, normalises them at the end and writes them back; the shared memory
+// it touches for all of this is its own rows' slice of X and of the output staging, so the warps never meet at a barrier.
 __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ FfnBars bars;
@@ -181,19 +188,19 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d = P.d, NJ = P.NJ;
-  const uint32_t x_bytes = kRows * d * 2, hs_bytes = kRows * kChunk * 2, w_bytes = kChunk * d * 2;
+  const uint32_t x_bytes = kRows * d * 2, w_bytes = kChunk * d * 2;
   uint8_t* Xs = smem_raw;                              // [2][128 x d]       K-major, K = d
-  uint8_t* Hs = Xs + 2 * x_bytes;                      // [2][128 x 128]     K-major, K = 128 hidden units
-  uint8_t* Ws = Hs + 2 * hs_bytes;                     // [kWStages][128 d]  one weight chunk each
+  uint8_t* Os = Xs + 2 * x_bytes;                      // [2][128 x d]       output rows on their way to global memory
+  uint8_t* Ws = Os + 2 * x_bytes;                      // [kWStages][128 d]  one weight chunk each
+  float* s_lnv = reinterpret_cast<float*>(Ws + kWStages * w_bytes);        // [3][d] b_2, gain, shift
+  bf16* s_b1 = reinterpret_cast<bf16*>(s_lnv + 3 * d);                      // [hid]
 
   if (tid == 0) {
     for (int i = 0; i < kWStages; ++i) { mbar_init(&bars.w_full[i], 1); mbar_init(&bars.w_empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.x_full[i], 4);
       mbar_init(&bars.a1_full[i], 1);
-      mbar_init(&bars.a1_free[i], 4);
-      mbar_init(&bars.hs_full[i], 4);
-      mbar_init(&bars.hs_free[i], 1);
+      mbar_init(&bars.hid_full[i], 4);
       mbar_init(&bars.a2_full[i], 1);
       mbar_init(&bars.a2_free[i], 4);
     }
@@ -210,15 +217,32 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
-  chain_wait();                         // H' rows, the row prefix and the weight images are complete
+  chain_wait();                         // H' rows, the row map and the weight images are complete
   chain_release();
 
+  for (int i = tid; i < 3 * d; i += kFfnThreads) s_lnv[i] = P.lnv[i];
+  for (int i = tid; i < P.hid; i += kFfnThreads) s_b1[i] = P.b1[i];
+  __syncthreads();
   const int total = P.counters[0];
   const int n_pairs = (total + kPairRows - 1) / kPairRows;
   const int G = gridDim.x, bidx = blockIdx.x;
   const int my_pairs = bidx < n_pairs ? (n_pairs - bidx + G - 1) / G : 0;
   auto wait_all = [&](uint64_t* bar, uint32_t parity) {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abortp)) != 0;
+  };
+  // Two barriers polled together (their round trips to shared memory overlap); bounded like mbar_wait.
+  auto wait_both = [&](uint64_t* b0, uint32_t p0, uint64_t* b1, uint32_t p1) {
+    bool done = false;
+    for (uint32_t i = 0; i < kSpinLimit && !done; ++i) {
+      const bool r0 = mbar_try_wait(b0, p0), r1 = mbar_try_wait(b1, p1);
+      done = r0 && r1;
+      if (!done && (i & 63u) == 63u) {
+        if (*abortp) break;
+        __nanosleep(64);
+      }
+    }
+    if (!done) *abortp = 1;
+    return __all_sync(0xffffffffu, done) != 0;
   };
 
   if (my_pairs > 0) {
@@ -229,14 +253,12 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         bool ok = true;
         for (int it = 0; it < my_pairs && ok; ++it) {
           for (int s = 0; s < 2 * NJ && ok; ++s, ++use) {
-            bool second;
-            int j;
-            ffn_step(s, NJ, second, j);
             const uint32_t slot = use % kWStages;
             ok = mbar_wait(&bars.w_empty[slot], ((use / kWStages) & 1) ^ 1, abortp);
             if (!ok) break;
             mbar_arrive_expect_tx(&bars.w_full[slot], w_bytes);
-            bulk_g2s(Ws + slot * w_bytes, (second ? P.img2 : P.img1) + (size_t)j * kChunk * d, w_bytes, &bars.w_full[slot]);
+            bulk_g2s(Ws + slot * w_bytes, ((s & 1) ? P.img2 : P.img1) + (size_t)(s >> 1) * kChunk * d, w_bytes,
+                     &bars.w_full[slot]);
           }
         }
         if (!ok) {                                       // let the copies in flight land before the block goes away
@@ -252,43 +274,49 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       const bool leader = elect_one();
       const uint32_t x_sbo = (d >> 3) * 128, h_sbo = (kChunk >> 3) * 128;
       const uint32_t id1 = idesc_bf16(128, kChunk), id2 = idesc_bf16(128, d);
-      const int ks1 = d >> 4, ks2 = kChunk >> 4;
-      const uint64_t xd0 = smem_desc(smem_u32(Xs), 128, x_sbo), hd0 = smem_desc(smem_u32(Hs), 128, h_sbo);
+      const int ks1 = d >> 4;
+      const uint64_t xd0 = smem_desc(smem_u32(Xs), 128, x_sbo);
       const uint64_t w1d0 = smem_desc(smem_u32(Ws), 128, x_sbo), w2d0 = smem_desc(smem_u32(Ws), 128, h_sbo);
-      uint32_t use = 0, slot = 0, w_par = 0;
+      uint32_t slot = 0, w_par = 0;
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
-        for (int s = 0; s < 2 * NJ && ok; ++s, ++use) {
-          bool second;
-          int j;
-          ffn_step(s, NJ, second, j);
-          ok = wait_all(&bars.w_full[slot], w_par);
-          if (!ok) break;
+        for (int j = 0; j < NJ && ok; ++j) {
           const uint32_t k = (uint32_t)it * NJ + j;
-          for (int t = 0; t < 2 && ok; ++t) {
-            if (!second) {
-              if (j == 0) ok = wait_all(&bars.x_full[t], it & 1);
-              ok = ok && wait_all(&bars.a1_free[t], (k & 1) ^ 1);
-              if (!ok) break;
-              tc_fence_after();
-              const uint64_t ad = xd0 + (uint64_t)(t * (x_bytes >> 4)), bd = w1d0 + (uint64_t)(slot * (w_bytes >> 4));
-              const uint32_t dcol = tmem + 256 + t * kChunk;
-              if (leader) {
-                for (int ks = 0; ks < ks1; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id1, ks > 0);
+          // ---- first layer of chunk j, both tiles
+          if (j == 0) ok = wait_both(&bars.x_full[0], it & 1, &bars.x_full[1], it & 1);
+          ok = ok && wait_all(&bars.w_full[slot], w_par);
+          if (!ok) break;
+          tc_fence_after();
+          {
+            const uint64_t bd = w1d0 + (uint64_t)(slot * (w_bytes >> 4));
+            if (leader) {
+              for (int t = 0; t < 2; ++t) {
+                const uint64_t ad = xd0 + (uint64_t)(t * (x_bytes >> 4));
+                for (int ks = 0; ks < ks1; ++ks) mma_ss(tmem + 256 + t * kChunk, ad + ks * 16, bd + ks * 16, id1, ks > 0);
                 tc_commit(&bars.a1_full[t]);
               }
-            } else {
-              ok = wait_all(&bars.hs_full[t], k & 1);
-              if (ok && j == 0) ok = wait_all(&bars.a2_free[t], (it & 1) ^ 1);
+              tc_commit(&bars.w_empty[slot]);
+            }
+            __syncwarp();
+            if (++slot == kWStages) { slot = 0; w_par ^= 1; }
+          }
+          // ---- second layer of chunk j: acc2[t] += hid[t] (TMEM) W_2j
+          ok = wait_both(&bars.w_full[slot], w_par, &bars.hid_full[0], k & 1);
+          if (ok && j == 0) ok = wait_both(&bars.a2_free[0], (it & 1) ^ 1, &bars.a2_free[1], (it & 1) ^ 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t bd = w2d0 + (uint64_t)(slot * (w_bytes >> 4));
+          for (int t = 0; t < 2; ++t) {
+            if (t == 1) {
+              ok = wait_all(&bars.hid_full[1], k & 1);
               if (!ok) break;
               tc_fence_after();
-              const uint64_t ad = hd0 + (uint64_t)(t * (hs_bytes >> 4)), bd = w2d0 + (uint64_t)(slot * (w_bytes >> 4));
-              const uint32_t dcol = tmem + t * 128;
-              if (leader) {
+            }
+            if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < kChunk / 16; ++ks) mma_ss(dcol, ad + ks * 16, bd + ks * 16, id2, (j | ks) != 0);
-                tc_commit(j == NJ - 1 ? &bars.a2_full[t] : &bars.hs_free[t]);   // a2_full also says "Hs[t] is free"
-              }
+              for (int ks = 0; ks < kChunk / 16; ++ks)
+                mma_ts(tmem + t * 128, tmem + 256 + t * kChunk + ks * 8, bd + ks * 16, id2, (j | ks) != 0);
+              if (j == NJ - 1) tc_commit(&bars.a2_full[t]);
             }
             __syncwarp();
           }
@@ -297,7 +325,6 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           if (++slot == kWStages) { slot = 0; w_par ^= 1; }
         }
       }
-      (void)ks2;
       if (leader) tc_commit(&bars.done);
       __syncwarp();
       wait_all(&bars.done, 0);
@@ -307,13 +334,12 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
       const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
       const int cpr = d >> 3;                              // 16-byte chunks per row
-      uint8_t* hs_row = Hs + t * hs_bytes + (r >> 3) * ((kChunk >> 3) * 128) + (r & 7) * 16;
       uint8_t* x_warp = Xs + t * x_bytes + (size_t)(quad * 4) * cpr * 128;    // this warp's four 8-row groups of X[t]
-      uint8_t* o_warp = Hs + t * hs_bytes + quad * (hs_bytes / 4);            // this warp's slice of Hs[t]: output staging
+      uint8_t* o_warp = Os + t * x_bytes + (size_t)quad * 32 * (d * 2);       // this warp's 32 rows of the output staging
       const float inv_d = 1.f / (float)d;
       const bool swz = (cpr & (cpr - 1)) == 0;             // XOR-swizzled staging rows when cpr is a power of two
       const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
-      // stage my warp's rows of the pair `it`: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
+      // stage my warp's rows of a pair: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
       auto stage = [&](int grow_mine) {
         for (int idx = lane >> 3; idx < 4 * cpr; idx += 4) {
           const int gq = idx / cpr, c = idx - gq * cpr;
@@ -328,49 +354,57 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars.x_full[t]);
       };
-      int grow = global_row(P, bidx * kPairRows + t * kRows + r, total);
+      auto row_of = [&](int pair) {
+        const int crow = pair * kPairRows + t * kRows + r;
+        return crow < total ? P.rowmap[crow] : -1;
+      };
+      int grow = row_of(bidx);
       stage(grow);
       publish_x();
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
-        const int grow_next = it + 1 < my_pairs ? global_row(P, (bidx + (it + 1) * G) * kPairRows + t * kRows + r, total) : -1;
-        // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> shared memory (A operand of the second layer)
+        const int grow_next = it + 1 < my_pairs ? row_of(bidx + (it + 1) * G) : -1;
+        const uint32_t tA = tmem + lane_base + 256 + t * kChunk;
+        // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> back into the first 64 columns of acc1 (A operand of the
+        // second layer)
         for (int j = 0; j < NJ && ok; ++j) {
           const uint32_t kh = (uint32_t)it * NJ + j;
           ok = wait_all(&bars.a1_full[t], kh & 1);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t tA = tmem + lane_base + 256 + t * kChunk;
-          const uint4* bias = reinterpret_cast<const uint4*>(P.b1 + (size_t)j * kChunk);
+          const uint4* bias = reinterpret_cast<const uint4*>(s_b1 + (size_t)j * kChunk);
           uint32_t o[kChunk / 2];                          // the whole chunk of my row, packed bf16
 #pragma unroll
-          for (int c = 0; c < kChunk / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tA + c * 32, v);
+          for (int c2 = 0; c2 < kChunk / 64; ++c2) {
+            uint32_t v[2][32];
+            tmem_ld32(tA + c2 * 64, v[0]);
+            tmem_ld32(tA + c2 * 64 + 32, v[1]);
             tc_wait_ld();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const uint4 bb = __ldg(bias + c * 4 + q);
-              const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+            for (int cc = 0; cc < 2; ++cc) {
+              const int c = c2 * 2 + cc;
 #pragma unroll
-              for (int e = 0; e < 4; ++e)                  // round the pair to bf16, then max(h + b_1, 0) on both halves at once
-                o[c * 16 + q * 4 + e] = relu_add_bf16x2(
-                    pack_bf16x2(__uint_as_float(v[q * 8 + 2 * e]), __uint_as_float(v[q * 8 + 2 * e + 1])), bw[e]);
+              for (int q = 0; q < 4; ++q) {
+                const uint4 bb = bias[c * 4 + q];
+                const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)                // round the pair to bf16, then max(h + b_1, 0) on both halves at once
+                  o[c * 16 + q * 4 + e] = relu_add_bf16x2(
+                      pack_bf16x2(__uint_as_float(v[cc][q * 8 + 2 * e]), __uint_as_float(v[cc][q * 8 + 2 * e + 1])), bw[e]);
+              }
             }
           }
-          tc_fence_before();                               // the accumulator is in registers: hand it back
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars.a1_free[t]);
-          // Hs[t] is free once the previous chunk's second-layer product has read it (for the first chunk of a pair
-          // that was the previous pair's last product, which this warp has already waited for through a2_full)
-          if (j > 0) ok = wait_all(&bars.hs_free[t], ((uint32_t)(it * (NJ - 1) + j - 1)) & 1);
-          if (!ok) break;
 #pragma unroll
-          for (int k8 = 0; k8 < kChunk / 8; ++k8)
-            *reinterpret_cast<uint4*>(hs_row + k8 * 128) = make_uint4(o[k8 * 4], o[k8 * 4 + 1], o[k8 * 4 + 2], o[k8 * 4 + 3]);
-          fence_proxy_async_smem();
+          for (int c = 0; c < kChunk / 32; ++c) {          // every column of acc1 is in registers: overwrite it
+            uint32_t w16[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) w16[e] = o[c * 16 + e];
+            tmem_st16(tA + c * 16, w16);
+          }
+          tc_wait_st();
+          tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&bars.hs_full[t]);
+          if (lane == 0) mbar_arrive(&bars.hid_full[t]);
         }
         if (!ok) break;
         // ---- the last first-layer product has read X[t] (its a1_full arrived): keep my row of s for the residual and
@@ -387,27 +421,35 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         if (!ok) break;
         tc_fence_after();
         const uint32_t tO = tmem + lane_base + t * 128;
-        const float4* vb2 = reinterpret_cast<const float4*>(P.lnv);
-        const float4* vg = reinterpret_cast<const float4*>(P.lnv + d);
-        const float4* vbeta = reinterpret_cast<const float4*>(P.lnv + 2 * d);
+        const float4* vb2 = reinterpret_cast<const float4*>(s_lnv);
+        const float4* vg = reinterpret_cast<const float4*>(s_lnv + d);
+        const float4* vbeta = reinterpret_cast<const float4*>(s_lnv + 2 * d);
         float sum = 0.f, sq = 0.f;
 #pragma unroll
-        for (int c16 = 0; c16 < 8; ++c16) {
-          if (c16 * 16 < d) {
-            uint32_t v[16];
-            tmem_ld16(tO + c16 * 16, v);
+        for (int h = 0; h < 4; ++h) {
+          if (h * 32 < d) {
+            uint32_t v[2][16];
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+              if (h * 32 + k * 16 < d) tmem_ld16(tO + h * 32 + k * 16, v[k]);
             tc_wait_ld();
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 bb = __ldg(vb2 + c16 * 4 + q);
-              const uint4 xx = xr[c16 * 2 + (q >> 1)];
-              const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
-              const float y0 = __uint_as_float(v[q * 4 + 0]) + bb.x + bf_lo(x0);
-              const float y1 = __uint_as_float(v[q * 4 + 1]) + bb.y + bf_hi(x0);
-              const float y2 = __uint_as_float(v[q * 4 + 2]) + bb.z + bf_lo(x1);
-              const float y3 = __uint_as_float(v[q * 4 + 3]) + bb.w + bf_hi(x1);
-              sum += (y0 + y1) + (y2 + y3);
-              sq = fmaf(y0, y0, fmaf(y1, y1, fmaf(y2, y2, fmaf(y3, y3, sq))));
+            for (int k = 0; k < 2; ++k) {
+              if (h * 32 + k * 16 < d) {
+                const int c16 = h * 2 + k;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float4 bb = vb2[c16 * 4 + q];
+                  const uint4 xx = xr[c16 * 2 + (q >> 1)];
+                  const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+                  const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
+                  const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
+                  const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
+                  const float y3 = __uint_as_float(v[k][q * 4 + 3]) + bb.w + bf_hi(x1);
+                  sum += (y0 + y1) + (y2 + y3);
+                  sq = fmaf(y0, y0, fmaf(y1, y1, fmaf(y2, y2, fmaf(y3, y3, sq))));
+                }
+              }
             }
           }
         }
@@ -415,36 +457,43 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         const float mean = sum * inv_d;
         const float rstd = rsqrtf(fmaxf(sq * inv_d - mean * mean, 0.f) + P.eps);
 #pragma unroll
-        for (int c16 = 0; c16 < 8; ++c16) {
-          if (c16 * 16 < d) {
-            uint32_t v[16];
-            tmem_ld16(tO + c16 * 16, v);
+        for (int h = 0; h < 4; ++h) {
+          if (h * 32 < d) {
+            uint32_t v[2][16];
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+              if (h * 32 + k * 16 < d) tmem_ld16(tO + h * 32 + k * 16, v[k]);
             tc_wait_ld();
-            if ((c16 + 1) * 16 >= d) {                     // last read of the accumulator: hand it back
+            if ((h + 1) * 32 >= d) {                       // last read of the accumulator: hand it back
               tc_fence_before();
               __syncwarp();
               if (lane == 0) mbar_arrive(&bars.a2_free[t]);
             }
-            uint32_t o[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 bb = __ldg(vb2 + c16 * 4 + q), gg = __ldg(vg + c16 * 4 + q), be = __ldg(vbeta + c16 * 4 + q);
-              const uint4 xx = xr[c16 * 2 + (q >> 1)];
-              const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
-              const float y0 = __uint_as_float(v[q * 4 + 0]) + bb.x + bf_lo(x0);
-              const float y1 = __uint_as_float(v[q * 4 + 1]) + bb.y + bf_hi(x0);
-              const float y2 = __uint_as_float(v[q * 4 + 2]) + bb.z + bf_lo(x1);
-              const float y3 = __uint_as_float(v[q * 4 + 3]) + bb.w + bf_hi(x1);
-              const float a0 = rstd * gg.x, a1 = rstd * gg.y, a2 = rstd * gg.z, a3 = rstd * gg.w;
-              o[q * 2] = pack_bf16x2(fmaf(y0, a0, fmaf(-mean, a0, be.x)), fmaf(y1, a1, fmaf(-mean, a1, be.y)));
-              o[q * 2 + 1] = pack_bf16x2(fmaf(y2, a2, fmaf(-mean, a2, be.z)), fmaf(y3, a3, fmaf(-mean, a3, be.w)));
+            for (int k = 0; k < 2; ++k) {
+              if (h * 32 + k * 16 < d) {
+                const int c16 = h * 2 + k;
+                uint32_t o[8];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  const float4 bb = vb2[c16 * 4 + q], gg = vg[c16 * 4 + q], be = vbeta[c16 * 4 + q];
+                  const uint4 xx = xr[c16 * 2 + (q >> 1)];
+                  const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+                  const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
+                  const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
+                  const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
+                  const float y3 = __uint_as_float(v[k][q * 4 + 3]) + bb.w + bf_hi(x1);
+                  const float a0 = rstd * gg.x, a1 = rstd * gg.y, a2 = rstd * gg.z, a3 = rstd * gg.w;
+                  o[q * 2] = pack_bf16x2(fmaf(y0, a0, fmaf(-mean, a0, be.x)), fmaf(y1, a1, fmaf(-mean, a1, be.y)));
+                  o[q * 2 + 1] = pack_bf16x2(fmaf(y2, a2, fmaf(-mean, a2, be.z)), fmaf(y3, a3, fmaf(-mean, a3, be.w)));
+                }
+                const int c0 = c16 * 2, c1 = c16 * 2 + 1;   // my row of the output, staged in my slice of Os[t]
+                *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c0 ^ (lane & (cpr - 1)) : c0) << 4)) =
+                    make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c1 ^ (lane & (cpr - 1)) : c1) << 4)) =
+                    make_uint4(o[4], o[5], o[6], o[7]);
+              }
             }
-            // my row of the output, staged in my slice of Hs[t] (free: the last second-layer product is complete)
-            const int c0 = c16 * 2, c1 = c16 * 2 + 1;
-            *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c0 ^ (lane & (cpr - 1)) : c0) << 4)) =
-                make_uint4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c1 ^ (lane & (cpr - 1)) : c1) << 4)) =
-                make_uint4(o[4], o[5], o[6], o[7]);
           }
         }
         __syncwarp();
@@ -461,7 +510,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
             }
           }
         }
-        __syncwarp();                                      // the staging slice is read: the next pair's E1 may overwrite it
+        __syncwarp();                                      // the staging slice is read: the next pair may overwrite it
         grow = grow_next;
       }
       cp_async_wait_all();
@@ -569,15 +618,15 @@ int ffn_sm_count() {
   return n;
 }
 
-size_t ffn_tc_smem(int d) {
-  return (size_t)2 * kRows * d * 2 + (size_t)2 * kRows * kChunk * 2 + (size_t)kWStages * kChunk * d * 2;
+size_t ffn_tc_smem(int d, int hid) {
+  return (size_t)4 * kRows * d * 2 + (size_t)kWStages * kChunk * d * 2 + (size_t)3 * d * sizeof(float) + (size_t)hid * 2;
 }
 
 bool ffn_tc_supported(const Plan& p, int hid) {
   if (p.dtype != LASER_BF16) return false;
   if (p.d % 16 || p.d < 16 || p.d > 128) return false;
   if (hid % kChunk || hid < kChunk) return false;
-  return ffn_tc_smem(p.d) + 1024 <= 227 * 1024;   // dynamic + static shared memory of one block
+  return ffn_tc_smem(p.d, hid) + 512 <= 227 * 1024;   // dynamic + static shared memory of one block
 }
 
 template <typename T>
@@ -614,7 +663,7 @@ int ffn_simt(const Plan& p, const laser_ffn_params* f, void* H, const int32_t* l
 
 size_t ffn_scratch_bytes(const Plan& p, int hid) {
   return kAlign + align_up(((size_t)p.U + 1) * sizeof(int)) + 2 * align_up((size_t)p.d * hid * 2) +
-         align_up((size_t)3 * p.d * sizeof(float));
+         align_up((size_t)3 * p.d * sizeof(float)) + align_up((size_t)p.N * p.Lp * sizeof(int));
 }
 
 bool ffn_supported(const Plan& p, int hid) {
@@ -646,13 +695,20 @@ int ffn_forward(const Plan& p, const laser_ffn_params* f, void* H, const int32_t
   P.img1 = (bf16*)(scratch + kAlign + align_up(((size_t)p.U + 1) * sizeof(int)));
   P.img2 = (bf16*)((char*)P.img1 + align_up((size_t)p.d * hid * 2));
   P.lnv = (float*)((char*)P.img2 + align_up((size_t)p.d * hid * 2));
+  P.rowmap = (int*)((char*)P.lnv + align_up((size_t)3 * p.d * sizeof(float)));
   P.status = (int*)(ws + p.off_status);
   {
     LaunchScope ls("ffn_prep", st);
     LASER_CUDA_OK(launch_chained(ffn_prep_kernel, dim3(1 + 16), dim3(1024), 0, st, P, 1));
   }
   {
-    const size_t smem = ffn_tc_smem(p.d);
+    const long long rows_max = (long long)p.N * p.Lp;
+    const int grid = (int)(rows_max < 256LL * 4 * ffn_sm_count() ? (rows_max + 255) / 256 : 4 * ffn_sm_count());
+    LaunchScope ls("ffn_map", st);
+    LASER_CUDA_OK(launch_chained(ffn_map_kernel, dim3(grid > 0 ? grid : 1), dim3(256), 0, st, P));
+  }
+  {
+    const size_t smem = ffn_tc_smem(p.d, hid);
     LASER_CUDA_OK(cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const long long pairs_max = ((long long)p.N * p.Lp + kPairRows - 1) / kPairRows;
     const int sms = ffn_sm_count();
