@@ -373,32 +373,22 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           if (!ok) break;
           tc_fence_after();
           const uint4* bias = reinterpret_cast<const uint4*>(s_b1 + (size_t)j * kChunk);
-          uint32_t o[kChunk / 2];                          // the whole chunk of my row, packed bf16
+          // 32 accumulator columns at a time; their 16 packed columns land on accumulator columns that are already in
+          // registers (packed columns 16 c .. 16 c + 15 lie inside the 32-column batch c / 2)
 #pragma unroll
-          for (int c2 = 0; c2 < kChunk / 64; ++c2) {
-            uint32_t v[2][32];
-            tmem_ld32(tA + c2 * 64, v[0]);
-            tmem_ld32(tA + c2 * 64 + 32, v[1]);
+          for (int c = 0; c < kChunk / 32; ++c) {
+            uint32_t v[32], w16[16];
+            tmem_ld32(tA + c * 32, v);
             tc_wait_ld();
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-              const int c = c2 * 2 + cc;
+            for (int q = 0; q < 4; ++q) {
+              const uint4 bb = bias[c * 4 + q];
+              const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                const uint4 bb = bias[c * 4 + q];
-                const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)                // round the pair to bf16, then max(h + b_1, 0) on both halves at once
-                  o[c * 16 + q * 4 + e] = relu_add_bf16x2(
-                      pack_bf16x2(__uint_as_float(v[cc][q * 8 + 2 * e]), __uint_as_float(v[cc][q * 8 + 2 * e + 1])), bw[e]);
-              }
+              for (int e = 0; e < 4; ++e)                  // round the pair to bf16, then max(h + b_1, 0) on both halves at once
+                w16[q * 4 + e] = relu_add_bf16x2(
+                    pack_bf16x2(__uint_as_float(v[q * 8 + 2 * e]), __uint_as_float(v[q * 8 + 2 * e + 1])), bw[e]);
             }
-          }
-#pragma unroll
-          for (int c = 0; c < kChunk / 32; ++c) {          // every column of acc1 is in registers: overwrite it
-            uint32_t w16[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) w16[e] = o[c * 16 + e];
             tmem_st16(tA + c * 16, w16);
           }
           tc_wait_st();
@@ -409,11 +399,11 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         if (!ok) break;
         // ---- the last first-layer product has read X[t] (its a1_full arrived): keep my row of s for the residual and
         // start fetching the next pair's rows into the same place
-        uint4 xr[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          xr[i] = i < cpr ? *reinterpret_cast<const uint4*>(x_warp + ((size_t)(lane >> 3) * cpr + i) * 128 + (lane & 7) * 16)
-                          : make_uint4(0, 0, 0, 0);
+        uint8_t* o_row = o_warp + (size_t)lane * (d * 2);   // my row of the output staging; chunk c sits at slot(c)
+        auto slot_of = [&](int c) { return (swz ? c ^ (lane & (cpr - 1)) : c) << 4; };
+        for (int i = 0; i < cpr; ++i)
+          *reinterpret_cast<uint4*>(o_row + slot_of(i)) =
+              *reinterpret_cast<const uint4*>(x_warp + ((size_t)(lane >> 3) * cpr + i) * 128 + (lane & 7) * 16);
         __syncwarp();
         if (it + 1 < my_pairs) stage(grow_next);
         // ---- second layer: y = acc2 + b_2 + s, layer norm over the row
@@ -440,8 +430,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                   const float4 bb = vb2[c16 * 4 + q];
-                  const uint4 xx = xr[c16 * 2 + (q >> 1)];
-                  const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+                  const uint2 xx = *reinterpret_cast<const uint2*>(o_row + slot_of(c16 * 2 + (q >> 1)) + (q & 1) * 8);
+                  const uint32_t x0 = xx.x, x1 = xx.y;
                   const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
                   const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
                   const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
@@ -477,8 +467,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                   const float4 bb = vb2[c16 * 4 + q], gg = vg[c16 * 4 + q], be = vbeta[c16 * 4 + q];
-                  const uint4 xx = xr[c16 * 2 + (q >> 1)];
-                  const uint32_t x0 = (q & 1) ? xx.z : xx.x, x1 = (q & 1) ? xx.w : xx.y;
+                  const uint2 xx = *reinterpret_cast<const uint2*>(o_row + slot_of(c16 * 2 + (q >> 1)) + (q & 1) * 8);
+                  const uint32_t x0 = xx.x, x1 = xx.y;
                   const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
                   const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
                   const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
@@ -487,11 +477,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
                   o[q * 2] = pack_bf16x2(fmaf(y0, a0, fmaf(-mean, a0, be.x)), fmaf(y1, a1, fmaf(-mean, a1, be.y)));
                   o[q * 2 + 1] = pack_bf16x2(fmaf(y2, a2, fmaf(-mean, a2, be.z)), fmaf(y3, a3, fmaf(-mean, a3, be.w)));
                 }
-                const int c0 = c16 * 2, c1 = c16 * 2 + 1;   // my row of the output, staged in my slice of Os[t]
-                *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c0 ^ (lane & (cpr - 1)) : c0) << 4)) =
-                    make_uint4(o[0], o[1], o[2], o[3]);
-                *reinterpret_cast<uint4*>(o_warp + (size_t)lane * (d * 2) + ((swz ? c1 ^ (lane & (cpr - 1)) : c1) << 4)) =
-                    make_uint4(o[4], o[5], o[6], o[7]);
+                // the output chunks replace the residual chunks they were computed from
+                *reinterpret_cast<uint4*>(o_row + slot_of(c16 * 2)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(o_row + slot_of(c16 * 2 + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
               }
             }
           }
