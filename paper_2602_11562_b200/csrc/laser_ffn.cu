@@ -341,8 +341,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
       // stage my warp's rows of a pair: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
       auto stage = [&](int grow_mine) {
-        for (int idx = lane >> 3; idx < 4 * cpr; idx += 4) {
-          const int gq = idx / cpr, c = idx - gq * cpr;
+        int gq = 0, c = lane >> 3;
+        for (int idx = lane >> 3; idx < 4 * cpr; idx += 4, c += 4) {
+          while (c >= cpr) { c -= cpr; ++gq; }
           const int grow = __shfl_sync(0xffffffffu, grow_mine, gq * 8 + (lane & 7));
           const bf16* src = grow >= 0 ? P.H + (size_t)grow * d + c * 8 : P.H;
           cp_async16(x_warp + (size_t)idx * 128 + (lane & 7) * 16, src, grow >= 0 ? 16u : 0u);
@@ -401,6 +402,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         // start fetching the next pair's rows into the same place
         uint8_t* o_row = o_warp + (size_t)lane * (d * 2);   // my row of the output staging; chunk c sits at slot(c)
         auto slot_of = [&](int c) { return (swz ? c ^ (lane & (cpr - 1)) : c) << 4; };
+#pragma unroll 4
         for (int i = 0; i < cpr; ++i)
           *reinterpret_cast<uint4*>(o_row + slot_of(i)) =
               *reinterpret_cast<const uint4*>(x_warp + ((size_t)(lane >> 3) * cpr + i) * 128 + (lane & 7) * 16);
@@ -414,7 +416,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         const float4* vb2 = reinterpret_cast<const float4*>(s_lnv);
         const float4* vg = reinterpret_cast<const float4*>(s_lnv + d);
         const float4* vbeta = reinterpret_cast<const float4*>(s_lnv + 2 * d);
-        float sum = 0.f, sq = 0.f;
+        // pass 1: y = acc2 + b_2 + s (two features at a time with the packed fp32 instructions), written back over the
+        // accumulator; row sums of y and y^2
+        float2 sum2 = make_float2(0.f, 0.f), sq2 = make_float2(0.f, 0.f);
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
           if (h * 32 < d) {
@@ -428,24 +432,33 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
               if (h * 32 + k * 16 < d) {
                 const int c16 = h * 2 + k;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float4 bb = vb2[c16 * 4 + q];
-                  const uint2 xx = *reinterpret_cast<const uint2*>(o_row + slot_of(c16 * 2 + (q >> 1)) + (q & 1) * 8);
-                  const uint32_t x0 = xx.x, x1 = xx.y;
-                  const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
-                  const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
-                  const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
-                  const float y3 = __uint_as_float(v[k][q * 4 + 3]) + bb.w + bf_hi(x1);
-                  sum += (y0 + y1) + (y2 + y3);
-                  sq = fmaf(y0, y0, fmaf(y1, y1, fmaf(y2, y2, fmaf(y3, y3, sq))));
+                for (int q = 0; q < 2; ++q) {                // 8 features: one 16-byte chunk of the residual
+                  const uint4 xx = *reinterpret_cast<const uint4*>(o_row + slot_of(c16 * 2 + q));
+                  const float4 b0 = vb2[c16 * 4 + q * 2], b1 = vb2[c16 * 4 + q * 2 + 1];
+                  const uint32_t xw[4] = {xx.x, xx.y, xx.z, xx.w};
+                  const float2 bb[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y),
+                                        make_float2(b1.z, b1.w)};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float2 acc = make_float2(__uint_as_float(v[k][q * 8 + 2 * e]), __uint_as_float(v[k][q * 8 + 2 * e + 1]));
+                    const float2 y = __fadd2_rn(__fadd2_rn(acc, bb[e]), make_float2(bf_lo(xw[e]), bf_hi(xw[e])));
+                    sum2 = __fadd2_rn(sum2, y);
+                    sq2 = __ffma2_rn(y, y, sq2);
+                    v[k][q * 8 + 2 * e] = __float_as_uint(y.x);
+                    v[k][q * 8 + 2 * e + 1] = __float_as_uint(y.y);
+                  }
                 }
+                tmem_st16(tO + c16 * 16, v[k]);
               }
             }
           }
         }
+        tc_wait_st();
         if (it + 1 < my_pairs) publish_x();                // the next pair's rows have landed by now
-        const float mean = sum * inv_d;
-        const float rstd = rsqrtf(fmaxf(sq * inv_d - mean * mean, 0.f) + P.eps);
+        const float mean = (sum2.x + sum2.y) * inv_d;
+        const float rstd = rsqrtf(fmaxf((sq2.x + sq2.y) * inv_d - mean * mean, 0.f) + P.eps);
+        const float2 rstd2 = make_float2(rstd, rstd), shift2 = make_float2(-mean * rstd, -mean * rstd);
+        // pass 2: ((y - mean) rstd) gain + shift -> bf16 -> my row of the output staging
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
           if (h * 32 < d) {
@@ -463,23 +476,23 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
             for (int k = 0; k < 2; ++k) {
               if (h * 32 + k * 16 < d) {
                 const int c16 = h * 2 + k;
-                uint32_t o[8];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float4 bb = vb2[c16 * 4 + q], gg = vg[c16 * 4 + q], be = vbeta[c16 * 4 + q];
-                  const uint2 xx = *reinterpret_cast<const uint2*>(o_row + slot_of(c16 * 2 + (q >> 1)) + (q & 1) * 8);
-                  const uint32_t x0 = xx.x, x1 = xx.y;
-                  const float y0 = __uint_as_float(v[k][q * 4 + 0]) + bb.x + bf_lo(x0);
-                  const float y1 = __uint_as_float(v[k][q * 4 + 1]) + bb.y + bf_hi(x0);
-                  const float y2 = __uint_as_float(v[k][q * 4 + 2]) + bb.z + bf_lo(x1);
-                  const float y3 = __uint_as_float(v[k][q * 4 + 3]) + bb.w + bf_hi(x1);
-                  const float a0 = rstd * gg.x, a1 = rstd * gg.y, a2 = rstd * gg.z, a3 = rstd * gg.w;
-                  o[q * 2] = pack_bf16x2(fmaf(y0, a0, fmaf(-mean, a0, be.x)), fmaf(y1, a1, fmaf(-mean, a1, be.y)));
-                  o[q * 2 + 1] = pack_bf16x2(fmaf(y2, a2, fmaf(-mean, a2, be.z)), fmaf(y3, a3, fmaf(-mean, a3, be.w)));
+                for (int q = 0; q < 2; ++q) {
+                  const float4 g0 = vg[c16 * 4 + q * 2], g1 = vg[c16 * 4 + q * 2 + 1];
+                  const float4 e0 = vbeta[c16 * 4 + q * 2], e1 = vbeta[c16 * 4 + q * 2 + 1];
+                  const float2 gg[4] = {make_float2(g0.x, g0.y), make_float2(g0.z, g0.w), make_float2(g1.x, g1.y),
+                                        make_float2(g1.z, g1.w)};
+                  const float2 be[4] = {make_float2(e0.x, e0.y), make_float2(e0.z, e0.w), make_float2(e1.x, e1.y),
+                                        make_float2(e1.z, e1.w)};
+                  uint32_t o[4];
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float2 y = make_float2(__uint_as_float(v[k][q * 8 + 2 * e]), __uint_as_float(v[k][q * 8 + 2 * e + 1]));
+                    const float2 r2 = __ffma2_rn(__ffma2_rn(y, rstd2, shift2), gg[e], be[e]);
+                    o[e] = pack_bf16x2(r2.x, r2.y);
+                  }
+                  *reinterpret_cast<uint4*>(o_row + slot_of(c16 * 2 + q)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
-                // the output chunks replace the residual chunks they were computed from
-                *reinterpret_cast<uint4*>(o_row + slot_of(c16 * 2)) = make_uint4(o[0], o[1], o[2], o[3]);
-                *reinterpret_cast<uint4*>(o_row + slot_of(c16 * 2 + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
               }
             }
           }
@@ -488,6 +501,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         // coalesced write-back: cpr consecutive lanes write one row, 32 / cpr rows per instruction
         {
           const int rr0 = lane / cpr, cc = lane - rr0 * cpr;
+#pragma unroll 4
           for (int base = 0; base < 32; base += rows_per) {
             const int rr = base + rr0;
             const int g_row = __shfl_sync(0xffffffffu, grow, rr & 31);
