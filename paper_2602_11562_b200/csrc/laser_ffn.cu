@@ -189,9 +189,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int d = P.d, NJ = P.NJ;
   const uint32_t x_bytes = kRows * d * 2, w_bytes = kChunk * d * 2;
-  uint8_t* Xs = smem_raw;                              // [2][128 x d]       K-major, K = d
-  uint8_t* Os = Xs + 2 * x_bytes;                      // [2][128 x d]       output rows on their way to global memory
-  uint8_t* Ws = Os + 2 * x_bytes;                      // [kWStages][128 d]  one weight chunk each
+  uint8_t* Xs = smem_raw;                              // [2 pairs][2 tiles][128 x d]  K-major, K = d; pair p in buffer p & 1
+  uint8_t* Ws = Xs + 4 * x_bytes;                      // [kWStages][128 d]  one weight chunk each
   float* s_lnv = reinterpret_cast<float*>(Ws + kWStages * w_bytes);        // [3][d] b_2, gain, shift
   bf16* s_b1 = reinterpret_cast<bf16*>(s_lnv + 3 * d);                      // [hid]
 
@@ -291,7 +290,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
             const uint64_t bd = w1d0 + (uint64_t)(slot * (w_bytes >> 4));
             if (leader) {
               for (int t = 0; t < 2; ++t) {
-                const uint64_t ad = xd0 + (uint64_t)(t * (x_bytes >> 4));
+                const uint64_t ad = xd0 + (uint64_t)((2 * (it & 1) + t) * (x_bytes >> 4));
                 for (int ks = 0; ks < ks1; ++ks) mma_ss(tmem + 256 + t * kChunk, ad + ks * 16, bd + ks * 16, id1, ks > 0);
                 tc_commit(&bars.a1_full[t]);
               }
@@ -334,19 +333,23 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
       const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
       const int cpr = d >> 3;                              // 16-byte chunks per row
-      uint8_t* x_warp = Xs + t * x_bytes + (size_t)(quad * 4) * cpr * 128;    // this warp's four 8-row groups of X[t]
-      uint8_t* o_warp = Os + t * x_bytes + (size_t)quad * 32 * (d * 2);       // this warp's 32 rows of the output staging
+      // this warp's four 8-row groups of X[t] in buffer b: 32 rows, first K-major (staged rows, read by the first
+      // layer and for the residual), at the end of the pair row-major (output rows on their way to global memory)
+      auto x_slice = [&](int b) { return Xs + (size_t)(2 * b + t) * x_bytes + (size_t)(quad * 4) * cpr * 128; };
       const float inv_d = 1.f / (float)d;
       const bool swz = (cpr & (cpr - 1)) == 0;             // XOR-swizzled staging rows when cpr is a power of two
       const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
       // stage my warp's rows of a pair: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
-      auto stage = [&](int grow_mine) {
-        int gq = 0, c = lane >> 3;
-        for (int idx = lane >> 3; idx < 4 * cpr; idx += 4, c += 4) {
+      // pieces [i0, i1) of the cpr this lane copies for one pair: piece i is (group, chunk) number (lane >> 3) + 4 i of
+      // row-in-group lane & 7
+      auto stage = [&](int grow_mine, uint8_t* xw, int i0, int i1) {
+        int idx = (lane >> 3) + 4 * i0;
+        int gq = idx / cpr, c = idx - gq * cpr;
+        for (int i = i0; i < i1; ++i, idx += 4, c += 4) {
           while (c >= cpr) { c -= cpr; ++gq; }
           const int grow = __shfl_sync(0xffffffffu, grow_mine, gq * 8 + (lane & 7));
           const bf16* src = grow >= 0 ? P.H + (size_t)grow * d + c * 8 : P.H;
-          cp_async16(x_warp + (size_t)idx * 128 + (lane & 7) * 16, src, grow >= 0 ? 16u : 0u);
+          cp_async16(xw + (size_t)idx * 128 + (lane & 7) * 16, src, grow >= 0 ? 16u : 0u);
         }
       };
       auto publish_x = [&]() {                             // my copies have landed: tell the issuer
@@ -360,16 +363,21 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         return crow < total ? P.rowmap[crow] : -1;
       };
       int grow = row_of(bidx);
-      stage(grow);
+      stage(grow, x_slice(0), 0, cpr);
       publish_x();
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
         const int grow_next = it + 1 < my_pairs ? row_of(bidx + (it + 1) * G) : -1;
         const uint32_t tA = tmem + lane_base + 256 + t * kChunk;
+        uint8_t* x_warp = x_slice(it & 1);
+        uint8_t* x_next = x_slice((it + 1) & 1);
         // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> back into the first 64 columns of acc1 (A operand of the
         // second layer)
         for (int j = 0; j < NJ && ok; ++j) {
           const uint32_t kh = (uint32_t)it * NJ + j;
+          // a share of the next pair's rows goes on its way while this chunk's first-layer product runs (the other
+          // buffer: its pair is written back)
+          if (it + 1 < my_pairs) stage(grow_next, x_next, (j * cpr) / NJ, ((j + 1) * cpr) / NJ);
           ok = wait_all(&bars.a1_full[t], kh & 1);
           if (!ok) break;
           tc_fence_after();
@@ -398,16 +406,10 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           if (lane == 0) mbar_arrive(&bars.hid_full[t]);
         }
         if (!ok) break;
-        // ---- the last first-layer product has read X[t] (its a1_full arrived): keep my row of s for the residual and
-        // start fetching the next pair's rows into the same place
-        uint8_t* o_row = o_warp + (size_t)lane * (d * 2);   // my row of the output staging; chunk c sits at slot(c)
+        if (it + 1 < my_pairs) publish_x();                // the next pair's rows are staged
+        uint8_t* o_row = x_warp + (size_t)lane * (d * 2);   // my row of the output staging; chunk c sits at slot(c)
         auto slot_of = [&](int c) { return (swz ? c ^ (lane & (cpr - 1)) : c) << 4; };
-#pragma unroll 4
-        for (int i = 0; i < cpr; ++i)
-          *reinterpret_cast<uint4*>(o_row + slot_of(i)) =
-              *reinterpret_cast<const uint4*>(x_warp + ((size_t)(lane >> 3) * cpr + i) * 128 + (lane & 7) * 16);
-        __syncwarp();
-        if (it + 1 < my_pairs) stage(grow_next);
+        const uint8_t* x_row = x_warp + (size_t)(lane >> 3) * cpr * 128 + (lane & 7) * 16;   // my staged row: chunk c at + 128 c
         // ---- second layer: y = acc2 + b_2 + s, layer norm over the row
         ok = wait_all(&bars.a2_full[t], it & 1);
         if (!ok) break;
@@ -433,7 +435,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
                 const int c16 = h * 2 + k;
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {                // 8 features: one 16-byte chunk of the residual
-                  const uint4 xx = *reinterpret_cast<const uint4*>(o_row + slot_of(c16 * 2 + q));
+                  const uint4 xx = *reinterpret_cast<const uint4*>(x_row + (c16 * 2 + q) * 128);
                   const float4 b0 = vb2[c16 * 4 + q * 2], b1 = vb2[c16 * 4 + q * 2 + 1];
                   const uint32_t xw[4] = {xx.x, xx.y, xx.z, xx.w};
                   const float2 bb[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y),
@@ -454,7 +456,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           }
         }
         tc_wait_st();
-        if (it + 1 < my_pairs) publish_x();                // the next pair's rows have landed by now
+        __syncwarp();                                      // every lane has read its residual: the slice becomes output staging
         const float mean = (sum2.x + sum2.y) * inv_d;
         const float rstd = rsqrtf(fmaxf((sq2.x + sq2.y) * inv_d - mean * mean, 0.f) + P.eps);
         const float2 rstd2 = make_float2(rstd, rstd), shift2 = make_float2(-mean * rstd, -mean * rstd);
@@ -507,12 +509,12 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
             const int g_row = __shfl_sync(0xffffffffu, grow, rr & 31);
             if (rr0 < rows_per && rr < 32 && g_row >= 0) {
               const uint4 val = *reinterpret_cast<const uint4*>(
-                  o_warp + (size_t)rr * (d * 2) + ((swz ? cc ^ (rr & (cpr - 1)) : cc) << 4));
+                  x_warp + (size_t)rr * (d * 2) + ((swz ? cc ^ (rr & (cpr - 1)) : cc) << 4));
               *reinterpret_cast<uint4*>(P.H + (size_t)g_row * d + cc * 8) = val;
             }
           }
         }
-        __syncwarp();                                      // the staging slice is read: the next pair may overwrite it
+        __syncwarp();                                      // the slice is read: the pair after the next may be staged into it
         grow = grow_next;
       }
       cp_async_wait_all();
