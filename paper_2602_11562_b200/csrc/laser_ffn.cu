@@ -22,8 +22,8 @@ using namespace ptx;
 constexpr int kRows = 128;            // rows per tile = MMA M = TMEM lanes
 constexpr int kChunk = 128;           // hidden units per step
 constexpr int kPairRows = 2 * kRows;  // two tiles share every weight chunk
-constexpr int kFfnThreads = 320;      // warp 0 weight producer + TMEM, warp 1 MMA issuer,
-                                      // warps 2-5 / 6-9 epilogue warpgroups of tile 0 / tile 1
+constexpr int kFfnThreads = 576;      // warp 0 weight producer + TMEM, warp 1 MMA issuer, warps 2-5 / 6-9 hidden-
+                                      // activation warpgroups of tile 0 / 1, warps 10-13 / 14-17 layer-norm warpgroups
 constexpr int kWStages = 3;
 constexpr int kFfnTmemCols = 512;     // acc2[t] at 128 t; acc1[t], then the hidden activations, at 256 + 128 t
 constexpr int kSimtRows = 8;
@@ -152,7 +152,8 @@ __global__ void __launch_bounds__(256) ffn_map_kernel(FfnParams P) {
 // ------------------------------------------------------------------------------------------------------- tensor kernel
 struct FfnBars {
   uint64_t w_full[kWStages], w_empty[kWStages];
-  uint64_t x_full[2];                   // X[t] staged (4 epilogue warps)
+  uint64_t x_full[2];                   // X[t] staged (4 hidden-activation warps)
+  uint64_t x_free[2];                   // X[t] of a finished pair written back (4 layer-norm warps)
   uint64_t a1_full[2];                  // first-layer product of tile t complete
   uint64_t hid_full[2];                 // hidden activations of tile t written to TMEM (4 epilogue warps)
   uint64_t a2_full[2], a2_free[2];      // second-layer accumulator of tile t complete / drained (4 epilogue warps)
@@ -198,6 +199,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
     for (int i = 0; i < kWStages; ++i) { mbar_init(&bars.w_full[i], 1); mbar_init(&bars.w_empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.x_full[i], 4);
+      mbar_init(&bars.x_free[i], 4);
       mbar_init(&bars.a1_full[i], 1);
       mbar_init(&bars.hid_full[i], 4);
       mbar_init(&bars.a2_full[i], 1);
@@ -327,19 +329,14 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
       if (leader) tc_commit(&bars.done);
       __syncwarp();
       wait_all(&bars.done, 0);
-    } else {
-      // ------------------------------------------------------------------ epilogue warp: rows 32 quad .. + 31 of tile t
+    } else if (warp < 10) {
+      // ------------------------------------------------------------------ hidden-activation warp: rows 32 quad .. + 31 of tile t
       const int t = (warp - 2) >> 2, quad = warp & 3;
       const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
       const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
       const int cpr = d >> 3;                              // 16-byte chunks per row
-      // this warp's four 8-row groups of X[t] in buffer b: 32 rows, first K-major (staged rows, read by the first
-      // layer and for the residual), at the end of the pair row-major (output rows on their way to global memory)
+      // this warp's four 8-row groups of X[t] in buffer b (32 rows, K-major)
       auto x_slice = [&](int b) { return Xs + (size_t)(2 * b + t) * x_bytes + (size_t)(quad * 4) * cpr * 128; };
-      const float inv_d = 1.f / (float)d;
-      const bool swz = (cpr & (cpr - 1)) == 0;             // XOR-swizzled staging rows when cpr is a power of two
-      const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
-      // stage my warp's rows of a pair: lane l copies pieces (group, chunk) = (l >> 3) + 4 i of row-in-group l & 7
       // pieces [i0, i1) of the cpr this lane copies for one pair: piece i is (group, chunk) number (lane >> 3) + 4 i of
       // row-in-group lane & 7
       auto stage = [&](int grow_mine, uint8_t* xw, int i0, int i1) {
@@ -362,22 +359,25 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         const int crow = pair * kPairRows + t * kRows + r;
         return crow < total ? P.rowmap[crow] : -1;
       };
-      int grow = row_of(bidx);
-      stage(grow, x_slice(0), 0, cpr);
+      stage(row_of(bidx), x_slice(0), 0, cpr);
       publish_x();
+      const int j_stage0 = NJ / 2;
       bool ok = true;
       for (int it = 0; it < my_pairs && ok; ++it) {
         const int grow_next = it + 1 < my_pairs ? row_of(bidx + (it + 1) * G) : -1;
         const uint32_t tA = tmem + lane_base + 256 + t * kChunk;
-        uint8_t* x_warp = x_slice(it & 1);
         uint8_t* x_next = x_slice((it + 1) & 1);
         // ---- first layer: acc1 -> + b_1, ReLU, bf16 -> back into the first 64 columns of acc1 (A operand of the
         // second layer)
         for (int j = 0; j < NJ && ok; ++j) {
           const uint32_t kh = (uint32_t)it * NJ + j;
-          // a share of the next pair's rows goes on its way while this chunk's first-layer product runs (the other
-          // buffer: its pair is written back)
-          if (it + 1 < my_pairs) stage(grow_next, x_next, (j * cpr) / NJ, ((j + 1) * cpr) / NJ);
+          // in the later chunks a share of the next pair's rows goes on its way while the first-layer product runs
+          if (it + 1 < my_pairs && j >= j_stage0) {
+            // (the other buffer: the layer-norm warps must have written its pair back)
+            if (j == j_stage0 && it > 0) ok = wait_all(&bars.x_free[t], (it - 1) & 1);
+            if (!ok) break;
+            stage(grow_next, x_next, ((j - j_stage0) * cpr) / (NJ - j_stage0), ((j - j_stage0 + 1) * cpr) / (NJ - j_stage0));
+          }
           ok = wait_all(&bars.a1_full[t], kh & 1);
           if (!ok) break;
           tc_fence_after();
@@ -407,6 +407,23 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
         }
         if (!ok) break;
         if (it + 1 < my_pairs) publish_x();                // the next pair's rows are staged
+      }
+      cp_async_wait_all();
+    } else {
+      // ------------------------------------------------------------------ layer-norm warp: rows 32 quad .. + 31 of tile t
+      const int t = (warp - 10) >> 2, quad = warp & 3;
+      const int r = quad * 32 + lane;                      // my row of the tile = my TMEM lane
+      const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+      const int cpr = d >> 3;                              // 16-byte chunks per row
+      const float inv_d = 1.f / (float)d;
+      const bool swz = (cpr & (cpr - 1)) == 0;             // XOR-swizzled staging rows when cpr is a power of two
+      const int rows_per = 32 / cpr;                       // rows covered by one coalesced store instruction
+      bool ok = true;
+      for (int it = 0; it < my_pairs && ok; ++it) {
+        const int crow = (bidx + it * G) * kPairRows + t * kRows + r;
+        const int grow = crow < total ? P.rowmap[crow] : -1;
+        // this warp's 32 rows of X[t]: K-major as staged (read for the residual), then row-major output staging
+        uint8_t* x_warp = Xs + (size_t)(2 * (it & 1) + t) * x_bytes + (size_t)(quad * 4) * cpr * 128;
         uint8_t* o_row = x_warp + (size_t)lane * (d * 2);   // my row of the output staging; chunk c sits at slot(c)
         auto slot_of = [&](int c) { return (swz ? c ^ (lane & (cpr - 1)) : c) << 4; };
         const uint8_t* x_row = x_warp + (size_t)(lane >> 3) * cpr * 128 + (lane & 7) * 16;   // my staged row: chunk c at + 128 c
@@ -515,9 +532,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) ffn_tc_kernel(FfnParams P) {
           }
         }
         __syncwarp();                                      // the slice is read: the pair after the next may be staged into it
-        grow = grow_next;
+        if (lane == 0) mbar_arrive(&bars.x_free[t]);
       }
-      cp_async_wait_all();
     }
   }
 
