@@ -1,15 +1,23 @@
 // Feed-forward refinement of the segment vectors (Eq. 6):  s <- LN(max(s W_1 + b_1, 0) W_2 + b_2 + s), applied in place
 // to the rows of H' that belong to non-empty segments.
 //
-//   ffn_prep_kernel   prefix of the valid rows per user (the "compact" row numbering the main kernel tiles over) and the
-//                     weights re-laid as MMA operand images, one 128-hidden-unit chunk after the other.
-//   ffn_tc_kernel     bf16, tcgen05: a persistent block owns pairs of 128-row tiles.  Per pair and per chunk j of 128
-//                     hidden units:   acc1 = X W_1[:, j]  (TMEM)  ->  registers: + b_1, ReLU, bf16  ->  shared memory
-//                     ->  acc2 += hidden_j W_2[j, :]  (TMEM).  The hidden activations never leave the SM; the weights
-//                     stream through a three-slot ring of bulk copies (from L2) and are shared by both tiles of the pair.
-//                     The last step adds b_2 and the residual, normalises each row (one thread owns one row of the
-//                     accumulator) and writes bf16.
+//   ffn_prep_kernel   prefix of the valid rows per user (the "compact" row numbering the main kernel tiles over), the
+//                     weights re-laid as MMA operand images (one 128-hidden-unit chunk after the other) and fp32 copies
+//                     of b_2 and of the layer norm's gain and shift.
+//   ffn_map_kernel    compact row -> row of H' for every valid row, so that the main kernel finds its rows with one
+//                     coalesced load.
+//   ffn_tc_kernel     bf16, tcgen05: a persistent block (one per SM) owns pairs of 128-row tiles.  Per pair and per chunk
+//                     j of 128 hidden units:  acc1 = X W_1[:, j] (shared-memory operands, TMEM accumulator)  ->  + b_1,
+//                     ReLU, bf16 in registers, written back over acc1  ->  acc2 += hidden_j W_2[j, :] with the hidden
+//                     activations read straight from TMEM.  Nothing of the hidden layer ever leaves the SM; the weights
+//                     stream through a three-slot ring of bulk copies (they stay in L2) and both tiles of the pair share
+//                     every chunk.  At the end of a pair the layer-norm warps add b_2 and the residual, normalise each row
+//                     (one thread owns one row of the accumulator) and write bf16 rows back, while the other warps are
+//                     already busy with the next pair.
 //   ffn_simt_kernel   FP32-ALU version for fp32 data and for shapes outside the tensor kernel's envelope.
+//
+// Roofline: 4 d d_hidden flops per valid row on the tensor cores (the H' rows themselves are read and written once,
+// 4 d bytes per row, far below the HBM bound at d_hidden = 4 d).
 #include "laser_common.cuh"
 #include "laser_ptx.cuh"
 
