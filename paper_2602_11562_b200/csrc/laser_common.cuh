@@ -73,7 +73,8 @@ int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const
 
 // Fused warp-MMA GSTA kernel for bf16 (laser_gsta.cu); needs gsta_mma_image_bytes(p) of scratch at off_gimg.
 bool gsta_mma_supported(const Plan& p);
-size_t gsta_mma_image_bytes(const Plan& p);
+size_t gsta_mma_image_bytes(const Plan& p);   // weight images, then the per-candidate segment counts
+size_t gsta_nseg_offset(const Plan& p);       // byte offset of the segment counts inside that scratch
 // images_ready: the weight images at off_gimg were already built for these weights earlier on the same stream.
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
              const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready);

@@ -37,6 +37,7 @@ struct GstaParams {
   const bf16 *Hp, *cands, *Wg;
   const int *lengths, *cand_offsets;
   uint4* img;                  // [M][3][d/16 k-tiles][d/16 column pairs][32 lanes]
+  int* nseg;                   // [N] non-empty segments per candidate (built with the images)
   bf16* z;
   int* status;
 };
@@ -45,6 +46,8 @@ __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
   chain_wait();
   chain_release();
   gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+  gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.nseg,
+                  blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
 }
 
 template <int D16>
@@ -66,29 +69,15 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   chain_wait();
   chain_release();
 
-  // ---- set-up: candidate -> user -> number of non-empty segments; T = candidates; zero row
-  if (tid < kGT) {
-    const int c = c_base + tid;
-    int nv = 0;
-    if (c < P.N) {
-      if (P.cand_offsets[0] > c || P.cand_offsets[P.U] <= c) {
-        report_status(P.status, LASER_ERR_BAD_INPUT);
-      } else {
-        int lo = 0, hi = P.U;   // cand_offsets[lo] <= c < cand_offsets[hi]
-        while (hi - lo > 1) {
-          const int mid = (lo + hi) >> 1;
-          if (P.cand_offsets[mid] <= c) lo = mid; else hi = mid;
-        }
-        const int len = P.lengths[lo];
-        if (len < 0 || len > P.L) report_status(P.status, LASER_ERR_BAD_INPUT);
-        else nv = min((len + P.S - 1) / P.S, P.Lp);
-      }
-    }
-    nv_s[tid] = nv;
-  }
-  for (int i = tid; i < kGT * d; i += kGThreads) {
-    const int r = i / d, c = i - r * d;
-    Ts[r * TS + c] = c_base + r < P.N ? __bfloat162float(P.cands[(size_t)(c_base + r) * d + c]) : 0.f;
+  // ---- set-up: number of non-empty segments per candidate (from the set-up kernel's map); T = candidates; zero row
+  if (tid < kGT) nv_s[tid] = (P.M > 0 && c_base + tid < P.N) ? min(max(P.nseg[c_base + tid], 0), P.Lp) : 0;
+  for (int i = tid; i < kGT * (d / 8); i += kGThreads) {     // 8 features (16 bytes) at a time
+    const int r = i / (d / 8), c8 = (i - r * (d / 8)) * 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (c_base + r < P.N) v = *reinterpret_cast<const uint4*>(P.cands + (size_t)(c_base + r) * d + c8);
+    float* dst = Ts + r * TS + c8;
+    dst[0] = bf16_lo(v.x); dst[1] = bf16_hi(v.x); dst[2] = bf16_lo(v.y); dst[3] = bf16_hi(v.y);
+    dst[4] = bf16_lo(v.z); dst[5] = bf16_hi(v.z); dst[6] = bf16_lo(v.w); dst[7] = bf16_hi(v.w);
   }
   for (int i = tid; i < RS / 4; i += kGThreads) reinterpret_cast<uint32_t*>(zrow)[i] = 0u;
   __syncthreads();
@@ -344,7 +333,8 @@ bool gsta_mma_supported(const Plan& p) {
   return true;
 }
 
-size_t gsta_mma_image_bytes(const Plan& p) { return (size_t)p.M * 3 * p.d * p.d * 2; }
+size_t gsta_nseg_offset(const Plan& p) { return align_up((size_t)p.M * 3 * p.d * p.d * 2); }
+size_t gsta_mma_image_bytes(const Plan& p) { return gsta_nseg_offset(p) + (size_t)p.N * sizeof(int); }
 
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
              const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready) {
@@ -355,6 +345,7 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   P.Hp = (const bf16*)Hprime; P.cands = (const bf16*)cands; P.Wg = (const bf16*)Wg;
   P.lengths = lengths; P.cand_offsets = cand_offsets;
   P.img = reinterpret_cast<uint4*>(ws + p.off_gimg);
+  P.nseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.z = (bf16*)z;
   P.status = reinterpret_cast<int*>(ws + p.off_status);
   if (p.M > 0 && !images_ready) {

@@ -9,6 +9,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include "laser.h"
+
 namespace laser {
 
 // Called by `n_workers` threads with ranks worker = 0 .. n_workers - 1; img has M * 3 * (d/16)^2 * 32 entries.
@@ -36,6 +38,29 @@ __device__ __forceinline__ void gsta_build_images(const __nv_bfloat16* Wg, uint4
       v[q] = lo | (hi << 16);
     }
     img[i] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+}
+
+// Per candidate: the number of non-empty segments of its user (what the GSTA kernel's softmax runs over), so that the
+// kernel's blocks need no search through the candidate offsets.  A candidate outside every user's range or a length
+// outside [0, L] is reported through `status` and gets 0 segments.
+__device__ __forceinline__ void gsta_build_nseg(const int* lengths, const int* cand_offsets, int U, int N, int L, int S,
+                                                int Lp, int* status, int* nseg, int worker, int n_workers) {
+  for (int c = worker; c < N; c += n_workers) {
+    int nv = 0;
+    if (cand_offsets[0] > c || cand_offsets[U] <= c) {
+      atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
+    } else {
+      int lo = 0, hi = U;   // cand_offsets[lo] <= c < cand_offsets[hi]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (cand_offsets[mid] <= c) lo = mid; else hi = mid;
+      }
+      const int len = lengths[lo];
+      if (len < 0 || len > L) atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
+      else nv = min((len + S - 1) / S, Lp);
+    }
+    nseg[c] = nv;
   }
 }
 

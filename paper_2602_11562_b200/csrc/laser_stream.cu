@@ -47,6 +47,7 @@ struct StreamParams {
   int zero_empty;                 // write zero rows for segments without valid items
   const bf16* Wg;                 // GSTA weights whose images the pre kernel also builds (null: none)
   uint4* gimg;
+  int* gnseg;                     // per-candidate segment counts for the GSTA kernel (built with the images)
   int M;
   int* status;
 };
@@ -92,9 +93,13 @@ __global__ void __launch_bounds__(kPreWarps * 32) stream_pre_kernel(StreamParams
   }
   // users 16 wg + g (MMA rows g) and 16 wg + g + 8 (rows g + 8); a user without a candidate is a zero row
   const int uA = wg * 16 + g, uB = uA + 8;
-  int len = 0;
-  const int cA = uA < P.U ? user_candidate(P, uA, &len) : -1;
-  const int cB = uB < P.U ? user_candidate(P, uB, &len) : -1;
+  int lenA = 0, lenB = 0;
+  const int cA = uA < P.U ? user_candidate(P, uA, &lenA) : -1;
+  const int cB = uB < P.U ? user_candidate(P, uB, &lenB) : -1;
+  if (P.Wg && t == 0) {                                  // segment counts of these users' candidates for the GSTA kernel
+    if (cA >= 0) P.gnseg[cA] = min((lenA + P.S - 1) / P.S, P.Lp);
+    if (cB >= 0) P.gnseg[cB] = min((lenB + P.S - 1) / P.S, P.Lp);
+  }
   uint32_t ta[D16][4];                                   // A fragments of T (bf16, exact)
 #pragma unroll
   for (int kt = 0; kt < D16; ++kt) {
@@ -376,6 +381,7 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   StreamParams P;
   P.Wg = (const bf16*)Wg_images;
   P.gimg = reinterpret_cast<uint4*>(ws + p.off_gimg);
+  P.gnseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.M = p.M;
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.inv_gamma = p.inv_gamma;

@@ -46,6 +46,7 @@ struct TcParams {
   int sta_grid, proj_grid;
   const bf16* Wg;                     // GSTA weights whose images this set-up also builds (null: none)
   uint4* gimg;
+  int* gnseg;                         // per-candidate segment counts for the GSTA kernel (built with the images)
   int M;
   bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
   int* status;
@@ -181,7 +182,10 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     const int k = i / kCandTile, j = i - k * kCandTile;
     P.imgV[canon_off(j, k, P.d)] = j < P.d ? P.Wv[(size_t)k * P.d + j] : __float2bfloat16_rn(0.f);
   }
-  if (P.Wg) gsta_build_images(P.Wg, P.gimg, P.d, P.M, g, nthreads);
+  if (P.Wg) {
+    gsta_build_images(P.Wg, P.gimg, P.d, P.M, g, nthreads);
+    gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.gnseg, g, nthreads);
+  }
 }
 
 // H' rows of segments without valid items are zero rows (only needed when the caller wants H').
@@ -946,6 +950,7 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   TcParams P = make_params(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws);
   P.Wg = (const bf16*)Wg_images;
   P.gimg = reinterpret_cast<uint4*>(ws + p.off_gimg);
+  P.gnseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.M = p.M;
   const int sms = sm_count();
   {
