@@ -69,6 +69,17 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   chain_wait();
   chain_release();
 
+  // Dense phases (A, B, D): warp p < d / 16 owns the 16 output columns 16 p .. 16 p + 15.  Its weight fragments come
+  // straight from L2; those of the next dense phase are requested before the block-wide barrier that precedes it, so the
+  // round trip overlaps the barrier and the stores around it.
+  static_assert(D16 <= kGW, "one column pair per warp");
+  const bool dense = warp < D16;
+  uint4 wpre[D16];
+  if (dense && P.M > 0) {
+#pragma unroll
+    for (int kt = 0; kt < D16; ++kt) wpre[kt] = __ldg(P.img + (kt * D16 + warp) * 32 + lane);
+  }
+
   // ---- set-up: number of non-empty segments per candidate (from the set-up kernel's map); T = candidates; zero row
   if (tid < kGT) nv_s[tid] = (P.M > 0 && c_base + tid < P.N) ? min(max(P.nseg[c_base + tid], 0), P.Lp) : 0;
   for (int i = tid; i < kGT * (d / 8); i += kGThreads) {     // 8 features (16 bytes) at a time
@@ -133,7 +144,6 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   const uint32_t ldsm_kc = lane >> 4;                             // 16-byte k-chunk supplied by this lane
 
   for (int l = 0; l < P.M; ++l) {
-    const uint4* imgq = P.img + (size_t)(l * 3 + 0) * D16 * D16 * 32;
     const uint4* imgk = P.img + (size_t)(l * 3 + 1) * D16 * D16 * 32;
     const uint4* imgv = P.img + (size_t)(l * 3 + 2) * D16 * D16 * 32;
 
@@ -151,14 +161,16 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
         ta[kt][2] = pack2(x2.x, x2.y);
         ta[kt][3] = pack2(x3.x, x3.y);
       }
-      for (int p = warp; p < D16; p += kGW) {
+      if (dense) {
+        const int p = warp;
         float acc[2][4] = {};
 #pragma unroll
         for (int kt = 0; kt < D16; ++kt) {
-          const uint4 b = __ldg(imgq + (kt * D16 + p) * 32 + lane);
-          mma16816(acc[0], ta[kt][0], ta[kt][1], ta[kt][2], ta[kt][3], b.x, b.y);
-          mma16816(acc[1], ta[kt][0], ta[kt][1], ta[kt][2], ta[kt][3], b.z, b.w);
+          mma16816(acc[0], ta[kt][0], ta[kt][1], ta[kt][2], ta[kt][3], wpre[kt].x, wpre[kt].y);
+          mma16816(acc[1], ta[kt][0], ta[kt][1], ta[kt][2], ta[kt][3], wpre[kt].z, wpre[kt].w);
         }
+#pragma unroll
+        for (int kt = 0; kt < D16; ++kt) wpre[kt] = __ldg(imgk + (kt * D16 + p) * 32 + lane);   // for phase B
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
           const int col = p * 16 + nt * 8 + 2 * t;
@@ -174,11 +186,12 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
       uint32_t qa[D16][4];
 #pragma unroll
       for (int kt = 0; kt < D16; ++kt) ldsm_x4(qa[kt], smem_addr(Qs + ldsm_row * RS + (kt * 2 + ldsm_kc) * 16));
-      for (int p = warp; p < D16; p += kGW) {
+      if (dense) {
+        const int p = warp;
         float acc[2][4] = {};
 #pragma unroll
         for (int kt = 0; kt < D16; ++kt) {
-          const uint4 b = __ldg(imgk + (kt * D16 + p) * 32 + lane);
+          const uint4 b = wpre[kt];
           mma16816(acc[0], qa[kt][0], qa[kt][1], qa[kt][2], qa[kt][3], b.x, b.y);
           mma16816(acc[1], qa[kt][0], qa[kt][1], qa[kt][2], qa[kt][3], b.z, b.w);
           if ((kt + 1) % KH == 0) {   // last k-tile of head h: store its Qt columns and start the next head
@@ -277,16 +290,23 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
     __syncthreads();
 
     // ---------------------------------------------------------------- D: o[:, head h] = m_h W_v[:, head h];  T += o
-    for (int p = warp; p < D16; p += kGW) {
+    if (dense) {
+      const int p = warp;
       const int h = (p * 16) / dvh;
       float acc[2][4] = {};
+#pragma unroll
+      for (int kt = 0; kt < D16; ++kt) wpre[kt] = __ldg(imgv + (kt * D16 + p) * 32 + lane);
 #pragma unroll
       for (int kt = 0; kt < D16; ++kt) {
         uint32_t a[4];
         ldsm_x4(a, smem_addr(Qt + ((int)ldsm_row * H + h) * RS + (kt * 2 + ldsm_kc) * 16));
-        const uint4 b = __ldg(imgv + (kt * D16 + p) * 32 + lane);
-        mma16816(acc[0], a[0], a[1], a[2], a[3], b.x, b.y);
-        mma16816(acc[1], a[0], a[1], a[2], a[3], b.z, b.w);
+        mma16816(acc[0], a[0], a[1], a[2], a[3], wpre[kt].x, wpre[kt].y);
+        mma16816(acc[1], a[0], a[1], a[2], a[3], wpre[kt].z, wpre[kt].w);
+      }
+      if (l + 1 < P.M) {                                   // next layer's W_q fragments for its phase A
+        const uint4* nq = P.img + (size_t)((l + 1) * 3) * D16 * D16 * 32;
+#pragma unroll
+        for (int kt = 0; kt < D16; ++kt) wpre[kt] = __ldg(nq + (kt * D16 + p) * 32 + lane);
       }
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
