@@ -361,32 +361,44 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     if (is_item && quad * 32 < d) {
       const int n16 = rows >> 4;
       const int lo16 = half ? (n16 + 1) >> 1 : 0, hi16 = half ? n16 : (n16 + 1) >> 1;
-      for (int c16 = lo16; c16 < hi16; ++c16) {
-        uint32_t v[16];
-        tmem_ld16(tmem_lane + 128 + c16 * 16, v);
+      auto store_v = [&](int c16, const uint32_t (&v)[16]) {
+        const int rr = c16 * 16;                          // unit row of the first of these 16 columns
+        const int tt = rr / IT, in_tile = rr - tt * IT;   // IT is a multiple of 16: the 16 columns share a tile
+        const int n_valid = pu.seg_items - ((pu.t0 + tt) * IT + in_tile);   // valid items among them (<= 0 .. >= 16)
+        bf16* dst = P.Vtblk + ((size_t)pu.u * P.n_tiles + pu.seg * P.NT + pu.t0 + tt) * ((size_t)IT * d) +
+                    (size_t)jh * IT * P.dvh + ((in_tile >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int cnt = n_valid - hf * 8;
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float a = __uint_as_float(v[hf * 8 + 2 * e]), b = __uint_as_float(v[hf * 8 + 2 * e + 1]);
+            if (cnt < 8) {                                // ragged end of the segment: masked items are exact zeros
+              if (2 * e >= cnt) a = 0.f;
+              if (2 * e + 1 >= cnt) b = 0.f;
+            }
+            pk[e] = pack_bf16x2(a, b);
+          }
+          *reinterpret_cast<uint4*>(dst + hf * npr * 64) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+      };
+      int c16 = lo16;
+      for (; c16 + 2 <= hi16; c16 += 2) {                   // two accumulator loads in flight per wait
+        uint32_t v0[16], v1[16];
+        tmem_ld16(tmem_lane + 128 + c16 * 16, v0);
+        tmem_ld16(tmem_lane + 128 + c16 * 16 + 16, v1);
         tc_wait_ld();
         if (j < d) {
-          const int rr = c16 * 16;                          // unit row of the first of these 16 columns
-          const int tt = rr / IT, in_tile = rr - tt * IT;   // IT is a multiple of 16: the 16 columns share a tile
-          const int n_valid = pu.seg_items - ((pu.t0 + tt) * IT + in_tile);   // valid items among them (<= 0 .. >= 16)
-          bf16* dst = P.Vtblk + ((size_t)pu.u * P.n_tiles + pu.seg * P.NT + pu.t0 + tt) * ((size_t)IT * d) +
-                      (size_t)jh * IT * P.dvh + ((in_tile >> 3) * npr + (jj >> 3)) * 64 + (jj & 7) * 8;
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const int cnt = n_valid - hf * 8;
-            uint32_t pk[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float a = __uint_as_float(v[hf * 8 + 2 * e]), b = __uint_as_float(v[hf * 8 + 2 * e + 1]);
-              if (cnt < 8) {                                // ragged end of the segment: masked items are exact zeros
-                if (2 * e >= cnt) a = 0.f;
-                if (2 * e + 1 >= cnt) b = 0.f;
-              }
-              pk[e] = pack_bf16x2(a, b);
-            }
-            *reinterpret_cast<uint4*>(dst + hf * npr * 64) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-          }
+          store_v(c16, v0);
+          store_v(c16 + 1, v1);
         }
+      }
+      if (c16 < hi16) {
+        uint32_t v0[16];
+        tmem_ld16(tmem_lane + 128 + c16 * 16, v0);
+        tc_wait_ld();
+        if (j < d) store_v(c16, v0);
       }
     }
     tc_fence_before();
