@@ -38,6 +38,7 @@ struct GstaParams {
   const int *lengths, *cand_offsets;
   uint4* img;                  // [M][3][d/16 k-tiles][d/16 column pairs][32 lanes]
   int* nseg;                   // [N] non-empty segments per candidate (built with the images)
+  int cpb;                     // candidates per block: 16, or 8 (one per warp) when that still fits one wave of blocks
   bf16* z;
   int* status;
 };
@@ -65,7 +66,8 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   uint8_t* stage = reinterpret_cast<uint8_t*>(nv_s + kGT);          // [kGW][2][kChunk] rows
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int c_base = blockIdx.x * kGT;
+  const int c_base = blockIdx.x * P.cpb;
+  const int c_end = min(c_base + P.cpb, P.N);          // rows of the 16-row tile past this are empty
   chain_wait();
   chain_release();
 
@@ -81,11 +83,11 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   }
 
   // ---- set-up: number of non-empty segments per candidate (from the set-up kernel's map); T = candidates; zero row
-  if (tid < kGT) nv_s[tid] = (P.M > 0 && c_base + tid < P.N) ? min(max(P.nseg[c_base + tid], 0), P.Lp) : 0;
+  if (tid < kGT) nv_s[tid] = (P.M > 0 && c_base + tid < c_end) ? min(max(P.nseg[c_base + tid], 0), P.Lp) : 0;
   for (int i = tid; i < kGT * (d / 8); i += kGThreads) {     // 8 features (16 bytes) at a time
     const int r = i / (d / 8), c8 = (i - r * (d / 8)) * 8;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (c_base + r < P.N) v = *reinterpret_cast<const uint4*>(P.cands + (size_t)(c_base + r) * d + c8);
+    if (c_base + r < c_end) v = *reinterpret_cast<const uint4*>(P.cands + (size_t)(c_base + r) * d + c8);
     float* dst = Ts + r * TS + c8;
     dst[0] = bf16_lo(v.x); dst[1] = bf16_hi(v.x); dst[2] = bf16_lo(v.y); dst[3] = bf16_hi(v.y);
     dst[4] = bf16_lo(v.z); dst[5] = bf16_hi(v.z); dst[6] = bf16_lo(v.w); dst[7] = bf16_hi(v.w);
@@ -326,7 +328,7 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
 
   for (int i = tid; i < kGT * (d / 2); i += kGThreads) {
     const int r = i / (d / 2), q = i - r * (d / 2);
-    if (c_base + r < P.N) {
+    if (c_base + r < c_end) {
       const float2 v = *reinterpret_cast<const float2*>(Ts + r * TS + 2 * q);
       *reinterpret_cast<uint32_t*>(P.z + (size_t)(c_base + r) * d + 2 * q) = pack2(v.x, v.y);
     }
@@ -340,7 +342,7 @@ int launch_gsta(const GstaParams& P, cudaStream_t st) {
                       (size_t)kGW * 2 * kChunk * RS;
   LASER_CUDA_OK(cudaFuncSetAttribute(gsta_mma_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   LaunchScope ls("gsta_mma", st);
-  LASER_CUDA_OK(launch_chained(gsta_mma_kernel<D16>, dim3((P.N + kGT - 1) / kGT), dim3(kGThreads), smem, st, P));
+  LASER_CUDA_OK(launch_chained(gsta_mma_kernel<D16>, dim3((P.N + P.cpb - 1) / P.cpb), dim3(kGThreads), smem, st, P));
   return LASER_OK;
 }
 
@@ -368,6 +370,13 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   P.nseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.z = (bf16*)z;
   P.status = reinterpret_cast<int*>(ws + p.off_status);
+  {
+    // Small batches: 8 candidates per block (every warp then has one candidate instead of two, which halves the
+    // per-candidate part of a block's latency) as long as all blocks still run at once, two per SM.
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    P.cpb = (p.N + 7) / 8 <= 2 * sms ? 8 : kGT;
+  }
   if (p.M > 0 && !images_ready) {
     const int total = p.M * 3 * (p.d / 16) * (p.d / 16) * 32;
     LaunchScope ls("gsta_prep", st);
