@@ -91,6 +91,7 @@ __device__ void scan_rows(const PT& P, int* status) {
   __shared__ int sa[1024];
   const int tid = threadIdx.x;
   const int per = (P.U + 1023) / 1024;
+  const int n_act = max(1, (P.U + per - 1) / per);        // threads that own users: the scan runs over these only
   const int u0 = min(tid * per, P.U), u1 = min(u0 + per, P.U);
   int a = 0;
   bool bad = false;
@@ -103,7 +104,7 @@ __device__ void scan_rows(const PT& P, int* status) {
   if (bad) report_status(status, LASER_ERR_BAD_INPUT);
   sa[tid] = a;
   __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {
+  for (int off = 1; off < n_act; off <<= 1) {
     const int v = tid >= off ? sa[tid - off] : 0;
     __syncthreads();
     sa[tid] += v;
@@ -115,9 +116,9 @@ __device__ void scan_rows(const PT& P, int* status) {
     P.prefix[u] = pa;
     pa += s.nc * s.nseg;
   }
-  if (tid == 1023) {
-    P.prefix[P.U] = sa[1023];
-    P.counters[0] = sa[1023];
+  if (tid == n_act - 1) {
+    P.prefix[P.U] = sa[n_act - 1];
+    P.counters[0] = sa[n_act - 1];
   }
 }
 

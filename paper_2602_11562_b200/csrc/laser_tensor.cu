@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
   if (blockIdx.x == 0) {
     __shared__ int sa[1024], sb[1024], sc[1024];
     const int per = (P.U + 1023) / 1024;
+    const int n_act = max(1, (P.U + per - 1) / per);      // threads that own users: the scan runs over these only
+    const int last = n_act - 1;
     const int u0 = min(tid * per, P.U), u1 = min(u0 + per, P.U);
     int a = 0, b = 0, c = 0;
     bool bad = false;
@@ -108,7 +110,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     sb[tid] = b;
     sc[tid] = c;
     __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
+    for (int off = 1; off < n_act; off <<= 1) {
       int va = 0, vb = 0, vc = 0;
       if (tid >= off) { va = sa[tid - off]; vb = sb[tid - off]; vc = sc[tid - off]; }
       __syncthreads();
@@ -127,17 +129,17 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
       pb += s.ctiles * s.nseg;
       pc += proj_units_of(P, s);
     }
-    if (tid == 1023) {
-      P.tile_off[P.U] = sa[1023];
-      P.unit_start[P.U] = sb[1023];
-      P.proj_start[P.U] = sc[1023];
-      P.counters[0] = sb[1023];
-      P.counters[1] = sa[1023];
-      P.counters[2] = sc[1023];
+    if (tid == last) {
+      P.tile_off[P.U] = sa[last];
+      P.unit_start[P.U] = sb[last];
+      P.proj_start[P.U] = sc[last];
+      P.counters[0] = sb[last];
+      P.counters[1] = sa[last];
+      P.counters[2] = sc[last];
     }
     // First unit of every block of the two main kernels (block b of G owns units [n b / G, n (b + 1) / G)): find the
     // scan chunk in shared memory, then the user inside the chunk.
-    const int n_att = sb[1023], n_proj = sc[1023];
+    const int n_att = sb[last], n_proj = sc[last];
     for (int b = tid; b < P.sta_grid + P.proj_grid; b += 1024) {
       const bool att = b < P.sta_grid;
       const int* incl = att ? sb : sc;
@@ -145,7 +147,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
       const int id = (int)(((long long)n * bb) / G);
       int4 out = make_int4(-1, 0, 0, 0);
       if (id < n) {
-        int lo = 0, hi = 1023;                     // smallest chunk k with incl[k] > id
+        int lo = 0, hi = last;                     // smallest chunk k with incl[k] > id
         while (lo < hi) {
           const int mid = (lo + hi) >> 1;
           if (incl[mid] > id) hi = mid; else lo = mid + 1;
