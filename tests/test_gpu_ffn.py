@@ -133,3 +133,35 @@ def test_ffn_rejects_bad_arguments():
         P.laser_ffn_forward(b.cfg, fw, Hd, b.lengths, b.cand_offsets, workspace=small)
     assert ei.value.status == -3
     assert P.laser_ffn_workspace_bytes(b.cfg, 0) == 0
+
+
+def test_ffn_many_users_and_no_rows_at_all():
+    # More users than the set-up scan has threads (several users per thread), a third of them empty; then a batch in
+    # which no segment holds an item (nothing to do, nothing touched).
+    rng = np.random.default_rng(760)
+    U, d, S, L = 2500, 32, 16, 64
+    lengths = rng.integers(0, L + 1, size=U)
+    lengths[rng.random(U) < 0.33] = 0
+    w = make_custom(U=U, C=1, L=L, d=d, H=2, S=S, M=1, dtype="bf16", seed=760, lengths=lengths.tolist())
+    fw = make_ffn_weights(d, 4, "bf16", seed=60)
+    Lp = w.spec.n_seg
+    Hp = round_to_dtype(rng.standard_normal((U, Lp, d)).astype(np.float32), "bf16")
+    live = np.arange(Lp)[None, :] < (-(-lengths // S))[:, None]
+    Hp[~live] = SENTINEL
+    ref = _oracle_ffn(np.where(live[..., None], Hp, 0.0), w, fw)
+    b = P.DeviceBatch.from_workload(w)
+    ws = torch.empty(P.laser_ffn_workspace_bytes(b.cfg, 4 * d), dtype=torch.uint8, device="cuda")
+    Hd = torch.from_numpy(Hp).to(torch.bfloat16).cuda()
+    P.laser_ffn_forward(b.cfg, _ffn_dev(fw, torch.bfloat16), Hd, b.lengths, b.cand_offsets, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    got = to_np(Hd)
+    assert np.all(got[~live] == SENTINEL)
+    assert err_metric(got[live], ref[live]) <= TOL["bf16"]
+
+    w0 = make_custom(U=3, C=4, L=L, d=d, H=2, S=S, M=1, dtype="bf16", seed=761, lengths=[0, 0, 0])
+    b0 = P.DeviceBatch.from_workload(w0)
+    H0 = torch.full((12, Lp, d), SENTINEL, dtype=torch.bfloat16, device="cuda")
+    ws0 = torch.empty(P.laser_ffn_workspace_bytes(b0.cfg, 4 * d), dtype=torch.uint8, device="cuda")
+    P.laser_ffn_forward(b0.cfg, _ffn_dev(fw, torch.bfloat16), H0, b0.lengths, b0.cand_offsets, workspace=ws0)
+    assert P.laser_check_status(ws0) == 0
+    assert bool((H0 == SENTINEL).all())
