@@ -86,6 +86,7 @@ int make_plan(const laser_config* c, Plan* p) {
     p->off_tv = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->d * 2);
     p->off_twork = off; off = align_up(off + ((size_t)p->U + 1) * 3 * sizeof(int));
     p->off_tcount = off; off = align_up(off + 64 * sizeof(int) + 2 * 1024 * 4 * sizeof(int));   // counters + per-block start tables
+    p->off_tctile = off; off = align_up(off + (size_t)g.cand_tiles_max * 4 * sizeof(int));       // (user, tile, first candidate, candidates) per candidate tile
     p->off_timg = off; off = align_up(off + ((size_t)2 * p->dqk * p->d + (size_t)128 * p->d) * 2);
     if (gsta_mma_supported(*p)) { p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p)); }
   } else if (path == LASER_PATH_STREAM) {

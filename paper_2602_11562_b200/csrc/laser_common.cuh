@@ -32,7 +32,7 @@ struct Plan {
   size_t off_hp;                   // internal H' [N,Lp,d] in the I/O dtype
   // tensor path
   TensorGeom tg;
-  size_t off_tq, off_tk, off_tv, off_twork, off_tcount, off_timg;
+  size_t off_tq, off_tk, off_tv, off_twork, off_tcount, off_tctile, off_timg;
   size_t off_gimg;                 // GSTA weight images in MMA fragment order (bf16 paths)
   // stream path
   size_t off_su;

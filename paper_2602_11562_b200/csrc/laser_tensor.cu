@@ -42,7 +42,8 @@ struct TcParams {
   int* proj_start;                    // [U+1] prefix of projection units (groups of item tiles that hold valid items)
   int* counters;                      // [0] attention units, [1] candidate tiles, [2] projection units
   int4* sta_begin;                    // [sta_grid]  first attention unit of every block: (user, candidate tile, segment, -)
-  int4* proj_begin;                   // [proj_grid] first projection unit of every block: (user, segment, tile group, -)
+  int4* proj_begin;                   // [proj_grid] first projection unit of every block: (user, segment, tile group, user's length)
+  int4* ctile;                        // [candidate tiles] (user, tile within the user, user's first candidate, its candidates)
   int sta_grid, proj_grid;
   const bf16* Wg;                     // GSTA weights whose images this set-up also builds (null: none)
   uint4* gimg;
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     int pa = sa[tid] - a, pb = sb[tid] - b, pc = sc[tid] - c;   // exclusive prefixes
     for (int u = u0; u < u1; ++u) {
       const UserShape s = user_shape(P, u);
+      for (int jt = 0; jt < s.ctiles; ++jt) P.ctile[pa + jt] = make_int4(u, jt, s.c0, s.nc);
       P.tile_off[u] = pa;
       P.unit_start[u] = pb;
       P.proj_start[u] = pc;
@@ -163,7 +165,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
         }
         const int local = id - base;
         if (att) out = make_int4(u, local / s.nseg, local % s.nseg, 0);
-        else out = make_int4(u, local / P.NG, local % P.NG, 0);
+        else out = make_int4(u, local / P.NG, local % P.NG, s.len);
       }
       if (att) P.sta_begin[bb] = out; else P.proj_begin[bb] = out;
     }
@@ -416,16 +418,17 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   if (ok && hi > lo) {
     // cursor over (user, segment, tile group)
     int cu, cseg, cgrp, c_nseg, c_len, c_last_groups;
-    auto load_user = [&]() {
-      const UserShape s = user_shape(P, cu);
-      c_nseg = s.nseg; c_len = s.len;
-      const int last_items = s.nseg > 0 ? s.len - (s.nseg - 1) * P.S : 0;
+    auto set_len = [&](int len) {
+      c_len = len;
+      c_nseg = (len + P.S - 1) / P.S;
+      const int last_items = c_nseg > 0 ? len - (c_nseg - 1) * P.S : 0;
       c_last_groups = (min(P.NT, (last_items + IT - 1) / IT) + P.NTG - 1) / P.NTG;
     };
+    auto load_user = [&]() { set_len(user_shape(P, cu).len); };
     {
-      const int4 b = P.proj_begin[bidx];                     // this block's first unit, as found by tc_prep_kernel
-      cu = b.x; cseg = b.y; cgrp = b.z;
-      load_user();
+      const int4 b = P.proj_begin[bidx];                     // this block's first unit and its user's (sanitised) length,
+      cu = b.x; cseg = b.y; cgrp = b.z;                      // as found by tc_prep_kernel: one load before the first copy
+      set_len(b.w);
     }
     auto make_unit = [&]() {
       ProjUnit pu;
@@ -473,24 +476,27 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   // ---- candidate tiles, dealt round-robin over the blocks (W_q^T replaces W_k^T in shared memory)
   const int n_ctiles = P.counters[1];
   if (ok && bidx < n_ctiles) {
-    __syncthreads();                      // every MMA that read W_k^T has completed (its accumulators were drained)
+    __syncthreads();                      // every MMA that read W_k^T or the staging buffer has completed (drained)
     if (tid == 0) {
       mbar_arrive_expect_tx(&bar_img, bK);
       bulk_g2s(imgK, P.imgQ, bK, &bar_img);
     }
+    auto cand_unit = [&](int ct) {          // (user, tile, first candidate, candidates), tabulated by tc_prep_kernel
+      const int4 e = P.ctile[ct];
+      ProjUnit pu;
+      pu.u = e.x; pu.seg = 0; pu.t0 = 0; pu.rows = kCandTile; pu.seg_items = 0;
+      pu.jt = e.y; pu.c0 = e.z; pu.nc = e.w;
+      return pu;
+    };
+    ProjUnit pu = cand_unit(bidx);
+    stage(pu, false, Xbuf);                 // the first tile's rows travel together with W_q^T
     ok = __syncthreads_and(mbar_wait(&bar_img, 1, abortp));
     for (int ct = bidx; ct < n_ctiles && ok; ct += G) {
-      int a = 0, b = P.U;                 // tile_off[a] <= ct < tile_off[b]
-      while (b - a > 1) {
-        const int mid = (a + b) >> 1;
-        if (P.tile_off[mid] <= ct) a = mid; else b = mid;
+      if (ct != bidx) {
+        pu = cand_unit(ct);
+        __syncthreads();                    // staging buffer and TMEM of the previous unit are free
+        stage(pu, false, Xbuf);
       }
-      const UserShape us = user_shape(P, a);
-      ProjUnit pu;
-      pu.u = a; pu.seg = 0; pu.t0 = 0; pu.rows = kCandTile; pu.seg_items = 0;
-      pu.jt = ct - P.tile_off[a]; pu.c0 = us.c0; pu.nc = us.nc;
-      __syncthreads();                    // staging buffer and TMEM of the previous unit are free
-      stage(pu, false, Xbuf);
       cp_async_wait_all();
       fence_proxy_async_smem();
       __syncthreads();
@@ -916,6 +922,7 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.counters = (int*)(ws + p.off_tcount);
   P.sta_begin = reinterpret_cast<int4*>(ws + p.off_tcount + 64 * sizeof(int));
   P.proj_begin = P.sta_begin + 1024;
+  P.ctile = reinterpret_cast<int4*>(ws + p.off_tctile);
   P.sta_grid = sm_count() < 1024 ? sm_count() : 1024;
   P.proj_grid = 2 * sm_count() < 1024 ? 2 * sm_count() : 1024;
   P.imgK = (bf16*)(ws + p.off_timg);
