@@ -267,8 +267,10 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
           for (int jt = 0; jt < D16; ++jt) {
             uint32_t a[4];
             ldsm_x4_t(a, sb + t_off + jt * 32);
-            macc[jt][0] *= sc0; macc[jt][1] *= sc1;
-            macc[jt][2] *= sc0; macc[jt][3] *= sc1;
+            if (ch > 0) {                       // (the first chunk starts from zero)
+              macc[jt][0] *= sc0; macc[jt][1] *= sc1;
+              macc[jt][2] *= sc0; macc[jt][3] *= sc1;
+            }
             mma16816(macc[jt], a[0], a[1], a[2], a[3], pb0, pb1);
           }
           __syncwarp();               // every lane is done with this buffer before the next iteration refills it
