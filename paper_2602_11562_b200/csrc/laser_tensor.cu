@@ -704,7 +704,10 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         uint64_t q_desc = q_desc0;
         bool ok = true;
 
-        auto issue_scores = [&](const Cursor& c) {
+        // Scores of a unit in two steps: everything that does not need the score buffer (the Q tile, the K tile, the
+        // descriptors) first, so that once the warpgroup hands the buffer back only the MMA itself remains.
+        uint64_t qd = 0, kd = 0;
+        auto prepare_scores = [&](const Cursor& c) {
           if (c.w.u != qu || c.w.j != qj) {               // first unit on a new candidate tile
             if (qu >= 0 && leader) tc_commit(&bars.q_empty[(qcount - 1) & 1]);   // my score MMAs on the old Q tile are issued
             ok = wait_all(&bars.q_full[qcount & 1], (qcount >> 1) & 1);
@@ -716,8 +719,11 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           }
           ok = wait_all(&bars.kv_full[c.st], c.kv_par);
           if (!ok) return;
+          qd = q_desc + c.h * q_head;
+          kd = k_desc0 + (uint64_t)(c.st * (k_bytes >> 4) + c.h * k_head);
+        };
+        auto fire_scores = [&]() {
           tc_fence_after();
-          const uint64_t qd = q_desc + c.h * q_head, kd = k_desc0 + (uint64_t)(c.st * (k_bytes >> 4) + c.h * k_head);
           if (leader) {
             for (int ks = 0; ks < ks1; ++ks) mma_ss(tS, qd + ks * 16, kd + ks * 16, id1, ks > 0);
             tc_commit(&bars.s_full[wgi]);
@@ -751,16 +757,18 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         Cursor cur;
         cur.w.init(P);
         cur.it = 0; cur.t = 0; cur.h = wgi; cur.nt = cur.w.ntiles(P); cur.st = 0; cur.kv_par = 0;
-        issue_scores(cur);
+        prepare_scores(cur);
+        if (ok) fire_scores();
         while (ok) {
           Cursor nxt = cur;
           const bool more = advance(nxt);
           if (more) {                                     // next scores as soon as the warpgroup has read the current ones
+            prepare_scores(nxt);
+            if (!ok) break;
             ok = wait_all(&bars.s_free[wgi], sf_par);
             if (!ok) break;
             sf_par ^= 1;
-            issue_scores(nxt);
-            if (!ok) break;
+            fire_scores();
           }
           issue_values(cur);
           if (!more) break;
