@@ -164,8 +164,9 @@ LASER_API size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hi
  *   Hprime  [N, L', d]  IN / OUT: rows of non-empty segments are replaced by LN(FFN(s) + s)
  *   workspace           at least laser_ffn_workspace_bytes(cfg, ffn->d_hidden) bytes, 256-byte aligned
  * BF16 with d a multiple of 16 (<= 128) and d_hidden a multiple of 128 runs on the tensor cores (bf16 operands and
- * hidden activations, fp32 accumulation and normalisation) unless cfg->path is LASER_PATH_SIMT; everything else runs
- * in fp32 on the ALUs.  LASER_ERR_UNSUPPORTED when neither kernel takes the shape. */
+ * hidden activations, fp32 accumulation and normalisation) unless cfg->path is LASER_PATH_SIMT or the bias / layer-norm
+ * vectors no longer fit beside the tiles in shared memory (at d = 128: d_hidden > 512); everything else runs in fp32
+ * on the ALUs.  LASER_ERR_UNSUPPORTED when neither kernel takes the shape. */
 LASER_API int laser_ffn_forward(const laser_config* cfg, const laser_ffn_params* ffn, void* Hprime,
                                 const int32_t* lengths, const int32_t* cand_offsets, void* workspace,
                                 size_t workspace_bytes, void* cuda_stream);
