@@ -51,10 +51,15 @@ fusion_kernel(const T* __restrict__ Hp, const T* __restrict__ z, const int* __re
   if (cand_offsets[0] > c || cand_offsets[U] <= c) {
     if (lane == 0) report_status(status, LASER_ERR_BAD_INPUT);
   } else {
-    int lo = 0, hi = U;   // cand_offsets[lo] <= c < cand_offsets[hi]
+    // the warp searches together, 32 probes per round trip: cand_offsets[lo] <= c < cand_offsets[hi]
+    int lo = 0, hi = U;
     while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (cand_offsets[mid] <= c) lo = mid; else hi = mid;
+      const int step = (hi - lo + 31) / 32;
+      const int idx = min(lo + lane * step, hi);
+      const unsigned le = __ballot_sync(0xffffffffu, idx < hi && cand_offsets[idx] <= c);   // a prefix of the lanes
+      const int k = __popc(le);                         // >= 1: lane 0 probes lo itself
+      lo = lo + (k - 1) * step;
+      hi = min(lo + step, hi);
     }
     const int len = lengths[lo];
     if (len < 0 || len > L) { if (lane == 0) report_status(status, LASER_ERR_BAD_INPUT); }
