@@ -311,3 +311,26 @@ def test_full_size_configs_sampled_users(name, n_users):
     assert P.laser_check_status(ws) == 0
     _, z_full = run_forward(w, "auto")
     assert torch.equal(z, z_full)
+
+
+@pytest.mark.parametrize("S", [5, 10, 20])
+def test_production_shape_segment_sizes_tensor_path(S):
+    # The paper's production shape (L = 1000, two heads of d_q = 16, d = 128, two GSTA layers) at the three segment
+    # sizes of its segment-size study, many candidates per user, at a batch the oracle finishes in seconds.
+    w = make_custom(dtype="bf16", seed=900 + S, U=2, C=140, L=1000, d=128, H=2, S=S, M=2, d_qh=16, lengths=[1000, 437])
+    check_against_oracle(w, "tensor")
+    # and with the FFN + LayerNorm of Eq. 6 between the two stages
+    from oracle import ffn_oracle, laser_oracle
+    from workloads import make_ffn_weights
+    s = w.spec
+    fw = make_ffn_weights(s.d, 4, "bf16", seed=S)
+    Hp = laser_oracle.sta_forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, s.S, s.H, w.gamma)
+    Hp = ffn_oracle.ffn_forward(Hp, w.lengths, w.cand_offsets, s.S, fw["W1"], fw["b1"], fw["W2"], fw["b2"], fw["ln_g"],
+                                fw["ln_b"])
+    z_ref = laser_oracle.gsta_forward(Hp, w.lengths, w.cand_offsets, w.cands, w.Wg, s.S, s.H, w.tau)
+    b = P.DeviceBatch.from_workload(w)
+    fdev = {k: torch.from_numpy(v).to(torch.bfloat16).cuda() for k, v in fw.items()}
+    ws = torch.empty(P.laser_ffn_workspace_bytes(b.cfg, 4 * s.d), dtype=torch.uint8, device="cuda")
+    z = P.laser_forward_ffn(b.cfg, *b.args(), b.Wg, fdev, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    assert err_metric(to_np(z), z_ref) <= TOL["bf16"]
