@@ -179,6 +179,18 @@ LASER_API int laser_forward_ffn(const laser_config* cfg, const void* items, cons
                                 const void* Wgsta, const laser_ffn_params* ffn, void* Hprime, void* z, void* workspace,
                                 size_t workspace_bytes, void* cuda_stream);
 
+/* The softmax-aggregation variant of STA, the paper's ablation of the sigmoid gate ("replacing sigmoid aggregation with
+ * the conventional softmax"): inside every segment the weights of the valid items are exp(q_h . k_{n,h} / gamma)
+ * normalised to sum to one per (candidate, head); everything else (projections of Eq. 4, heads, ragged lengths, zero
+ * rows for empty segments) is as in laser_sta_forward.  Runs on the FP32-ALU kernels for either dtype, whatever
+ * cfg->path says (an ablation, not a production path).
+ *   workspace  at least laser_sta_softmax_workspace_bytes(cfg) bytes, 256-byte aligned */
+LASER_API size_t laser_sta_softmax_workspace_bytes(const laser_config* cfg);
+LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const int32_t* lengths,
+                                        const void* cands, const int32_t* cand_offsets, const void* Wq, const void* Wk,
+                                        const void* Wv, void* Hprime, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream);
+
 /* STA without any workspace argument, for callers that cannot allocate device memory (no counterpart in the
  * paper: this is a deployment convenience of this library).  Think of a plug-in inside a serving process
  * whose GPU memory belongs entirely to the host framework's pool, or of a request thread that must never hit

@@ -19,6 +19,8 @@ from .binding import (  # noqa: F401
     laser_sta_forward_static,
     laser_gsta_forward,
     laser_fusion_forward,
+    laser_sta_softmax_workspace_bytes,
+    laser_sta_softmax_forward,
     laser_ffn_workspace_bytes,
     laser_ffn_forward,
     laser_forward_ffn,

@@ -82,6 +82,10 @@ def load_library() -> ctypes.CDLL:
     lib.laser_sta_forward_static.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp]
     lib.laser_fusion_forward.restype = ctypes.c_int
     lib.laser_fusion_forward.argtypes = [cfgp, vp, vp, i32p, i32p, ctypes.c_int32, vp, vp, sz, vp]
+    lib.laser_sta_softmax_workspace_bytes.restype = sz
+    lib.laser_sta_softmax_workspace_bytes.argtypes = [cfgp]
+    lib.laser_sta_softmax_forward.restype = ctypes.c_int
+    lib.laser_sta_softmax_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, sz, vp]
     ffnp = ctypes.POINTER(LaserFfnParams)
     lib.laser_ffn_workspace_bytes.restype = sz
     lib.laser_ffn_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
@@ -241,6 +245,28 @@ def laser_fusion_forward(cfg, Hprime, z, lengths, cand_offsets, num_recent, fuse
                                   _stream_ptr(stream))
     _check(rc, "laser_fusion_forward")
     return fused
+
+
+def laser_sta_softmax_workspace_bytes(cfg: LaserConfig) -> int:
+    return int(load_library().laser_sta_softmax_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_sta_softmax_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime=None, workspace=None,
+                              stream=None):
+    """The softmax-aggregation variant of STA (the paper's ablation): returns H' [N, L', d]."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    need = laser_sta_softmax_workspace_bytes(cfg)
+    if need == 0:
+        raise LaserError(-1, "laser_sta_softmax_workspace_bytes (invalid or unsupported configuration)")
+    ws = torch.empty(need, dtype=torch.uint8, device=items.device) if workspace is None else workspace
+    if Hprime is None:
+        Hprime = torch.empty((cfg.total_cands, cfg.n_seg, cfg.d_model), dtype=dt, device=items.device)
+    rc = lib.laser_sta_softmax_forward(ctypes.byref(cfg), _dev(items, dt, "items"), _dev(lengths, torch.int32, "lengths"),
+                                       _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                                       _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"),
+                                       _dev(Hprime, dt, "Hprime"), ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_sta_softmax_forward")
+    return Hprime
 
 
 def laser_ffn_workspace_bytes(cfg: LaserConfig, d_hidden: int) -> int:

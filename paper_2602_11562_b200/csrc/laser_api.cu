@@ -235,6 +235,36 @@ int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void
   return fusion_forward(p, Hprime, z, lengths, cand_offsets, num_recent, fused, ws, st);
 }
 
+static int softmax_plan(const laser_config* cfg, Plan* p) {
+  if (!cfg) return LASER_ERR_INVALID_ARG;
+  laser_config c = *cfg;
+  c.path = LASER_PATH_SIMT;
+  return make_plan(&c, p);
+}
+
+size_t laser_sta_softmax_workspace_bytes(const laser_config* cfg) {
+  Plan p;
+  if (softmax_plan(cfg, &p) != LASER_OK) return 0;
+  return p.total;
+}
+
+int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                              const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = softmax_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({items, cands, Wq, Wk, Wv, Hprime})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  if (p.N == 0) return LASER_OK;
+  return simt_sta_softmax(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
+}
+
 size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hidden) {
   Plan p;
   if (make_plan(cfg, &p) != LASER_OK || d_hidden < 1) return 0;

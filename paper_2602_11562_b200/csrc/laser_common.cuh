@@ -59,6 +59,10 @@ class LaunchScope {
 // --- per-path launchers (each returns LASER_OK / LASER_ERR_*) -------------------------------------------------------
 int simt_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
              const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st);
+// Softmax-aggregation variant of STA (the paper's ablation of the sigmoid gate); FP32-ALU kernels, same scratch as simt_sta.
+int simt_sta_softmax(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                     const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws,
+                     cudaStream_t st);
 int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
               const void* Wg, void* z, char* ws, cudaStream_t st);
 

@@ -61,9 +61,22 @@ __device__ __forceinline__ float sigmoid_accurate(float x) {
   return 1.f / (1.f + expf(-x));
 }
 
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
 // One block = (segment, 32-candidate tile, user).  Gates (Eq. 5 / Eq. 10) for a 32x32 (candidate, item) chunk go to
 // shared memory, then every thread accumulates gate * value for its candidate and its interleaved columns (Eq. 12).
-template <typename T>
+// kSoftmax selects the ablation variant: the weights of a segment's valid items are exp(score) normalised to sum to one
+// per (candidate, head), computed online over the 32-item chunks (running maximum, running sum, rescaled accumulators).
+template <typename T, bool kSoftmax>
 __global__ void __launch_bounds__(kStaThreads)
 sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const float* __restrict__ V,
                 const int* __restrict__ lengths, const int* __restrict__ cand_offsets, T* __restrict__ Hp,
@@ -85,6 +98,9 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
   float* Ks = Qs + kStaCands * qld;            // [32][dqk+1]
   float* Vs = Ks + kStaItems * qld;            // [32][d]
   float* G = Vs + kStaItems * d;               // [H][32][33]
+  float* st_m = G + H * kStaCands * 33;        // softmax variant: running maximum   [H][32]
+  float* st_z = st_m + H * kStaCands;          //                  running sum       [H][32]
+  float* st_s = st_z + H * kStaCands;          //                  this chunk's rescale factor [H][32]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int c = tid >> 2, cg = tid & 3;        // accumulate phase: candidate, column group
@@ -101,6 +117,12 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
   for (int idx = tid; idx < kStaCands * dqk; idx += kStaThreads) {
     int r = idx / dqk, a = idx - r * dqk;
     Qs[r * qld + a] = r < nc ? Q[(size_t)(c0 + r) * dqk + a] : 0.f;
+  }
+  if (kSoftmax) {
+    for (int idx = tid; idx < H * kStaCands; idx += kStaThreads) {
+      st_m[idx] = -INFINITY;
+      st_z[idx] = 0.f;
+    }
   }
 
   const int n_begin = seg * S;
@@ -124,10 +146,30 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
       for (int h = 0; h < H; ++h) {
         float dot = 0.f;
         for (int a = 0; a < dqh; ++a) dot = fmaf(Qs[cc * qld + h * dqh + a], Ks[lane * qld + h * dqh + a], dot);
-        G[(h * kStaCands + cc) * 33 + lane] = lane < cnt ? sigmoid_accurate(dot) : 0.f;
+        if (!kSoftmax) {
+          G[(h * kStaCands + cc) * 33 + lane] = lane < cnt ? sigmoid_accurate(dot) : 0.f;
+        } else {
+          const float m_old = st_m[h * kStaCands + cc], z_old = st_z[h * kStaCands + cc];
+          const float m_new = fmaxf(m_old, warp_max(lane < cnt ? dot : -INFINITY));   // finite: the chunk has an item
+          const float pw = lane < cnt ? expf(dot - m_new) : 0.f;
+          const float psum = warp_sum(pw);
+          G[(h * kStaCands + cc) * 33 + lane] = pw;
+          __syncwarp();
+          if (lane == 0) {
+            const float sc = expf(m_old - m_new);           // 0 on the first chunk (m_old = -inf)
+            st_s[h * kStaCands + cc] = sc;
+            st_z[h * kStaCands + cc] = z_old * sc + psum;
+            st_m[h * kStaCands + cc] = m_new;
+          }
+        }
       }
     }
     __syncthreads();
+    if (kSoftmax) {
+#pragma unroll
+      for (int j = 0; j < kStaMaxJ; ++j)
+        if (j < nj) acc[j] *= st_s[goff[j] / 33];
+    }
     for (int n = 0; n < cnt; ++n) {
 #pragma unroll
       for (int j = 0; j < kStaMaxJ; ++j) {
@@ -138,21 +180,19 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
   if (c < nc) {
     T* out = Hp + ((size_t)(c0 + c) * Lp + seg) * d;
 #pragma unroll
-    for (int j = 0; j < kStaMaxJ; ++j)
-      if (j < nj) out[cg + 4 * j] = from_f32<T>(acc[j]);
+    for (int j = 0; j < kStaMaxJ; ++j) {
+      if (j < nj) {
+        float v = acc[j];
+        if (kSoftmax) {
+          const float z = st_z[goff[j] / 33];
+          v = z > 0.f ? v / z : 0.f;                        // a segment without valid items stays a zero row
+        }
+        out[cg + 4 * j] = from_f32<T>(v);
+      }
+    }
   }
 }
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
 
 // One block per candidate.  Eq. 7 in the reassociated form (exact in real arithmetic):
 //   q = t W_q;  qt_h = W_k[:, head h] q_h  (so that (s_j W_k)_h . q_h = s_j . qt_h);  e_{j,h} = s_j . qt_h / tau;
@@ -264,7 +304,7 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
 
 template <typename T>
 int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
-               const T* Wq, const T* Wk, const T* Wv, T* Hp, char* ws, cudaStream_t st) {
+               const T* Wq, const T* Wk, const T* Wv, T* Hp, char* ws, cudaStream_t st, bool softmax) {
   int* status = reinterpret_cast<int*>(ws + p.off_status);
   float* Qf = reinterpret_cast<float*>(ws + p.off_q);
   float* Kf = reinterpret_cast<float*>(ws + p.off_k);
@@ -285,13 +325,20 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   }
   {
     const size_t smem = ((size_t)(kStaCands + kStaItems) * (p.dqk + 1) + (size_t)kStaItems * p.d +
-                         (size_t)p.H * kStaCands * 33) * sizeof(float);
+                         (size_t)p.H * kStaCands * (33 + 3)) * sizeof(float);
     if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
-    LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid(p.Lp, (p.maxC + kStaCands - 1) / kStaCands, p.U);
-    LaunchScope ls("sta_simt", st);
-    sta_simt_kernel<T><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk, p.H,
-                                                       p.S, p.Lp, p.N, status);
+    if (softmax) {
+      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      LaunchScope ls("sta_simt_softmax", st);
+      sta_simt_kernel<T, true><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
+                                                               p.H, p.S, p.Lp, p.N, status);
+    } else {
+      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      LaunchScope ls("sta_simt", st);
+      sta_simt_kernel<T, false><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
+                                                                p.H, p.S, p.Lp, p.N, status);
+    }
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
@@ -316,15 +363,27 @@ int simt_gsta_t(const Plan& p, const T* Hp, const int32_t* lengths, const int32_
 
 }  // namespace
 
-int simt_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
-             const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+static int simt_sta_any(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                        const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime,
+                        char* ws, cudaStream_t st, bool softmax) {
   if (p.d > 4 * kStaMaxJ) return LASER_ERR_UNSUPPORTED;
   if (p.dtype == LASER_F32)
     return simt_sta_t<float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
-                             (const float*)Wk, (const float*)Wv, (float*)Hprime, ws, st);
+                             (const float*)Wk, (const float*)Wv, (float*)Hprime, ws, st, softmax);
   using B = __nv_bfloat16;
   return simt_sta_t<B>(p, (const B*)items, lengths, (const B*)cands, cand_offsets, (const B*)Wq, (const B*)Wk,
-                       (const B*)Wv, (B*)Hprime, ws, st);
+                       (const B*)Wv, (B*)Hprime, ws, st, softmax);
+}
+
+int simt_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+             const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st) {
+  return simt_sta_any(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st, false);
+}
+
+int simt_sta_softmax(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
+                     const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws,
+                     cudaStream_t st) {
+  return simt_sta_any(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st, true);
 }
 
 int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
