@@ -199,7 +199,8 @@ NCU_TRAFFIC = {
 }
 KERNEL_SOURCE = {"sta_tc": "laser_tensor.cu", "tc_proj": "laser_tensor.cu", "gsta_mma": "laser_gsta.cu",
                  "stream_sta": "laser_stream.cu", "ffn_tc": "laser_ffn.cu"}
-MAIN_KERNELS = ("sta_tc", "tc_proj", "gsta_mma", "stream_sta")   # kernels of the timed step (roofline candidates)
+MAIN_KERNELS = ("sta_tc", "tc_proj", "gsta_mma", "stream_sta",      # kernels of the timed step (roofline candidates)
+                "proj_simt_q", "proj_simt_kv", "sta_simt", "gsta_simt")
 
 
 def _source_digest(fname):
@@ -226,6 +227,17 @@ def kernel_roofline(w, name, ms, peaks):
     sec = ms * 1e-3
     src = "of measured" if peaks["_source"] == "measured" else "of fallback"
     traffic = ncu_traffic(name, w.spec.name)
+    if name.endswith("_simt") or "_simt_" in name:
+        # FP32-ALU path (the fp32 configuration): plain FMA arithmetic.  Peak = 148 SMs x 128 FP32 lanes x 2 flops x the
+        # maximum SM clock (1965 MHz) = 74.4 TFLOP/s, derived from the unit counts, not measured.
+        s = w.spec
+        flops = {"proj_simt_q": 2 * w.N * s.d * s.d_qk, "proj_simt_kv": work["proj_flops"], "sta_simt": work["attn_flops"],
+                 "gsta_simt": work["gsta_flops"]}.get(name, 0)
+        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        achieved = flops / sec / 1e12
+        return {"kernel": name, "bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+                "ms": ms}
     if name.startswith("stream") or name.startswith("gsta"):
         nbytes = work["io_bytes"] if name.startswith("stream") else work["gsta_bytes"]
         achieved = nbytes / sec / 1e9
