@@ -329,6 +329,37 @@ def ffn_row(P, w, b, Hp, flush, stream, steps, peaks, dev):
             "parity": {"err": err, "tol": tol, "rows_checked": sum(n for _, n in before.values())}}
 
 
+def packed_row(P, w, b, z_padded, ws, flush, stream, steps, dev):
+    """Another row of the scope: the same forward on items stored without padding (laser_forward_packed); its z must
+    equal the padded layout's bit for bit, and it is timed like the main step."""
+    import torch
+    s = w.spec
+    lens = w.lengths.astype(np.int64)
+    offs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    rows = torch.cat([b.items[u, :int(lens[u])] for u in range(s.U)], dim=0) if int(lens.sum()) > 0 else \
+        torch.zeros((1, s.d), dtype=b.items.dtype, device=dev)
+    rows = rows.contiguous()
+    offs_d = torch.from_numpy(offs).to(dev)
+    z2 = torch.empty_like(z_padded)
+    P.laser_forward_packed(b.cfg, rows, offs_d, b.lengths, b.cands, b.cand_offsets, b.Wq, b.Wk, b.Wv, b.Wg, z=z2,
+                           workspace=ws, stream=stream)
+    assert P.laser_check_status(ws) == 0
+    if not torch.equal(z2, z_padded):
+        raise SystemExit("packed layout: z differs from the padded layout's")
+    tot = 0.0
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        P.laser_forward_packed(b.cfg, rows, offs_d, b.lengths, b.cands, b.cand_offsets, b.Wq, b.Wk, b.Wv, b.Wg, z=z2,
+                               workspace=ws, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1) / steps
+    return {"ms_per_step": tot, "value": w.N / (tot * 1e-3), "unit": UNIT, "item_bytes": int(rows.numel() * rows.element_size()),
+            "padded_item_bytes": int(b.items.numel() * b.items.element_size()), "z_identical_to_padded": True}
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -424,6 +455,7 @@ def run_ours(args, rank, world, local_rank):
     # next row of the scope: multi-resolution fusion outputs on the H' and z of this batch (outside the timed step)
     fusion = None
     ffn = None
+    packed = None
     if rank == 0:
         r_recent = 2
         Hp_full = torch.empty((b.cfg.total_cands, b.cfg.n_seg, s.d), dtype=b.items.dtype, device=dev)
@@ -447,6 +479,7 @@ def run_ours(args, rank, world, local_rank):
                   "frac": f_bytes / (f_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del fused
         ffn = ffn_row(P, w, b, Hp_full, flush, stream, args.steps, peaks, dev)
+        packed = packed_row(P, w, b, z, ws, flush, stream, args.steps, dev)
         del Hp_full
 
     # end to end: pinned host buffers in, z out, through laser_forward_host
@@ -499,6 +532,7 @@ def run_ours(args, rank, world, local_rank):
                 "kernels_ms": prof,
                 "fusion": fusion,
                 "ffn": ffn,
+                "packed_layout": packed,
                 "kernel_rooflines": [kernel_roofline(w, k, v, peaks) for k, v in prof.items() if k in MAIN_KERNELS],
                 "cpu_baseline": cpu_base,
                 "parity": parity,

@@ -125,6 +125,18 @@ LASER_API int laser_forward(const laser_config* cfg, const void* items, const in
                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
                   void* Hprime, void* z, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* laser_forward for item embeddings stored without padding (a packed, CSR-style layout): user u's rows are
+ * items_packed[item_offsets[u] .. item_offsets[u] + lengths[u]), so a batch of ragged sequences costs memory for its
+ * valid items only.  The paper does not fix a memory layout; everything computed is as for laser_forward.
+ *   items_packed  [item_offsets[U], d]
+ *   item_offsets  [U+1] int32 (DEVICE), non-decreasing; user u's valid prefix must fit before item_offsets[U]
+ *                 (a violation is reported as LASER_ERR_BAD_INPUT through the status word and that user is skipped)
+ * cfg->max_len still bounds every length and fixes L' = ceil(max_len / S). */
+LASER_API int laser_forward_packed(const laser_config* cfg, const void* items_packed, const int32_t* item_offsets,
+                                   const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+                                   const void* Wq, const void* Wk, const void* Wv, const void* Wgsta, void* Hprime,
+                                   void* z, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Multi-resolution feature fusion (section "Multi-resolution Feature Fusion"): per candidate the concatenation
  *   fused = [ z | max over the non-empty segments j of s_j (element-wise) | s_0 | ... | s_{r-1} ]     in R^{(2 + r) d}
  * of the GSTA output, the max-pooled compact sequence and the r most recent segment vectors.  Segment 0 holds the most

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     laser_forward_ffn,
     LaserFfnParams,
     laser_forward,
+    laser_forward_packed,
     laser_forward_host,
     laser_check_status,
     laser_last_launch_count,

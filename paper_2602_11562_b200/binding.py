@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.laser_gsta_forward.argtypes = [cfgp, vp, i32p, i32p, vp, vp, vp, vp, sz, vp]
     lib.laser_forward.restype = ctypes.c_int
     lib.laser_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.laser_forward_packed.restype = ctypes.c_int
+    lib.laser_forward_packed.argtypes = [cfgp, vp, i32p, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.laser_forward_host.restype = ctypes.c_int
     lib.laser_forward_host.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, sz, vp, ctypes.c_int]
     lib.laser_sta_forward_static.restype = ctypes.c_int
@@ -229,6 +231,25 @@ def laser_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, H
                            None if Hprime is None else _dev(Hprime, dt, "Hprime"), _dev(z, dt, "z"),
                            ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     _check(rc, "laser_forward")
+    return (Hprime, z) if Hprime is not None else z
+
+
+def laser_forward_packed(cfg, items_packed, item_offsets, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, Hprime=None,
+                         z=None, workspace=None, stream=None, want_hprime=False):
+    """laser_forward on items stored without padding: items_packed [item_offsets[U], d], item_offsets [U + 1] int32."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    ws = _workspace(cfg, workspace, items_packed.device)
+    if z is None:
+        z = torch.empty((cfg.total_cands, cfg.d_model), dtype=dt, device=items_packed.device)
+    if Hprime is None and want_hprime:
+        Hprime = torch.empty((cfg.total_cands, cfg.n_seg, cfg.d_model), dtype=dt, device=items_packed.device)
+    rc = lib.laser_forward_packed(ctypes.byref(cfg), _dev(items_packed, dt, "items_packed"),
+                                  _dev(item_offsets, torch.int32, "item_offsets"), _dev(lengths, torch.int32, "lengths"),
+                                  _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                                  _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Wgsta, dt, "Wgsta"),
+                                  None if Hprime is None else _dev(Hprime, dt, "Hprime"), _dev(z, dt, "z"),
+                                  ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_forward_packed")
     return (Hprime, z) if Hprime is not None else z
 
 

@@ -217,6 +217,24 @@ int laser_forward(const laser_config* cfg, const void* items, const int32_t* len
                       static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
 }
 
+int laser_forward_packed(const laser_config* cfg, const void* items_packed, const int32_t* item_offsets,
+                         const int32_t* lengths, const void* cands, const int32_t* cand_offsets, const void* Wq,
+                         const void* Wk, const void* Wv, const void* Wgsta, void* Hprime, void* z, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if ((rc = check_ws(p, workspace, workspace_bytes)) != LASER_OK) return rc;
+  if (!lengths || !cand_offsets || !item_offsets) return LASER_ERR_INVALID_ARG;
+  if (p.N > 0 && (rc = check_ptrs({items_packed, cands, Wq, Wk, Wv, z})) != LASER_OK) return rc;
+  if (p.N > 0 && p.M > 0 && (rc = check_ptrs({Wgsta})) != LASER_OK) return rc;
+  if (Hprime && !aligned16(Hprime)) return LASER_ERR_INVALID_ARG;
+  p.item_offsets = item_offsets;
+  return forward_impl(p, items_packed, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, Hprime, z,
+                      static_cast<char*>(workspace), static_cast<cudaStream_t>(cuda_stream));
+}
+
 int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void* z, const int32_t* lengths,
                          const int32_t* cand_offsets, int32_t num_recent, void* fused, void* workspace,
                          size_t workspace_bytes, void* cuda_stream) {

@@ -26,6 +26,7 @@ struct Plan {
   int Lp, dqh, dvh;
   float inv_gamma, inv_tau;
   size_t esize;
+  const int32_t* item_offsets;     // packed item layout: first row of every user ([U + 1]); null = padded [U, L, d]
   // workspace byte offsets
   size_t off_status;
   size_t off_q, off_k, off_v;      // SIMT: fp32 Q [N,dqk], K [U,L,dqk], V [U,L,d]

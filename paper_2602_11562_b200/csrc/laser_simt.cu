@@ -20,7 +20,8 @@ template <typename T>
 __global__ void __launch_bounds__(kProjThreads)
 proj_simt_kernel(const T* __restrict__ X, int rows_per_group, const int* __restrict__ lengths, int d,
                  const T* __restrict__ W0, int n0, float* __restrict__ Y0, float scale0,
-                 const T* __restrict__ W1, int n1, float* __restrict__ Y1) {
+                 const T* __restrict__ W1, int n1, float* __restrict__ Y1, const int* __restrict__ row_off, int n_groups,
+                 int* __restrict__ status) {
   extern __shared__ float xs[];   // [kProjRows][d]
   const int g = blockIdx.y;
   const int r0 = blockIdx.x * kProjRows;
@@ -28,13 +29,18 @@ proj_simt_kernel(const T* __restrict__ X, int rows_per_group, const int* __restr
   if (lengths) {
     int len = lengths[g];
     nrows = len < 0 ? 0 : (len > rows_per_group ? 0 : len);   // out-of-range lengths are reported by the STA kernel
+    if (row_off && nrows > 0 && (row_off[g] < 0 || row_off[g] > row_off[n_groups] - nrows)) {   // packed rows out of range
+      if (threadIdx.x == 0 && blockIdx.x == 0) report_status(status, LASER_ERR_BAD_INPUT);
+      nrows = 0;
+    }
   }
   if (r0 >= nrows) return;
   const int rcount = min(kProjRows, nrows - r0);
-  const size_t base = (size_t)g * rows_per_group + r0;
+  const size_t base = (size_t)g * rows_per_group + r0;                       // rows of the (padded) outputs
+  const size_t in_base = row_off ? (size_t)row_off[g] + r0 : base;          // rows of the input (packed or padded)
   for (int idx = threadIdx.x; idx < kProjRows * d; idx += kProjThreads) {
     int r = idx / d, c = idx - r * d;
-    xs[idx] = r < rcount ? to_f32<T>(X[(base + r) * d + c]) : 0.f;
+    xs[idx] = r < rcount ? to_f32<T>(X[(in_base + r) * d + c]) : 0.f;
   }
   __syncthreads();
   for (int col = threadIdx.x; col < n0 + n1; col += kProjThreads) {
@@ -315,13 +321,13 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     dim3 grid((p.N + kProjRows - 1) / kProjRows, 1);
     LaunchScope ls("proj_simt_q", st);
     proj_simt_kernel<T><<<grid, kProjThreads, proj_smem, st>>>(cands, p.N, nullptr, p.d, Wq, p.dqk, Qf, p.inv_gamma,
-                                                              nullptr, 0, nullptr);
+                                                              nullptr, 0, nullptr, nullptr, 0, status);
   }
   {
     dim3 grid((p.L + kProjRows - 1) / kProjRows, p.U);
     LaunchScope ls("proj_simt_kv", st);
     proj_simt_kernel<T><<<grid, kProjThreads, proj_smem, st>>>(items, p.L, lengths, p.d, Wk, p.dqk, Kf, 1.f, Wv, p.d,
-                                                              Vf);
+                                                              Vf, p.item_offsets, p.U, status);
   }
   {
     const size_t smem = ((size_t)(kStaCands + kStaItems) * (p.dqk + 1) + (size_t)kStaItems * p.d +

@@ -41,6 +41,7 @@ struct StreamParams {
   float inv_gamma;
   const bf16 *items, *cands, *Wq, *Wk, *Wv;
   const int *lengths, *cand_offsets;
+  const int* item_off;            // packed item layout: first row of every user ([U + 1]); null = padded [U, L, d]
   float* u;                       // [U, H, d]
   uint4* imgv;                    // W_v as MMA B fragments: [d/16 k-tiles][d/16 column pairs][32 lanes]
   bf16* Hp;                       // [N, Lp, d]
@@ -55,7 +56,9 @@ struct StreamParams {
 // Candidate of user u, or -1 when it has none (or its offsets / length are invalid).
 __device__ __forceinline__ int user_candidate(const StreamParams& P, int u, int* len_out) {
   const int c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1], len = P.lengths[u];
-  if (c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > 1 || len < 0 || len > P.L) {
+  bool bad = c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > 1 || len < 0 || len > P.L;
+  if (!bad && P.item_off) bad = P.item_off[u] < 0 || P.item_off[u] > P.item_off[P.U] - len;
+  if (bad) {
     report_status(P.status, LASER_ERR_BAD_INPUT);
     return -1;
   }
@@ -198,7 +201,7 @@ __global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
         }
       }
     }
-    const bf16* xu = P.items + (size_t)u * P.L * d;
+    const bf16* xu = P.items + (P.item_off ? (size_t)P.item_off[u] : (size_t)u * P.L) * d;
 
     // fetch cursor over this warp's (segment, 16-row group) sequence.  A stage is kSRows rows of 2 D16 16-byte
     // pieces; lane l copies pieces l, l + 32, ...: their row, source offset and destination offset never change.
@@ -388,6 +391,7 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   P.items = (const bf16*)items; P.cands = (const bf16*)cands;
   P.Wq = (const bf16*)Wq; P.Wk = (const bf16*)Wk; P.Wv = (const bf16*)Wv;
   P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.item_off = p.item_offsets;
   P.u = reinterpret_cast<float*>(ws + p.off_su);
   P.imgv = reinterpret_cast<uint4*>(ws + p.off_su + align_up((size_t)p.U * p.H * p.d * sizeof(float)));
   P.Hp = (bf16*)Hprime;

@@ -37,6 +37,7 @@ struct TcParams {
   float q_scale;                      // 1 / (2 gamma)
   const bf16 *items, *cands, *Wq, *Wk, *Wv;
   const int *lengths, *cand_offsets;
+  const int* item_off;                // packed item layout: first row of every user ([U + 1]); null = padded [U, L, d]
   bf16 *Qblk, *Kblk, *Vtblk;
   int *unit_start, *tile_off;         // [U+1] prefix of attention units / candidate tiles per user
   int* proj_start;                    // [U+1] prefix of projection units (groups of item tiles that hold valid items)
@@ -61,7 +62,11 @@ struct UserShape {
 __device__ __forceinline__ UserShape user_shape(const TcParams& P, int u) {
   UserShape s;
   int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
-  const bool bad = len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+  bool bad = len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
+  if (!bad && P.item_off) {                      // packed rows: the user's valid prefix must lie inside the array
+    const int r0 = P.item_off[u];
+    bad = r0 < 0 || r0 > P.item_off[P.U] - len;
+  }
   s.len = bad ? 0 : len;
   s.c0 = bad ? 0 : c0;
   s.nc = bad ? 0 : c1 - c0;
@@ -102,6 +107,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
       const int len = P.lengths[u], c0 = P.cand_offsets[u], c1 = P.cand_offsets[u + 1];
       bad |= len < 0 || len > P.L || c0 < 0 || c1 < c0 || c1 > P.N || c1 - c0 > P.maxC;
       const UserShape s = user_shape(P, u);
+      bad |= s.len != len && len >= 0 && len <= P.L;      // (the packed-row check of user_shape)
       a += s.ctiles;
       b += s.ctiles * s.nseg;
       c += proj_units_of(P, s);
@@ -276,8 +282,13 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     int row_limit;                                         // rows at or past it are staged as zeros
     if (is_item) {
       const int n0 = pu.seg * P.S + pu.t0 * IT;            // unit row r is item n0 + r
-      base = P.items + ((size_t)pu.u * P.L + n0) * d;
-      row_limit = P.L - n0;
+      if (P.item_off) {                                    // packed rows: never read past the user's valid prefix
+        base = P.items + ((size_t)P.item_off[pu.u] + n0) * d;
+        row_limit = pu.seg_items - pu.t0 * IT;
+      } else {
+        base = P.items + ((size_t)pu.u * P.L + n0) * d;
+        row_limit = P.L - n0;
+      }
     } else {
       base = P.cands + (size_t)(pu.c0 + pu.jt * kCandTile) * d;
       row_limit = pu.nc - pu.jt * kCandTile;
@@ -923,6 +934,7 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.items = (const bf16*)items; P.cands = (const bf16*)cands;
   P.Wq = (const bf16*)Wq; P.Wk = (const bf16*)Wk; P.Wv = (const bf16*)Wv;
   P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.item_off = p.item_offsets;
   P.Qblk = (bf16*)(ws + p.off_tq); P.Kblk = (bf16*)(ws + p.off_tk); P.Vtblk = (bf16*)(ws + p.off_tv);
   P.unit_start = (int*)(ws + p.off_twork);
   P.tile_off = P.unit_start + (p.U + 1);
