@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
   chain_release();
   gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
   gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.nseg,
-                  blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+                  (blockIdx.x * blockDim.x + threadIdx.x) >> 5, (gridDim.x * blockDim.x) >> 5, threadIdx.x & 31);
 }
 
 template <int D16>

@@ -42,25 +42,22 @@ __device__ __forceinline__ void gsta_build_images(const __nv_bfloat16* Wg, uint4
 }
 
 // Per candidate: the number of non-empty segments of its user (what the GSTA kernel's softmax runs over), so that the
-// kernel's blocks need no search through the candidate offsets.  A candidate outside every user's range or a length
-// outside [0, L] is reported through `status` and gets 0 segments.
+// kernel's blocks need no search through the candidate offsets.  Filled user by user: warp `warp_id` of `n_warps` takes
+// users warp_id, warp_id + n_warps, ... and its lanes write that user's candidates.  A user with an invalid length or
+// offsets is reported through `status` and skipped (its candidates keep whatever the scratch held; the GSTA kernel
+// clamps what it reads to [0, L']); so are offsets that do not cover candidates 0 .. N - 1.
 __device__ __forceinline__ void gsta_build_nseg(const int* lengths, const int* cand_offsets, int U, int N, int L, int S,
-                                                int Lp, int* status, int* nseg, int worker, int n_workers) {
-  for (int c = worker; c < N; c += n_workers) {
-    int nv = 0;
-    if (cand_offsets[0] > c || cand_offsets[U] <= c) {
-      atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
-    } else {
-      int lo = 0, hi = U;   // cand_offsets[lo] <= c < cand_offsets[hi]
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (cand_offsets[mid] <= c) lo = mid; else hi = mid;
-      }
-      const int len = lengths[lo];
-      if (len < 0 || len > L) atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
-      else nv = min((len + S - 1) / S, Lp);
+                                                int Lp, int* status, int* nseg, int warp_id, int n_warps, int lane) {
+  if (warp_id == 0 && lane == 0 && N > 0 && (cand_offsets[0] != 0 || cand_offsets[U] < N))
+    atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
+  for (int u = warp_id; u < U; u += n_warps) {
+    const int len = lengths[u], c0 = cand_offsets[u], c1 = cand_offsets[u + 1];
+    if (len < 0 || len > L || c0 < 0 || c1 < c0 || c1 > N) {
+      if (lane == 0) atomicCAS(status, 0, LASER_ERR_BAD_INPUT);
+      continue;
     }
-    nseg[c] = nv;
+    const int nv = min((len + S - 1) / S, Lp);
+    for (int c = c0 + lane; c < c1; c += 32) nseg[c] = nv;
   }
 }
 

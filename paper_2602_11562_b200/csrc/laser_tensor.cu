@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
   }
   if (P.Wg) {
     gsta_build_images(P.Wg, P.gimg, P.d, P.M, g, nthreads);
-    gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.gnseg, g, nthreads);
+    gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.gnseg, g >> 5, nthreads >> 5, tid & 31);
   }
 }
 
