@@ -33,7 +33,8 @@ struct TcParams {
   int U, L, d, dqk, H, S, Lp, N, dqh, dvh, maxC;
   int IT, NT, NTG, NG, n_tiles;       // items per tile, tiles per segment, tiles per projection unit, units per segment
   int cand_tiles_max;
-  int n_obuf;                         // output accumulators in TMEM (2 when they fit beside the gate buffers, else 1)
+  int n_obuf;                         // output accumulators in TMEM (2 when a second one fits, else 1)
+  int o_col1;                         // TMEM column of the second output accumulator
   float q_scale;                      // 1 / (2 gamma)
   const bf16 *items, *cands, *Wq, *Wk, *Wv;
   const int *lengths, *cand_offsets;
@@ -750,7 +751,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
             if (!ok) return;
           }
           tc_fence_after();
-          const uint32_t dO = tmem + kColO + ob * d + c.h * P.dvh;
+          const uint32_t dO = tmem + (ob ? (uint32_t)P.o_col1 : kColO) + c.h * P.dvh;
           const uint64_t vd = v_desc0 + (uint64_t)(c.st * (v_bytes >> 4) + c.h * v_head);
           const int ks2 = c.w.tile_cols(P, c.t) >> 4;     // k-steps that hold valid items
           const bool last = c.t == c.nt - 1 && c.h + kGateGroups >= H;      // my last unit of the segment
@@ -873,7 +874,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], o_par, abortp));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tO = tmem + lane_base + kColO + ob * d;
+        const uint32_t tO = tmem + lane_base + (ob ? (uint32_t)P.o_col1 : kColO);
         for (int c = 0; c < d; c += 16) {
           uint32_t v[16];
           tmem_ld16(tO + c, v);
@@ -927,7 +928,11 @@ TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, c
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.dqh = p.dqh; P.dvh = p.dvh; P.maxC = p.maxC;
   P.IT = p.tg.IT; P.NT = p.tg.NT; P.n_tiles = p.tg.n_tiles; P.cand_tiles_max = p.tg.cand_tiles_max;
-  P.n_obuf = (int)kColO + 2 * p.d <= kStaTmemCols ? 2 : 1;
+  // a second output accumulator: behind the first when both fit, else (at most two heads: warpgroups 2 and 3 idle) in
+  // the score buffers those warpgroups would use
+  if ((int)kColO + 2 * p.d <= kStaTmemCols) { P.n_obuf = 2; P.o_col1 = (int)kColO + p.d; }
+  else if (p.H <= 2 && p.d <= 2 * kItMax) { P.n_obuf = 2; P.o_col1 = 2 * kItMax; }
+  else { P.n_obuf = 1; P.o_col1 = (int)kColO; }
   P.NTG = P.IT <= 64 ? (128 / P.IT < P.NT ? 128 / P.IT : P.NT) : 1;
   P.NG = (P.NT + P.NTG - 1) / P.NTG;
   P.q_scale = 0.5f * p.inv_gamma;
