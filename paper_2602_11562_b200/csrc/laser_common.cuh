@@ -80,6 +80,9 @@ int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const
 bool gsta_mma_supported(const Plan& p);
 size_t gsta_mma_image_bytes(const Plan& p);   // weight images, then the per-candidate segment counts
 size_t gsta_nseg_offset(const Plan& p);       // byte offset of the segment counts inside that scratch
+size_t gsta_order_offset(const Plan& p);      // byte offset of the block launch order (n ints) and its sort keys (n ints), n = ceil(N / 8)
+int gsta_candidates_per_block(const Plan& p);
+bool gsta_wants_order(const Plan& p);         // the kernel runs its blocks longest first (a set-up kernel must build the order)
 // images_ready: the weight images at off_gimg were already built for these weights earlier on the same stream.
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
              const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready);

@@ -39,6 +39,9 @@ struct GstaParams {
   uint4* img;                  // [M][3][d/16 k-tiles][d/16 column pairs][32 lanes]
   int* nseg;                   // [N] non-empty segments per candidate (built with the images)
   int cpb;                     // candidates per block: 16, or 8 (one per warp) when that still fits one wave of blocks
+  int* order;                  // [blocks] launch order, longest first (null: blocks run in candidate order)
+  int* order_keys;             // [blocks] scratch of the sort that builds `order`
+  int build_order;             // the set-up kernel's last block builds `order`
   bf16* z;
   int* status;
 };
@@ -46,9 +49,14 @@ struct GstaParams {
 __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
   chain_wait();
   chain_release();
-  gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+  const int n_blocks = gridDim.x - (P.build_order ? 1 : 0);          // blocks that build images and segment counts
+  if ((int)blockIdx.x == n_blocks) {
+    gsta_build_order(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.cpb, P.order, P.order_keys);
+    return;
+  }
+  gsta_build_images(P.Wg, P.img, P.d, P.M, blockIdx.x * blockDim.x + threadIdx.x, n_blocks * blockDim.x);
   gsta_build_nseg(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.status, P.nseg,
-                  (blockIdx.x * blockDim.x + threadIdx.x) >> 5, (gridDim.x * blockDim.x) >> 5, threadIdx.x & 31);
+                  (blockIdx.x * blockDim.x + threadIdx.x) >> 5, (n_blocks * blockDim.x) >> 5, threadIdx.x & 31);
 }
 
 template <int D16>
@@ -66,10 +74,12 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   uint8_t* stage = reinterpret_cast<uint8_t*>(nv_s + kGT);          // [kGW][2][kChunk] rows
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int c_base = blockIdx.x * P.cpb;
-  const int c_end = min(c_base + P.cpb, P.N);          // rows of the 16-row tile past this are empty
   chain_wait();
   chain_release();
+  // which 16 (or 8) candidates: in launch order when the set-up kernel sorted the blocks, else in candidate order
+  const int blk = P.order ? min(max(P.order[blockIdx.x], 0), (int)gridDim.x - 1) : (int)blockIdx.x;
+  const int c_base = blk * P.cpb;
+  const int c_end = min(c_base + P.cpb, P.N);          // rows of the 16-row tile past this are empty
 
   // Dense phases (A, B, D): warp p < d / 16 owns the 16 output columns 16 p .. 16 p + 15.  Its weight fragments come
   // straight from L2; those of the next dense phase are requested before the block-wide barrier that precedes it, so the
@@ -358,7 +368,26 @@ bool gsta_mma_supported(const Plan& p) {
 }
 
 size_t gsta_nseg_offset(const Plan& p) { return align_up((size_t)p.M * 3 * p.d * p.d * 2); }
-size_t gsta_mma_image_bytes(const Plan& p) { return gsta_nseg_offset(p) + (size_t)p.N * sizeof(int); }
+size_t gsta_order_offset(const Plan& p) { return align_up(gsta_nseg_offset(p) + (size_t)p.N * sizeof(int)); }
+size_t gsta_mma_image_bytes(const Plan& p) {       // the order table and its sort keys: one int each per block of >= 8
+  return gsta_order_offset(p) + 2 * (size_t)((p.N + 7) / 8) * sizeof(int);
+}
+
+// Small batches: 8 candidates per block (every warp then has one candidate instead of two, which halves the
+// per-candidate part of a block's latency) as long as all blocks still run at once, two per SM.
+int gsta_candidates_per_block(const Plan& p) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return (p.N + 7) / 8 <= 2 * sms ? 8 : kGT;
+}
+
+// Sorting the blocks pays only when the grid runs in more than one wave (two blocks per SM).
+bool gsta_wants_order(const Plan& p) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int cpb = gsta_candidates_per_block(p);
+  return p.M > 0 && (p.N + cpb - 1) / cpb > 2 * sms;
+}
 
 int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
              const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready) {
@@ -372,17 +401,18 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   P.nseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.z = (bf16*)z;
   P.status = reinterpret_cast<int*>(ws + p.off_status);
-  {
-    // Small batches: 8 candidates per block (every warp then has one candidate instead of two, which halves the
-    // per-candidate part of a block's latency) as long as all blocks still run at once, two per SM.
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    P.cpb = (p.N + 7) / 8 <= 2 * sms ? 8 : kGT;
-  }
+  P.cpb = gsta_candidates_per_block(p);
+  // The block order exists when this call's own set-up kernel builds it, or when the tensor-core STA path's set-up
+  // kernel built it beside the images; the one-candidate path builds none (its batches are one wave of blocks).
+  const bool ordered = gsta_wants_order(p) && (!images_ready || p.path == LASER_PATH_TENSOR);
+  int* order = reinterpret_cast<int*>(ws + p.off_gimg + gsta_order_offset(p));
+  P.order = ordered ? order : nullptr;
+  P.order_keys = order + (p.N + 7) / 8;
+  P.build_order = ordered && !images_ready;
   if (p.M > 0 && !images_ready) {
     const int total = p.M * 3 * (p.d / 16) * (p.d / 16) * 32;
     LaunchScope ls("gsta_prep", st);
-    LASER_CUDA_OK(launch_chained(gsta_prep_kernel, dim3((total + 255) / 256), dim3(256), 0, st, P));
+    LASER_CUDA_OK(launch_chained(gsta_prep_kernel, dim3((total + 255) / 256 + P.build_order), dim3(256), 0, st, P));
   }
   int rc;
   switch (p.d / 16) {

@@ -50,6 +50,9 @@ struct TcParams {
   const bf16* Wg;                     // GSTA weights whose images this set-up also builds (null: none)
   uint4* gimg;
   int* gnseg;                         // per-candidate segment counts for the GSTA kernel (built with the images)
+  int* gorder;                        // launch order of the GSTA kernel's blocks (null: not wanted), its sort keys, and
+  int* gorder_keys;                   // the candidates per block of that kernel
+  int gcpb;
   int M;
   bf16 *imgK, *imgQ, *imgV;           // W_k^T, W_q^T [dqk x d], W_v^T [128 x d] in canonical K-major layout
   int* status;
@@ -178,8 +181,12 @@ __global__ void __launch_bounds__(1024) tc_prep_kernel(TcParams P) {
     }
     return;
   }
+  if (P.gorder && blockIdx.x == gridDim.x - 1) {   // one extra block when the GSTA kernel wants its blocks sorted
+    gsta_build_order(P.lengths, P.cand_offsets, P.U, P.N, P.L, P.S, P.Lp, P.gcpb, P.gorder, P.gorder_keys);
+    return;
+  }
   // remaining blocks: weight images, grid-stride
-  const int nthreads = (gridDim.x - 1) * blockDim.x;
+  const int nthreads = (gridDim.x - 1 - (P.gorder ? 1 : 0)) * blockDim.x;
   const int g = (blockIdx.x - 1) * blockDim.x + tid;
   const int nK = P.dqk * P.d;
   for (int i = g; i < nK; i += nthreads) {       // i = k * dqk + j  (coalesced read of W[k][j])
@@ -924,7 +931,7 @@ int sm_count() {
 
 TcParams make_params(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
                      const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, void* Hp, char* ws) {
-  TcParams P;
+  TcParams P = {};
   P.U = p.U; P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.dqh = p.dqh; P.dvh = p.dvh; P.maxC = p.maxC;
   P.IT = p.tg.IT; P.NT = p.tg.NT; P.n_tiles = p.tg.n_tiles; P.cand_tiles_max = p.tg.cand_tiles_max;
@@ -998,10 +1005,16 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   P.gimg = reinterpret_cast<uint4*>(ws + p.off_gimg);
   P.gnseg = reinterpret_cast<int*>(ws + p.off_gimg + gsta_nseg_offset(p));
   P.M = p.M;
+  P.gorder = nullptr;
+  if (P.Wg && gsta_wants_order(p)) {
+    P.gorder = reinterpret_cast<int*>(ws + p.off_gimg + gsta_order_offset(p));
+    P.gorder_keys = P.gorder + (p.N + 7) / 8;
+    P.gcpb = gsta_candidates_per_block(p);
+  }
   const int sms = sm_count();
   {
     LaunchScope ls("tc_prep", st);
-    LASER_CUDA_OK(launch_chained(tc_prep_kernel, dim3(1 + 32), dim3(1024), 0, st, P));
+    LASER_CUDA_OK(launch_chained(tc_prep_kernel, dim3(1 + 32 + (P.gorder ? 1 : 0)), dim3(1024), 0, st, P));
   }
   {
     const size_t smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;   // W_k^T | W_q^T, W_v^T, two staging buffers

@@ -334,3 +334,25 @@ def test_production_shape_segment_sizes_tensor_path(S):
     z = P.laser_forward_ffn(b.cfg, *b.args(), b.Wg, fdev, workspace=ws)
     assert P.laser_check_status(ws) == 0
     assert err_metric(to_np(z), z_ref) <= TOL["bf16"]
+
+
+def test_gsta_blocks_in_sorted_order_cover_every_candidate():
+    # More 16-candidate GSTA blocks (330) than run at once (two per SM), so the kernel takes them longest first from the
+    # order that the set-up kernels build; every candidate of every user is compared, after the full forward (order
+    # built by the STA set-up kernel) and for the GSTA entry point alone (order built by its own set-up kernel).
+    rng = np.random.default_rng(77)
+    lengths = rng.integers(0, 65, size=48).tolist()
+    lengths[3], lengths[17], lengths[40] = 0, 64, 1
+    w = make_custom(dtype="bf16", seed=977, U=48, C=110, L=64, d=16, H=1, S=16, M=2, d_qh=16, lengths=lengths)
+    check_against_oracle(w, "tensor")
+    s = w.spec
+    Hp_ref, _ = oracle_forward(w)
+    Hp_in = round_to_dtype(Hp_ref.astype(np.float32), "bf16")
+    z_ref = laser_oracle.gsta_forward(Hp_in, w.lengths, w.cand_offsets, w.cands, w.Wg, s.S, s.H, w.tau)
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
+    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)                                           # stale scratch must not matter
+    z = P.laser_gsta_forward(b.cfg, torch.from_numpy(Hp_in).to(torch.bfloat16).cuda(), b.lengths, b.cand_offsets,
+                             b.cands, b.Wg, workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    assert err_metric(to_np(z), z_ref) <= TOL["bf16"]
