@@ -231,7 +231,11 @@ LASER_API int laser_sta_forward_static(const laser_config* cfg, const void* item
 LASER_API size_t laser_host_workspace_bytes(const laser_config* cfg);
 
 /* laser_forward for callers whose data lives in HOST memory (the end-to-end path): copies the inputs to
- * the device, runs laser_forward without H' output, copies z back.
+ * the device, runs laser_forward without H' output, copies z back.  Rows of items_h at or past a user's length
+ * need not cross the bus: when that saves enough, only each user's valid prefix travels, into a gap-free
+ * device array that the kernels read as in laser_forward_packed.  If items_h is pinned (or registered) host
+ * memory, one kernel reads the valid rows straight from it; otherwise there is one copy per run of users whose
+ * valid rows are contiguous in items_h.  z is bit-identical whatever the route.
  *   items_h, lengths_h, cands_h, cand_offsets_h, Wq_h, Wk_h, Wv_h, Wgsta_h : HOST pointers, same shapes
  *       and dtype as above (pinned memory makes the copies asynchronous; pageable memory also works)
  *   z_h        HOST pointer, OUT [N, d]
@@ -243,6 +247,16 @@ LASER_API int laser_forward_host(const laser_config* cfg, const void* items_h, c
                        const void* cands_h, const int32_t* cand_offsets_h, const void* Wq_h, const void* Wk_h,
                        const void* Wv_h, const void* Wgsta_h, void* z_h, void* workspace, size_t workspace_bytes,
                        void* cuda_stream, int blocking);
+
+/* Bytes laser_forward_host moves for this batch: host to device (every input; of the items only what the
+ * route chosen for this pointer and these lengths transfers) and device to host (z).  Launches nothing.
+ *   items_h    HOST pointer as it would be passed to laser_forward_host (only its kind and alignment matter;
+ *              null: treated as pageable memory)
+ *   lengths_h  HOST pointer, [U]
+ *   h2d_bytes, d2h_bytes  HOST pointers, OUT
+ * Returns LASER_OK, or LASER_ERR_INVALID_ARG / LASER_ERR_UNSUPPORTED as laser_forward_host would. */
+LASER_API int laser_host_transfer_bytes(const laser_config* cfg, const void* items_h, const int32_t* lengths_h,
+                                        size_t* h2d_bytes, size_t* d2h_bytes);
 
 /* Waits for `cuda_stream`, reads the device status word at the start of `workspace` and returns it
  * (LASER_OK, LASER_ERR_TIMEOUT, LASER_ERR_BAD_INPUT) or LASER_ERR_CUDA if the stream reports an error. */

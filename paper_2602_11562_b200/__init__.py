@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     library_path,
     make_config,
     laser_workspace_bytes,
+    laser_host_transfer_bytes,
     laser_host_workspace_bytes,
     laser_sta_forward,
     laser_sta_forward_static,

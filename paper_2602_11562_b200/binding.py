@@ -70,6 +70,8 @@ def load_library() -> ctypes.CDLL:
     lib.laser_workspace_bytes.argtypes = [cfgp]
     lib.laser_host_workspace_bytes.restype = sz
     lib.laser_host_workspace_bytes.argtypes = [cfgp]
+    lib.laser_host_transfer_bytes.restype = ctypes.c_int
+    lib.laser_host_transfer_bytes.argtypes = [cfgp, vp, i32p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
     lib.laser_sta_forward.restype = ctypes.c_int
     lib.laser_sta_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, sz, vp]
     lib.laser_gsta_forward.restype = ctypes.c_int
@@ -127,6 +129,21 @@ def laser_workspace_bytes(cfg: LaserConfig) -> int:
 
 def laser_host_workspace_bytes(cfg: LaserConfig) -> int:
     return int(load_library().laser_host_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_host_transfer_bytes(cfg: LaserConfig, lengths_h, items_h=None) -> tuple:
+    """(host-to-device bytes, device-to-host bytes) that laser_forward_host moves for these HOST lengths and this HOST
+    items tensor (None: as for pageable memory)."""
+    if lengths_h.is_cuda or lengths_h.dtype != torch.int32 or not lengths_h.is_contiguous():
+        raise LaserError(-1, "laser_host_transfer_bytes (lengths must be a contiguous int32 HOST tensor)")
+    if items_h is not None and items_h.is_cuda:
+        raise LaserError(-1, "laser_host_transfer_bytes (items must be a HOST tensor)")
+    h2d, d2h = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(load_library().laser_host_transfer_bytes(ctypes.byref(cfg),
+                                                    ctypes.c_void_p(items_h.data_ptr() if items_h is not None else 0),
+                                                    ctypes.c_void_p(lengths_h.data_ptr()), ctypes.byref(h2d),
+                                                    ctypes.byref(d2h)), "laser_host_transfer_bytes")
+    return int(h2d.value), int(d2h.value)
 
 
 def laser_last_launch_count() -> int:

@@ -2,6 +2,10 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
+#include <utility>
+#include <vector>
+
 #include "laser_common.cuh"
 
 namespace laser {
@@ -345,7 +349,7 @@ int laser_forward_ffn(const laser_config* cfg, const void* items, const int32_t*
 
 namespace {
 struct HostStage {
-  size_t items, lengths, cands, offs, wq, wk, wv, wg, z, total;
+  size_t items, lengths, cands, offs, item_offs, wq, wk, wv, wg, z, total;
   size_t b_items, b_lengths, b_cands, b_offs, b_wq, b_wk, b_wv, b_wg, b_z;
 };
 HostStage host_stage(const Plan& p) {
@@ -363,6 +367,7 @@ HostStage host_stage(const Plan& p) {
   s.lengths = off; off = align_up(off + s.b_lengths);
   s.cands = off; off = align_up(off + s.b_cands);
   s.offs = off; off = align_up(off + s.b_offs);
+  s.item_offs = off; off = align_up(off + s.b_offs);
   s.wq = off; off = align_up(off + s.b_wq);
   s.wk = off; off = align_up(off + s.b_wk);
   s.wv = off; off = align_up(off + s.b_wv);
@@ -371,7 +376,100 @@ HostStage host_stage(const Plan& p) {
   s.total = off;
   return s;
 }
+
+// How the item rows travel to the device.  The lengths are known on the host, so rows past a user's valid prefix need
+// not cross the bus; the valid rows land in a gap-free device array, which the kernels then read through per-user row
+// offsets exactly as for laser_forward_packed.  Three routes:
+//   kGather  items_h is pinned (or registered) host memory with a device alias: one kernel reads the valid rows straight
+//            from it.  Taken when it saves at least kGatherWorth bytes.
+//   kRuns    one copy per run of users whose valid rows are contiguous in the padded host array (a run ends after the
+//            first user shorter than L).  Every copy has a fixed cost on the host (several microseconds, i.e. some
+//            hundred KB of bus time), so this is taken only when it saves at least kCopyWorth bytes per copy.
+//   kPadded  the padded array travels in one piece.
+enum HostRouteKind { kPadded, kRuns, kGather };
+struct HostItemRoute {
+  HostRouteKind kind;
+  size_t bytes;                          // item bytes that travel
+  const void* alias;                     // kGather: device alias of items_h
+  std::vector<int32_t> row_off;          // [U + 1] first packed row per user (kRuns, kGather)
+};
+constexpr size_t kCopyWorth = 384 * 1024, kGatherWorth = 256 * 1024;
+constexpr int kGatherThreads = 256;
+
+HostItemRoute host_item_route(const Plan& p, const void* items_h, const int32_t* lengths_h) {
+  HostItemRoute r;
+  const size_t row = (size_t)p.d * p.esize, padded = (size_t)p.U * p.L * row;
+  r.kind = kPadded;
+  r.bytes = padded;
+  r.alias = nullptr;
+  if (p.U == 0 || p.N == 0) return r;
+  std::vector<int32_t> off((size_t)p.U + 1);
+  long long rows = 0;
+  size_t copies = 0;
+  bool contiguous = false;               // the previous user's rows end where this user's begin
+  for (int u = 0; u < p.U; ++u) {
+    const int len = std::min(std::max(lengths_h[u], 0), p.L);   // invalid lengths are reported by the device
+    off[u] = (int32_t)rows;
+    if (len > 0 && !contiguous) ++copies;
+    contiguous = len == p.L;
+    rows += len;
+  }
+  off[p.U] = (int32_t)rows;
+  if (rows > 0x7fffffffLL) return r;
+  const size_t need = (size_t)rows * row;
+  if (items_h && row % 16 == 0 && (reinterpret_cast<uintptr_t>(items_h) & 15) == 0 && need + kGatherWorth < padded) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, items_h) == cudaSuccess) {
+      if (attr.type == cudaMemoryTypeHost && attr.devicePointer) {
+        r.kind = kGather;
+        r.alias = attr.devicePointer;
+      }
+    } else {
+      cudaGetLastError();                // (no device, or a runtime that rejects pageable pointers: not an error here)
+    }
+  }
+  if (r.kind == kPadded && need + copies * kCopyWorth < padded) r.kind = kRuns;
+  if (r.kind == kPadded) return r;
+  r.bytes = need;
+  r.row_off = std::move(off);
+  return r;
+}
+
+// kGather: block (u, j) copies rows j * rows_per_block ... of user u's valid prefix, 16 bytes per thread and step, from
+// the padded host array (through its device alias) to the user's place in the gap-free device array.
+__global__ void __launch_bounds__(kGatherThreads) host_gather_kernel(const uint4* __restrict__ src,
+                                                                     uint4* __restrict__ dst, const int32_t* lengths,
+                                                                     const int32_t* row_off, int L, int vec,
+                                                                     int rows_per_block) {
+  chain_wait();                          // (the next kernel starts once this grid has drained: nothing to overlap with)
+  const int u = blockIdx.x;
+  const int len = min(max(lengths[u], 0), L);              // as the host clamped it when it built row_off
+  const int r0 = blockIdx.y * rows_per_block;
+  if (r0 >= len) return;
+  const int n = min(rows_per_block, len - r0) * vec;
+  const uint4* s = src + ((size_t)u * L + r0) * vec;
+  uint4* d = dst + ((size_t)row_off[u] + r0) * vec;
+#pragma unroll 4
+  for (int i = threadIdx.x; i < n; i += kGatherThreads) d[i] = s[i];
+}
 }  // namespace
+
+int laser_host_transfer_bytes(const laser_config* cfg, const void* items_h, const int32_t* lengths_h,
+                              size_t* h2d_bytes, size_t* d2h_bytes) {
+  Plan p;
+  int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (!lengths_h || !h2d_bytes || !d2h_bytes) return LASER_ERR_INVALID_ARG;
+  const HostStage s = host_stage(p);
+  *h2d_bytes = s.b_lengths + s.b_offs;
+  *d2h_bytes = 0;
+  if (p.N > 0) {
+    const HostItemRoute r = host_item_route(p, items_h, lengths_h);
+    *h2d_bytes += r.bytes + (r.kind != kPadded ? s.b_offs : 0) + s.b_cands + s.b_wq + s.b_wk + s.b_wv + s.b_wg;
+    *d2h_bytes = s.b_z;
+  }
+  return LASER_OK;
+}
 
 size_t laser_host_workspace_bytes(const laser_config* cfg) {
   Plan p;
@@ -402,7 +500,31 @@ int laser_forward_host(const laser_config* cfg, const void* items_h, const int32
   LASER_CUDA_OK(h2d(s.lengths, lengths_h, s.b_lengths));
   LASER_CUDA_OK(h2d(s.offs, cand_offsets_h, s.b_offs));
   if (p.N > 0) {
-    LASER_CUDA_OK(h2d(s.items, items_h, s.b_items));
+    const HostItemRoute route = host_item_route(p, items_h, lengths_h);
+    if (route.kind == kPadded) LASER_CUDA_OK(h2d(s.items, items_h, s.b_items));
+    else {
+      // (the offsets live in pageable memory: the runtime stages such a source before the call returns)
+      LASER_CUDA_OK(h2d(s.item_offs, route.row_off.data(), s.b_offs));
+      const size_t row = (size_t)p.d * p.esize;
+      if (route.kind == kGather) {
+        const int per = std::max(64, (p.L + 65534) / 65535);            // rows per block; grid.y <= 65535
+        LaunchScope ls("host_gather", st);
+        LASER_CUDA_OK(launch_chained(host_gather_kernel, dim3(p.U, (p.L + per - 1) / per), dim3(kGatherThreads), 0, st,
+                                     static_cast<const uint4*>(route.alias), reinterpret_cast<uint4*>(ws + s.items),
+                                     reinterpret_cast<const int32_t*>(ws + s.lengths),
+                                     reinterpret_cast<const int32_t*>(ws + s.item_offs), p.L, (int)(row / 16), per));
+      } else {
+        const char* src = static_cast<const char*>(items_h);
+        for (int u = 0; u < p.U;) {        // one copy per run of users whose valid rows are contiguous on the host
+          int e = u;
+          while (e + 1 < p.U && route.row_off[e + 1] - route.row_off[e] == p.L) ++e;
+          const size_t rows = (size_t)(route.row_off[e + 1] - route.row_off[u]);
+          LASER_CUDA_OK(h2d(s.items + (size_t)route.row_off[u] * row, src + (size_t)u * p.L * row, rows * row));
+          u = e + 1;
+        }
+      }
+      p.item_offsets = reinterpret_cast<const int32_t*>(ws + s.item_offs);
+    }
     LASER_CUDA_OK(h2d(s.cands, cands_h, s.b_cands));
     LASER_CUDA_OK(h2d(s.wq, Wq_h, s.b_wq));
     LASER_CUDA_OK(h2d(s.wk, Wk_h, s.b_wk));

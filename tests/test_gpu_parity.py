@@ -296,6 +296,51 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert torch.equal(z_h, z_dev.cpu())
 
 
+@pytest.mark.parametrize("path", ["simt", "tensor", "auto"])
+def test_host_buffer_entry_point_sends_only_valid_rows_when_that_pays(path):
+    # Long padded rows, short valid prefixes: the host entry point moves the prefixes alone (pinned memory: one kernel
+    # reads them from the host array; pageable memory: two copies here, since users 0 and 1 are contiguous on the host,
+    # user 2 has no items and user 3 starts a new run) and must give the bits of the device entry point on the padded
+    # batch; the padding on the host is NaN, which no kernel may ever see.
+    lengths = [2048, 10, 0, 700]
+    w = make_custom(U=4, C=5, L=2048, d=64, H=2, S=64, M=2, dtype="bf16", seed=23, lengths=lengths)
+    z_dev = run_forward(w, path, want_hprime=False).cpu()
+    row = 64 * 2
+    for pinned in (True, False):
+        hb = P.DeviceBatch.from_workload(w, path=PATHS[path], device="cpu", pin_host=pinned)
+        h2d, d2h = P.laser_host_transfer_bytes(hb.cfg, hb.lengths, hb.items)
+        every = sum(t.numel() * t.element_size() for t in (*hb.args(), hb.Wg))
+        if pinned:                                              # the valid rows and the row-offset table instead
+            assert h2d == every - (4 * 2048 - sum(lengths)) * row + 5 * 4
+        else:                                                   # two more copies would cost more than they save here
+            assert h2d == every
+        assert d2h == 20 * row
+        for u, n in enumerate(lengths):
+            hb.items[u, n:] = float("nan") if pinned else 7.0
+        ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
+        z_h = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype)
+        z_h = z_h.pin_memory() if pinned else z_h
+        P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
+        assert torch.equal(z_h, z_dev)
+
+
+def test_host_buffer_entry_point_pageable_memory_copies_runs_of_users():
+    # Pageable host memory and much padding: one copy per run of users whose valid rows are contiguous on the host.
+    lengths = [8192, 8192, 100, 0, 0, 3000, 8192, 1]
+    w = make_custom(U=8, C=2, L=8192, d=64, H=2, S=128, M=1, dtype="bf16", seed=24, lengths=lengths)
+    z_dev = run_forward(w, "auto", want_hprime=False).cpu()
+    hb = P.DeviceBatch.from_workload(w, device="cpu")
+    h2d, _ = P.laser_host_transfer_bytes(hb.cfg, hb.lengths, hb.items)
+    every = sum(t.numel() * t.element_size() for t in (*hb.args(), hb.Wg))
+    assert h2d == every - (8 * 8192 - sum(lengths)) * 128 + 9 * 4
+    for u, n in enumerate(lengths):
+        hb.items[u, n:] = float("nan")
+    ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
+    z_h = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype)
+    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
+    assert torch.equal(z_h, z_dev)
+
+
 # ------------------------------------------------------------------ full-size configurations, sampled users
 @pytest.mark.parametrize("name,n_users", [("cfg3", 3), ("cfg4", 2), ("cfg5", 48)])
 def test_full_size_configs_sampled_users(name, n_users):

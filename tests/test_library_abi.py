@@ -56,6 +56,26 @@ def test_workspace_query_and_validation(lib):
     assert "workspace" in P.laser_status_string(-3)
 
 
+def test_host_transfer_size_query(lib):
+    import torch
+    # 4 users x 4096 rows of 128 bf16 features (256 bytes each): everything else is small next to the items.  Without
+    # a pinned items pointer the route is the one for pageable memory: one copy per run of contiguous users.
+    cfg = _cfg(num_users=4, max_len=4096, d_model=128, d_qk=32, seg_size=128, dtype="bf16", total_cands=8,
+               max_cands_per_user=2)
+    row = 256
+    other = 4 * 4 + 5 * 4 + 8 * row + 2 * 128 * 32 * 2 + 128 * 128 * 2 + 3 * 128 * 128 * 2
+    full = torch.full((4,), 4096, dtype=torch.int32)
+    assert P.laser_host_transfer_bytes(cfg, full) == (4 * 4096 * row + other, 8 * row)      # one padded copy
+    short = torch.tensor([4096, 100, 0, 4096], dtype=torch.int32)                           # two runs
+    assert P.laser_host_transfer_bytes(cfg, short) == ((4096 + 100 + 4096) * row + 5 * 4 + other, 8 * row)
+    # lengths outside [0, L] are clamped for the copy (the device reports them)
+    bad = torch.tensor([-5, 100, 9999, 7], dtype=torch.int32)                               # two runs
+    assert P.laser_host_transfer_bytes(cfg, bad) == ((100 + 4096 + 7) * row + 5 * 4 + other, 8 * row)
+    # saving less than the fixed cost of the extra copies: the padded array travels in one piece
+    nearly = torch.tensor([3000, 3000, 3000, 3000], dtype=torch.int32)
+    assert P.laser_host_transfer_bytes(cfg, nearly)[0] == 4 * 4096 * row + other
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     from paper_2602_11562_b200 import binding
     monkeypatch.setattr(binding, "_LIB", None)
