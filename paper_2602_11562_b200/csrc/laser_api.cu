@@ -3,8 +3,6 @@
 #include <string.h>
 
 #include <algorithm>
-#include <utility>
-#include <vector>
 
 #include "laser_common.cuh"
 
@@ -391,7 +389,6 @@ struct HostItemRoute {
   HostRouteKind kind;
   size_t bytes;                          // item bytes that travel
   const void* alias;                     // kGather: device alias of items_h
-  std::vector<int32_t> row_off;          // [U + 1] first packed row per user (kRuns, kGather)
 };
 constexpr size_t kCopyWorth = 384 * 1024, kGatherWorth = 256 * 1024;
 constexpr int kGatherThreads = 256;
@@ -403,18 +400,15 @@ HostItemRoute host_item_route(const Plan& p, const void* items_h, const int32_t*
   r.bytes = padded;
   r.alias = nullptr;
   if (p.U == 0 || p.N == 0) return r;
-  std::vector<int32_t> off((size_t)p.U + 1);
   long long rows = 0;
   size_t copies = 0;
   bool contiguous = false;               // the previous user's rows end where this user's begin
   for (int u = 0; u < p.U; ++u) {
     const int len = std::min(std::max(lengths_h[u], 0), p.L);   // invalid lengths are reported by the device
-    off[u] = (int32_t)rows;
     if (len > 0 && !contiguous) ++copies;
     contiguous = len == p.L;
     rows += len;
   }
-  off[p.U] = (int32_t)rows;
   if (rows > 0x7fffffffLL) return r;
   const size_t need = (size_t)rows * row;
   if (items_h && row % 16 == 0 && (reinterpret_cast<uintptr_t>(items_h) & 15) == 0 && need + kGatherWorth < padded) {
@@ -429,10 +423,34 @@ HostItemRoute host_item_route(const Plan& p, const void* items_h, const int32_t*
     }
   }
   if (r.kind == kPadded && need + copies * kCopyWorth < padded) r.kind = kRuns;
-  if (r.kind == kPadded) return r;
-  r.bytes = need;
-  r.row_off = std::move(off);
+  if (r.kind != kPadded) r.bytes = need;
   return r;
+}
+
+// First row of every user in the gap-free array: exclusive prefix sums of the lengths, clamped to [0, L] as the host
+// clamps them when it sizes its copies.  One block; computed on the device so that the host never has to hand a
+// pageable table to an asynchronous copy (which would make it wait for the stream on every call).
+__global__ void __launch_bounds__(1024) host_row_offsets_kernel(const int32_t* lengths, int U, int L, int32_t* row_off) {
+  chain_wait();
+  __shared__ int part[1024];
+  const int tid = threadIdx.x, per = (U + 1023) / 1024;
+  const int u0 = min(tid * per, U), u1 = min(u0 + per, U);
+  int sum = 0;
+  for (int u = u0; u < u1; ++u) sum += min(max(lengths[u], 0), L);
+  part[tid] = sum;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {
+    const int v = tid >= off ? part[tid - off] : 0;
+    __syncthreads();
+    part[tid] += v;
+    __syncthreads();
+  }
+  int run = part[tid] - sum;
+  for (int u = u0; u < u1; ++u) {
+    row_off[u] = run;
+    run += min(max(lengths[u], 0), L);
+  }
+  if (tid == 1023) row_off[U] = part[1023];
 }
 
 // kGather: block (u, j) copies rows j * rows_per_block ... of user u's valid prefix, 16 bytes per thread and step, from
@@ -465,7 +483,7 @@ int laser_host_transfer_bytes(const laser_config* cfg, const void* items_h, cons
   *d2h_bytes = 0;
   if (p.N > 0) {
     const HostItemRoute r = host_item_route(p, items_h, lengths_h);
-    *h2d_bytes += r.bytes + (r.kind != kPadded ? s.b_offs : 0) + s.b_cands + s.b_wq + s.b_wk + s.b_wv + s.b_wg;
+    *h2d_bytes += r.bytes + s.b_cands + s.b_wq + s.b_wk + s.b_wv + s.b_wg;
     *d2h_bytes = s.b_z;
   }
   return LASER_OK;
@@ -503,8 +521,12 @@ int laser_forward_host(const laser_config* cfg, const void* items_h, const int32
     const HostItemRoute route = host_item_route(p, items_h, lengths_h);
     if (route.kind == kPadded) LASER_CUDA_OK(h2d(s.items, items_h, s.b_items));
     else {
-      // (the offsets live in pageable memory: the runtime stages such a source before the call returns)
-      LASER_CUDA_OK(h2d(s.item_offs, route.row_off.data(), s.b_offs));
+      {
+        LaunchScope ls("host_row_offsets", st);
+        LASER_CUDA_OK(launch_chained(host_row_offsets_kernel, dim3(1), dim3(1024), 0, st,
+                                     reinterpret_cast<const int32_t*>(ws + s.lengths), p.U, p.L,
+                                     reinterpret_cast<int32_t*>(ws + s.item_offs)));
+      }
       const size_t row = (size_t)p.d * p.esize;
       if (route.kind == kGather) {
         const int per = std::max(64, (p.L + 65534) / 65535);            // rows per block; grid.y <= 65535
@@ -515,11 +537,17 @@ int laser_forward_host(const laser_config* cfg, const void* items_h, const int32
                                      reinterpret_cast<const int32_t*>(ws + s.item_offs), p.L, (int)(row / 16), per));
       } else {
         const char* src = static_cast<const char*>(items_h);
+        size_t first_row = 0;              // of the run in the gap-free array
         for (int u = 0; u < p.U;) {        // one copy per run of users whose valid rows are contiguous on the host
+          size_t rows = 0;
           int e = u;
-          while (e + 1 < p.U && route.row_off[e + 1] - route.row_off[e] == p.L) ++e;
-          const size_t rows = (size_t)(route.row_off[e + 1] - route.row_off[u]);
-          LASER_CUDA_OK(h2d(s.items + (size_t)route.row_off[u] * row, src + (size_t)u * p.L * row, rows * row));
+          for (;; ++e) {
+            const int len = std::min(std::max(lengths_h[e], 0), p.L);
+            rows += (size_t)len;
+            if (len != p.L || e + 1 == p.U) break;
+          }
+          LASER_CUDA_OK(h2d(s.items + first_row * row, src + (size_t)u * p.L * row, rows * row));
+          first_row += rows;
           u = e + 1;
         }
       }

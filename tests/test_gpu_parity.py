@@ -310,8 +310,8 @@ def test_host_buffer_entry_point_sends_only_valid_rows_when_that_pays(path):
         hb = P.DeviceBatch.from_workload(w, path=PATHS[path], device="cpu", pin_host=pinned)
         h2d, d2h = P.laser_host_transfer_bytes(hb.cfg, hb.lengths, hb.items)
         every = sum(t.numel() * t.element_size() for t in (*hb.args(), hb.Wg))
-        if pinned:                                              # the valid rows and the row-offset table instead
-            assert h2d == every - (4 * 2048 - sum(lengths)) * row + 5 * 4
+        if pinned:                                              # the valid rows alone
+            assert h2d == every - (4 * 2048 - sum(lengths)) * row
         else:                                                   # two more copies would cost more than they save here
             assert h2d == every
         assert d2h == 20 * row
@@ -332,7 +332,7 @@ def test_host_buffer_entry_point_pageable_memory_copies_runs_of_users():
     hb = P.DeviceBatch.from_workload(w, device="cpu")
     h2d, _ = P.laser_host_transfer_bytes(hb.cfg, hb.lengths, hb.items)
     every = sum(t.numel() * t.element_size() for t in (*hb.args(), hb.Wg))
-    assert h2d == every - (8 * 8192 - sum(lengths)) * 128 + 9 * 4
+    assert h2d == every - (8 * 8192 - sum(lengths)) * 128
     for u, n in enumerate(lengths):
         hb.items[u, n:] = float("nan")
     ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
