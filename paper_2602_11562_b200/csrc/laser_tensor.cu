@@ -11,6 +11,9 @@
 //                    and H' = O / 2.  Uses Sigmoid(x) = (1 + tanh(x/2)) / 2 with 1 / (2 gamma) folded into Q: one
 //                    transcendental and one add per gate.  Masked items have zero K and V rows, so they contribute
 //                    exactly nothing.  No score ever leaves the SM.
+#include <cuda.h>
+#include <string.h>
+
 #include "laser_common.cuh"
 #include "laser_gsta_img.cuh"
 #include "laser_ptx.cuh"
@@ -232,9 +235,10 @@ struct ProjUnit {
   int jt, c0, nc;                       // candidate unit: tile jt of user u, whose candidates are [c0, c0 + nc)
 };
 
-__global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
-  extern __shared__ __align__(128) uint8_t smem_raw[];
-  __shared__ uint64_t bar_img, bar_mma;
+__global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P, const __grid_constant__ CUtensorMap tmap_items,
+                                                              int use_tma) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ uint64_t bar_img, bar_mma, bar_x[2];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ int s_kcol[16];            // per 8-column group of K / Q: (head << 8) | (8-column chunk within the head)
@@ -249,6 +253,8 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   if (tid == 0) {
     mbar_init(&bar_img, 1);
     mbar_init(&bar_mma, 1);
+    mbar_init(&bar_x[0], 1);
+    mbar_init(&bar_x[1], 1);
     s_abort = 0;
     fence_mbar_init();
   }
@@ -266,6 +272,7 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
   const uint32_t bK = dqk * d * 2, bV = kCandTile * d * 2;
+  if (smem_u32(Xbuf) & 1023u) use_tma = 0;   // (the swizzled layout needs 1024-byte aligned buffers; else plain copies)
   chain_wait();                         // the set-up kernel's images, prefixes and start cursors are complete
   chain_release();
 
@@ -322,17 +329,25 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
   const int npr = P.dvh >> 3;                          // 8-row groups per head
 
   // multiply the staged unit and drain the accumulators
-  auto run_unit = [&](const ProjUnit& pu, bool is_item, bf16* X) -> bool {
+  // x_bar: null when the rows were staged with cp.async (canonical layout, already complete); else the mbarrier of
+  // the TMA copies that bring them in the 128-byte swizzled layout (two 64-column halves of 128 rows, 16 KB apart).
+  auto run_unit = [&](const ProjUnit& pu, bool is_item, bf16* X, uint64_t* x_bar, uint32_t x_phase) -> bool {
     if (warp == 0) {                                         // warp-uniform loop, one elected lane issues
+      const bool staged = x_bar == nullptr || mbar_wait(x_bar, x_phase, abortp);
+      __syncwarp();
       tc_fence_after();
-      const uint64_t xd = smem_desc(smem_u32(X), lbo, sbo), wd = smem_desc(smem_u32(imgK), lbo, sbo);
-      const uint64_t vd = smem_desc(smem_u32(imgV), lbo, sbo);
+      const uint32_t xa = smem_u32(X);
+      const uint64_t wd = smem_desc(smem_u32(imgK), lbo, sbo), vd = smem_desc(smem_u32(imgV), lbo, sbo);
       const int ksteps = d >> 4;
       const uint32_t id1 = idesc_bf16(128, dqk), id2 = idesc_bf16(128, pu.rows);
-      if (elect_one()) {
-        for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem, xd + ks * 16, wd + ks * 16, id1, ks > 0);
+      auto xdesc = [&](int ks) -> uint64_t {
+        return x_bar ? smem_desc_sw128(xa + (uint32_t)(ks >> 2) * (kCandTile * 128)) + (uint64_t)((ks & 3) * 2)
+                     : smem_desc(xa, lbo, sbo) + (uint64_t)(ks * 16);
+      };
+      if (staged && elect_one()) {
+        for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem, xdesc(ks), wd + ks * 16, id1, ks > 0);
         if (is_item)
-          for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem + 128, vd + ks * 16, xd + ks * 16, id2, ks > 0);
+          for (int ks = 0; ks < ksteps; ++ks) mma_ss(tmem + 128, vd + ks * 16, xdesc(ks), id2, ks > 0);
         tc_commit(&bar_mma);
       }
       __syncwarp();
@@ -428,13 +443,13 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
     return true;
   };
 
-  bool ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
-
   // ---- item units: this block's contiguous range, two-deep pipeline
+  bool ok = true;
   const int n_proj = P.counters[2];
   const int G = gridDim.x, bidx = blockIdx.x;
   const int lo = (int)(((long long)n_proj * bidx) / G), hi = (int)(((long long)n_proj * (bidx + 1)) / G);
-  if (ok && hi > lo) {
+  if (hi <= lo) ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
+  else {
     // cursor over (user, segment, tile group)
     int cu, cseg, cgrp, c_nseg, c_len, c_last_groups;
     auto set_len = [&](int len) {
@@ -473,22 +488,58 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
 
     ProjUnit cur = make_unit();
     int buf = 0;
-    stage(cur, true, Xbuf);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int n = lo; n < hi && ok; ++n) {
-      ProjUnit nxt = cur;
-      if (n + 1 < hi) {
-        step();
-        nxt = make_unit();
-        stage(nxt, true, Xbuf + (size_t)(buf ^ 1) * kCandTile * d);
+    if (use_tma) {
+      // One thread asks the TMA unit for the rows of a unit: per item tile and 64-column half one tiled copy (IT rows of
+      // 128 bytes, 128-byte swizzle), all completing on the buffer's mbarrier.  Rows past the end of the item array
+      // arrive as zeros; rows past the user's block are another user's (finite) rows and are masked like padding.
+      auto fetch = [&](const ProjUnit& pu, int b) {
+        const uint32_t dst = smem_u32(Xbuf + (size_t)b * kCandTile * d);
+        const int row0 = pu.u * P.L + pu.seg * P.S + pu.t0 * IT;
+        mbar_arrive_expect_tx(&bar_x[b], (uint32_t)pu.rows * d * 2);
+        for (int t = 0; t * IT < pu.rows; ++t)
+          for (int kh = 0; kh * 64 < d; ++kh)
+            tma_load_2d(dst + kh * (kCandTile * 128) + t * IT * 128, &tmap_items, kh * 64, row0 + t * IT, &bar_x[b]);
+      };
+      uint32_t x_phase[2] = {0, 0};
+      bool in_flight = true;                // a unit was requested and not yet multiplied
+      if (tid == 0) fetch(cur, 0);          // (before the wait for the weight images: the two round trips overlap)
+      ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
+      for (int n = lo; n < hi && ok; ++n) {
+        ProjUnit nxt = cur;
+        in_flight = n + 1 < hi;
+        if (in_flight) {
+          step();
+          nxt = make_unit();
+          if (tid == 0) fetch(nxt, buf ^ 1);   // (its last readers, the MMAs of unit n - 1, have completed)
+        }
+        __syncthreads();                    // TMEM of unit n - 1 drained
+        ok = run_unit(cur, true, Xbuf + (size_t)buf * kCandTile * d, &bar_x[buf], x_phase[buf]);
+        x_phase[buf] ^= 1;
+        cur = nxt;
+        buf ^= 1;
       }
+      // giving up with a copy still on its way: let it land (bounded) before the block may exit
+      if (!ok && in_flight && tid == 0)
+        for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(&bar_x[buf], x_phase[buf]); ++i) __nanosleep(64);
+    } else {
+      ok = __syncthreads_and(mbar_wait(&bar_img, 0, abortp));
+      if (ok) stage(cur, true, Xbuf);
       asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 1;" ::: "memory");
-      fence_proxy_async_smem();
-      __syncthreads();                    // unit n staged by every thread; TMEM of unit n - 1 drained
-      ok = run_unit(cur, true, Xbuf + (size_t)buf * kCandTile * d);
-      cur = nxt;
-      buf ^= 1;
+      for (int n = lo; n < hi && ok; ++n) {
+        ProjUnit nxt = cur;
+        if (n + 1 < hi) {
+          step();
+          nxt = make_unit();
+          stage(nxt, true, Xbuf + (size_t)(buf ^ 1) * kCandTile * d);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        fence_proxy_async_smem();
+        __syncthreads();                    // unit n staged by every thread; TMEM of unit n - 1 drained
+        ok = run_unit(cur, true, Xbuf + (size_t)buf * kCandTile * d, nullptr, 0);
+        cur = nxt;
+        buf ^= 1;
+      }
     }
   }
 
@@ -519,7 +570,7 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P) {
       cp_async_wait_all();
       fence_proxy_async_smem();
       __syncthreads();
-      ok = run_unit(pu, false, Xbuf);
+      ok = run_unit(pu, false, Xbuf, nullptr, 0);
     }
   }
 
@@ -995,6 +1046,34 @@ void tensor_geometry(const Plan& p, TensorGeom* g) {
   g->cand_tiles_max = (int)(a < b ? a : b);
 }
 
+namespace {
+// Tensor map of the padded item array as a [U * L, d] bf16 matrix for tc_proj_kernel's tiled TMA loads: boxes of 64
+// columns (128 bytes, the swizzle span) by IT rows, 128-byte swizzle, zeros outside the array.  False when the driver
+// entry point is missing or refuses the shape; the kernel then stages the rows with plain asynchronous copies.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool encode_item_map(const Plan& p, int IT, const void* items, CUtensorMap* map) {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  if (!fn || p.d % 64 || (reinterpret_cast<uintptr_t>(items) & 15)) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.U * p.L};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)IT}, elem[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(items), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
                const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
                const void* Wg_images) {
@@ -1020,7 +1099,11 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     const size_t smem = ((size_t)p.dqk * p.d + 3 * (size_t)kCandTile * p.d) * 2;   // W_k^T | W_q^T, W_v^T, two staging buffers
     LASER_CUDA_OK(cudaFuncSetAttribute(tc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("tc_proj", st);
-    LASER_CUDA_OK(launch_chained(tc_proj_kernel, dim3(P.proj_grid), dim3(kProjThreads), smem, st, P));
+    alignas(64) CUtensorMap item_map;
+    memset(&item_map, 0, sizeof(item_map));
+    // (packed rows, and item tiles under 32 rows, i.e. copies under 4 KB, stay on plain asynchronous copies)
+    const int use_tma = !P.item_off && P.IT >= 32 && encode_item_map(p, P.IT, items, &item_map) ? 1 : 0;
+    LASER_CUDA_OK(launch_chained(tc_proj_kernel, dim3(P.proj_grid), dim3(kProjThreads), smem, st, P, item_map, use_tma));
   }
   if (user_wants_hp) {
     LaunchScope ls("tc_zero_empty", st);
