@@ -228,8 +228,8 @@ __global__ void __launch_bounds__(256) tc_zero_empty_kernel(TcParams P) {
 // tile (Q rows).  Every block takes a contiguous range of the item units (no empty ones: tc_prep_kernel counted them)
 // and runs them through a two-deep pipeline: while unit n is multiplied (two MMA groups into TMEM: rows x d_qk for K,
 // d x rows for V^T) and drained by the eight warps (warp w reads TMEM lanes 32 (w mod 4) .. +31 and one half of the
-// columns), the rows of unit n + 1 are already on their way into the other staging buffer (cp.async, canonical K-major
-// layout).  Afterwards the blocks share out the candidate tiles (Q = T W_q / 2 gamma) the same way.
+// columns), the rows of unit n + 1 are already on their way into the other staging buffer: tiled TMA loads in the
+// 128-byte swizzled layout when the item layout allows, else cp.async into the canonical K-major layout.  Afterwards the blocks share out the candidate tiles (Q = T W_q / 2 gamma) the same way.
 struct ProjUnit {
   int u, seg, t0, rows, seg_items;      // item unit: tiles t0.. of segment seg; rows = staged rows; valid items of seg
   int jt, c0, nc;                       // candidate unit: tile jt of user u, whose candidates are [c0, c0 + nc)
