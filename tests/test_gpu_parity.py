@@ -324,6 +324,26 @@ def test_host_buffer_entry_point_sends_only_valid_rows_when_that_pays(path):
         assert torch.equal(z_h, z_dev)
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_entry_point_reports_lengths_out_of_range(pinned):
+    # Lengths below 0 or above L: the host clamps them when it sizes what it moves, the device treats such users as
+    # empty and reports the batch; the next call on the same workspace is clean again.
+    lengths = [2048, 10, 0, 700]
+    w = make_custom(U=4, C=5, L=2048, d=64, H=2, S=64, M=2, dtype="bf16", seed=23, lengths=lengths)
+    z_dev = run_forward(w, "auto", want_hprime=False).cpu()
+    hb = P.DeviceBatch.from_workload(w, device="cpu", pin_host=pinned)
+    ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
+    z_h = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype)
+    z_h = z_h.pin_memory() if pinned else z_h
+    bad = torch.tensor([-3, 3000, 0, 700], dtype=torch.int32)
+    bad = bad.pin_memory() if pinned else bad
+    with pytest.raises(P.binding.LaserError) as err:
+        P.laser_forward_host(hb.cfg, hb.items, bad, hb.cands, hb.cand_offsets, hb.Wq, hb.Wk, hb.Wv, hb.Wg, z_h, ws)
+    assert err.value.status == -6
+    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
+    assert torch.equal(z_h, z_dev)
+
+
 def test_host_buffer_entry_point_pageable_memory_copies_runs_of_users():
     # Pageable host memory and much padding: one copy per run of users whose valid rows are contiguous on the host.
     lengths = [8192, 8192, 100, 0, 0, 3000, 8192, 1]
