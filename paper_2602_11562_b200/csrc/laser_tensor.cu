@@ -1065,6 +1065,7 @@ bool encode_item_map(const Plan& p, int IT, const void* items, CUtensorMap* map)
     return reinterpret_cast<EncodeTiledFn>(f);
   }();
   if (!fn || p.d % 64 || (reinterpret_cast<uintptr_t>(items) & 15)) return false;
+  if ((long long)p.U * p.L > 0x7fffff00LL) return false;          // row coordinates are 32-bit
   const cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.U * p.L};
   const cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
   const cuuint32_t box[2] = {64, (cuuint32_t)IT}, elem[2] = {1, 1};
