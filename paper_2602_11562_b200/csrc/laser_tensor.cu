@@ -933,15 +933,12 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         if (!ok) break;
         tc_fence_after();
         const uint32_t tO = tmem + lane_base + (ob ? (uint32_t)P.o_col1 : kColO);
-        for (int c = 0; c < d; c += 16) {
-          uint32_t v[16];
-          tmem_ld16(tO + c, v);
-          tc_wait_ld();
-          if (c + 16 >= d) {                               // the accumulator is in registers: hand it back
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
-          }
+        auto hand_back = [&]() {                           // the accumulator is in registers
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
+        };
+        auto stage16 = [&](int c, const uint32_t (&v)[16]) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             uint4 o;
@@ -951,6 +948,23 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
             o.w = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 6]), 0.5f * __uint_as_float(v[half * 8 + 7]));
             *reinterpret_cast<uint4*>(row + (c + half * 8) * 2) = o;
           }
+        };
+        int c = 0;
+        for (; c + 32 <= d; c += 32) {                     // two accumulator loads in flight per wait
+          uint32_t v0[16], v1[16];
+          tmem_ld16(tO + c, v0);
+          tmem_ld16(tO + c + 16, v1);
+          tc_wait_ld();
+          if (c + 32 >= d) hand_back();
+          stage16(c, v0);
+          stage16(c + 16, v1);
+        }
+        if (c < d) {
+          uint32_t v0[16];
+          tmem_ld16(tO + c, v0);
+          tc_wait_ld();
+          hand_back();
+          stage16(c, v0);
         }
         const int ci = w.j * kCandTile + m;
         if (ci < w.nc) {                                   // my candidate's row of this segment: one contiguous store
