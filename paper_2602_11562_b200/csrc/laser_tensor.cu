@@ -237,7 +237,7 @@ struct ProjUnit {
 
 __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P, const __grid_constant__ CUtensorMap tmap_items,
                                                               int use_tma) {
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t proj_smem[];
   __shared__ uint64_t bar_img, bar_mma, bar_x[2];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(kProjThreads) tc_proj_kernel(TcParams P, const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int quad = warp & 3, half = warp >> 2;
   const int d = P.d, dqk = P.dqk, IT = P.IT;
-  bf16* imgK = reinterpret_cast<bf16*>(smem_raw);          // W_k^T, later W_q^T
+  bf16* imgK = reinterpret_cast<bf16*>(proj_smem);          // W_k^T, later W_q^T
   bf16* imgV = imgK + dqk * d;
   bf16* Xbuf = imgV + kCandTile * d;                       // [2][128 x d]
 
