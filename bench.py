@@ -118,14 +118,14 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(w, budget_users=None):
+def oracle_sample(w, budget_users=None, target=4e10):
     """Users forming a bounded sample for the CPU oracle (a prefix of the batch), sized by a rough cost model so
-    that the run takes on the order of 10-30 s."""
+    that the run takes on the order of 10-30 s at the default target (flop-equivalents of numpy float64 work)."""
     s = w.spec
     cost = w.lengths.astype(np.float64) * 0 + s.L  # the oracle projects and gates all L rows of a user
     ncand = (w.cand_offsets[1:] - w.cand_offsets[:-1]).astype(np.float64)
     per_user = cost * (ncand * s.H * 40.0 + s.d * (s.d_qk + s.d) * 2.0) + ncand * s.M * s.n_seg * 4.0 * s.d * s.d
-    target = 4e10 if budget_users is None else None   # ~ flop-equivalents for roughly 10-30 s of numpy float64
+    target = target if budget_users is None else None
     users, acc = [], 0.0
     for u in range(s.U):
         if budget_users is not None and len(users) >= budget_users:
@@ -146,6 +146,19 @@ def time_oracle(w, users):
     dt = time.perf_counter() - t0
     scores = int(sum(int(w.cand_offsets[u + 1] - w.cand_offsets[u]) for u in users))
     return dt, scores
+
+
+def parity_figures(got, ref):
+    """The three error figures reported per tensor: the pass/fail metric max |g - r| / max(1, |r|), the raw maximum
+    absolute error, and that maximum divided by the root mean square of the reference (error relative to the signal)."""
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    if got.size == 0:
+        return {"err": 0.0, "max_abs": 0.0, "max_abs_over_rms": 0.0}
+    diff = np.abs(got - ref)
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    return {"err": float(np.max(diff / np.maximum(1.0, np.abs(ref)))), "max_abs": float(diff.max()),
+            "max_abs_over_rms": float(diff.max() / rms) if rms > 0 else 0.0}
 
 
 def host_cores() -> int:
@@ -199,6 +212,7 @@ NCU_TRAFFIC = {
 }
 KERNEL_SOURCE = {"sta_tc": "laser_tensor.cu", "tc_proj": "laser_tensor.cu", "gsta_mma": "laser_gsta.cu",
                  "stream_sta": "laser_stream.cu", "ffn_tc": "laser_ffn.cu"}
+OTHER_WORKLOADS = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "prod")      # entries of the `configs` array
 MAIN_KERNELS = ("sta_tc", "tc_proj", "gsta_mma", "stream_sta",      # kernels of the timed step (roofline candidates)
                 "proj_simt_q", "proj_simt_kv", "sta_simt", "gsta_simt")
 
@@ -251,12 +265,29 @@ def kernel_roofline(w, name, ms, peaks):
     out = {"kernel": name, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
            "frac": achieved / peak, "traffic": traffic, "peak_source": src, "ms": ms,
            "frac_of_nominal": achieved / NOMINAL["bf16_tflops"]}
+    if name == "tc_proj":
+        # the projection moves more than it computes at these widths: 2 d bytes read and 2 (d_qk + d) bytes written per
+        # valid item, so its bytes-based fraction is reported beside the flop-based one
+        s = w.spec
+        nbytes = work["valid_items"] * 2 * (s.d + s.d_qk + s.d)
+        out["hbm_bytes"] = nbytes
+        out["hbm_achieved_gbs"] = nbytes / sec / 1e9
+        out["hbm_frac"] = nbytes / sec / 1e9 / peaks["hbm_gbs"]
     if name.startswith("sta"):
         # the gate (one MUFU tanh per candidate x item x head) is what bounds this kernel: 15.8 / clk / SM measured
         gates = work["gate_evals"] / sec
         out["gate_evals_per_s"] = gates
         out["gate_frac_of_mufu_peak"] = gates / (15.8 * 148 * 1.965e9)
     return out
+
+
+def sta_kernel_roofline(w, prof, peaks):
+    """Roofline entry of the fused segment-attention kernel of the path that ran (the kernel the tensor-peak and
+    HBM-bandwidth targets are stated for), or None."""
+    for name in ("sta_tc", "stream_sta", "sta_simt"):
+        if name in prof:
+            return kernel_roofline(w, name, prof[name], peaks)
+    return None
 
 
 def dominant_kernel_roofline(w, prof, peaks):
@@ -394,11 +425,6 @@ def run_ours(args, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = make_workload(args.workload, seed_offset=rank)
-    s = w.spec
-    b = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device=dev)
-    ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device=dev)
-    z = torch.empty((b.cfg.total_cands, s.d), dtype=b.items.dtype, device=dev)
     class _L2Flush:
         """Evicts L2 between timed steps: writes a 256 MB buffer (> 126 MB L2), then reads a second 256 MB buffer so that
         the dirty lines of the write are back in HBM before the timed region starts (otherwise their write-back would be
@@ -416,56 +442,96 @@ def run_ours(args, rank, world, local_rank):
     flush = _L2Flush()
     stream = torch.cuda.current_stream()
 
+    def measure(name, steps, oracle_target, sync_ranks, before_timing=None):
+        """One configuration: parity of z against the oracle on a bounded sample of users (rank 0, before any timing;
+        the same run is the timed CPU baseline), `steps` timed forward calls with an L2 flush before each, and a second
+        pass of the same steps with the library's per-kernel CUDA events."""
+        w = make_workload(name, seed_offset=rank)
+        s = w.spec
+        b = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device=dev)
+        ws = torch.empty(P.laser_workspace_bytes(b.cfg), dtype=torch.uint8, device=dev)
+        z = torch.empty((b.cfg.total_cands, s.d), dtype=b.items.dtype, device=dev)
+
+        def step():
+            P.laser_forward(b.cfg, *b.args(), b.Wg, z=z, workspace=ws, stream=stream)
+
+        parity = cpu_base = None
+        if rank == 0:
+            step()
+            assert P.laser_check_status(ws) == 0
+            users = oracle_sample(w, target=oracle_target)
+            from oracle import laser_oracle
+            t0 = time.perf_counter()
+            _, z_ref = laser_oracle.forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S,
+                                            s.H, w.gamma, w.tau, users=users, return_hprime=False)
+            dt = time.perf_counter() - t0
+            scores = int(sum(int(w.cand_offsets[u + 1] - w.cand_offsets[u]) for u in users))
+            rows = np.concatenate([np.arange(int(w.cand_offsets[u]), int(w.cand_offsets[u + 1])) for u in users])
+            got = z.float().cpu().numpy().astype(np.float64)[rows]
+            tol = 1e-4 if s.dtype == "f32" else 2e-2
+            fig = parity_figures(got, z_ref[rows])
+            if not (np.isfinite(got).all() and fig["err"] <= tol):
+                raise SystemExit(f"parity failure before timing ({s.name}): z error {fig['err']:.3e} > {tol}")
+            parity = {"z_err": fig["err"], "z_max_abs": fig["max_abs"], "z_max_abs_over_rms": fig["max_abs_over_rms"],
+                      "tol": tol, "users_checked": len(users), "scores_checked": int(rows.size)}
+            cpu_base = {"value": scores / dt, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+                        "sample": f"users 0..{len(users) - 1} of {s.U} ({scores} scores) of {s.name}, {dt:.1f} s"}
+
+        for _ in range(max(3, args.warmup)):
+            flush.fill_(1)
+            step()
+        launches = P.laser_last_launch_count()
+        if sync_ranks:
+            barrier()
+        else:
+            torch.cuda.synchronize()
+        if before_timing:
+            before_timing()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for e0, e1 in evs:
+            flush.fill_(1)          # evict the previous step's data from L2 (outside the timed bracket)
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        if sync_ranks:
+            barrier()
+        else:
+            torch.cuda.synchronize()
+        times = [e0.elapsed_time(e1) for e0, e1 in evs]
+
+        # per-kernel durations (CUDA events recorded by the library around each launch), same step, same flush
+        P.laser_profile_enable(True)
+        prof = {}
+        for _ in range(steps):
+            flush.fill_(1)
+            step()
+            for kname, ms in P.laser_profile_read():
+                prof[kname] = prof.get(kname, 0.0) + ms / steps
+        P.laser_profile_enable(False)
+        return {"w": w, "b": b, "ws": ws, "z": z, "times": times, "prof": prof, "parity": parity,
+                "cpu_baseline": cpu_base, "launches": launches}
+
+    def summary(m):
+        """The per-configuration entry of the `configs` array."""
+        w, prof = m["w"], m["prof"]
+        mean = sum(m["times"]) / len(m["times"])
+        return {"workload": w.spec.name, "value": w.N / (mean * 1e-3), "unit": UNIT, "ms_per_step": mean,
+                "ms_per_step_median": statistics.median(m["times"]), "steps": len(m["times"]), "kernels_ms": prof,
+                "roofline": dominant_kernel_roofline(w, prof, peaks), "sta_roofline": sta_kernel_roofline(w, prof, peaks),
+                "parity": m["parity"], "cpu_baseline": m["cpu_baseline"], "gpu_launches": m["launches"] * len(m["times"])}
+
+    sampler = ClockSampler(local_rank)       # clocks from the start of the timed region to the end of the e2e timing
+    head = measure(args.workload, args.steps, 4e10, True, before_timing=sampler.start)
+    w, b, ws, z = head["w"], head["b"], head["ws"], head["z"]
+    s = w.spec
+    step_times = list(head["times"])
+    dev_ms = sum(step_times)
+    prof = head["prof"]
+    parity, cpu_base = head["parity"], head["cpu_baseline"]
+    launches_per_step = head["launches"]
+
     def step():
         P.laser_forward(b.cfg, *b.args(), b.Wg, z=z, workspace=ws, stream=stream)
-
-    # parity on sampled users before any timing (rank 0 only; the oracle runs on the host)
-    parity = None
-    cpu_base = None
-    if rank == 0:
-        step()
-        assert P.laser_check_status(ws) == 0
-        users = oracle_sample(w)
-        dt, scores = time_oracle(w, users)
-        from oracle import laser_oracle
-        _, z_ref = laser_oracle.forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
-                                        w.gamma, w.tau, users=users[:2], return_hprime=False)
-        rows = np.arange(int(w.cand_offsets[0]), int(w.cand_offsets[min(2, len(users))]))
-        got = z.float().cpu().numpy().astype(np.float64)[rows]
-        err = float(np.max(np.abs(got - z_ref[rows]) / np.maximum(1.0, np.abs(z_ref[rows])))) if rows.size else 0.0
-        tol = 1e-4 if s.dtype == "f32" else 2e-2
-        if not (err <= tol):
-            raise SystemExit(f"parity failure before timing: z error {err:.3e} > {tol}")
-        parity = {"z_err": err, "tol": tol, "users_checked": min(2, len(users))}
-        cpu_base = {"value": scores / dt, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
-                    "sample": f"users 0..{len(users) - 1} of {s.U} ({scores} scores) of {s.name}, {dt:.1f} s"}
-
-    for _ in range(max(3, args.warmup)):
-        flush.fill_(1)
-        step()
-    launches_per_step = P.laser_last_launch_count()
-
-    sampler = ClockSampler(local_rank)
-    barrier()
-    sampler.start()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for e0, e1 in evs:
-        flush.fill_(1)          # evict the previous step's data from L2 (outside the timed bracket)
-        e0.record(stream)
-        step()
-        e1.record(stream)
-    barrier()
-    dev_ms = sum(e0.elapsed_time(e1) for e0, e1 in evs)
-
-    # per-kernel durations (CUDA events recorded by the library around each launch), same step, same flush
-    P.laser_profile_enable(True)
-    prof = {}
-    for _ in range(args.steps):
-        flush.fill_(1)
-        step()
-        for name, ms in P.laser_profile_read():
-            prof[name] = prof.get(name, 0.0) + ms / args.steps
-    P.laser_profile_enable(False)
 
     # next row of the scope: multi-resolution fusion outputs on the H' and z of this batch (outside the timed step)
     fusion = None
@@ -511,7 +577,6 @@ def run_ours(args, rank, world, local_rank):
         P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, hws, stream=stream, blocking=True)
     barrier()
     e2e_steps = max(1, min(args.steps, 20))
-    t0 = time.perf_counter()
     ee = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(e2e_steps)]
     for e0, e1 in ee:
         e0.record(stream)
@@ -520,6 +585,17 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     e2e_ms = sum(e0.elapsed_time(e1) for e0, e1 in ee)
     clocks = sampler.stop()
+
+    # the other configurations (one GPU only: each rank of a multi-GPU run times the headline workload alone)
+    others = []
+    if world == 1 and not args.headline_only:
+        del hb, hws, z_h
+        del b, ws, z, head
+        for name in OTHER_WORKLOADS:
+            if name == args.workload:
+                continue
+            torch.cuda.empty_cache()
+            others.append(summary(measure(name, min(args.steps, 20), 4e10, False)))
 
     if world > 1:
         t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
@@ -537,6 +613,7 @@ def run_ours(args, rank, world, local_rank):
         roof = dominant_kernel_roofline(w, prof, peaks)
         line = {"metric": METRIC, "value": total_scores / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
                 "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_per_step,
+                "ms_per_step_median": statistics.median(step_times),
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32" if s.dtype == "f32" else "bf16", "data": "synthetic",
                 "config": {"workload": s.name, "users": s.U, "cands_per_user": s.C, "L": s.L, "d": s.d, "heads": s.H,
@@ -548,6 +625,7 @@ def run_ours(args, rank, world, local_rank):
                 "gpu_launches": launches_per_step * args.steps,
                 "clocks": clocks,
                 "roofline": roof,
+                "sta_roofline": sta_kernel_roofline(w, prof, peaks),
                 "kernels_ms": prof,
                 "fusion": fusion,
                 "ffn": ffn,
@@ -555,7 +633,8 @@ def run_ours(args, rank, world, local_rank):
                 "kernel_rooflines": [kernel_roofline(w, k, v, peaks) for k, v in prof.items() if k in MAIN_KERNELS],
                 "cpu_baseline": cpu_base,
                 "parity": parity,
-                "work": work}
+                "work": work,
+                "configs": others}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -567,7 +646,9 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "prod"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "prod"],
+                    help="the headline configuration (value, roofline, e2e); the others follow in `configs`")
+    ap.add_argument("--headline-only", action="store_true", help="skip the `configs` array of the other configurations")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -52,6 +52,14 @@ def test_roofline_entries_divide_work_by_time_and_peak():
     assert abs(r["gate_evals_per_s"] - work["gate_evals"] / 4e-6) < 1e-3
     r = b.kernel_roofline(w, "sta_simt", 0.004, dict(peaks, _source="fallback"))
     assert r["bound"] == "alu" and abs(r["peak"] - 148 * 128 * 2 * 1.965e9 / 1e12) < 1e-9 and r["traffic"] is None
+    # the projection also carries a bytes-based fraction: 2 d read + 2 (d_qk + d) written per valid item
+    r = b.kernel_roofline(w, "tc_proj", 0.001, peaks)
+    assert r["bound"] == "tensor" and r["hbm_bytes"] == 47 * 2 * (32 + 32 + 32)
+    assert abs(r["hbm_frac"] - r["hbm_bytes"] / 1e-6 / 1e9 / 1000.0) < 1e-12
+    # the segment-attention kernel of whichever path ran
+    assert b.sta_kernel_roofline(w, {"tc_prep": 0.5, "sta_tc": 0.2, "gsta_mma": 0.3}, peaks)["kernel"] == "sta_tc"
+    assert b.sta_kernel_roofline(w, {"stream_pre": 0.1, "stream_sta": 0.2}, peaks)["bound"] == "hbm"
+    assert b.sta_kernel_roofline(w, {"gsta_mma": 0.3}, peaks) is None
     # the dominant kernel is the one with the largest time among the step's own kernels
     dom = b.dominant_kernel_roofline(w, {"tc_prep": 0.5, "sta_tc": 0.2, "gsta_mma": 0.3, "fusion": 9.0}, peaks)
     assert dom["kernel"] == "gsta_mma"
@@ -67,3 +75,15 @@ def test_ncu_traffic_is_null_once_the_kernel_source_changed(monkeypatch):
     monkeypatch.setattr(b, "_source_digest", lambda f: "0" * 12)
     assert b.ncu_traffic(kernel, workload) is None
     assert b.ncu_traffic("no_such_kernel", workload) is None
+
+
+def test_parity_figures_report_the_bar_metric_the_raw_error_and_the_error_over_the_signal():
+    b = _bench()
+    ref = np.array([0.1, -0.2, 4.0, 0.0])
+    got = np.array([0.11, -0.2, 4.4, 0.0])
+    f = b.parity_figures(got, ref)
+    assert abs(f["err"] - 0.1) < 1e-12                   # 0.4 / max(1, 4.0): relative above 1, absolute below
+    assert abs(f["max_abs"] - 0.4) < 1e-12
+    rms = np.sqrt((0.01 + 0.04 + 16.0) / 4)
+    assert abs(f["max_abs_over_rms"] - 0.4 / rms) < 1e-12
+    assert b.parity_figures(np.zeros((0, 3)), np.zeros((0, 3))) == {"err": 0.0, "max_abs": 0.0, "max_abs_over_rms": 0.0}
