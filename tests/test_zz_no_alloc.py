@@ -5,6 +5,7 @@ import pytest
 import torch
 
 import paper_2602_11562_b200 as P
+from oracle import laser_oracle
 from workloads import make_custom
 
 from _util import TOL, err_metric, to_np
@@ -32,6 +33,10 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice_in_a_row
         ref, out = _both(w)
         assert err_metric(to_np(out), to_np(ref)) <= TOL[w.spec.dtype]
         assert torch.equal(out, ref)                   # same kernels, same arithmetic: identical bits
+        s = w.spec                                     # and against the float64 oracle itself, not only its sibling
+        Hp_ref = laser_oracle.sta_forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, s.S, s.H,
+                                          w.gamma)
+        assert err_metric(to_np(out), Hp_ref) <= TOL[s.dtype]
 
 
 def test_static_scratch_rejects_problems_beyond_its_fixed_size():

@@ -13,6 +13,6 @@ from .configs import (  # noqa: F401
     make_workload,
     make_custom,
     make_ffn_weights,
+    make_gsta_inputs,
     round_to_dtype,
-    shard_users,
 )

@@ -214,16 +214,6 @@ def make_custom(*, U, C, L, d, H, S, M, dtype="f32", seed=0, d_qh=16, lengths=No
     return _generate(spec, lengths=None if lengths is None else np.asarray(lengths, dtype=np.int32))
 
 
-def shard_users(num_users: int, rank: int, world_size: int) -> range:
-    """Contiguous block partition of users over ranks: rank r owns users [lo, hi); sizes differ by at most 1."""
-    if not (0 <= rank < world_size):
-        raise ValueError("rank out of range")
-    base, rem = divmod(num_users, world_size)
-    lo = rank * base + min(rank, rem)
-    hi = lo + base + (1 if rank < rem else 0)
-    return range(lo, hi)
-
-
 def make_ffn_weights(d: int, r: int = 4, dtype: str = "bf16", seed: int = 0) -> dict:
     """Seeded weights of the feed-forward refinement (Eq. 6): W1 [d, r d], b1 [r d], W2 [r d, d], b2 [d] and the
     layer norm's gain / shift [d], all rounded to `dtype` and returned as float32 arrays."""
@@ -238,3 +228,21 @@ def make_ffn_weights(d: int, r: int = 4, dtype: str = "bf16", seed: int = 0) -> 
         "ln_b": (0.1 * rng.standard_normal(d)).astype(np.float32),
     }
     return {k: round_to_dtype(v, dtype) for k, v in w.items()}
+
+
+def make_gsta_inputs(*, counts, segments, Lp, d, M, seed=0, hp_std=0.5):
+    """Seeded inputs for the GSTA stage alone (tests): per user u `counts[u]` candidates whose first `segments[u]` of
+    `Lp` segment vectors are non-empty.  Returns (cand_offsets [U+1] int32, Hp [N, Lp, d], cands [N, d],
+    Wg [M, 3, d, d]) as float32 arrays of bf16-representable values; rows of empty segments hold NaN (a consumer must
+    never use them)."""
+    rng = np.random.Generator(np.random.PCG64(55_000 + seed))
+    counts = np.asarray(counts, dtype=np.int64)
+    offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    N = int(offs[-1])
+    Hp = (hp_std * rng.standard_normal((N, Lp, d), dtype=np.float32)).astype(np.float32)
+    cands = rng.standard_normal((N, d), dtype=np.float32) * np.float32(1.0 / math.sqrt(d))
+    Wg = _xavier_uniform(rng, d, d, (M, 3, d, d))
+    Hp, cands, Wg = (round_to_dtype(a, "bf16") for a in (Hp, cands, Wg))
+    for u, nv in enumerate(segments):
+        Hp[int(offs[u]):int(offs[u + 1]), int(nv):, :] = np.float32("nan")
+    return offs, Hp, cands, Wg
