@@ -191,8 +191,8 @@ LASER_API int laser_forward_ffn(const laser_config* cfg, const void* items, cons
                                 const void* Wgsta, const laser_ffn_params* ffn, void* Hprime, void* z, void* workspace,
                                 size_t workspace_bytes, void* cuda_stream);
 
-/* The softmax-aggregation variant of STA, the paper's ablation of the sigmoid gate ("replacing sigmoid aggregation with
- * the conventional softmax"): inside every segment the weights of the valid items are exp(q_h . k_{n,h} / gamma)
+/* The softmax-aggregation variant of STA (the component-ablation table's row on the sigmoid aggregation, where the
+ * gate is swapped for an ordinary softmax over the segment): inside every segment the weights of the valid items are exp(q_h . k_{n,h} / gamma)
  * normalised to sum to one per (candidate, head); everything else (projections of Eq. 4, heads, ragged lengths, zero
  * rows for empty segments) is as in laser_sta_forward.  Runs on the FP32-ALU kernels for either dtype, whatever
  * cfg->path says (an ablation, not a production path).
@@ -257,6 +257,26 @@ LASER_API int laser_forward_host(const laser_config* cfg, const void* items_h, c
  * Returns LASER_OK, or LASER_ERR_INVALID_ARG / LASER_ERR_UNSUPPORTED as laser_forward_host would. */
 LASER_API int laser_host_transfer_bytes(const laser_config* cfg, const void* items_h, const int32_t* lengths_h,
                                         size_t* h2d_bytes, size_t* d2h_bytes);
+
+/* Diagnostics.
+ *
+ * laser_workspace_regions: the regions of the carve-up of a laser_workspace_bytes(cfg) workspace, in order, as byte
+ * offsets and bytes in use.  A call with this configuration writes inside these regions only: each is followed by at
+ * least 256 bytes that no kernel touches, so a test can fill the workspace with a pattern, run a call and find the
+ * pattern intact everywhere else (the place of a memory checker on machines that have none).
+ *   offsets, sizes  HOST pointers, OUT, room for max_regions entries each (may be null when max_regions is 0)
+ * Returns the number of regions (which may exceed max_regions), or a negative status for an invalid configuration.
+ *
+ * laser_selftest_wait_timeout: exercises the give-up path of the bounded device-side waits (every wait on a copy or on
+ * the tensor cores in this library has a poll budget).  One small block waits, with a budget of poll_limit polls
+ * (1 .. 4096), for a barrier that nothing ever completes, gives up, releases its tensor memory and reports
+ * LASER_ERR_TIMEOUT through the status word exactly as a production block would; the context stays usable and the next
+ * call on the same workspace runs normally.  Nothing faults, traps or hangs.
+ *   workspace  DEVICE pointer, 256-byte aligned, at least 256 bytes; its first word receives the status
+ * Returns LASER_OK once the block is enqueued (LASER_ERR_INVALID_ARG / LASER_ERR_WORKSPACE / LASER_ERR_CUDA otherwise);
+ * laser_check_status(workspace, stream) then returns LASER_ERR_TIMEOUT. */
+LASER_API int laser_workspace_regions(const laser_config* cfg, int max_regions, size_t* offsets, size_t* sizes);
+LASER_API int laser_selftest_wait_timeout(void* workspace, size_t workspace_bytes, int32_t poll_limit, void* cuda_stream);
 
 /* Waits for `cuda_stream`, reads the device status word at the start of `workspace` and returns it
  * (LASER_OK, LASER_ERR_TIMEOUT, LASER_ERR_BAD_INPUT) or LASER_ERR_CUDA if the stream reports an error. */

@@ -2,7 +2,7 @@
 
 TEST INFRASTRUCTURE ONLY, like the rest of oracle/: imported by tests, never by the CUDA library or its binding.
 
-The ablation study replaces the sigmoid aggregation of Eq. 5 by "the conventional softmax": inside every segment the
+The component-ablation study swaps the sigmoid aggregation of Eq. 5 for an ordinary softmax: inside every segment the
 weights of the items are normalised to sum to one.  Written out, per candidate t, segment i and head h, over the valid
 items n of the segment,
 

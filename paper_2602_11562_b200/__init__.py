@@ -14,6 +14,8 @@ from .binding import (  # noqa: F401
     library_path,
     make_config,
     laser_workspace_bytes,
+    laser_workspace_regions,
+    laser_selftest_wait_timeout,
     laser_host_transfer_bytes,
     laser_host_workspace_bytes,
     laser_sta_forward,

@@ -99,6 +99,10 @@ def load_library() -> ctypes.CDLL:
     lib.laser_forward_ffn.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, ffnp, vp, vp, vp, sz, vp]
     lib.laser_check_status.restype = ctypes.c_int
     lib.laser_check_status.argtypes = [vp, vp]
+    lib.laser_workspace_regions.restype = ctypes.c_int
+    lib.laser_workspace_regions.argtypes = [cfgp, ctypes.c_int, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.laser_selftest_wait_timeout.restype = ctypes.c_int
+    lib.laser_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_int32, vp]
     lib.laser_last_launch_count.restype = ctypes.c_int
     lib.laser_last_launch_count.argtypes = []
     lib.laser_profile_enable.restype = ctypes.c_int
@@ -125,6 +129,25 @@ def laser_status_string(status: int) -> str:
 
 def laser_workspace_bytes(cfg: LaserConfig) -> int:
     return int(load_library().laser_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_workspace_regions(cfg: LaserConfig) -> list:
+    """[(byte offset, bytes in use)] of the regions a call with this configuration may write inside its workspace."""
+    lib = load_library()
+    n = lib.laser_workspace_regions(ctypes.byref(cfg), 0, None, None)
+    _check(min(n, 0), "laser_workspace_regions")
+    offs, sizes = (ctypes.c_size_t * n)(), (ctypes.c_size_t * n)()
+    _check(min(lib.laser_workspace_regions(ctypes.byref(cfg), n, offs, sizes), 0), "laser_workspace_regions")
+    return [(int(offs[i]), int(sizes[i])) for i in range(n)]
+
+
+def laser_selftest_wait_timeout(workspace: torch.Tensor, poll_limit: int = 1024, stream=None) -> None:
+    """Enqueues the bounded-wait self-test block; laser_check_status(workspace) then returns LASER_ERR_TIMEOUT (-5)."""
+    if not workspace.is_cuda or workspace.dtype != torch.uint8:
+        raise LaserError(-1, "laser_selftest_wait_timeout (workspace must be a uint8 device tensor)")
+    _check(load_library().laser_selftest_wait_timeout(ctypes.c_void_p(workspace.data_ptr()), workspace.numel(),
+                                                      int(poll_limit), ctypes.c_void_p(_stream_ptr(stream))),
+           "laser_selftest_wait_timeout")
 
 
 def laser_host_workspace_bytes(cfg: LaserConfig) -> int:

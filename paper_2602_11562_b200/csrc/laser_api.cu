@@ -72,28 +72,39 @@ int make_plan(const laser_config* c, Plan* p) {
   if (path < 0) return path;
   p->path = path;
 
+  // carve-up: every region starts 256-byte aligned and is followed by kGuardBytes that nothing may touch
   size_t off = 0;
-  p->off_status = off; off = align_up(off + kStatusWords * sizeof(int));
-  p->off_hp = off; off = align_up(off + (size_t)p->N * p->Lp * p->d * p->esize);
+  auto carve = [&](size_t bytes) {
+    const size_t at = off;
+    if (p->n_regions < kMaxRegions) {
+      p->reg_off[p->n_regions] = at;
+      p->reg_size[p->n_regions] = bytes;
+      ++p->n_regions;
+    }
+    off = align_up(off + bytes) + kGuardBytes;
+    return at;
+  };
+  p->off_status = carve(kStatusWords * sizeof(int));
+  p->off_hp = carve((size_t)p->N * p->Lp * p->d * p->esize);
   if (path == LASER_PATH_SIMT) {
-    p->off_q = off; off = align_up(off + (size_t)p->N * p->dqk * sizeof(float));
-    p->off_k = off; off = align_up(off + (size_t)p->U * p->L * p->dqk * sizeof(float));
-    p->off_v = off; off = align_up(off + (size_t)p->U * p->L * p->d * sizeof(float));
+    p->off_q = carve((size_t)p->N * p->dqk * sizeof(float));
+    p->off_k = carve((size_t)p->U * p->L * p->dqk * sizeof(float));
+    p->off_v = carve((size_t)p->U * p->L * p->d * sizeof(float));
   } else if (path == LASER_PATH_TENSOR) {
     tensor_geometry(*p, &p->tg);
     const TensorGeom& g = p->tg;
     const size_t q_tiles = (size_t)g.cand_tiles_max;
-    p->off_tq = off; off = align_up(off + q_tiles * 128 * p->dqk * 2);
-    p->off_tk = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->dqk * 2);
-    p->off_tv = off; off = align_up(off + (size_t)p->U * g.n_tiles * g.IT * p->d * 2);
-    p->off_twork = off; off = align_up(off + ((size_t)p->U + 1) * 3 * sizeof(int));
-    p->off_tcount = off; off = align_up(off + 64 * sizeof(int) + 2 * 1024 * 4 * sizeof(int));   // counters + per-block start tables
-    p->off_tctile = off; off = align_up(off + (size_t)g.cand_tiles_max * 4 * sizeof(int));       // (user, tile, first candidate, candidates) per candidate tile
-    p->off_timg = off; off = align_up(off + ((size_t)2 * p->dqk * p->d + (size_t)128 * p->d) * 2);
-    if (gsta_mma_supported(*p)) { p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p)); }
+    p->off_tq = carve(q_tiles * 128 * p->dqk * 2);
+    p->off_tk = carve((size_t)p->U * g.n_tiles * g.IT * p->dqk * 2);
+    p->off_tv = carve((size_t)p->U * g.n_tiles * g.IT * p->d * 2);
+    p->off_twork = carve(((size_t)p->U + 1) * 3 * sizeof(int));
+    p->off_tcount = carve(64 * sizeof(int) + 2 * 1024 * 4 * sizeof(int));   // counters + per-block start tables
+    p->off_tctile = carve((size_t)g.cand_tiles_max * 4 * sizeof(int));       // (user, tile, first candidate, candidates) per candidate tile
+    p->off_timg = carve(((size_t)2 * p->dqk * p->d + (size_t)128 * p->d) * 2);
+    if (gsta_mma_supported(*p)) p->off_gimg = carve(gsta_mma_image_bytes(*p));
   } else if (path == LASER_PATH_STREAM) {
-    p->off_su = off; off = align_up(off + stream_scratch_bytes(*p));
-    p->off_gimg = off; off = align_up(off + gsta_mma_image_bytes(*p));
+    p->off_su = carve(stream_scratch_bytes(*p));
+    p->off_gimg = carve(gsta_mma_image_bytes(*p));
   }
   p->total = off;
   return LASER_OK;
@@ -593,6 +604,28 @@ int laser_profile_read(int max_kernels, float* ms_out, const char** names_out) {
     names_out[i] = g_prof_name[i];
   }
   return n;
+}
+
+int laser_workspace_regions(const laser_config* cfg, int max_regions, size_t* offsets, size_t* sizes) {
+  Plan p;
+  const int rc = make_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (max_regions < 0 || (max_regions > 0 && (!offsets || !sizes))) return LASER_ERR_INVALID_ARG;
+  for (int i = 0; i < p.n_regions && i < max_regions; ++i) {
+    offsets[i] = p.reg_off[i];
+    sizes[i] = p.reg_size[i];
+  }
+  return p.n_regions;
+}
+
+int laser_selftest_wait_timeout(void* workspace, size_t workspace_bytes, int32_t poll_limit, void* cuda_stream) {
+  reset_launch_count();
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
+  if (workspace_bytes < kStatusWords * sizeof(int)) return LASER_ERR_WORKSPACE;
+  if (poll_limit < 1 || poll_limit > 4096) return LASER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  LASER_CUDA_OK(cudaMemsetAsync(workspace, 0, kStatusWords * sizeof(int), st));
+  return tensor_wait_selftest(static_cast<char*>(workspace), poll_limit, st);
 }
 
 const char* laser_status_string(int status) {

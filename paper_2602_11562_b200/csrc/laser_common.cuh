@@ -12,6 +12,8 @@ namespace laser {
 
 constexpr int kStatusWords = 64;          // int32 words reserved at the start of every workspace
 constexpr size_t kAlign = 256;
+constexpr size_t kGuardBytes = 256;       // left unused after every workspace region (overruns show up there)
+constexpr int kMaxRegions = 24;
 
 // Tile geometry of the tensor-core path (defined by laser_tensor.cu, used by the plan for sizing).
 struct TensorGeom {
@@ -38,6 +40,9 @@ struct Plan {
   // stream path
   size_t off_su;
   size_t total;
+  // every region of the carve-up (byte offset, bytes in use), in order: what a call may write inside the workspace
+  int n_regions;
+  size_t reg_off[kMaxRegions], reg_size[kMaxRegions];
 };
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -73,6 +78,8 @@ void tensor_geometry(const Plan& p, TensorGeom* g);
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
                const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
                const void* Wg_images);
+// Launches the bounded-wait self-test block (laser_tensor.cu); the status word is the first word of ws.
+int tensor_wait_selftest(char* ws, int poll_limit, cudaStream_t st);
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,
                 const void* cands, const void* Wg, void* z, char* ws, cudaStream_t st, bool images_ready);
 

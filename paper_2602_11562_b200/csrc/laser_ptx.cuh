@@ -42,10 +42,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 constexpr uint32_t kSpinLimit = 1u << 20;   // polls; each try_wait may itself suspend for a while
 
-// Waits for the phase with the given parity to complete.  Gives up (returns false) when the poll budget runs out
-// or when another thread of the block has raised *abort.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Waits for the phase with the given parity to complete.  Gives up (returns false) when the poll budget `limit` runs
+// out or when another thread of the block has raised *abort.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u) {
       if (*abort_flag) return false;
@@ -53,6 +54,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
   }
   *abort_flag = 1;
+  return false;
+}
+// For a block that has given up: waits, within the same poll budget but whatever the abort flag says, for an operation
+// that is already on its way (a bulk copy into this block's shared memory, MMAs into its tensor memory) to complete,
+// so that nothing still writes to the block's resources when it releases them.
+__device__ __forceinline__ bool mbar_drain(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u) __nanosleep(64);
+  }
   return false;
 }
 

@@ -91,7 +91,8 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
   const int u = blockIdx.z, seg = blockIdx.x;
   const int off0 = cand_offsets[u], off1 = cand_offsets[u + 1];
   const int len = lengths[u];
-  if (off0 < 0 || off1 < off0 || off1 > N || len < 0 || len > L) {
+  // (a user with more candidates than the grid was sized for, i.e. than max_cands_per_user, would leave rows unwritten)
+  if (off0 < 0 || off1 < off0 || off1 > N || len < 0 || len > L || off1 - off0 > (int)gridDim.y * kStaCands) {
     if (threadIdx.x == 0) report_status(status, LASER_ERR_BAD_INPUT);
     return;
   }
@@ -316,6 +317,8 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   float* Kf = reinterpret_cast<float*>(ws + p.off_k);
   float* Vf = reinterpret_cast<float*>(ws + p.off_v);
   if (p.N == 0 || p.U == 0) return LASER_OK;
+  // users and candidate tiles index grid.y / grid.z of the launches below
+  if (p.U > 65535 || (p.maxC + kStaCands - 1) / kStaCands > 65535) return LASER_ERR_UNSUPPORTED;
   const size_t proj_smem = (size_t)kProjRows * p.d * sizeof(float);
   {
     dim3 grid((p.N + kProjRows - 1) / kProjRows, 1);

@@ -17,6 +17,7 @@
 #include "laser_common.cuh"
 #include "laser_gsta_img.cuh"
 #include "laser_ptx.cuh"
+#include "laser_tmap.cuh"
 
 namespace laser {
 namespace {
@@ -706,6 +707,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         w.init(P);
         int pu = -1, pj = -1;
         uint32_t qcount = 0, st = 0, kv_par = 1;      // kv_par: parity that means "stage st is free"
+        uint32_t kv_armed = 0, kv_full_par = 0;       // per stage (bit): requested at least once; parity of its last request
         bool ok = true;
         for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
           if (w.u != pu || w.j != pj) {
@@ -727,7 +729,19 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
             mbar_arrive_expect_tx(&bars.kv_full[st], k_bytes + v_bytes);
             bulk_g2s(Ks + st * k_bytes, P.Kblk + (tile0 + t) * ((size_t)IT * dqk), k_bytes, &bars.kv_full[st]);
             bulk_g2s(Vs + st * v_bytes, P.Vtblk + (tile0 + t) * ((size_t)IT * d), v_bytes, &bars.kv_full[st]);
+            kv_armed |= 1u << st;
+            kv_full_par = (kv_full_par & ~(1u << st)) | ((kv_par ^ 1u) << st);
             if (++st == kKvStages) { st = 0; kv_par ^= 1; }
+          }
+        }
+        if (!ok) {
+          // giving up with copies possibly still on their way into this block's shared memory: let every requested
+          // stage and Q tile land (bounded) before the block releases its resources
+          for (uint32_t i = 0; i < (uint32_t)kKvStages; ++i)
+            if (kv_armed >> i & 1u) mbar_drain(&bars.kv_full[i], kv_full_par >> i & 1u);
+          for (uint32_t i = 0; i < 2 && i < qcount; ++i) {
+            const uint32_t n = qcount - 1 - i;                    // the last two Q requests: buffer n & 1, round n >> 1
+            mbar_drain(&bars.q_full[n & 1], (n >> 1) & 1);
           }
         }
       }
@@ -844,10 +858,11 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           if (!more) break;
           cur = nxt;
         }
-        // every MMA issued by the leader has completed once `done` flips
+        // every MMA issued by the leader has completed once `done` flips (also awaited, bounded, by a block that gave up:
+        // its tensor memory must not be released under MMAs that still write to it)
         if (leader) tc_commit(&bars.done[wgi]);
         __syncwarp();
-        wait_all(&bars.done[wgi], 0);
+        mbar_drain(&bars.done[wgi], 0);
       }
     } else if (warp >= 8 && warp < kProducerWarp) {
       // ------------------------------------------------------------------ gate warps: P = 1 + tanh(scores)
@@ -984,13 +999,40 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   if (tid == 0 && s_abort) report_status(P.status, LASER_ERR_TIMEOUT);
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+// Self-test of the give-up path of the bounded waits: one block sets itself up like the kernels above (an mbarrier,
+// tensor memory), then every warp waits, with a poll budget of `poll_limit`, for a barrier phase that nothing will ever
+// complete.  The wait runs out by construction; the block then leaves the way an aborting production block does: flag
+// raised, tensor memory released, LASER_ERR_TIMEOUT in the status word.
+__global__ void __launch_bounds__(128) tc_wait_selftest_kernel(int* status, uint32_t poll_limit) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid == 0) {
+    mbar_init(&bar, 1);
+    s_abort = 0;
+    fence_mbar_init();
   }
+  if (warp == 0) {
+    tmem_alloc(&s_tmem, 32);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  volatile int* abortp = &s_abort;
+  mbar_wait(&bar, 0, abortp, poll_limit);      // no arrival, no copy: gives up after poll_limit polls
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 32);
+  if (tid == 0 && s_abort) report_status(status, LASER_ERR_TIMEOUT);
+}
+
+int sm_count() {                         // of the current device (a process may drive several)
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
   return n;
 }
 
@@ -1064,28 +1106,8 @@ namespace {
 // Tensor map of the padded item array as a [U * L, d] bf16 matrix for tc_proj_kernel's tiled TMA loads: boxes of 64
 // columns (128 bytes, the swizzle span) by IT rows, 128-byte swizzle, zeros outside the array.  False when the driver
 // entry point is missing or refuses the shape; the kernel then stages the rows with plain asynchronous copies.
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 bool encode_item_map(const Plan& p, int IT, const void* items, CUtensorMap* map) {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess) {
-      cudaGetLastError();
-      return nullptr;
-    }
-    return reinterpret_cast<EncodeTiledFn>(f);
-  }();
-  if (!fn || p.d % 64 || (reinterpret_cast<uintptr_t>(items) & 15)) return false;
-  if ((long long)p.U * p.L > 0x7fffff00LL) return false;          // row coordinates are 32-bit
-  const cuuint64_t dims[2] = {(cuuint64_t)p.d, (cuuint64_t)p.U * p.L};
-  const cuuint64_t strides[1] = {(cuuint64_t)p.d * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)IT}, elem[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(items), dims, strides, box, elem,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_bf16_rows_map(items, (unsigned long long)p.U * p.L, p.d, IT, map);
 }
 }  // namespace
 
@@ -1132,6 +1154,13 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     LaunchScope ls("sta_tc", st);
     LASER_CUDA_OK(launch_chained(tc_sta_kernel, dim3(P.sta_grid), dim3(kStaThreads), smem, st, P));
   }
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+int tensor_wait_selftest(char* ws, int poll_limit, cudaStream_t st) {
+  LaunchScope ls("tc_wait_selftest", st);
+  tc_wait_selftest_kernel<<<1, 128, 0, st>>>(reinterpret_cast<int*>(ws), (uint32_t)poll_limit);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
 }

@@ -56,6 +56,27 @@ def test_workspace_query_and_validation(lib):
     assert "workspace" in P.laser_status_string(-3)
 
 
+def test_workspace_regions_are_disjoint_and_followed_by_a_guard_gap(lib):
+    for kw in (dict(), dict(dtype="bf16", path=P.PATH_SIMT),
+               dict(num_users=3, max_len=512, d_model=64, d_qk=64, num_heads=4, seg_size=64, num_gsta_layers=2, dtype="bf16",
+                    total_cands=600, max_cands_per_user=200, path=P.PATH_TENSOR),
+               dict(num_users=40, max_len=256, d_model=64, d_qk=32, num_heads=2, seg_size=64, dtype="bf16", total_cands=40,
+                    max_cands_per_user=1, path=P.PATH_STREAM)):
+        cfg = _cfg(**kw)
+        total = P.laser_workspace_bytes(cfg)
+        regions = P.laser_workspace_regions(cfg)
+        assert total > 0 and len(regions) >= 3 and regions[0][0] == 0
+        end = 0
+        for i, (off, size) in enumerate(regions):
+            assert off % 256 == 0
+            assert off >= end + (256 if i else 0)          # at least 256 untouched bytes after the previous region
+            end = off + size
+        assert end + 256 <= total
+    assert P.laser_workspace_regions(_cfg())[0][1] == 256   # the status block comes first
+    with pytest.raises(P.LaserError):
+        P.laser_workspace_regions(_cfg(num_heads=3))
+
+
 def test_host_transfer_size_query(lib):
     import torch
     # 4 users x 4096 rows of 128 bf16 features (256 bytes each): everything else is small next to the items.  Without

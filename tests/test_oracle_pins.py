@@ -242,6 +242,15 @@ def test_cost_model_reproduces_paper_numbers(repo_root):
     # the closed total equals the sum of its stages up to the dropped lower-order terms
     parts = cost_model.c_sta(L, d, d_q, w, r) + cost_model.c_gsta(L, d, w, M)
     assert parts == pytest.approx(cost_model.c_laser(L, d, d_q, w, r, M), rel=0.01)
+    # the three stage costs of the "Computational Complexity" section, counted by hand from the shapes of the products
+    # at a small size: K [L x d_q] and V [L x d] from X [L x d]; one score and one weighted value per item and target;
+    # two d x r d products per compressed vector
+    Ls, ds, dqs, ws, rs = 12, 8, 4, 3, 2
+    assert cost_model.c_proj(Ls, ds, dqs) == sum(ds for _ in range(Ls) for _ in range(dqs + ds))
+    assert cost_model.c_attn(Ls, ds, dqs) == sum(dqs + ds for _ in range(Ls))
+    assert cost_model.c_ffn(Ls, ds, ws, rs) == sum(ds * rs * ds + rs * ds * ds for _ in range(Ls // ws))
+    # and the stage total the paper prints drops only the per-target term
+    assert cost_model.c_sta(Ls, ds, dqs, ws, rs) == cost_model.c_proj(Ls, ds, dqs) + cost_model.c_ffn(Ls, ds, ws, rs)
 
 
 # ---------------------------------------------------------------- the duplicate-item workload exercises the gate
