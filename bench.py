@@ -212,7 +212,7 @@ NCU_TRAFFIC = {
 }
 KERNEL_SOURCE = {"sta_tc": "laser_tensor.cu", "tc_proj": "laser_tensor.cu", "gsta_mma": "laser_gsta.cu",
                  "stream_sta": "laser_stream.cu", "ffn_tc": "laser_ffn.cu"}
-OTHER_WORKLOADS = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "prod")      # entries of the `configs` array
+OTHER_WORKLOADS = ("cfg1", "cfg2", "cfg2x32", "cfg3", "cfg4", "cfg5", "prod")      # entries of the `configs` array
 MAIN_KERNELS = ("sta_tc", "tc_proj", "gsta_mma", "stream_sta",      # kernels of the timed step (roofline candidates)
                 "proj_simt_q", "proj_simt_kv", "sta_simt", "gsta_simt")
 
@@ -288,6 +288,18 @@ def sta_kernel_roofline(w, prof, peaks):
         if name in prof:
             return kernel_roofline(w, name, prof[name], peaks)
     return None
+
+
+def request_batching(entries):
+    """Throughput of 32 serving-shaped requests in one call over that of one request per call (from the `configs`
+    entries), or None when either was not measured."""
+    by = {e["workload"]: e for e in entries}
+    one, many = by.get("cfg2_serving_bf16"), by.get("cfg2_serving_bf16_x32_requests")
+    if not one or not many:
+        return None
+    return {"single_request_us": one["ms_per_step"] * 1e3, "requests_per_call": 32,
+            "batched_call_us": many["ms_per_step"] * 1e3, "single_scores_per_s": one["value"],
+            "batched_scores_per_s": many["value"], "speedup": many["value"] / one["value"]}
 
 
 def dominant_kernel_roofline(w, prof, peaks):
@@ -634,7 +646,8 @@ def run_ours(args, rank, world, local_rank):
                 "cpu_baseline": cpu_base,
                 "parity": parity,
                 "work": work,
-                "configs": others}
+                "configs": others,
+                "request_batching": request_batching(others)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -646,7 +659,7 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "prod"],
+    ap.add_argument("--workload", default="cfg3", choices=["cfg1", "cfg2", "cfg2x32", "cfg3", "cfg4", "cfg5", "prod"],
                     help="the headline configuration (value, roofline, e2e); the others follow in `configs`")
     ap.add_argument("--headline-only", action="store_true", help="skip the `configs` array of the other configurations")
     args = ap.parse_args()

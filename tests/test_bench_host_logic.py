@@ -87,3 +87,12 @@ def test_parity_figures_report_the_bar_metric_the_raw_error_and_the_error_over_t
     rms = np.sqrt((0.01 + 0.04 + 16.0) / 4)
     assert abs(f["max_abs_over_rms"] - 0.4 / rms) < 1e-12
     assert b.parity_figures(np.zeros((0, 3)), np.zeros((0, 3))) == {"err": 0.0, "max_abs": 0.0, "max_abs_over_rms": 0.0}
+
+
+def test_request_batching_ratio_comes_from_the_two_serving_entries():
+    b = _bench()
+    one = {"workload": "cfg2_serving_bf16", "ms_per_step": 0.04, "value": 1.0e7}
+    many = {"workload": "cfg2_serving_bf16_x32_requests", "ms_per_step": 0.1, "value": 1.6e8}
+    r = b.request_batching([one, many, {"workload": "cfg4_lifelong_bf16", "ms_per_step": 1.0, "value": 1.0}])
+    assert r["speedup"] == 16.0 and r["requests_per_call"] == 32 and abs(r["batched_call_us"] - 100.0) < 1e-9
+    assert b.request_batching([one]) is None

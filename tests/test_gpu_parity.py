@@ -385,10 +385,11 @@ def test_host_buffer_entry_point_pageable_memory_copies_runs_of_users():
 MAX_ABS_OVER_RMS = {"hp": 0.06, "z": 0.06}
 
 
-@pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5"])
+@pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5", "cfg2x32"])
 def test_full_size_configs_every_user(name):
     """H' and z of EVERY user of the full-size configurations against the oracle, in the launch configuration the
-    benchmark times (AUTO path).  The oracle runs user by user, so that its float64 arrays stay small."""
+    benchmark times (AUTO path).  The oracle runs user by user, so that its float64 arrays stay small.  cfg2x32 is the
+    multi-request case: 32 serving-shaped requests go through one call, each as a user of the batch."""
     w = make_workload(name)
     s = w.spec
     tol = TOL[s.dtype]

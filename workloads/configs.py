@@ -74,6 +74,10 @@ CONFIGS = {
     # One candidate per user (memory-bound) bf16
     "cfg5": WorkloadSpec("cfg5_onecand_bf16", U=4096, C=1, L=2048, d=64, H=2, S=64, M=1, dtype="bf16", seed=4,
                          length_kind="uniform", len_lo=256, len_hi=2048),
+    # 32 serving-shaped requests (cfg2) handed to the library in ONE call, each request a user of the batch; not one of
+    # the five benchmark configurations
+    "cfg2x32": WorkloadSpec("cfg2_serving_bf16_x32_requests", U=32, C=512, L=2048, d=64, H=4, S=64, M=2, dtype="bf16",
+                            seed=6, length_kind="uniform", len_lo=1024, len_hi=2048),
     # The paper's production shape (experiment set-up: L = 1000, w = 10, 2 heads of d_q = 16, d = 128, two GSTA layers),
     # batched like cfg3; not one of the five benchmark configurations
     "prod": WorkloadSpec("prod_w10_bf16", U=64, C=256, L=1000, d=128, H=2, S=10, M=2, dtype="bf16", seed=5,
