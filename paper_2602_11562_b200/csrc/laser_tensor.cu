@@ -635,6 +635,7 @@ constexpr uint32_t kColO = kColP + kGateGroups * (kItMax / 2);   // outputs [n_o
 // Roles of the 25 warps of a block (one block per SM):
 //   warps 0-3   MMA issuers, one per gate warpgroup (the warp runs the loop, one elected lane issues)
 //   warps 4-7   epilogue: H' = O / 2 per finished segment, staged in shared memory, written by bulk stores
+//               (with at most two heads, warps 16-19 are a second epilogue group: one group per output accumulator)
 //   warps 8-23  four gate warpgroups: P = 1 + tanh(S)
 //   warp 24     bulk-copy producer (Q tile per (user, candidate tile), K / V^T tile per item tile, mbarrier rings) and
 //               TMEM allocation
@@ -689,6 +690,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   const uint32_t tmem = s_tmem;
   volatile int* abortp = &s_abort;
   const int n_obuf = P.n_obuf;
+  const bool two_epilogues = n_groups <= 2 && n_obuf == 2;    // gate warpgroup 2 has no head: it drains accumulator 1
   chain_wait();                         // K, V^T and Q tiles are complete
   chain_release();
 
@@ -864,7 +866,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         __syncwarp();
         mbar_drain(&bars.done[wgi], 0);
       }
-    } else if (warp >= 8 && warp < kProducerWarp) {
+    } else if (warp >= 8 && warp < kProducerWarp && !(two_epilogues && ((warp - 8) >> 2) == 2)) {
       // ------------------------------------------------------------------ gate warps: P = 1 + tanh(scores)
       const int wg = (warp - 8) >> 2;                       // warpgroup wg owns buffers wg and heads wg, wg + 4, ...
       const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -933,16 +935,20 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
       }
     } else if (warp >= 4) {
       // ------------------------------------------------------------------ epilogue: H' = O / 2
-      const int q = warp - 4;
+      // Warps 4-7; with at most two heads, warps 16-19 (whose gate warpgroup has no head) are a second epilogue group:
+      // the two output accumulators alternate segment by segment, so group e drains accumulator e, every other unit.
+      const int q = warp & 3, eg = warp >= 8 ? 1 : 0;
       const uint32_t lane_base = (uint32_t)(q * 32) << 16;
       const int m = q * 32 + lane;
       UnitWalker w;
       w.init(P);
-      uint32_t ob = 0, o_par = 0;
+      uint32_t ob = two_epilogues ? (uint32_t)eg : 0u, o_par = 0;
       bool ok = true;
       for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
+        if (two_epilogues && (it & 1) != eg) continue;
         uint8_t* row = Os + ((size_t)(it & 1) * kCandTile + m) * out_row;
-        bulk_wait_read<1>();                               // my store from this staging buffer (two units ago) has left it
+        if (two_epilogues) bulk_wait_read<0>();            // my previous store has left this group's staging buffer
+        else bulk_wait_read<1>();                          // my store from this staging buffer (two units ago) has left it
         __syncwarp();
         ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full[ob], o_par, abortp));
         if (!ok) break;
@@ -987,7 +993,8 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           bulk_s2g(P.Hp + ((size_t)(w.c0 + ci) * P.Lp + w.seg) * d, row, d * 2);
         }
         bulk_commit();
-        if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
+        if (two_epilogues) o_par ^= 1;                     // (this group's accumulator again, next phase)
+        else if ((int)++ob == n_obuf) { ob = 0; o_par ^= 1; }
       }
       bulk_wait<0>();
     }
