@@ -42,6 +42,7 @@ struct GstaParams {
   int* order;                  // [blocks] launch order, longest first (null: blocks run in candidate order)
   int* order_keys;             // [blocks] scratch of the sort that builds `order`
   int build_order;             // the set-up kernel's last block builds `order`
+  int early_setup;             // images, counts and order come from a kernel at least two launches back (see the kernel)
   bf16* z;
   int* status;
 };
@@ -74,8 +75,15 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
   uint8_t* stage = reinterpret_cast<uint8_t*>(nv_s + kGT);          // [kGW][2][kChunk] rows
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  chain_wait();
-  chain_release();
+  // The block's set-up reads the candidates (an input) and what the set-up kernel built.  After a full forward call that
+  // kernel lies at least two launches back: every kernel of the chain waits for its predecessor before it lets its
+  // successor start, so those results are complete whenever this block runs, and the set-up can overlap the tail of the
+  // attention kernel in front of this one; only H' has to wait for it.  Called on its own, the set-up kernel is the direct
+  // predecessor and the wait comes first.
+  if (!P.early_setup) {
+    chain_wait();
+    chain_release();
+  }
   // which 16 (or 8) candidates: in launch order when the set-up kernel sorted the blocks, else in candidate order
   const int blk = P.order ? min(max(P.order[blockIdx.x], 0), (int)gridDim.x - 1) : (int)blockIdx.x;
   const int c_base = blk * P.cpb;
@@ -149,6 +157,10 @@ __global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
     }
   };
   int buf = 0;
+  if (P.early_setup) {
+    chain_wait();
+    chain_release();
+  }
   if (f_valid) issue(0);
   cp_commit();
 
@@ -409,6 +421,7 @@ int gsta_mma(const Plan& p, const void* Hprime, const int32_t* lengths, const in
   P.order = ordered ? order : nullptr;
   P.order_keys = order + (p.N + 7) / 8;
   P.build_order = ordered && !images_ready;
+  P.early_setup = images_ready ? 1 : 0;
   if (p.M > 0 && !images_ready) {
     const int total = p.M * 3 * (p.d / 16) * (p.d / 16) * 32;
     LaunchScope ls("gsta_prep", st);
