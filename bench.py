@@ -389,6 +389,58 @@ def ffn_row(P, w, b, Hp, flush, stream, steps, peaks, dev):
                            "unit": UNIT}}
 
 
+def softmax_row(P, w, b, flush, stream, steps, peaks, dev):
+    """Another row of the scope: the softmax-aggregation variant of STA (the paper's ablation of the sigmoid gate) on
+    this batch, checked on the first two users with candidates against its oracle, then timed on its own."""
+    import torch
+    from oracle import softmax_sta_oracle
+    s = w.spec
+    need = P.laser_sta_softmax_workspace_bytes(b.cfg)
+    if need == 0:
+        return None
+    sws = torch.empty(need, dtype=torch.uint8, device=dev)
+    Hs = torch.empty((b.cfg.total_cands, b.cfg.n_seg, s.d), dtype=b.items.dtype, device=dev)
+    P.laser_sta_softmax_forward(b.cfg, *b.args(), Hprime=Hs, workspace=sws, stream=stream)
+    torch.cuda.synchronize()
+    assert P.laser_check_status(sws) == 0
+    fig, checked = {"err": 0.0, "max_abs": 0.0, "max_abs_over_rms": 0.0}, 0
+    for u in [u for u in range(s.U) if w.cand_offsets[u + 1] > w.cand_offsets[u]][:2]:
+        c0, c1 = int(w.cand_offsets[u]), int(w.cand_offsets[u + 1])
+        ref = softmax_sta_oracle.sta_softmax_user(w.items[u], w.lengths[u], w.cands[c0:c1], w.Wq, w.Wk, w.Wv, s.S, s.H,
+                                                  w.gamma)
+        f = parity_figures(Hs[c0:c1].float().cpu().numpy().astype(np.float64), ref)
+        fig = {k: max(fig[k], f[k]) for k in fig}
+        checked += c1 - c0
+    tol = 1e-4 if s.dtype == "f32" else 2e-2
+    if not (fig["err"] <= tol):
+        raise SystemExit(f"softmax-aggregation parity failure before timing: error {fig['err']:.3e} > {tol}")
+    P.laser_profile_enable(True)
+    prof, tot = {}, 0.0
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        P.laser_sta_softmax_forward(b.cfg, *b.args(), Hprime=Hs, workspace=sws, stream=stream)
+        e1.record(stream)
+        for name, ms in P.laser_profile_read():
+            prof[name] = prof.get(name, 0.0) + ms / steps
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1) / steps
+    P.laser_profile_enable(False)
+    main = "sta_tc_softmax" if "sta_tc_softmax" in prof else "sta_simt_softmax"
+    work = algorithmic_work(w)
+    sec = prof[main] * 1e-3
+    out = {"kernel": main, "ms": tot, "kernels_ms": prof, "parity": dict(fig, tol=tol, scores_checked=checked),
+           "weight_evals_per_s": work["gate_evals"] / sec}
+    if main == "sta_tc_softmax":
+        # one MUFU exponential per (candidate, item, head): the same 15.8 / clk / SM bound as the sigmoid gate
+        ach = work["attn_flops"] / sec / 1e12
+        out.update({"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["bf16_tflops"],
+                    "weight_frac_of_mufu_peak": work["gate_evals"] / sec / (15.8 * 148 * 1.965e9)})
+    return out
+
+
 def packed_row(P, w, b, z_padded, ws, flush, stream, steps, dev):
     """Another row of the scope: the same forward on items stored without padding (laser_forward_packed); its z must
     equal the padded layout's bit for bit, and it is timed like the main step."""
@@ -551,6 +603,7 @@ def run_ours(args, rank, world, local_rank):
     fusion = None
     ffn = None
     packed = None
+    softmax = None
     if rank == 0:
         r_recent = 2
         Hp_full = torch.empty((b.cfg.total_cands, b.cfg.n_seg, s.d), dtype=b.items.dtype, device=dev)
@@ -576,6 +629,7 @@ def run_ours(args, rank, world, local_rank):
         ffn = ffn_row(P, w, b, Hp_full, flush, stream, args.steps, peaks, dev)
         packed = packed_row(P, w, b, z, ws, flush, stream, args.steps, dev)
         del Hp_full
+        softmax = softmax_row(P, w, b, flush, stream, min(args.steps, 10), peaks, dev)
 
     # end to end: pinned host buffers in, z out, through laser_forward_host
     hb = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device="cpu", pin_host=True)
@@ -644,6 +698,7 @@ def run_ours(args, rank, world, local_rank):
                 "fusion": fusion,
                 "ffn": ffn,
                 "packed_layout": packed,
+                "softmax_sta": softmax,
                 "kernel_rooflines": [kernel_roofline(w, k, v, peaks) for k, v in prof.items() if k in MAIN_KERNELS],
                 "cpu_baseline": cpu_base,
                 "parity": parity,

@@ -194,8 +194,12 @@ LASER_API int laser_forward_ffn(const laser_config* cfg, const void* items, cons
 /* The softmax-aggregation variant of STA (the component-ablation table's row on the sigmoid aggregation, where the
  * gate is swapped for an ordinary softmax over the segment): inside every segment the weights of the valid items are exp(q_h . k_{n,h} / gamma)
  * normalised to sum to one per (candidate, head); everything else (projections of Eq. 4, heads, ragged lengths, zero
- * rows for empty segments) is as in laser_sta_forward.  Runs on the FP32-ALU kernels for either dtype, whatever
- * cfg->path says (an ablation, not a production path).
+ * rows for empty segments) is as in laser_sta_forward.  Two versions: on the tensor cores (bf16 shapes the tensor
+ * path supports; cfg->path LASER_PATH_AUTO or LASER_PATH_TENSOR, the latter answering LASER_ERR_UNSUPPORTED for other
+ * shapes) and on the FP32 ALUs (every other case, LASER_PATH_STREAM included: the variant has no one-candidate
+ * version).  The tensor-core version rounds Q and K to bf16 before the product and evaluates exp with the row's
+ * maximum over the first 32 valid items of the segment as the shift; a logit more than 41 nats above that shift is
+ * treated as 41 nats above it.
  *   workspace  at least laser_sta_softmax_workspace_bytes(cfg) bytes, 256-byte aligned */
 LASER_API size_t laser_sta_softmax_workspace_bytes(const laser_config* cfg);
 LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const int32_t* lengths,

@@ -266,9 +266,18 @@ int laser_fusion_forward(const laser_config* cfg, const void* Hprime, const void
   return fusion_forward(p, Hprime, z, lengths, cand_offsets, num_recent, fused, ws, st);
 }
 
+// The variant has a tensor-core version (bf16 shapes the tensor path supports) and the FP32-ALU one; there is no
+// one-candidate streaming version, so LASER_PATH_AUTO means "tensor cores if supported" and LASER_PATH_STREAM falls back
+// to the FP32 ALUs.
 static int softmax_plan(const laser_config* cfg, Plan* p) {
   if (!cfg) return LASER_ERR_INVALID_ARG;
   laser_config c = *cfg;
+  if (c.path == LASER_PATH_AUTO || c.path == LASER_PATH_TENSOR) {
+    const int requested = c.path;
+    c.path = LASER_PATH_TENSOR;
+    if (make_plan(&c, p) == LASER_OK && tensor_softmax_supported(*p)) return LASER_OK;
+    if (requested == LASER_PATH_TENSOR) return LASER_ERR_UNSUPPORTED;
+  }
   c.path = LASER_PATH_SIMT;
   return make_plan(&c, p);
 }
@@ -293,6 +302,8 @@ int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const 
   char* ws = static_cast<char*>(workspace);
   if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
+  if (p.path == LASER_PATH_TENSOR)
+    return tensor_sta(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st, nullptr, true);
   return simt_sta_softmax(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
 }
 

@@ -75,9 +75,11 @@ int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const i
 bool tensor_supported(const Plan& p);
 void tensor_geometry(const Plan& p, TensorGeom* g);
 // Wg_images: when non-null (and the fused GSTA kernel will follow), the set-up kernel also builds the GSTA weight images.
+// softmax: the softmax-aggregation variant (the paper's ablation of the sigmoid gate); needs tensor_softmax_supported(p).
+bool tensor_softmax_supported(const Plan& p);
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
                const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
-               const void* Wg_images);
+               const void* Wg_images, bool softmax = false);
 // Launches the bounded-wait self-test block (laser_tensor.cu); the status word is the first word of ws.
 int tensor_wait_selftest(char* ws, int poll_limit, cudaStream_t st);
 int tensor_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets,

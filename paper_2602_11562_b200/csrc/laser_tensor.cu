@@ -612,10 +612,10 @@ struct UnitWalker {
   // tiles of the current segment that hold at least one valid item
   __device__ int ntiles(const TcParams& P) const { return seg == nseg - 1 ? last_tiles : P.NT; }
   // columns of tile t that can hold a non-zero gate: its valid items rounded up to the MMA k-step (16)
-  __device__ int tile_cols(const TcParams& P, int t) const {
-    const int items = min(P.IT, (seg == nseg - 1 ? last_items : P.S) - t * P.IT);
-    return (items + 15) & ~15;
+  __device__ int tile_items(const TcParams& P, int t) const {
+    return min(P.IT, (seg == nseg - 1 ? last_items : P.S) - t * P.IT);
   }
+  __device__ int tile_cols(const TcParams& P, int t) const { return (tile_items(P, t) + 15) & ~15; }
 };
 
 struct StaBars {
@@ -643,6 +643,16 @@ constexpr uint32_t kColO = kColP + kGateGroups * (kItMax / 2);   // outputs [n_o
 // and one gate buffer in TMEM.  Per unit: the issuer writes S = Q_h K_h^T; the warpgroup reads it (releasing the score
 // buffer for the issuer's next unit as soon as the last column is in registers), writes P = 1 + tanh(S) as packed bf16;
 // the issuer accumulates O_h += P V_h.  All MMAs into a head's accumulator come from one thread, in order.
+//
+// kSoftmax selects the softmax-aggregation variant (the paper's ablation of the sigmoid gate): the weights of a segment's
+// valid items are exp(q_h . k_{n,h} / gamma) normalised to one per (candidate, head).  A gate thread owns one candidate
+// row of the score buffer, so the row sums are plain per-thread accumulations over the tiles of the segment; they reach
+// the epilogue through shared memory (a ring of four segments), and the epilogue divides each head's columns by its sum
+// instead of halving them.  The exponent is shifted by the row's maximum over the first 32 valid items of the segment
+// (any shift cancels in the quotient; this one keeps the sum >= 1) and capped at 2^60 above that shift.
+constexpr int kSumSlots = 4;
+constexpr float kExpCap = 60.f;
+template <bool kSoftmax>
 __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ StaBars bars;
@@ -658,6 +668,7 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
   uint8_t* Ks = Qs + 2 * q_bytes;                 // [kKvStages][k_bytes]
   uint8_t* Vs = Ks + kKvStages * k_bytes;         // [kKvStages][v_bytes]
   uint8_t* Os = Vs + kKvStages * v_bytes;         // [2][kCandTile][out_row]  staged H' rows
+  float* Sums = reinterpret_cast<float*>(Os + 2 * kCandTile * out_row);   // [kSumSlots][H][kCandTile] (kSoftmax only)
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
@@ -883,25 +894,62 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars.s_free[wg]);
       };
+      // softmax variant: per head of this warpgroup (at most two), this row's exponent shift and running sum
+      const float k2 = 2.f * 1.4426950408889634f;           // the scores hold q.k / (2 gamma); weights are 2^(k2 s - shift)
+      float sh0 = 0.f, sh1 = 0.f, rs0 = 0.f, rs1 = 0.f;
+      const int row = (warp & 3) * 32 + lane;
       for (int it = 0; it < my_units && ok; ++it, w.next(P)) {
         const int nt = w.ntiles(P);
         for (int t = 0; t < nt && ok; ++t) {
           const int cols = w.tile_cols(P, t);               // columns past this hold zero K rows: their gates are 0
+          const int items = w.tile_items(P, t);
           for (int hh = 0; hh < my_heads && ok; ++hh) {
             ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[wg], s_par, abortp));
             if (!ok) break;
             s_par ^= 1;
             tc_fence_after();
             bool first = true;
+            float shift = hh ? sh1 : sh0, rsum = (t == 0) ? 0.f : (hh ? rs1 : rs0);
+            // weights of `n` score columns starting at column c: packed bf16 pairs, summed as the MMA will see them
+            auto weights = [&](const uint32_t* v, uint32_t* o, int c, int n) {
+              if (t == 0 && c == 0) {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) if (e < n && e < items) mx = fmaxf(mx, __uint_as_float(v[e]));
+#pragma unroll
+                for (int e = 16; e < 32; ++e) if (e < n && e < items) mx = fmaxf(mx, __uint_as_float(v[e]));
+                shift = mx * k2;
+              }
+              const bool whole = c + n <= items;
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                if (2 * e < n) {
+                  float p0, p1;
+                  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p0) : "f"(fminf(fmaf(__uint_as_float(v[2 * e]), k2, -shift), kExpCap)));
+                  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p1) : "f"(fminf(fmaf(__uint_as_float(v[2 * e + 1]), k2, -shift), kExpCap)));
+                  if (!whole) {                             // padding columns of the segment's last 16-column group
+                    if (c + 2 * e >= items) p0 = 0.f;
+                    if (c + 2 * e + 1 >= items) p1 = 0.f;
+                  }
+                  const uint32_t pk = pack_bf16x2(p0, p1);
+                  rsum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xFFFF0000u);
+                  o[e] = pk;
+                }
+              }
+            };
             int c = 0;
             for (; c + 32 <= cols; c += 32) {
               uint32_t v[32], o[16];
               tmem_ld32(tS + c, v);
               tc_wait_ld();
               if (c + 32 >= cols) release_scores();
+              if (kSoftmax) {
+                weights(v, o, c, 32);
+              } else {
 #pragma unroll
-              for (int e = 0; e < 16; ++e)
-                o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
+                for (int e = 0; e < 16; ++e)
+                  o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
+              }
               if (first) {                                  // the previous unit's gates have been multiplied
                 ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
                 pf_par ^= 1;
@@ -911,20 +959,36 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
               tmem_st16(tP + (c >> 1), o);
             }
             if (c < cols) {   // 16-column tail
-              uint32_t v[16], o[8];
-              tmem_ld16(tS + c, v);
-              tc_wait_ld();
-              release_scores();
+              uint32_t v[32], o[16];
+              {
+                uint32_t v16[16];
+                tmem_ld16(tS + c, v16);
+                tc_wait_ld();
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
-                o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
+                for (int e = 0; e < 16; ++e) v[e] = v16[e];
+              }
+              release_scores();
+              if (kSoftmax) {
+                weights(v, o, c, 16);
+              } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                  o[e] = pack_bf16x2(1.f + tanh_approx(__uint_as_float(v[2 * e])), 1.f + tanh_approx(__uint_as_float(v[2 * e + 1])));
+              }
               if (first) {
                 ok = __all_sync(0xffffffffu, mbar_wait(&bars.p_free[wg], pf_par, abortp));
                 pf_par ^= 1;
                 first = false;
                 tc_fence_after();
               }
-              tmem_st8(tP + (c >> 1), o);
+              uint32_t o8[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) o8[e] = o[e];
+              tmem_st8(tP + (c >> 1), o8);
+            }
+            if (kSoftmax) {
+              if (hh) { sh1 = shift; rs1 = rsum; } else { sh0 = shift; rs0 = rsum; }
+              if (t == nt - 1) Sums[((it & (kSumSlots - 1)) * H + wg + kGateGroups * hh) * kCandTile + row] = rsum;
             }
             tc_wait_st();
             tc_fence_before();
@@ -959,33 +1023,38 @@ __global__ void __launch_bounds__(kStaThreads, 1) tc_sta_kernel(TcParams P) {
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.o_empty[ob]);
         };
-        auto stage16 = [&](int c, const uint32_t (&v)[16]) {
+        // sigmoid gates: H' = O / 2; softmax variant: the 16 columns' head divides by its row sum
+        const float* sums = Sums + (size_t)((it & (kSumSlots - 1)) * H) * kCandTile + m;
+        auto factor = [&](int c) { return kSoftmax ? 1.f / sums[(c / P.dvh) * kCandTile] : 0.5f; };
+        auto stage16 = [&](int c, const uint32_t (&v)[16], float f) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             uint4 o;
-            o.x = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 0]), 0.5f * __uint_as_float(v[half * 8 + 1]));
-            o.y = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 2]), 0.5f * __uint_as_float(v[half * 8 + 3]));
-            o.z = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 4]), 0.5f * __uint_as_float(v[half * 8 + 5]));
-            o.w = pack_bf16x2(0.5f * __uint_as_float(v[half * 8 + 6]), 0.5f * __uint_as_float(v[half * 8 + 7]));
+            o.x = pack_bf16x2(f * __uint_as_float(v[half * 8 + 0]), f * __uint_as_float(v[half * 8 + 1]));
+            o.y = pack_bf16x2(f * __uint_as_float(v[half * 8 + 2]), f * __uint_as_float(v[half * 8 + 3]));
+            o.z = pack_bf16x2(f * __uint_as_float(v[half * 8 + 4]), f * __uint_as_float(v[half * 8 + 5]));
+            o.w = pack_bf16x2(f * __uint_as_float(v[half * 8 + 6]), f * __uint_as_float(v[half * 8 + 7]));
             *reinterpret_cast<uint4*>(row + (c + half * 8) * 2) = o;
           }
         };
         int c = 0;
         for (; c + 32 <= d; c += 32) {                     // two accumulator loads in flight per wait
           uint32_t v0[16], v1[16];
+          const float f0 = factor(c), f1 = factor(c + 16);   // (the sums are read before the accumulator is handed back)
           tmem_ld16(tO + c, v0);
           tmem_ld16(tO + c + 16, v1);
           tc_wait_ld();
           if (c + 32 >= d) hand_back();
-          stage16(c, v0);
-          stage16(c + 16, v1);
+          stage16(c, v0, f0);
+          stage16(c + 16, v1, f1);
         }
         if (c < d) {
           uint32_t v0[16];
+          const float f0 = factor(c);
           tmem_ld16(tO + c, v0);
           tc_wait_ld();
           hand_back();
-          stage16(c, v0);
+          stage16(c, v0, f0);
         }
         const int ci = w.j * kCandTile + m;
         if (ci < w.nc) {                                   // my candidate's row of this segment: one contiguous store
@@ -1118,9 +1187,23 @@ bool encode_item_map(const Plan& p, int IT, const void* items, CUtensorMap* map)
 }
 }  // namespace
 
+// Shared memory of the attention kernel: Q double buffer, K / V^T ring, staged output rows, and for the softmax variant
+// the ring of row sums.
+static size_t sta_smem_bytes(const Plan& p, int IT, bool softmax) {
+  return (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * IT * (p.dqk + p.d) * 2 +
+         (size_t)2 * kCandTile * (p.d * 2 + 16) + (softmax ? (size_t)kSumSlots * p.H * kCandTile * sizeof(float) : 0);
+}
+
+bool tensor_softmax_supported(const Plan& p) {
+  if (!tensor_supported(p)) return false;
+  TensorGeom g;
+  tensor_geometry(p, &g);
+  return sta_smem_bytes(p, g.IT, true) <= 220 * 1024;
+}
+
 int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
                const void* Wq, const void* Wk, const void* Wv, void* Hprime, char* ws, cudaStream_t st,
-               const void* Wg_images) {
+               const void* Wg_images, bool softmax) {
   if (p.N == 0 || p.U == 0) return LASER_OK;
   const bool user_wants_hp = Hprime != (void*)(ws + p.off_hp);
   TcParams P = make_params(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws);
@@ -1154,12 +1237,12 @@ int tensor_sta(const Plan& p, const void* items, const int32_t* lengths, const v
     LASER_CUDA_OK(launch_chained(tc_zero_empty_kernel, dim3(p.Lp, p.U), dim3(256), 0, st, P));
   }
   {
-    const size_t smem = (size_t)2 * kCandTile * p.dqk * 2 + (size_t)kKvStages * P.IT * (p.dqk + p.d) * 2 +
-                        (size_t)2 * kCandTile * (p.d * 2 + 16);
+    const size_t smem = sta_smem_bytes(p, P.IT, softmax);
     if (smem > 220 * 1024) return LASER_ERR_UNSUPPORTED;
-    LASER_CUDA_OK(cudaFuncSetAttribute(tc_sta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    LaunchScope ls("sta_tc", st);
-    LASER_CUDA_OK(launch_chained(tc_sta_kernel, dim3(P.sta_grid), dim3(kStaThreads), smem, st, P));
+    auto kernel = softmax ? tc_sta_kernel<true> : tc_sta_kernel<false>;
+    LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LaunchScope ls(softmax ? "sta_tc_softmax" : "sta_tc", st);
+    LASER_CUDA_OK(launch_chained(kernel, dim3(P.sta_grid), dim3(kStaThreads), smem, st, P));
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;

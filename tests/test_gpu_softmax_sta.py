@@ -27,7 +27,7 @@ def test_softmax_sta_matches_oracle(case):
     s = w.spec
     ref = softmax_sta_oracle.sta_softmax_forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, s.S, s.H,
                                                  w.gamma)
-    b = P.DeviceBatch.from_workload(w)                       # whatever path the config selects: the variant ignores it
+    b = P.DeviceBatch.from_workload(w)                       # automatic choice: tensor cores where the shape allows
     ws = torch.empty(P.laser_sta_softmax_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
     Hp = P.laser_sta_softmax_forward(b.cfg, *b.args(), workspace=ws)
     assert P.laser_check_status(ws) == 0
@@ -37,3 +37,58 @@ def test_softmax_sta_matches_oracle(case):
     Hs = P.laser_sta_forward(b.cfg, *b.args())
     if case < 4:
         assert err_metric(to_np(Hs), ref) > 10 * TOL[s.dtype]
+
+
+# bf16 shapes that the tensor-core version takes: several candidate tiles, segments of one and of two item tiles with a
+# ragged last tile, one to eight heads, the paper's production shape, a one-item last segment
+TENSOR_CASES = [
+    dict(U=3, C=200, L=512, d=128, H=4, S=128, M=1, dtype="bf16", lengths=[512, 300, 77]),
+    dict(U=2, C=130, L=1000, d=64, H=4, S=100, M=1, dtype="bf16", lengths=[1000, 555]),
+    dict(U=2, C=70, L=256, d=128, H=8, S=32, M=1, dtype="bf16", lengths=[256, 129]),
+    dict(U=2, C=300, L=1000, d=128, H=2, S=10, M=1, dtype="bf16", lengths=[1000, 431]),
+    dict(U=4, C=33, L=512, d=64, H=4, S=64, M=1, dtype="bf16", lengths=[512, 1, 0, 65]),
+    dict(U=2, C=129, L=192, d=64, H=1, S=96, M=1, dtype="bf16", lengths=[192, 100], d_qh=64),
+    # logits with a spread of several nats (unit-variance embeddings, gamma = 1, |logit| up to ~15): near one-hot weights.
+    # The tensor-core version rounds Q and K to bf16 before the product, which moves a logit s by up to ~2^-8 |s| = 0.06
+    # nats, i.e. a weight by up to 6 %, and the outputs here are O(1): the bound for this case is 8e-2 (on the other
+    # cases the logits stay within a nat or two and the usual bf16 bound holds).
+    dict(U=2, C=64, L=256, d=64, H=4, S=128, M=1, dtype="bf16", lengths=[256, 200], emb_std="one", gamma=1.0, tol=8e-2),
+]
+
+
+def _profiled_softmax(b, ws):
+    P.laser_profile_enable(True)
+    try:
+        Hp = P.laser_sta_softmax_forward(b.cfg, *b.args(), workspace=ws)
+        names = [n for n, _ in P.laser_profile_read()]
+    finally:
+        P.laser_profile_enable(False)
+    return Hp, names
+
+
+@pytest.mark.parametrize("case", range(len(TENSOR_CASES)))
+def test_softmax_sta_tensor_path_matches_oracle(case):
+    kw = dict(TENSOR_CASES[case])
+    tol = kw.pop("tol", TOL["bf16"])
+    w = make_custom(seed=900 + case, **kw)
+    s = w.spec
+    ref = softmax_sta_oracle.sta_softmax_forward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, s.S, s.H,
+                                                 w.gamma)
+    b = P.DeviceBatch.from_workload(w)
+    ws = torch.empty(P.laser_sta_softmax_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    Hp, names = _profiled_softmax(b, ws)
+    assert "sta_tc_softmax" in names, names                  # the tensor-core kernel is what ran
+    assert P.laser_check_status(ws) == 0
+    got = to_np(Hp)
+    assert np.isfinite(got).all()
+    e = err_metric(got, ref)
+    assert e <= tol, f"case {case}: err {e}"
+    # a second call on the same workspace gives the same bits (the ring of row sums carries nothing over)
+    Hp2 = P.laser_sta_softmax_forward(b.cfg, *b.args(), workspace=ws)
+    assert torch.equal(Hp, Hp2)
+    # the FP32-ALU version on request, against the same oracle
+    bs = P.DeviceBatch.from_workload(w, path=P.PATH_SIMT)
+    ws2 = torch.empty(P.laser_sta_softmax_workspace_bytes(bs.cfg), dtype=torch.uint8, device="cuda")
+    Hs, names2 = _profiled_softmax(bs, ws2)
+    assert "sta_tc_softmax" not in names2
+    assert err_metric(to_np(Hs), ref) <= TOL["bf16"]
