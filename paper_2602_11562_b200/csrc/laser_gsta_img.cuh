@@ -61,38 +61,37 @@ __device__ __forceinline__ void gsta_build_nseg(const int* lengths, const int* c
   }
 }
 
-// Launch order of the GSTA kernel's blocks, longest first: block b of the kernel takes candidates
-// order[b] * cpb .. order[b] * cpb + cpb - 1.  A block's time grows with the number of segments of its candidates, and a
-// grid of several waves that ends on long blocks leaves most SMs idle during the last of them; started longest first,
-// the tail is made of the shortest blocks.  A counting sort by the segment count of each block's first candidate (counts
-// above kGstaOrderBins - 1 share the last bin), run by ONE thread block (all of its threads call this);
-// blocks of equal count land in arbitrary order.  keys: n_blocks ints of scratch.  Invalid lengths or offsets are
-// reported elsewhere; here they are clamped, so `order` is a permutation of 0 .. n_blocks - 1 whatever the inputs hold.
+// Counting sort, largest key first: order[0 .. n - 1] = the indices 0 .. n - 1 by descending key(i) (keys in
+// 0 .. kGstaOrderBins - 1; equal keys land in arbitrary order).  Run by ONE thread block (all of its threads call this, at
+// least one warp); keys: n ints of scratch.
 constexpr int kGstaOrderBins = 1024;
-__device__ __forceinline__ void gsta_build_order(const int* lengths, const int* cand_offsets, int U, int N, int L, int S,
-                                                 int Lp, int cpb, int* order, int* keys) {
+template <class KeyFn>
+__device__ __forceinline__ void sort_desc_by_key(int n, KeyFn key_of, int* order, int* keys) {
   __shared__ int bins[kGstaOrderBins + kGstaOrderBins / 32];      // bin k at k + k / 32: lane-strided walks stay conflict-free
   const int tid = threadIdx.x, nt = blockDim.x;
-  const int n_blocks = (N + cpb - 1) / cpb;
   for (int i = tid; i < kGstaOrderBins + kGstaOrderBins / 32; i += nt) bins[i] = 0;
   __syncthreads();
-  for (int b = tid; b < n_blocks; b += nt) {
-    const int c = b * cpb;
-    int lo = 0, hi = U - 1;                      // the last user whose first candidate is <= c
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (cand_offsets[mid] <= c) lo = mid; else hi = mid - 1;
+  constexpr int kBatch = 8;                      // independent loads first, then the atomics: the passes are latency-bound
+  for (int b0 = tid; b0 < n; b0 += kBatch * nt) {
+    int key[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const int b = b0 + j * nt;
+      key[j] = b < n ? min(max(key_of(b), 0), kGstaOrderBins - 1) : -1;
     }
-    const int len = min(max(lengths[lo], 0), L);
-    const int key = min(min((len + S - 1) / S, Lp), kGstaOrderBins - 1);
-    keys[b] = key;
-    atomicAdd(&bins[key + (key >> 5)], 1);
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      if (key[j] >= 0) {
+        keys[b0 + j * nt] = key[j];
+        atomicAdd(&bins[key[j] + (key[j] >> 5)], 1);
+      }
+    }
   }
   __syncthreads();
-  if (tid < 32) {                                // bins[k] <- number of blocks with a larger key (lane `tid` owns 32 bins)
+  if (tid < 32) {                                // bins[k] <- number of items with a larger key (lane `tid` owns 32 bins)
     int mine = 0;
     for (int j = 0; j < 32; ++j) mine += bins[tid * 33 + j];
-    int incl = mine;                             // blocks in this lane's bins and in those of the lanes above
+    int incl = mine;                             // items in this lane's bins and in those of the lanes above
     for (int off = 1; off < 32; off <<= 1) {
       const int v = __shfl_down_sync(0xffffffffu, incl, off);
       if (tid + off < 32) incl += v;
@@ -105,10 +104,36 @@ __device__ __forceinline__ void gsta_build_order(const int* lengths, const int* 
     }
   }
   __syncthreads();
-  for (int b = tid; b < n_blocks; b += nt) {
-    const int key = keys[b];
-    order[atomicAdd(&bins[key + (key >> 5)], 1)] = b;
+  for (int b0 = tid; b0 < n; b0 += kBatch * nt) {
+    int key[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) key[j] = b0 + j * nt < n ? keys[b0 + j * nt] : -1;
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j)
+      if (key[j] >= 0) order[atomicAdd(&bins[key[j] + (key[j] >> 5)], 1)] = b0 + j * nt;
   }
+}
+
+// Launch order of the GSTA kernel's blocks, longest first: block b of the kernel takes candidates
+// order[b] * cpb .. order[b] * cpb + cpb - 1.  A block's time grows with the number of segments of its candidates, and a
+// grid of several waves that ends on long blocks leaves most SMs idle during the last of them; started longest first,
+// the tail is made of the shortest blocks.  Sorted by the segment count of each block's first candidate (counts
+// above kGstaOrderBins - 1 share the last bin), by ONE thread block.  keys: n_blocks ints of scratch.  Invalid lengths
+// or offsets are reported elsewhere; here they are clamped, so `order` is a permutation of 0 .. n_blocks - 1 whatever
+// the inputs hold.
+__device__ __forceinline__ void gsta_build_order(const int* lengths, const int* cand_offsets, int U, int N, int L, int S,
+                                                 int Lp, int cpb, int* order, int* keys) {
+  const int n_blocks = (N + cpb - 1) / cpb;
+  sort_desc_by_key(n_blocks, [&](int b) {
+    const int c = b * cpb;
+    int lo = 0, hi = U - 1;                      // the last user whose first candidate is <= c
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (cand_offsets[mid] <= c) lo = mid; else hi = mid - 1;
+    }
+    const int len = min(max(lengths[lo], 0), L);
+    return min((len + S - 1) / S, Lp);
+  }, order, keys);
 }
 
 }  // namespace laser

@@ -50,6 +50,8 @@ struct StreamParams {
   uint4* gimg;
   int* gnseg;                     // per-candidate segment counts for the GSTA kernel (built with the images)
   int M;
+  int* order;                     // [U] users by descending length (null: blocks take the users in index order)
+  int* order_keys;                // [U] scratch of the sort
   int* status;
 };
 
@@ -74,10 +76,19 @@ __global__ void __launch_bounds__(kPreWarps * 32) stream_pre_kernel(StreamParams
   const int dqk = P.dqk, H = P.H, dqh = dqk / H;
   chain_wait();
   chain_release();
+  if (P.order && blockIdx.x == gridDim.x - 1) {
+    // the last block sorts the users by length, longest first: the attention kernel's grid runs in several waves of
+    // blocks whose time is proportional to the user's length, and its last wave should be made of the shortest
+    const float per_row = (float)(kGstaOrderBins - 1) / (float)P.L;
+    sort_desc_by_key(P.U, [&](int u) { return (int)((float)min(max(P.lengths[u], 0), P.L) * per_row); }, P.order,
+                     P.order_keys);
+    return;
+  }
   if (wg >= user_warps) {
     // spare warps: W_v image, entry (kt, p, lane) = {b0, b1 of column tile 2p, b0, b1 of column tile 2p+1},
     // B[k][n] = W_v[k][n]; and the GSTA weight images when GSTA follows
-    const int worker = (wg - user_warps) * 32 + lane, n_workers = (gridDim.x * kPreWarps - user_warps) * 32;
+    const int worker = (wg - user_warps) * 32 + lane;
+    const int n_workers = (((int)gridDim.x - (P.order ? 1 : 0)) * kPreWarps - user_warps) * 32;
     const int total = D16 * D16 * 32;
     const uint16_t* W = reinterpret_cast<const uint16_t*>(P.Wv);
     for (int i = worker; i < total; i += n_workers) {
@@ -171,9 +182,9 @@ __global__ void __launch_bounds__(kSThreads) stream_sta_kernel(StreamParams P) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int H = P.H, dvh = d / H;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int u = blockIdx.x;
   chain_wait();
   chain_release();
+  const int u = P.order ? min(max(P.order[blockIdx.x], 0), P.U - 1) : (int)blockIdx.x;
   int len = 0;
   const int cand = user_candidate(P, u, &len);
   if (cand < 0) return;
@@ -373,8 +384,16 @@ bool stream_supported(const Plan& p) {
   return stream_smem_bytes(p.d, p.H, p.Lp) <= 200 * 1024;
 }
 
-size_t stream_scratch_bytes(const Plan& p) {
-  return align_up((size_t)p.U * p.H * p.d * sizeof(float)) + align_up((size_t)p.d * p.d * 2);
+size_t stream_scratch_bytes(const Plan& p) {   // u, the W_v image, the launch order of the users and its sort keys
+  return align_up((size_t)p.U * p.H * p.d * sizeof(float)) + align_up((size_t)p.d * p.d * 2) +
+         align_up(2 * (size_t)p.U * sizeof(int));
+}
+
+// Sorting the users pays only when the attention grid runs in more than one wave (four blocks per SM).
+static bool stream_wants_order(const Plan& p) {
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return p.U > 4 * sms;
 }
 
 int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
@@ -397,9 +416,16 @@ int stream_sta(const Plan& p, const void* items, const int32_t* lengths, const v
   P.Hp = (bf16*)Hprime;
   P.zero_empty = Hprime != (void*)(ws + p.off_hp);
   P.status = reinterpret_cast<int*>(ws + p.off_status);
+  P.order = nullptr;
+  P.order_keys = nullptr;
+  if (stream_wants_order(p)) {
+    P.order = reinterpret_cast<int*>(ws + p.off_su + align_up((size_t)p.U * p.H * p.d * sizeof(float)) +
+                                     align_up((size_t)p.d * p.d * 2));
+    P.order_keys = P.order + p.U;
+  }
   {
     const int user_warps = (p.U + 15) / 16;
-    const dim3 grid((user_warps + kPreWarps - 1) / kPreWarps + 2), block(kPreWarps * 32);
+    const dim3 grid((user_warps + kPreWarps - 1) / kPreWarps + 2 + (P.order ? 1 : 0)), block(kPreWarps * 32);
     LaunchScope ls("stream_pre", st);
     cudaError_t e;
     switch (p.d / 16) {
