@@ -207,6 +207,28 @@ LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* ite
                                         const void* Wv, void* Hprime, void* workspace, size_t workspace_bytes,
                                         void* cuda_stream);
 
+/* Backward pass of laser_forward: given dz = dLoss/dz [N, d], the gradients of the loss with respect to every input of
+ * the forward, i.e. the chain rule through Eq. 7 and its residual updates (layers last to first), then through the
+ * segment sums and gates (Eq. 10-12) and the projections (Eq. 8-9).  The paper trains the model (section "Experimental
+ * Settings") and prints no backward formulas; readings are those of the forward (an item at or past its user's length
+ * receives a zero gradient row, an empty segment passes no gradient).  All gradients are fp32 device arrays, whatever
+ * cfg->dtype; the inputs are read in cfg->dtype.  Runs on the FP32 ALUs whatever cfg->path says (a first version: it
+ * recomputes the forward in fp32 and keeps every intermediate), padded item layout only.
+ *   dz          [N, d] fp32            IN
+ *   d_items     [U, L, d] fp32         OUT (rows of padding are zero)
+ *   d_cands     [N, d] fp32            OUT
+ *   dWq, dWk    [d, d_qk] fp32         OUT
+ *   dWv         [d, d] fp32            OUT
+ *   dWgsta      [M, 3, d, d] fp32      OUT (may be NULL when M = 0)
+ *   workspace   at least laser_backward_workspace_bytes(cfg) bytes, 256-byte aligned; its first word is the status word
+ * Sums over candidates that end in one weight matrix (and the query-side part of d_cands) are finished with
+ * floating-point atomics: their last bits may differ from call to call. */
+LASER_API size_t laser_backward_workspace_bytes(const laser_config* cfg);
+LASER_API int laser_backward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                             const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv,
+                             const void* Wgsta, const float* dz, float* d_items, float* d_cands, float* dWq, float* dWk,
+                             float* dWv, float* dWgsta, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* STA without any workspace argument, for callers that cannot allocate device memory (no counterpart in the
  * paper: this is a deployment convenience of this library).  Think of a plug-in inside a serving process
  * whose GPU memory belongs entirely to the host framework's pool, or of a request thread that must never hit

@@ -24,6 +24,8 @@ from .binding import (  # noqa: F401
     laser_fusion_forward,
     laser_sta_softmax_workspace_bytes,
     laser_sta_softmax_forward,
+    laser_backward_workspace_bytes,
+    laser_backward,
     laser_ffn_workspace_bytes,
     laser_ffn_forward,
     laser_forward_ffn,

@@ -90,6 +90,10 @@ def load_library() -> ctypes.CDLL:
     lib.laser_sta_softmax_workspace_bytes.argtypes = [cfgp]
     lib.laser_sta_softmax_forward.restype = ctypes.c_int
     lib.laser_sta_softmax_forward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, sz, vp]
+    lib.laser_backward_workspace_bytes.restype = sz
+    lib.laser_backward_workspace_bytes.argtypes = [cfgp]
+    lib.laser_backward.restype = ctypes.c_int
+    lib.laser_backward.argtypes = [cfgp, vp, i32p, vp, i32p, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     ffnp = ctypes.POINTER(LaserFfnParams)
     lib.laser_ffn_workspace_bytes.restype = sz
     lib.laser_ffn_workspace_bytes.argtypes = [cfgp, ctypes.c_int32]
@@ -328,6 +332,36 @@ def laser_sta_softmax_forward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, 
                                        _dev(Hprime, dt, "Hprime"), ws.data_ptr(), ws.numel(), _stream_ptr(stream))
     _check(rc, "laser_sta_softmax_forward")
     return Hprime
+
+
+def laser_backward_workspace_bytes(cfg: LaserConfig) -> int:
+    return int(load_library().laser_backward_workspace_bytes(ctypes.byref(cfg)))
+
+
+def laser_backward(cfg, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wg, dz, workspace=None, stream=None):
+    """Backward pass of laser_forward for the upstream gradient dz [N, d] (float32).  Returns a dict of float32
+    tensors: d_items [U, L, d], d_cands [N, d], dWq, dWk [d, d_qk], dWv [d, d], dWg [M, 3, d, d]."""
+    lib, dt = load_library(), cfg.torch_dtype()
+    need = laser_backward_workspace_bytes(cfg)
+    if need == 0:
+        raise LaserError(-1, "laser_backward_workspace_bytes (invalid or unsupported configuration)")
+    dev = items.device
+    ws = torch.empty(need, dtype=torch.uint8, device=dev) if workspace is None else workspace
+    f32 = torch.float32
+    out = {"d_items": torch.empty((cfg.num_users, cfg.max_len, cfg.d_model), dtype=f32, device=dev),
+           "d_cands": torch.empty((cfg.total_cands, cfg.d_model), dtype=f32, device=dev),
+           "dWq": torch.empty((cfg.d_model, cfg.d_qk), dtype=f32, device=dev),
+           "dWk": torch.empty((cfg.d_model, cfg.d_qk), dtype=f32, device=dev),
+           "dWv": torch.empty((cfg.d_model, cfg.d_model), dtype=f32, device=dev),
+           "dWg": torch.empty((cfg.num_gsta_layers, 3, cfg.d_model, cfg.d_model), dtype=f32, device=dev)}
+    rc = lib.laser_backward(ctypes.byref(cfg), _dev(items, dt, "items"), _dev(lengths, torch.int32, "lengths"),
+                            _dev(cands, dt, "cands"), _dev(cand_offsets, torch.int32, "cand_offsets"),
+                            _dev(Wq, dt, "Wq"), _dev(Wk, dt, "Wk"), _dev(Wv, dt, "Wv"), _dev(Wg, dt, "Wg"),
+                            _dev(dz, f32, "dz"), out["d_items"].data_ptr(), out["d_cands"].data_ptr(),
+                            out["dWq"].data_ptr(), out["dWk"].data_ptr(), out["dWv"].data_ptr(), out["dWg"].data_ptr(),
+                            ws.data_ptr(), ws.numel(), _stream_ptr(stream))
+    _check(rc, "laser_backward")
+    return out
 
 
 def laser_ffn_workspace_bytes(cfg: LaserConfig, d_hidden: int) -> int:

@@ -307,6 +307,42 @@ int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const 
   return simt_sta_softmax(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
 }
 
+// The backward pass runs on the FP32 ALUs whatever cfg->path says, on the padded item layout.
+static int backward_plan(const laser_config* cfg, Plan* p) {
+  if (!cfg) return LASER_ERR_INVALID_ARG;
+  laser_config c = *cfg;
+  c.path = LASER_PATH_SIMT;
+  return make_plan(&c, p);
+}
+
+size_t laser_backward_workspace_bytes(const laser_config* cfg) {
+  Plan p;
+  if (backward_plan(cfg, &p) != LASER_OK) return 0;
+  return p.total + backward_scratch_bytes(p);
+}
+
+int laser_backward(const laser_config* cfg, const void* items, const int32_t* lengths, const void* cands,
+                   const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wgsta,
+                   const float* dz, float* d_items, float* d_cands, float* dWq, float* dWk, float* dWv, float* dWgsta,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  reset_launch_count();
+  Plan p;
+  int rc = backward_plan(cfg, &p);
+  if (rc != LASER_OK) return rc;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
+  if (workspace_bytes < p.total + backward_scratch_bytes(p)) return LASER_ERR_WORKSPACE;
+  if (!lengths || !cand_offsets) return LASER_ERR_INVALID_ARG;
+  if ((rc = check_ptrs({Wq, Wk, Wv, dWq, dWk, dWv})) != LASER_OK) return rc;
+  if (p.U > 0 && (rc = check_ptrs({items, d_items})) != LASER_OK) return rc;
+  if (p.N > 0 && (rc = check_ptrs({cands, dz, d_cands})) != LASER_OK) return rc;
+  if (p.M > 0 && (rc = check_ptrs({Wgsta, dWgsta})) != LASER_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* ws = static_cast<char*>(workspace);
+  if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
+  return backward(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, dz, d_items, d_cands, dWq, dWk, dWv, dWgsta,
+                  ws, st);
+}
+
 size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hidden) {
   Plan p;
   if (make_plan(cfg, &p) != LASER_OK || d_hidden < 1) return 0;

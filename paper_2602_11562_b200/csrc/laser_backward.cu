@@ -1,0 +1,459 @@
+// Backward pass of STA + GSTA: the vector-Jacobian product of z with respect to the items, the candidates and every
+// weight matrix.  The paper trains the model (section "Experimental Settings") without printing backward formulas; what
+// is computed here is the chain rule through Eq. 7 (layers last to first) and then through Eq. 10-12 and Eq. 8-9.
+//
+// FP32-ALU implementation for either I/O dtype (inputs are read in their dtype, everything else is fp32): a first,
+// correctness-oriented version.  The forward intermediates are recomputed in fp32 (projections, H', and per GSTA layer
+// the running target, Q, the key-folded query Qt_h = W_k[:, h] Q_h / tau, the attention weights and the weighted sums
+// m_h = sum_j a_j s_j), all dense steps are batched matrix products over the N candidates (or the U L item rows), and
+// three kernels do what is not a matrix product:
+//   gsta_attn_fwd   per candidate: e_{j,h} = s_j . Qt_h, a = softmax_j, m_h = sum_j a_{j,h} s_j
+//   gsta_attn_bwd   per candidate: da_j = s_j . dm_h, de = a (da - sum a da), dQt_h = sum_j de_j s_j,
+//                   ds_j += de_j Qt_h + a_j dm_h
+//   sta_bwd         per (user, 32 items of a segment), looping over the user's candidates: gate g = Sigmoid(q_h . k_n),
+//                   dg = ds_i[h] . v_n, dv_n += g ds_i[h], de = dg g (1 - g), dk_n += de q_h, dq_h += de k_n
+// With the re-association of the forward (keys and values of a segment vector are never formed):
+//   o_h = m_h W_v[:, h]  =>  dm_h = do_h W_v[:, h]^T,  dW_v[:, h] += m_h^T do_h
+//   Qt_h = Q_h W_k[:, h]^T / tau  =>  dQ_h = dQt_h W_k[:, h] / tau,  dW_k[:, h] += dQt_h^T Q_h / tau
+// Sums over candidates that end in one weight matrix are split over blocks and finished with floating-point atomics, so
+// the last bits of the weight gradients and of d_cands' STA part depend on the order in which blocks finish.
+#include "laser_common.cuh"
+
+namespace laser {
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+// ------------------------------------------------------------------------------------------------ batched products
+// C[m][n] (+)= alpha * sum_k A(m, k) B(k, n);  A(m, k) = ta ? A[k lda + m] : A[m lda + k],  B(k, n) = tb ? B[n ldb + k]
+// : B[k ldb + n].  64 x 64 tiles of C, k-steps of 16; gridDim.z splits K and the partial sums are added atomically
+// (C then has to hold its initial value before the launch).
+constexpr int kTM = 64, kTN = 64, kTK = 16, kGemmThreads = 256;
+
+template <typename TA, typename TB>
+__global__ void __launch_bounds__(kGemmThreads)
+gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
+            float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split) {
+  __shared__ float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.y * kTM, n0 = blockIdx.x * kTN;
+  const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
+  float acc[4][4] = {};
+  for (int k0 = k_lo; k0 < k_hi; k0 += kTK) {
+    for (int i = tid; i < kTK * kTM; i += kGemmThreads) {
+      int kk, mm;
+      if (ta) { kk = i / kTM; mm = i - kk * kTM; } else { mm = i / kTK; kk = i - mm * kTK; }
+      const int m = m0 + mm, k = k0 + kk;
+      float v = 0.f;
+      if (m < M && k < k_hi) v = to_f32<TA>(ta ? A[(size_t)k * lda + m] : A[(size_t)m * lda + k]);
+      As[kk][mm] = v;
+    }
+    for (int i = tid; i < kTK * kTN; i += kGemmThreads) {
+      int kk, nn;
+      if (tb) { nn = i / kTK; kk = i - nn * kTK; } else { kk = i / kTN; nn = i - kk * kTN; }
+      const int n = n0 + nn, k = k0 + kk;
+      float v = 0.f;
+      if (n < N && k < k_hi) v = to_f32<TB>(tb ? B[(size_t)n * ldb + k] : B[(size_t)k * ldb + n]);
+      Bs[kk][nn] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kTK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + ty * 4 + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= N) continue;
+      float* c = C + (size_t)m * ldc + n;
+      const float v = alpha * acc[i][j];
+      if (gridDim.z > 1) atomicAdd(c, v);
+      else *c = accumulate ? *c + v : v;
+    }
+  }
+}
+
+template <typename TA, typename TB>
+int gemm(cudaStream_t st, int M, int N, int K, const TA* A, int lda, bool ta, const TB* B, int ldb, bool tb, float* C,
+         int ldc, float alpha, bool accumulate, bool split_k) {
+  if (M <= 0 || N <= 0 || K <= 0) return LASER_OK;
+  int splits = 1, per = K;
+  if (split_k) {                     // reductions over many rows into a small matrix (C must hold its initial value)
+    per = 2048;
+    splits = (K + per - 1) / per;
+    if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kTK - 1) / kTK * kTK; splits = (K + per - 1) / per; }
+  }
+  const dim3 grid((N + kTN - 1) / kTN, (M + kTM - 1) / kTM, splits);
+  if (grid.y > 65535) return LASER_ERR_UNSUPPORTED;
+  LaunchScope ls("bwd_gemm", st);
+  gemm_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
+                                                    accumulate ? 1 : 0, per);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+template <typename T>
+__global__ void to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = to_f32<T>(src[i]);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+constexpr int kAttnThreads = 128;
+
+// Non-empty segments of candidate c's user (0 for invalid shapes, which the forward kernels report).
+__device__ __forceinline__ int segments_of(const int* lengths, const int* cand_offsets, int U, int L, int S, int Lp, int c) {
+  int lo = 0, hi = U - 1;
+  while (lo < hi) {                               // the last user whose first candidate is <= c
+    const int mid = (lo + hi + 1) >> 1;
+    if (cand_offsets[mid] <= c) lo = mid; else hi = mid - 1;
+  }
+  const int len = lengths[lo];
+  if (len <= 0 || len > L) return 0;
+  return min((len + S - 1) / S, Lp);
+}
+
+// One block per candidate: e_{j,h} = s_j . Qt_h (Qt holds W_k[:, h] Q_h / tau), a = softmax over the non-empty segments,
+// m_h = sum_j a_{j,h} s_j.  Writes a [N, H, Lp] and m [N, H, d].
+__global__ void __launch_bounds__(kAttnThreads)
+gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const int* __restrict__ lengths,
+                     const int* __restrict__ cand_offsets, float* __restrict__ Aw, float* __restrict__ Mh, int U, int L,
+                     int S, int Lp, int H, int d) {
+  extern __shared__ float sm[];
+  float* qt = sm;                 // [H][d]
+  float* e = qt + H * d;          // [H][Lp]
+  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = kAttnThreads / 32;
+  const int nv = segments_of(lengths, cand_offsets, U, L, S, Lp, c);
+  const float* s = Hp + (size_t)c * Lp * d;
+  for (int i = tid; i < H * d; i += kAttnThreads) qt[i] = Qt[(size_t)c * H * d + i];
+  __syncthreads();
+  for (int p = warp; p < nv * H; p += nw) {
+    const int j = p / H, h = p - j * H;
+    float dot = 0.f;
+    for (int x = lane; x < d; x += 32) dot = fmaf(s[(size_t)j * d + x], qt[h * d + x], dot);
+    dot = warp_sum(dot);
+    if (lane == 0) e[h * Lp + j] = dot;
+  }
+  __syncthreads();
+  for (int h = warp; h < H; h += nw) {
+    float mx = -INFINITY;
+    for (int j = lane; j < nv; j += 32) mx = fmaxf(mx, e[h * Lp + j]);
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int j = lane; j < nv; j += 32) {
+      const float pw = expf(e[h * Lp + j] - mx);
+      e[h * Lp + j] = pw;
+      sum += pw;
+    }
+    sum = warp_sum(sum);
+    const float inv = sum > 0.f ? 1.f / sum : 0.f;
+    for (int j = lane; j < Lp; j += 32) {
+      const float a = j < nv ? e[h * Lp + j] * inv : 0.f;
+      e[h * Lp + j] = a;
+      Aw[((size_t)c * H + h) * Lp + j] = a;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < H * d; i += kAttnThreads) {
+    const int h = i / d, x = i - h * d;
+    float acc = 0.f;
+    for (int j = 0; j < nv; ++j) acc = fmaf(e[h * Lp + j], s[(size_t)j * d + x], acc);
+    Mh[(size_t)c * H * d + i] = acc;
+  }
+}
+
+// One block per candidate: the backward of the kernel above.  dM = dLoss/dm [N, H, d] in; dQt = dLoss/dQt [N, H, d] out;
+// dHp [N, Lp, d] accumulates dLoss/ds_j over the layers.
+__global__ void __launch_bounds__(kAttnThreads)
+gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const float* __restrict__ Aw,
+                     const float* __restrict__ dM, const int* __restrict__ lengths, const int* __restrict__ cand_offsets,
+                     float* __restrict__ dQt, float* __restrict__ dHp, int U, int L, int S, int Lp, int H, int d) {
+  extern __shared__ float sm[];
+  float* qt = sm;                 // [H][d]
+  float* dm = qt + H * d;         // [H][d]
+  float* a = dm + H * d;          // [H][Lp]
+  float* de = a + H * Lp;         // [H][Lp]: first da, then de
+  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = kAttnThreads / 32;
+  const int nv = segments_of(lengths, cand_offsets, U, L, S, Lp, c);
+  const float* s = Hp + (size_t)c * Lp * d;
+  for (int i = tid; i < H * d; i += kAttnThreads) {
+    qt[i] = Qt[(size_t)c * H * d + i];
+    dm[i] = dM[(size_t)c * H * d + i];
+  }
+  for (int i = tid; i < H * Lp; i += kAttnThreads) a[i] = Aw[(size_t)c * H * Lp + i];
+  __syncthreads();
+  for (int p = warp; p < nv * H; p += nw) {
+    const int j = p / H, h = p - j * H;
+    float dot = 0.f;
+    for (int x = lane; x < d; x += 32) dot = fmaf(s[(size_t)j * d + x], dm[h * d + x], dot);
+    dot = warp_sum(dot);
+    if (lane == 0) de[h * Lp + j] = dot;
+  }
+  __syncthreads();
+  for (int h = warp; h < H; h += nw) {
+    float dotp = 0.f;
+    for (int j = lane; j < nv; j += 32) dotp = fmaf(a[h * Lp + j], de[h * Lp + j], dotp);
+    dotp = warp_sum(dotp);
+    for (int j = lane; j < nv; j += 32) de[h * Lp + j] = a[h * Lp + j] * (de[h * Lp + j] - dotp);
+  }
+  __syncthreads();
+  for (int i = tid; i < H * d; i += kAttnThreads) {
+    const int h = i / d, x = i - h * d;
+    float acc = 0.f;
+    for (int j = 0; j < nv; ++j) acc = fmaf(de[h * Lp + j], s[(size_t)j * d + x], acc);
+    dQt[(size_t)c * H * d + i] = acc;
+  }
+  for (int i = tid; i < nv * d; i += kAttnThreads) {
+    const int j = i / d, x = i - j * d;
+    float acc = 0.f;
+    for (int h = 0; h < H; ++h) acc += de[h * Lp + j] * qt[h * d + x] + a[h * Lp + j] * dm[h * d + x];
+    dHp[((size_t)c * Lp + j) * d + x] += acc;
+  }
+}
+
+// One block per (user, 32 consecutive items of one segment), thread (item n, head h); the block walks the user's
+// candidates.  Qf holds q / gamma, so the score is Qf_h . k_n and dQf is the gradient with respect to q / gamma.
+// dK, dV rows of this chunk are written once (no other block touches them); dQf is summed over the chunks atomically.
+constexpr int kChunk = 32;
+__global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __restrict__ Kf, const float* __restrict__ Vf,
+                               const float* __restrict__ dHp, const int* __restrict__ lengths,
+                               const int* __restrict__ cand_offsets, float* __restrict__ dQf, float* __restrict__ dKf,
+                               float* __restrict__ dVf, int L, int d, int dqk, int H, int S, int Lp, int N,
+                               int chunks_per_seg) {
+  extern __shared__ float sm[];
+  const int u = blockIdx.y, seg = blockIdx.x / chunks_per_seg, ck = blockIdx.x - seg * chunks_per_seg;
+  const int len = lengths[u], off0 = cand_offsets[u], off1 = cand_offsets[u + 1];
+  if (len <= 0 || len > L || off0 < 0 || off1 <= off0 || off1 > N) return;
+  const int n0 = seg * S + ck * kChunk, n_end = min(min((seg + 1) * S, L), len);
+  if (n0 >= n_end) return;
+  const int cnt = min(kChunk, n_end - n0);
+  const int dqh = dqk / H, dvh = d / H, kld = dqk + 1, vld = d + 1;
+  float* Ks = sm;                          // [32][dqk + 1]
+  float* Vs = Ks + kChunk * kld;           // [32][d + 1]
+  float* dKs = Vs + kChunk * vld;          // [32][dqk + 1]
+  float* dVs = dKs + kChunk * kld;         // [32][d + 1]
+  float* qs = dVs + kChunk * vld;          // [dqk]
+  float* ds = qs + dqk;                    // [d]
+  const int tid = threadIdx.x, nt = blockDim.x, n = tid & 31, h = tid >> 5;
+  for (int i = tid; i < kChunk * dqk; i += nt) {
+    const int r = i / dqk, a = i - r * dqk;
+    Ks[r * kld + a] = r < cnt ? Kf[((size_t)u * L + n0 + r) * dqk + a] : 0.f;
+    dKs[r * kld + a] = 0.f;
+  }
+  for (int i = tid; i < kChunk * d; i += nt) {
+    const int r = i / d, a = i - r * d;
+    Vs[r * vld + a] = r < cnt ? Vf[((size_t)u * L + n0 + r) * d + a] : 0.f;
+    dVs[r * vld + a] = 0.f;
+  }
+  for (int c = off0; c < off1; ++c) {
+    __syncthreads();
+    for (int i = tid; i < dqk; i += nt) qs[i] = Qf[(size_t)c * dqk + i];
+    for (int i = tid; i < d; i += nt) ds[i] = dHp[((size_t)c * Lp + seg) * d + i];
+    __syncthreads();
+    if (h < H) {
+      float e = 0.f, dg = 0.f;
+      for (int a = 0; a < dqh; ++a) e = fmaf(qs[h * dqh + a], Ks[n * kld + h * dqh + a], e);
+      for (int v = 0; v < dvh; ++v) dg = fmaf(ds[h * dvh + v], Vs[n * vld + h * dvh + v], dg);
+      const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
+      const float de = dg * g * (1.f - g);
+      for (int v = 0; v < dvh; ++v) dVs[n * vld + h * dvh + v] = fmaf(g, ds[h * dvh + v], dVs[n * vld + h * dvh + v]);
+      for (int a = 0; a < dqh; ++a) {
+        dKs[n * kld + h * dqh + a] = fmaf(de, qs[h * dqh + a], dKs[n * kld + h * dqh + a]);
+        const float dq = warp_sum(de * Ks[n * kld + h * dqh + a]);     // over the 32 items of this warp's head
+        if (n == 0) atomicAdd(dQf + (size_t)c * dqk + h * dqh + a, dq);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < cnt * dqk; i += nt) {
+    const int r = i / dqk, a = i - r * dqk;
+    dKf[((size_t)u * L + n0 + r) * dqk + a] = dKs[r * kld + a];
+  }
+  for (int i = tid; i < cnt * d; i += nt) {
+    const int r = i / d, a = i - r * d;
+    dVf[((size_t)u * L + n0 + r) * d + a] = dVs[r * vld + a];
+  }
+}
+
+struct BwdScratch {
+  float *Hp, *dHp, *T, *Q, *Qt, *A, *Mh, *dT, *dM, *dQt, *dQ, *dQf, *dK, *dV;
+  size_t total;
+};
+
+// Carves the backward's own scratch (after the forward plan's regions).
+BwdScratch carve_scratch(const Plan& p, char* base) {
+  BwdScratch s;
+  size_t off = 0;
+  auto take = [&](size_t n_floats) {
+    float* ptr = base ? reinterpret_cast<float*>(base + off) : nullptr;
+    off = align_up(off + n_floats * sizeof(float)) + kGuardBytes;
+    return ptr;
+  };
+  const size_t N = p.N, d = p.d, H = p.H, Lp = p.Lp, M = p.M, UL = (size_t)p.U * p.L;
+  s.Hp = take(N * Lp * d);
+  s.dHp = take(N * Lp * d);
+  s.T = take((M + 1) * N * d);
+  s.Q = take(M * N * d);
+  s.Qt = take(M * N * H * d);
+  s.A = take(M * N * H * Lp);
+  s.Mh = take(M * N * H * d);
+  s.dT = take(N * d);
+  s.dM = take(N * H * d);
+  s.dQt = take(N * H * d);
+  s.dQ = take(N * d);
+  s.dQf = take(N * p.dqk);
+  s.dK = take(UL * p.dqk);
+  s.dV = take(UL * d);
+  s.total = off;
+  return s;
+}
+
+template <typename T>
+int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
+               const T* Wq, const T* Wk, const T* Wv, const T* Wg, const float* dz, float* d_items, float* d_cands,
+               float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st) {
+  const int N = p.N, d = p.d, H = p.H, Lp = p.Lp, M = p.M, dqk = p.dqk, dvh = p.dvh, U = p.U, L = p.L;
+  const size_t UL = (size_t)U * L;
+  LASER_CUDA_OK(cudaMemsetAsync(d_items, 0, UL * d * sizeof(float), st));
+  LASER_CUDA_OK(cudaMemsetAsync(dWq, 0, (size_t)d * dqk * sizeof(float), st));
+  LASER_CUDA_OK(cudaMemsetAsync(dWk, 0, (size_t)d * dqk * sizeof(float), st));
+  LASER_CUDA_OK(cudaMemsetAsync(dWv, 0, (size_t)d * d * sizeof(float), st));
+  if (M > 0) LASER_CUDA_OK(cudaMemsetAsync(dWg, 0, (size_t)M * 3 * d * d * sizeof(float), st));
+  if (N == 0 || U == 0) return LASER_OK;
+  BwdScratch s = carve_scratch(p, ws + p.total);
+  float* Qf = reinterpret_cast<float*>(ws + p.off_q);
+  float* Kf = reinterpret_cast<float*>(ws + p.off_k);
+  float* Vf = reinterpret_cast<float*>(ws + p.off_v);
+  int rc;
+#define BWD_OK(...) do { rc = (__VA_ARGS__); if (rc != LASER_OK) return rc; } while (0)
+
+  // ---- forward, kept in fp32: projections and H' (the FP32-ALU forward kernels), then the GSTA layers
+  BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
+  const size_t Nd = (size_t)N * d, NHd = Nd * H;
+  {
+    LaunchScope ls("bwd_to_f32", st);
+    to_f32_kernel<T><<<296, 256, 0, st>>>(cands, s.T, Nd);
+  }
+  const size_t attn_smem_f = ((size_t)H * d + (size_t)H * Lp) * sizeof(float);
+  const size_t attn_smem_b = (2 * (size_t)H * d + 2 * (size_t)H * Lp) * sizeof(float);
+  if (attn_smem_b > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+  LASER_CUDA_OK(cudaFuncSetAttribute(gsta_attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_f));
+  LASER_CUDA_OK(cudaFuncSetAttribute(gsta_attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_b));
+  for (int l = 0; l < M; ++l) {
+    const T *Wql = Wg + (size_t)(l * 3) * d * d, *Wkl = Wql + (size_t)d * d, *Wvl = Wkl + (size_t)d * d;
+    float *Tl = s.T + l * Nd, *Tn = Tl + Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
+          *Ml = s.Mh + l * NHd;
+    BWD_OK(gemm<float, T>(st, N, d, d, Tl, d, false, Wql, d, false, Ql, d, 1.f, false, false));
+    for (int h = 0; h < H; ++h)
+      BWD_OK(gemm<float, T>(st, N, d, dvh, Ql + h * dvh, d, false, Wkl + h * dvh, d, true, Qtl + (size_t)h * d, H * d,
+                            p.inv_tau, false, false));
+    {
+      LaunchScope ls("bwd_attn_fwd", st);
+      gsta_attn_fwd_kernel<<<N, kAttnThreads, attn_smem_f, st>>>(s.Hp, Qtl, lengths, cand_offsets, Al, Ml, U, L, p.S, Lp,
+                                                                 H, d);
+    }
+    LASER_CUDA_OK(cudaMemcpyAsync(Tn, Tl, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    for (int h = 0; h < H; ++h)
+      BWD_OK(gemm<float, T>(st, N, dvh, d, Ml + (size_t)h * d, H * d, false, Wvl + h * dvh, d, false, Tn + h * dvh, d, 1.f,
+                            true, false));
+  }
+
+  // ---- backward through the GSTA layers
+  LASER_CUDA_OK(cudaMemcpyAsync(s.dT, dz, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
+  LASER_CUDA_OK(cudaMemsetAsync(s.dHp, 0, (size_t)N * Lp * d * sizeof(float), st));
+  for (int l = M - 1; l >= 0; --l) {
+    const T *Wql = Wg + (size_t)(l * 3) * d * d, *Wkl = Wql + (size_t)d * d, *Wvl = Wkl + (size_t)d * d;
+    float *Tl = s.T + l * Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
+          *Ml = s.Mh + l * NHd;
+    float *gWq = dWg + (size_t)(l * 3) * d * d, *gWk = gWq + (size_t)d * d, *gWv = gWk + (size_t)d * d;
+    for (int h = 0; h < H; ++h) {
+      // dW_v[:, h] += m_h^T do_h;  dm_h = do_h W_v[:, h]^T
+      BWD_OK(gemm<float, float>(st, d, dvh, N, Ml + (size_t)h * d, H * d, true, s.dT + h * dvh, d, false, gWv + h * dvh, d,
+                                1.f, true, true));
+      BWD_OK(gemm<float, T>(st, N, d, dvh, s.dT + h * dvh, d, false, Wvl + h * dvh, d, true, s.dM + (size_t)h * d, H * d,
+                            1.f, false, false));
+    }
+    {
+      LaunchScope ls("bwd_attn_bwd", st);
+      gsta_attn_bwd_kernel<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
+                                                                 U, L, p.S, Lp, H, d);
+    }
+    for (int h = 0; h < H; ++h) {
+      // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau
+      BWD_OK(gemm<float, T>(st, N, dvh, d, s.dQt + (size_t)h * d, H * d, false, Wkl + h * dvh, d, false, s.dQ + h * dvh, d,
+                            p.inv_tau, false, false));
+      BWD_OK(gemm<float, float>(st, d, dvh, N, s.dQt + (size_t)h * d, H * d, true, Ql + h * dvh, d, false, gWk + h * dvh, d,
+                                p.inv_tau, true, true));
+    }
+    BWD_OK(gemm<float, float>(st, d, d, N, Tl, d, true, s.dQ, d, false, gWq, d, 1.f, true, true));        // dW_q += T^T dQ
+    BWD_OK(gemm<float, T>(st, N, d, d, s.dQ, d, false, Wql, d, true, s.dT, d, 1.f, true, false));            // dT += dQ W_q^T
+  }
+
+  // ---- backward through the segment aggregation and the gates
+  LASER_CUDA_OK(cudaMemsetAsync(s.dQf, 0, (size_t)N * dqk * sizeof(float), st));
+  LASER_CUDA_OK(cudaMemsetAsync(s.dK, 0, UL * dqk * sizeof(float), st));
+  LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
+  {
+    const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
+    const size_t smem = (2 * (size_t)kChunk * (dqk + 1 + d + 1) + dqk + d) * sizeof(float);
+    if (smem > 200 * 1024 || (long long)Lp * cps > 0x7fffffffLL || U > 65535 || H > 32) return LASER_ERR_UNSUPPORTED;
+    LASER_CUDA_OK(cudaFuncSetAttribute(sta_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    LaunchScope ls("bwd_sta", st);
+    sta_bwd_kernel<<<dim3(Lp * cps, U), 32 * H, smem, st>>>(Qf, Kf, Vf, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, L,
+                                                            d, dqk, H, p.S, Lp, N, cps);
+    LASER_CUDA_OK(cudaGetLastError());
+  }
+
+  // ---- backward through the projections (Qf = T W_q / gamma)
+  BWD_OK(gemm<T, float>(st, d, dqk, N, cands, d, true, s.dQf, dqk, false, dWq, dqk, p.inv_gamma, true, true));
+  BWD_OK(gemm<float, T>(st, N, d, dqk, s.dQf, dqk, false, Wq, dqk, true, s.dT, d, p.inv_gamma, true, false));
+  BWD_OK(gemm<T, float>(st, d, dqk, (int)UL, items, d, true, s.dK, dqk, false, dWk, dqk, 1.f, true, true));
+  BWD_OK(gemm<T, float>(st, d, d, (int)UL, items, d, true, s.dV, d, false, dWv, d, 1.f, true, true));
+  BWD_OK(gemm<float, T>(st, (int)UL, d, dqk, s.dK, dqk, false, Wk, dqk, true, d_items, d, 1.f, false, false));
+  BWD_OK(gemm<float, T>(st, (int)UL, d, d, s.dV, d, false, Wv, d, true, d_items, d, 1.f, true, false));
+  LASER_CUDA_OK(cudaMemcpyAsync(d_cands, s.dT, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
+#undef BWD_OK
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+}  // namespace
+
+size_t backward_scratch_bytes(const Plan& p) { return carve_scratch(p, nullptr).total; }
+
+int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+             const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,
+             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st) {
+  if ((unsigned long long)p.U * p.L > 0x7fffffffULL) return LASER_ERR_UNSUPPORTED;
+  if (p.dtype == LASER_F32)
+    return backward_t<float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
+                             (const float*)Wk, (const float*)Wv, (const float*)Wg, dz, d_items, d_cands, dWq, dWk, dWv,
+                             dWg, ws, st);
+  return backward_t<bf16>(p, (const bf16*)items, lengths, (const bf16*)cands, cand_offsets, (const bf16*)Wq,
+                          (const bf16*)Wk, (const bf16*)Wv, (const bf16*)Wg, dz, d_items, d_cands, dWq, dWk, dWv, dWg, ws,
+                          st);
+}
+
+}  // namespace laser

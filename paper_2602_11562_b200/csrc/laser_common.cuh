@@ -71,6 +71,16 @@ int simt_sta_softmax(const Plan& p, const void* items, const int32_t* lengths, c
                      cudaStream_t st);
 int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
               const void* Wg, void* z, char* ws, cudaStream_t st);
+// STA on the FP32 ALUs with an fp32 H' whatever the I/O dtype; leaves fp32 Q / gamma, K, V at off_q, off_k, off_v.
+int simt_sta_f32(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+                 const void* Wq, const void* Wk, const void* Wv, float* Hprime32, char* ws, cudaStream_t st);
+
+// Backward pass (laser_backward.cu): p is a plan of the FP32-ALU path; the workspace holds p.total bytes of the forward
+// plan followed by backward_scratch_bytes(p).  Gradients are fp32.
+size_t backward_scratch_bytes(const Plan& p);
+int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+             const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,
+             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st);
 
 bool tensor_supported(const Plan& p);
 void tensor_geometry(const Plan& p, TensorGeom* g);

@@ -309,9 +309,10 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
   for (int i = tid; i < d; i += kGstaThreads) z[(size_t)cand * d + i] = from_f32<T>(t[i]);
 }
 
-template <typename T>
+// T: dtype of the inputs; TO: dtype of H' (T itself, or float when the caller keeps fp32 intermediates)
+template <typename T, typename TO>
 int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
-               const T* Wq, const T* Wk, const T* Wv, T* Hp, char* ws, cudaStream_t st, bool softmax) {
+               const T* Wq, const T* Wk, const T* Wv, TO* Hp, char* ws, cudaStream_t st, bool softmax) {
   int* status = reinterpret_cast<int*>(ws + p.off_status);
   float* Qf = reinterpret_cast<float*>(ws + p.off_q);
   float* Kf = reinterpret_cast<float*>(ws + p.off_k);
@@ -338,14 +339,14 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     if (smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
     dim3 grid(p.Lp, (p.maxC + kStaCands - 1) / kStaCands, p.U);
     if (softmax) {
-      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<TO, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       LaunchScope ls("sta_simt_softmax", st);
-      sta_simt_kernel<T, true><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
+      sta_simt_kernel<TO, true><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
                                                                p.H, p.S, p.Lp, p.N, status);
     } else {
-      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<TO, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       LaunchScope ls("sta_simt", st);
-      sta_simt_kernel<T, false><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
+      sta_simt_kernel<TO, false><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
                                                                 p.H, p.S, p.Lp, p.N, status);
     }
   }
@@ -377,11 +378,24 @@ static int simt_sta_any(const Plan& p, const void* items, const int32_t* lengths
                         char* ws, cudaStream_t st, bool softmax) {
   if (p.d > 4 * kStaMaxJ) return LASER_ERR_UNSUPPORTED;
   if (p.dtype == LASER_F32)
-    return simt_sta_t<float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
-                             (const float*)Wk, (const float*)Wv, (float*)Hprime, ws, st, softmax);
+    return simt_sta_t<float, float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
+                                    (const float*)Wk, (const float*)Wv, (float*)Hprime, ws, st, softmax);
   using B = __nv_bfloat16;
-  return simt_sta_t<B>(p, (const B*)items, lengths, (const B*)cands, cand_offsets, (const B*)Wq, (const B*)Wk,
-                       (const B*)Wv, (B*)Hprime, ws, st, softmax);
+  return simt_sta_t<B, B>(p, (const B*)items, lengths, (const B*)cands, cand_offsets, (const B*)Wq, (const B*)Wk,
+                          (const B*)Wv, (B*)Hprime, ws, st, softmax);
+}
+
+// STA with H' kept in fp32 whatever the I/O dtype (the backward pass recomputes the forward this way); the projections
+// stay in the workspace as fp32 Q / gamma, K, V.
+int simt_sta_f32(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
+                 const void* Wq, const void* Wk, const void* Wv, float* Hprime32, char* ws, cudaStream_t st) {
+  if (p.d > 4 * kStaMaxJ) return LASER_ERR_UNSUPPORTED;
+  if (p.dtype == LASER_F32)
+    return simt_sta_t<float, float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
+                                    (const float*)Wk, (const float*)Wv, Hprime32, ws, st, false);
+  using B = __nv_bfloat16;
+  return simt_sta_t<B, float>(p, (const B*)items, lengths, (const B*)cands, cand_offsets, (const B*)Wq, (const B*)Wk,
+                              (const B*)Wv, Hprime32, ws, st, false);
 }
 
 int simt_sta(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
