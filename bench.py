@@ -441,6 +441,63 @@ def softmax_row(P, w, b, flush, stream, steps, peaks, dev):
     return out
 
 
+def backward_row(P, w, b, flush, stream, steps, peaks, dev):
+    """Another row of the scope: the backward pass (laser_backward) of this batch for a seeded upstream gradient,
+    checked on the first two users with candidates against the backward oracle (their rows of d_cands and d_items
+    depend on no other user), then timed on its own.  FP32-ALU kernels: reported against the derived FP32 peak."""
+    import torch
+    from oracle import backward_oracle
+    s = w.spec
+    need = P.laser_backward_workspace_bytes(b.cfg)
+    if need == 0:
+        return None
+    rng = np.random.default_rng(4242)
+    dz = rng.standard_normal((w.N, s.d)).astype(np.float32)
+    dz_d = torch.from_numpy(dz).to(dev)
+    bws = torch.empty(need, dtype=torch.uint8, device=dev)
+    try:
+        g = P.laser_backward(b.cfg, *b.args(), b.Wg, dz_d, workspace=bws, stream=stream)
+    except P.LaserError:
+        return None
+    torch.cuda.synchronize()
+    assert P.laser_check_status(bws) == 0
+    users = [u for u in range(s.U) if w.cand_offsets[u + 1] > w.cand_offsets[u]][:2]
+    ref = backward_oracle.backward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
+                                   dz.astype(np.float64), w.gamma, w.tau, users=users)
+    err, checked = 0.0, 0
+    for u in users:
+        c0, c1 = int(w.cand_offsets[u]), int(w.cand_offsets[u + 1])
+        for got, want in ((g["d_cands"][c0:c1], ref["d_cands"][c0:c1]), (g["d_items"][u], ref["d_items"][u])):
+            want = np.asarray(want)
+            scale = max(float(np.max(np.abs(want))), 1e-30)
+            err = max(err, float(np.max(np.abs(got.cpu().numpy().astype(np.float64) - want))) / scale)
+        checked += c1 - c0
+    tol = 1e-4
+    if not (err <= tol):
+        raise SystemExit(f"backward parity failure before timing: error {err:.3e} of the largest entry > {tol}")
+    del g
+    tot = 0.0
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        P.laser_backward(b.cfg, *b.args(), b.Wg, dz_d, workspace=bws, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1) / steps
+    launches = P.laser_last_launch_count()
+    work = algorithmic_work(w)
+    # forward recomputed once, then about two products per forward product: three times the forward's flops
+    flops = 3.0 * (work["proj_flops"] + 2 * w.N * s.d * s.d_qk + work["attn_flops"] + work["gsta_flops"])
+    peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    ach = flops / (tot * 1e-3) / 1e12
+    return {"call": "laser_backward", "ms": tot, "launches": launches, "value": w.N / (tot * 1e-3), "unit": UNIT,
+            "bound": "alu", "flops": flops, "achieved": ach, "peak": peak, "achieved_unit": "TFLOP/s", "frac": ach / peak,
+            "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+            "parity": {"err_over_max": err, "tol": tol, "users_checked": len(users), "scores_checked": checked},
+            "workspace_bytes": need}
+
+
 def packed_row(P, w, b, z_padded, ws, flush, stream, steps, dev):
     """Another row of the scope: the same forward on items stored without padding (laser_forward_packed); its z must
     equal the padded layout's bit for bit, and it is timed like the main step."""
@@ -604,6 +661,7 @@ def run_ours(args, rank, world, local_rank):
     ffn = None
     packed = None
     softmax = None
+    bwd = None
     if rank == 0:
         r_recent = 2
         Hp_full = torch.empty((b.cfg.total_cands, b.cfg.n_seg, s.d), dtype=b.items.dtype, device=dev)
@@ -630,6 +688,7 @@ def run_ours(args, rank, world, local_rank):
         packed = packed_row(P, w, b, z, ws, flush, stream, args.steps, dev)
         del Hp_full
         softmax = softmax_row(P, w, b, flush, stream, min(args.steps, 10), peaks, dev)
+        bwd = backward_row(P, w, b, flush, stream, min(args.steps, 3), peaks, dev)
 
     # end to end: pinned host buffers in, z out, through laser_forward_host
     hb = P.DeviceBatch.from_workload(w, path=P.PATH_AUTO, device="cpu", pin_host=True)
@@ -699,6 +758,7 @@ def run_ours(args, rank, world, local_rank):
                 "ffn": ffn,
                 "packed_layout": packed,
                 "softmax_sta": softmax,
+                "backward": bwd,
                 "kernel_rooflines": [kernel_roofline(w, k, v, peaks) for k, v in prof.items() if k in MAIN_KERNELS],
                 "cpu_baseline": cpu_base,
                 "parity": parity,

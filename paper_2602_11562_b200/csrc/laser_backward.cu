@@ -91,7 +91,7 @@ int gemm(cudaStream_t st, int M, int N, int K, const TA* A, int lda, bool ta, co
   if (M <= 0 || N <= 0 || K <= 0) return LASER_OK;
   int splits = 1, per = K;
   if (split_k) {                     // reductions over many rows into a small matrix (C must hold its initial value)
-    per = 2048;
+    per = 256;
     splits = (K + per - 1) / per;
     if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kTK - 1) / kTK * kTK; splits = (K + per - 1) / per; }
   }
@@ -234,9 +234,12 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
 }
 
 // One block per (user, 32 consecutive items of one segment), thread (item n, head h); the block walks the user's
-// candidates.  Qf holds q / gamma, so the score is Qf_h . k_n and dQf is the gradient with respect to q / gamma.
-// dK, dV rows of this chunk are written once (no other block touches them); dQf is summed over the chunks atomically.
+// candidates, kCandsPerStep at a time between two block-wide barriers.  Qf holds q / gamma, so the score is Qf_h . k_n
+// and dQf is the gradient with respect to q / gamma.  dK, dV rows of this chunk are written once (no other block touches
+// them); dQf is summed over the chunks atomically: the per-item terms de_n of a step go through shared memory and thread
+// (candidate, head, component) adds up its 32 items while the next step's rows are loaded.
 constexpr int kChunk = 32;
+constexpr int kCandsPerStep = 4;
 __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __restrict__ Kf, const float* __restrict__ Vf,
                                const float* __restrict__ dHp, const int* __restrict__ lengths,
                                const int* __restrict__ cand_offsets, float* __restrict__ dQf, float* __restrict__ dKf,
@@ -254,8 +257,9 @@ __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __rest
   float* Vs = Ks + kChunk * kld;           // [32][d + 1]
   float* dKs = Vs + kChunk * vld;          // [32][dqk + 1]
   float* dVs = dKs + kChunk * kld;         // [32][d + 1]
-  float* qs = dVs + kChunk * vld;          // [dqk]
-  float* ds = qs + dqk;                    // [d]
+  float* qs = dVs + kChunk * vld;          // [kCandsPerStep][dqk]
+  float* ds = qs + kCandsPerStep * dqk;    // [kCandsPerStep][d]
+  float* des = ds + kCandsPerStep * d;     // [kCandsPerStep][H][33]: de of (candidate, head, item)
   const int tid = threadIdx.x, nt = blockDim.x, n = tid & 31, h = tid >> 5;
   for (int i = tid; i < kChunk * dqk; i += nt) {
     const int r = i / dqk, a = i - r * dqk;
@@ -267,26 +271,47 @@ __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __rest
     Vs[r * vld + a] = r < cnt ? Vf[((size_t)u * L + n0 + r) * d + a] : 0.f;
     dVs[r * vld + a] = 0.f;
   }
-  for (int c = off0; c < off1; ++c) {
-    __syncthreads();
-    for (int i = tid; i < dqk; i += nt) qs[i] = Qf[(size_t)c * dqk + i];
-    for (int i = tid; i < d; i += nt) ds[i] = dHp[((size_t)c * Lp + seg) * d + i];
-    __syncthreads();
+  // the query-side sums of the step whose de terms sit in `des`: candidates c_lo .. c_lo + n_c - 1
+  auto reduce_dq = [&](int c_lo, int n_c) {
+    for (int i = tid; i < n_c * dqk; i += nt) {
+      const int cc = i / dqk, col = i - cc * dqk, hh = col / dqh;
+      const float* e = des + (cc * H + hh) * 33;
+      float acc = 0.f;
+#pragma unroll 8
+      for (int r = 0; r < kChunk; ++r) acc = fmaf(e[r], Ks[r * kld + col], acc);
+      atomicAdd(dQf + (size_t)(c_lo + cc) * dqk + col, acc);
+    }
+  };
+  int prev_lo = 0, prev_n = 0;
+  for (int c = off0; c < off1; c += kCandsPerStep) {
+    const int n_c = min(kCandsPerStep, off1 - c);
+    __syncthreads();                       // the previous step's de terms are complete; its q and ds rows are free
+    if (prev_n > 0) reduce_dq(prev_lo, prev_n);
+    for (int i = tid; i < n_c * dqk; i += nt) qs[i] = Qf[(size_t)c * dqk + i];
+    for (int i = tid; i < n_c * d; i += nt) {
+      const int cc = i / d, x = i - cc * d;
+      ds[i] = dHp[((size_t)(c + cc) * Lp + seg) * d + x];
+    }
+    __syncthreads();                       // (also: the previous step's sums have been read out of `des`)
     if (h < H) {
-      float e = 0.f, dg = 0.f;
-      for (int a = 0; a < dqh; ++a) e = fmaf(qs[h * dqh + a], Ks[n * kld + h * dqh + a], e);
-      for (int v = 0; v < dvh; ++v) dg = fmaf(ds[h * dvh + v], Vs[n * vld + h * dvh + v], dg);
-      const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
-      const float de = dg * g * (1.f - g);
-      for (int v = 0; v < dvh; ++v) dVs[n * vld + h * dvh + v] = fmaf(g, ds[h * dvh + v], dVs[n * vld + h * dvh + v]);
-      for (int a = 0; a < dqh; ++a) {
-        dKs[n * kld + h * dqh + a] = fmaf(de, qs[h * dqh + a], dKs[n * kld + h * dqh + a]);
-        const float dq = warp_sum(de * Ks[n * kld + h * dqh + a]);     // over the 32 items of this warp's head
-        if (n == 0) atomicAdd(dQf + (size_t)c * dqk + h * dqh + a, dq);
+      for (int cc = 0; cc < n_c; ++cc) {
+        const float* q = qs + cc * dqk + h * dqh;
+        const float* g_out = ds + cc * d + h * dvh;
+        float e = 0.f, dg = 0.f;
+        for (int a = 0; a < dqh; ++a) e = fmaf(q[a], Ks[n * kld + h * dqh + a], e);
+        for (int v = 0; v < dvh; ++v) dg = fmaf(g_out[v], Vs[n * vld + h * dvh + v], dg);
+        const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
+        const float de = dg * g * (1.f - g);
+        for (int v = 0; v < dvh; ++v) dVs[n * vld + h * dvh + v] = fmaf(g, g_out[v], dVs[n * vld + h * dvh + v]);
+        for (int a = 0; a < dqh; ++a) dKs[n * kld + h * dqh + a] = fmaf(de, q[a], dKs[n * kld + h * dqh + a]);
+        des[(cc * H + h) * 33 + n] = de;
       }
     }
+    prev_lo = c;
+    prev_n = n_c;
   }
   __syncthreads();
+  if (prev_n > 0) reduce_dq(prev_lo, prev_n);
   for (int i = tid; i < cnt * dqk; i += nt) {
     const int r = i / dqk, a = i - r * dqk;
     dKf[((size_t)u * L + n0 + r) * dqk + a] = dKs[r * kld + a];
@@ -417,7 +442,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
   {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
-    const size_t smem = (2 * (size_t)kChunk * (dqk + 1 + d + 1) + dqk + d) * sizeof(float);
+    const size_t smem = (2 * (size_t)kChunk * (dqk + 1 + d + 1) + (size_t)kCandsPerStep * (dqk + d + H * 33)) * sizeof(float);
     if (smem > 200 * 1024 || (long long)Lp * cps > 0x7fffffffLL || U > 65535 || H > 32) return LASER_ERR_UNSUPPORTED;
     LASER_CUDA_OK(cudaFuncSetAttribute(sta_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("bwd_sta", st);
