@@ -240,36 +240,64 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
 // (candidate, head, component) adds up its 32 items while the next step's rows are loaded.
 constexpr int kChunk = 32;
 constexpr int kCandsPerStep = 4;
+// DQH, DVH > 0: the head widths are compile-time constants and thread (item, head) keeps its key / value slices and
+// their gradient accumulators in registers (shared memory then holds only the keys for the query-side sums and the
+// step's candidate rows); 0, 0: any widths, everything in shared memory.
+template <int DQH, int DVH>
 __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __restrict__ Kf, const float* __restrict__ Vf,
                                const float* __restrict__ dHp, const int* __restrict__ lengths,
                                const int* __restrict__ cand_offsets, float* __restrict__ dQf, float* __restrict__ dKf,
                                float* __restrict__ dVf, int L, int d, int dqk, int H, int S, int Lp, int N,
                                int chunks_per_seg) {
-  extern __shared__ float sm[];
+  constexpr bool kRegs = DQH > 0;
+  constexpr int kR = kRegs ? DQH : 1, kV = kRegs ? DVH : 1;
+  extern __shared__ __align__(16) float sm[];
   const int u = blockIdx.y, seg = blockIdx.x / chunks_per_seg, ck = blockIdx.x - seg * chunks_per_seg;
   const int len = lengths[u], off0 = cand_offsets[u], off1 = cand_offsets[u + 1];
   if (len <= 0 || len > L || off0 < 0 || off1 <= off0 || off1 > N) return;
   const int n0 = seg * S + ck * kChunk, n_end = min(min((seg + 1) * S, L), len);
   if (n0 >= n_end) return;
   const int cnt = min(kChunk, n_end - n0);
-  const int dqh = dqk / H, dvh = d / H, kld = dqk + 1, vld = d + 1;
-  float* Ks = sm;                          // [32][dqk + 1]
-  float* Vs = Ks + kChunk * kld;           // [32][d + 1]
-  float* dKs = Vs + kChunk * vld;          // [32][dqk + 1]
-  float* dVs = dKs + kChunk * kld;         // [32][d + 1]
-  float* qs = dVs + kChunk * vld;          // [kCandsPerStep][dqk]
-  float* ds = qs + kCandsPerStep * dqk;    // [kCandsPerStep][d]
-  float* des = ds + kCandsPerStep * d;     // [kCandsPerStep][H][33]: de of (candidate, head, item)
+  const int dqh = kRegs ? DQH : dqk / H, dvh = kRegs ? DVH : d / H, kld = dqk + 1, vld = d + 1;
+  float* Ks = sm;                                                  // [32][dqk + 1]
+  float* Vs = Ks + kChunk * kld;                                   // [32][d + 1]      (shared-memory variant only)
+  float* dKs = Vs + (kRegs ? 0 : kChunk * vld);                    // [32][dqk + 1]    (shared-memory variant only)
+  float* dVs = dKs + (kRegs ? 0 : kChunk * kld);                   // [32][d + 1]      (shared-memory variant only)
+  float* qs = dVs + (kRegs ? 0 : kChunk * vld);                    // [kCandsPerStep][dqk]
+  float* ds = qs + kCandsPerStep * dqk;                            // [kCandsPerStep][d]
+  float* des = ds + kCandsPerStep * d;                             // [kCandsPerStep][H][33]: de of (candidate, head, item)
   const int tid = threadIdx.x, nt = blockDim.x, n = tid & 31, h = tid >> 5;
   for (int i = tid; i < kChunk * dqk; i += nt) {
     const int r = i / dqk, a = i - r * dqk;
     Ks[r * kld + a] = r < cnt ? Kf[((size_t)u * L + n0 + r) * dqk + a] : 0.f;
-    dKs[r * kld + a] = 0.f;
+    if (!kRegs) dKs[r * kld + a] = 0.f;
   }
-  for (int i = tid; i < kChunk * d; i += nt) {
-    const int r = i / d, a = i - r * d;
-    Vs[r * vld + a] = r < cnt ? Vf[((size_t)u * L + n0 + r) * d + a] : 0.f;
-    dVs[r * vld + a] = 0.f;
+  if (!kRegs) {
+    for (int i = tid; i < kChunk * d; i += nt) {
+      const int r = i / d, a = i - r * d;
+      Vs[r * vld + a] = r < cnt ? Vf[((size_t)u * L + n0 + r) * d + a] : 0.f;
+      dVs[r * vld + a] = 0.f;
+    }
+  }
+  float kreg[kR], vreg[kV], dk[kR], dv[kV];
+  if (kRegs) {
+    const bool live = h < H && n < cnt;
+    const float4* kp = reinterpret_cast<const float4*>(Kf + ((size_t)u * L + n0 + n) * dqk + h * dqh);
+    const float4* vp = reinterpret_cast<const float4*>(Vf + ((size_t)u * L + n0 + n) * d + h * dvh);
+#pragma unroll
+    for (int a = 0; a < kR / 4; ++a) {
+      const float4 x = live ? kp[a] : make_float4(0.f, 0.f, 0.f, 0.f);
+      kreg[4 * a] = x.x; kreg[4 * a + 1] = x.y; kreg[4 * a + 2] = x.z; kreg[4 * a + 3] = x.w;
+    }
+#pragma unroll
+    for (int v = 0; v < kV / 4; ++v) {
+      const float4 x = live ? vp[v] : make_float4(0.f, 0.f, 0.f, 0.f);
+      vreg[4 * v] = x.x; vreg[4 * v + 1] = x.y; vreg[4 * v + 2] = x.z; vreg[4 * v + 3] = x.w;
+    }
+#pragma unroll
+    for (int a = 0; a < kR; ++a) dk[a] = 0.f;
+#pragma unroll
+    for (int v = 0; v < kV; ++v) dv[v] = 0.f;
   }
   // the query-side sums of the step whose de terms sit in `des`: candidates c_lo .. c_lo + n_c - 1
   auto reduce_dq = [&](int c_lo, int n_c) {
@@ -298,13 +326,38 @@ __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __rest
         const float* q = qs + cc * dqk + h * dqh;
         const float* g_out = ds + cc * d + h * dvh;
         float e = 0.f, dg = 0.f;
-        for (int a = 0; a < dqh; ++a) e = fmaf(q[a], Ks[n * kld + h * dqh + a], e);
-        for (int v = 0; v < dvh; ++v) dg = fmaf(g_out[v], Vs[n * vld + h * dvh + v], dg);
-        const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
-        const float de = dg * g * (1.f - g);
-        for (int v = 0; v < dvh; ++v) dVs[n * vld + h * dvh + v] = fmaf(g, g_out[v], dVs[n * vld + h * dvh + v]);
-        for (int a = 0; a < dqh; ++a) dKs[n * kld + h * dqh + a] = fmaf(de, q[a], dKs[n * kld + h * dqh + a]);
-        des[(cc * H + h) * 33 + n] = de;
+        if (kRegs) {
+          float qv[kR], gv[kV];
+#pragma unroll
+          for (int a = 0; a < kR / 4; ++a) {
+            const float4 x = reinterpret_cast<const float4*>(q)[a];
+            qv[4 * a] = x.x; qv[4 * a + 1] = x.y; qv[4 * a + 2] = x.z; qv[4 * a + 3] = x.w;
+          }
+#pragma unroll
+          for (int v = 0; v < kV / 4; ++v) {
+            const float4 x = reinterpret_cast<const float4*>(g_out)[v];
+            gv[4 * v] = x.x; gv[4 * v + 1] = x.y; gv[4 * v + 2] = x.z; gv[4 * v + 3] = x.w;
+          }
+#pragma unroll
+          for (int a = 0; a < kR; ++a) e = fmaf(qv[a], kreg[a], e);
+#pragma unroll
+          for (int v = 0; v < kV; ++v) dg = fmaf(gv[v], vreg[v], dg);
+          const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
+          const float de = dg * g * (1.f - g);
+#pragma unroll
+          for (int v = 0; v < kV; ++v) dv[v] = fmaf(g, gv[v], dv[v]);
+#pragma unroll
+          for (int a = 0; a < kR; ++a) dk[a] = fmaf(de, qv[a], dk[a]);
+          des[(cc * H + h) * 33 + n] = de;
+        } else {
+          for (int a = 0; a < dqh; ++a) e = fmaf(q[a], Ks[n * kld + h * dqh + a], e);
+          for (int v = 0; v < dvh; ++v) dg = fmaf(g_out[v], Vs[n * vld + h * dvh + v], dg);
+          const float g = n < cnt ? 1.f / (1.f + expf(-e)) : 0.f;
+          const float de = dg * g * (1.f - g);
+          for (int v = 0; v < dvh; ++v) dVs[n * vld + h * dvh + v] = fmaf(g, g_out[v], dVs[n * vld + h * dvh + v]);
+          for (int a = 0; a < dqh; ++a) dKs[n * kld + h * dqh + a] = fmaf(de, q[a], dKs[n * kld + h * dqh + a]);
+          des[(cc * H + h) * 33 + n] = de;
+        }
       }
     }
     prev_lo = c;
@@ -312,13 +365,24 @@ __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __rest
   }
   __syncthreads();
   if (prev_n > 0) reduce_dq(prev_lo, prev_n);
-  for (int i = tid; i < cnt * dqk; i += nt) {
-    const int r = i / dqk, a = i - r * dqk;
-    dKf[((size_t)u * L + n0 + r) * dqk + a] = dKs[r * kld + a];
-  }
-  for (int i = tid; i < cnt * d; i += nt) {
-    const int r = i / d, a = i - r * d;
-    dVf[((size_t)u * L + n0 + r) * d + a] = dVs[r * vld + a];
+  if (kRegs) {
+    if (h < H && n < cnt) {
+      float4* kp = reinterpret_cast<float4*>(dKf + ((size_t)u * L + n0 + n) * dqk + h * dqh);
+      float4* vp = reinterpret_cast<float4*>(dVf + ((size_t)u * L + n0 + n) * d + h * dvh);
+#pragma unroll
+      for (int a = 0; a < kR / 4; ++a) kp[a] = make_float4(dk[4 * a], dk[4 * a + 1], dk[4 * a + 2], dk[4 * a + 3]);
+#pragma unroll
+      for (int v = 0; v < kV / 4; ++v) vp[v] = make_float4(dv[4 * v], dv[4 * v + 1], dv[4 * v + 2], dv[4 * v + 3]);
+    }
+  } else {
+    for (int i = tid; i < cnt * dqk; i += nt) {
+      const int r = i / dqk, a = i - r * dqk;
+      dKf[((size_t)u * L + n0 + r) * dqk + a] = dKs[r * kld + a];
+    }
+    for (int i = tid; i < cnt * d; i += nt) {
+      const int r = i / d, a = i - r * d;
+      dVf[((size_t)u * L + n0 + r) * d + a] = dVs[r * vld + a];
+    }
   }
 }
 
@@ -442,12 +506,17 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
   {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
-    const size_t smem = (2 * (size_t)kChunk * (dqk + 1 + d + 1) + (size_t)kCandsPerStep * (dqk + d + H * 33)) * sizeof(float);
+    const int dqh = dqk / H;
+    const int variant = (dqh == 16 && dvh == 32) ? 2 : (dqh == 16 && dvh == 16) ? 1 : 0;   // register-resident head slices
+    const size_t step_floats = (size_t)kCandsPerStep * (dqk + d + H * 33);
+    const size_t smem = ((variant ? (size_t)kChunk * (dqk + 1) : 2 * (size_t)kChunk * (dqk + 1 + d + 1)) + step_floats) *
+                        sizeof(float);
     if (smem > 200 * 1024 || (long long)Lp * cps > 0x7fffffffLL || U > 65535 || H > 32) return LASER_ERR_UNSUPPORTED;
-    LASER_CUDA_OK(cudaFuncSetAttribute(sta_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    auto kernel = variant == 2 ? sta_bwd_kernel<16, 32> : variant == 1 ? sta_bwd_kernel<16, 16> : sta_bwd_kernel<0, 0>;
+    LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     LaunchScope ls("bwd_sta", st);
-    sta_bwd_kernel<<<dim3(Lp * cps, U), 32 * H, smem, st>>>(Qf, Kf, Vf, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, L,
-                                                            d, dqk, H, p.S, Lp, N, cps);
+    kernel<<<dim3(Lp * cps, U), 32 * H, smem, st>>>(Qf, Kf, Vf, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, L, d, dqk,
+                                                    H, p.S, Lp, N, cps);
     LASER_CUDA_OK(cudaGetLastError());
   }
 
