@@ -36,7 +36,7 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, cons
             float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split) {
   __shared__ float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int m0 = blockIdx.y * kTM, n0 = blockIdx.x * kTN;
+  const int m0 = blockIdx.x * kTM, n0 = blockIdx.y * kTN;       // (row tiles on grid.x: there may be millions of rows)
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
   float acc[4][4] = {};
   for (int k0 = k_lo; k0 < k_hi; k0 += kTK) {
@@ -95,7 +95,7 @@ int gemm(cudaStream_t st, int M, int N, int K, const TA* A, int lda, bool ta, co
     splits = (K + per - 1) / per;
     if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kTK - 1) / kTK * kTK; splits = (K + per - 1) / per; }
   }
-  const dim3 grid((N + kTN - 1) / kTN, (M + kTM - 1) / kTM, splits);
+  const dim3 grid((M + kTM - 1) / kTM, (N + kTN - 1) / kTN, splits);
   if (grid.y > 65535) return LASER_ERR_UNSUPPORTED;
   LaunchScope ls("bwd_gemm", st);
   gemm_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
