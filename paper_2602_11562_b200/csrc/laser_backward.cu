@@ -386,6 +386,82 @@ __global__ void sta_bwd_kernel(const float* __restrict__ Qf, const float* __rest
   }
 }
 
+// H' in fp32 for the backward's forward recomputation, head widths known at compile time: one block per (segment, 32
+// candidates, user), thread (candidate, head) with its query slice and its accumulators in registers; the segment's
+// items pass through shared memory 32 at a time and every lane reads them as 128-bit broadcasts.  (Other head widths
+// use the forward's own FP32 kernel.)
+template <int DQH, int DVH>
+__global__ void sta_fwd32_kernel(const float* __restrict__ Qf, const float* __restrict__ Kf, const float* __restrict__ Vf,
+                                 const int* __restrict__ lengths, const int* __restrict__ cand_offsets,
+                                 float* __restrict__ Hp, int L, int d, int dqk, int H, int S, int Lp, int N) {
+  extern __shared__ __align__(16) float sm[];
+  float* Ks = sm;                        // [32][dqk]
+  float* Vs = Ks + kChunk * dqk;         // [32][d]
+  const int u = blockIdx.z, seg = blockIdx.x;
+  const int len = lengths[u], off0 = cand_offsets[u], off1 = cand_offsets[u + 1];
+  if (len < 0 || len > L || off0 < 0 || off1 < off0 || off1 > N) return;
+  const int c0 = off0 + blockIdx.y * 32;
+  if (c0 >= off1) return;
+  const int tid = threadIdx.x, nt = blockDim.x, ci = tid & 31, h = tid >> 5, c = c0 + ci;
+  const bool live = c < off1 && h < H;
+  float q[DQH], acc[DVH];
+#pragma unroll
+  for (int a = 0; a < DQH / 4; ++a) {
+    const float4 x = live ? reinterpret_cast<const float4*>(Qf + (size_t)c * dqk + h * DQH)[a] : make_float4(0.f, 0.f, 0.f, 0.f);
+    q[4 * a] = x.x; q[4 * a + 1] = x.y; q[4 * a + 2] = x.z; q[4 * a + 3] = x.w;
+  }
+#pragma unroll
+  for (int v = 0; v < DVH; ++v) acc[v] = 0.f;
+  const int n_begin = seg * S, n_end = min(min(n_begin + S, L), len);
+  for (int nb = n_begin; nb < n_end; nb += kChunk) {
+    const int cnt = min(kChunk, n_end - nb);
+    __syncthreads();
+    for (int i = tid; i < cnt * dqk / 4; i += nt)
+      reinterpret_cast<float4*>(Ks)[i] = reinterpret_cast<const float4*>(Kf + ((size_t)u * L + nb) * dqk)[i];
+    for (int i = tid; i < cnt * d / 4; i += nt)
+      reinterpret_cast<float4*>(Vs)[i] = reinterpret_cast<const float4*>(Vf + ((size_t)u * L + nb) * d)[i];
+    __syncthreads();
+    if (live) {
+      for (int n = 0; n < cnt; ++n) {
+        const float4* kp = reinterpret_cast<const float4*>(Ks + n * dqk + h * DQH);
+        const float4* vp = reinterpret_cast<const float4*>(Vs + n * d + h * DVH);
+        float e = 0.f;
+#pragma unroll
+        for (int a = 0; a < DQH / 4; ++a) {
+          const float4 x = kp[a];
+          e = fmaf(q[4 * a], x.x, e); e = fmaf(q[4 * a + 1], x.y, e); e = fmaf(q[4 * a + 2], x.z, e); e = fmaf(q[4 * a + 3], x.w, e);
+        }
+        const float g = 1.f / (1.f + expf(-e));
+#pragma unroll
+        for (int v = 0; v < DVH / 4; ++v) {
+          const float4 x = vp[v];
+          acc[4 * v] = fmaf(g, x.x, acc[4 * v]); acc[4 * v + 1] = fmaf(g, x.y, acc[4 * v + 1]);
+          acc[4 * v + 2] = fmaf(g, x.z, acc[4 * v + 2]); acc[4 * v + 3] = fmaf(g, x.w, acc[4 * v + 3]);
+        }
+      }
+    }
+  }
+  if (live) {
+    float4* out = reinterpret_cast<float4*>(Hp + ((size_t)c * Lp + seg) * d + h * DVH);
+#pragma unroll
+    for (int v = 0; v < DVH / 4; ++v) out[v] = make_float4(acc[4 * v], acc[4 * v + 1], acc[4 * v + 2], acc[4 * v + 3]);
+  }
+}
+
+template <int DQH, int DVH>
+int launch_sta_fwd32(const Plan& p, const float* Qf, const float* Kf, const float* Vf, const int32_t* lengths,
+                     const int32_t* cand_offsets, float* Hp, cudaStream_t st) {
+  const size_t smem = (size_t)kChunk * (p.dqk + p.d) * sizeof(float);
+  const int ctiles = (p.maxC + 31) / 32;
+  if (p.U > 65535 || ctiles > 65535 || smem > 200 * 1024) return LASER_ERR_UNSUPPORTED;
+  LASER_CUDA_OK(cudaFuncSetAttribute(sta_fwd32_kernel<DQH, DVH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LaunchScope ls("bwd_sta_fwd", st);
+  sta_fwd32_kernel<DQH, DVH><<<dim3(p.Lp, ctiles, p.U), 32 * p.H, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L,
+                                                                               p.d, p.dqk, p.H, p.S, p.Lp, p.N);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
 struct BwdScratch {
   float *Hp, *dHp, *T, *Q, *Qt, *A, *Mh, *dT, *dM, *dQt, *dQ, *dQf, *dK, *dV;
   size_t total;
@@ -439,7 +515,15 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 #define BWD_OK(...) do { rc = (__VA_ARGS__); if (rc != LASER_OK) return rc; } while (0)
 
   // ---- forward, kept in fp32: projections and H' (the FP32-ALU forward kernels), then the GSTA layers
-  BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
+  if (p.dqh == 16 && (dvh == 16 || dvh == 32) && p.H <= 32) {
+    // (a candidate tile of a user with more candidates than max_cands_per_user declares would stay unwritten: zero first)
+    LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
+    BWD_OK(simt_project(p, items, lengths, cands, Wq, Wk, Wv, ws, st));
+    if (dvh == 16) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
+    else BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
+  } else {
+    BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
+  }
   const size_t Nd = (size_t)N * d, NHd = Nd * H;
   {
     LaunchScope ls("bwd_to_f32", st);

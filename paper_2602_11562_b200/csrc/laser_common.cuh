@@ -71,6 +71,9 @@ int simt_sta_softmax(const Plan& p, const void* items, const int32_t* lengths, c
                      cudaStream_t st);
 int simt_gsta(const Plan& p, const void* Hprime, const int32_t* lengths, const int32_t* cand_offsets, const void* cands,
               const void* Wg, void* z, char* ws, cudaStream_t st);
+// Eq. 8-9 on the FP32 ALUs: leaves fp32 Q / gamma, K, V at off_q, off_k, off_v.
+int simt_project(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const void* Wq,
+                 const void* Wk, const void* Wv, char* ws, cudaStream_t st);
 // STA on the FP32 ALUs with an fp32 H' whatever the I/O dtype; leaves fp32 Q / gamma, K, V at off_q, off_k, off_v.
 int simt_sta_f32(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
                  const void* Wq, const void* Wk, const void* Wv, float* Hprime32, char* ws, cudaStream_t st);

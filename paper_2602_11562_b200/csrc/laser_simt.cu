@@ -310,16 +310,16 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
 }
 
 // T: dtype of the inputs; TO: dtype of H' (T itself, or float when the caller keeps fp32 intermediates)
-template <typename T, typename TO>
-int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
-               const T* Wq, const T* Wk, const T* Wv, TO* Hp, char* ws, cudaStream_t st, bool softmax) {
+// Eq. 8-9 in fp32: Q / gamma, K, V into the workspace (off_q, off_k, off_v).
+template <typename T>
+int simt_project_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const T* Wq, const T* Wk,
+                   const T* Wv, char* ws, cudaStream_t st) {
   int* status = reinterpret_cast<int*>(ws + p.off_status);
   float* Qf = reinterpret_cast<float*>(ws + p.off_q);
   float* Kf = reinterpret_cast<float*>(ws + p.off_k);
   float* Vf = reinterpret_cast<float*>(ws + p.off_v);
   if (p.N == 0 || p.U == 0) return LASER_OK;
-  // users and candidate tiles index grid.y / grid.z of the launches below
-  if (p.U > 65535 || (p.maxC + kStaCands - 1) / kStaCands > 65535) return LASER_ERR_UNSUPPORTED;
+  if (p.U > 65535) return LASER_ERR_UNSUPPORTED;           // users index grid.y of the second launch
   const size_t proj_smem = (size_t)kProjRows * p.d * sizeof(float);
   {
     dim3 grid((p.N + kProjRows - 1) / kProjRows, 1);
@@ -333,6 +333,22 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     proj_simt_kernel<T><<<grid, kProjThreads, proj_smem, st>>>(items, p.L, lengths, p.d, Wk, p.dqk, Kf, 1.f, Wv, p.d,
                                                               Vf, p.item_offsets, p.U, status);
   }
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+template <typename T, typename TO>
+int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
+               const T* Wq, const T* Wk, const T* Wv, TO* Hp, char* ws, cudaStream_t st, bool softmax) {
+  int* status = reinterpret_cast<int*>(ws + p.off_status);
+  float* Qf = reinterpret_cast<float*>(ws + p.off_q);
+  float* Kf = reinterpret_cast<float*>(ws + p.off_k);
+  float* Vf = reinterpret_cast<float*>(ws + p.off_v);
+  if (p.N == 0 || p.U == 0) return LASER_OK;
+  // users and candidate tiles index grid.y / grid.z of the launches below
+  if (p.U > 65535 || (p.maxC + kStaCands - 1) / kStaCands > 65535) return LASER_ERR_UNSUPPORTED;
+  const int rc = simt_project_t<T>(p, items, lengths, cands, Wq, Wk, Wv, ws, st);
+  if (rc != LASER_OK) return rc;
   {
     const size_t smem = ((size_t)(kStaCands + kStaItems) * (p.dqk + 1) + (size_t)kStaItems * p.d +
                          (size_t)p.H * kStaCands * (33 + 3)) * sizeof(float);
@@ -383,6 +399,16 @@ static int simt_sta_any(const Plan& p, const void* items, const int32_t* lengths
   using B = __nv_bfloat16;
   return simt_sta_t<B, B>(p, (const B*)items, lengths, (const B*)cands, cand_offsets, (const B*)Wq, (const B*)Wk,
                           (const B*)Wv, (B*)Hprime, ws, st, softmax);
+}
+
+// The projections alone (fp32 Q / gamma, K, V in the workspace), for callers with an attention kernel of their own.
+int simt_project(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const void* Wq,
+                 const void* Wk, const void* Wv, char* ws, cudaStream_t st) {
+  if (p.dtype == LASER_F32)
+    return simt_project_t<float>(p, (const float*)items, lengths, (const float*)cands, (const float*)Wq, (const float*)Wk,
+                                 (const float*)Wv, ws, st);
+  using B = __nv_bfloat16;
+  return simt_project_t<B>(p, (const B*)items, lengths, (const B*)cands, (const B*)Wq, (const B*)Wk, (const B*)Wv, ws, st);
 }
 
 // STA with H' kept in fp32 whatever the I/O dtype (the backward pass recomputes the forward this way); the projections
