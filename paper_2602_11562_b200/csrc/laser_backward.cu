@@ -34,7 +34,7 @@ template <typename TA, typename TB>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
             float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split) {
-  __shared__ float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
+  __shared__ __align__(16) float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int m0 = blockIdx.x * kTM, n0 = blockIdx.y * kTN;       // (row tiles on grid.x: there may be millions of rows)
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
@@ -59,9 +59,9 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, cons
     __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < kTK; ++kk) {
-      float a[4], b[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; b[i] = Bs[kk][tx * 4 + i]; }
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
