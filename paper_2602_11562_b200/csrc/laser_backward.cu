@@ -176,11 +176,19 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
     }
   }
   __syncthreads();
-  for (int i = tid; i < H * d; i += kAttnThreads) {
-    const int h = i / d, x = i - h * d;
-    float acc = 0.f;
-    for (int j = 0; j < nv; ++j) acc = fmaf(e[h * Lp + j], s[(size_t)j * d + x], acc);
-    Mh[(size_t)c * H * d + i] = acc;
+  for (int x = tid; x < d; x += kAttnThreads) {            // feature x of every head: the segment vectors are read once
+    for (int h0 = 0; h0 < H; h0 += 4) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int j = 0; j < nv; ++j) {
+        const float sv = s[(size_t)j * d + x];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (h0 + k < H) acc[k] = fmaf(e[(h0 + k) * Lp + j], sv, acc[k]);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (h0 + k < H) Mh[((size_t)c * H + h0 + k) * d + x] = acc[k];
+    }
   }
 }
 
@@ -219,17 +227,31 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
     for (int j = lane; j < nv; j += 32) de[h * Lp + j] = a[h * Lp + j] * (de[h * Lp + j] - dotp);
   }
   __syncthreads();
-  for (int i = tid; i < H * d; i += kAttnThreads) {
-    const int h = i / d, x = i - h * d;
-    float acc = 0.f;
-    for (int j = 0; j < nv; ++j) acc = fmaf(de[h * Lp + j], s[(size_t)j * d + x], acc);
-    dQt[(size_t)c * H * d + i] = acc;
-  }
-  for (int i = tid; i < nv * d; i += kAttnThreads) {
-    const int j = i / d, x = i - j * d;
-    float acc = 0.f;
-    for (int h = 0; h < H; ++h) acc += de[h * Lp + j] * qt[h * d + x] + a[h * Lp + j] * dm[h * d + x];
-    dHp[((size_t)c * Lp + j) * d + x] += acc;
+  for (int x = tid; x < d; x += kAttnThreads) {            // feature x: one pass over the segment vectors for both sums
+    for (int h0 = 0; h0 < H; h0 += 4) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f}, qx[4], mx[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        qx[k] = h0 + k < H ? qt[(h0 + k) * d + x] : 0.f;
+        mx[k] = h0 + k < H ? dm[(h0 + k) * d + x] : 0.f;
+      }
+      for (int j = 0; j < nv; ++j) {
+        const float sv = s[(size_t)j * d + x];
+        float g = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (h0 + k < H) {
+            const float dej = de[(h0 + k) * Lp + j];
+            acc[k] = fmaf(dej, sv, acc[k]);
+            g += dej * qx[k] + a[(h0 + k) * Lp + j] * mx[k];
+          }
+        }
+        dHp[((size_t)c * Lp + j) * d + x] += g;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (h0 + k < H) dQt[((size_t)c * H + h0 + k) * d + x] = acc[k];
+    }
   }
 }
 
