@@ -60,8 +60,12 @@ __global__ void __launch_bounds__(256) gsta_prep_kernel(GstaParams P) {
                   (blockIdx.x * blockDim.x + threadIdx.x) >> 5, (n_blocks * blockDim.x) >> 5, threadIdx.x & 31);
 }
 
-template <int D16>
-__global__ void __launch_bounds__(kGThreads, 2) gsta_mma_kernel(GstaParams P) {
+// BPS = blocks per SM the registers are budgeted for: two (127 registers), or three at d <= 64 (80 registers, ~57 KB of
+// shared memory per block) for grids of several waves, where the kernel is latency-bound and a third block's warps fill
+// issue slots (cfg4 49.5 -> 47.6 us); a grid of one wave keeps the two-block budget, whose code has the shorter
+// dependency chains.
+template <int D16, int BPS>
+__global__ void __launch_bounds__(kGThreads, BPS) gsta_mma_kernel(GstaParams P) {
   constexpr int d = D16 * 16;
   constexpr int RS = 2 * d + 16;            // bytes per staged bf16 row (16 bytes of padding: conflict-free ldmatrix)
   constexpr int TS = d + 8;                 // floats per row of the running target
@@ -364,9 +368,13 @@ int launch_gsta(const GstaParams& P, cudaStream_t st) {
   constexpr int d = D16 * 16, RS = 2 * d + 16, TS = d + 8;
   const size_t smem = (size_t)kGT * TS * 4 + (size_t)kGT * RS + (size_t)kGT * P.H * RS + RS + kGT * sizeof(int) +
                       (size_t)kGW * 2 * kChunk * RS;
-  LASER_CUDA_OK(cudaFuncSetAttribute(gsta_mma_kernel<D16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int blocks = (P.N + P.cpb - 1) / P.cpb;
+  auto kernel = (D16 <= 4 && blocks > 2 * sms) ? gsta_mma_kernel<D16, (D16 <= 4 ? 3 : 2)> : gsta_mma_kernel<D16, 2>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   LaunchScope ls("gsta_mma", st);
-  LASER_CUDA_OK(launch_chained(gsta_mma_kernel<D16>, dim3((P.N + P.cpb - 1) / P.cpb), dim3(kGThreads), smem, st, P));
+  LASER_CUDA_OK(launch_chained(kernel, dim3(blocks), dim3(kGThreads), smem, st, P));
   return LASER_OK;
 }
 
@@ -386,14 +394,14 @@ size_t gsta_mma_image_bytes(const Plan& p) {       // the order table and its so
 }
 
 // Small batches: 8 candidates per block (every warp then has one candidate instead of two, which halves the
-// per-candidate part of a block's latency) as long as all blocks still run at once, two per SM.
+// per-candidate part of a block's latency) as long as all blocks still run at once.
 int gsta_candidates_per_block(const Plan& p) {
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   return (p.N + 7) / 8 <= 2 * sms ? 8 : kGT;
 }
 
-// Sorting the blocks pays only when the grid runs in more than one wave (two blocks per SM).
+// Sorting the blocks pays only when the grid runs in more than one wave.
 bool gsta_wants_order(const Plan& p) {
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
