@@ -23,6 +23,8 @@ proj_simt_kernel(const T* __restrict__ X, int rows_per_group, const int* __restr
                  const T* __restrict__ W1, int n1, float* __restrict__ Y1, const int* __restrict__ row_off, int n_groups,
                  int* __restrict__ status) {
   extern __shared__ float xs[];   // [kProjRows][d]
+  chain_wait();                   // (the kernels of this path are chained like the others: launch latencies overlap)
+  chain_release();
   const int g = blockIdx.y;
   const int r0 = blockIdx.x * kProjRows;
   int nrows = rows_per_group;
@@ -53,6 +55,7 @@ proj_simt_kernel(const T* __restrict__ X, int rows_per_group, const int* __restr
     float acc[kProjRows];
 #pragma unroll
     for (int r = 0; r < kProjRows; ++r) acc[r] = 0.f;
+#pragma unroll 8                    // (eight weight loads in flight: the loop is latency-bound at small d)
     for (int k = 0; k < d; ++k) {
       const float w = to_f32<T>(W[(size_t)k * n + cc]);
 #pragma unroll
@@ -88,6 +91,8 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
                 const int* __restrict__ lengths, const int* __restrict__ cand_offsets, T* __restrict__ Hp,
                 int L, int d, int dqk, int H, int S, int Lp, int N, int* __restrict__ status) {
   extern __shared__ float sm[];
+  chain_wait();
+  chain_release();
   const int u = blockIdx.z, seg = blockIdx.x;
   const int off0 = cand_offsets[u], off1 = cand_offsets[u + 1];
   const int len = lengths[u];
@@ -177,10 +182,31 @@ sta_simt_kernel(const float* __restrict__ Q, const float* __restrict__ K, const 
       for (int j = 0; j < kStaMaxJ; ++j)
         if (j < nj) acc[j] *= st_s[goff[j] / 33];
     }
-    for (int n = 0; n < cnt; ++n) {
+    // (the column loop is unrolled over the accumulator registers; its bound follows the width in use, so that a narrow
+    // d does not pay for 64 predicated steps per item)
+    if (nj <= 8) {
+      for (int n = 0; n < cnt; ++n) {
 #pragma unroll
-      for (int j = 0; j < kStaMaxJ; ++j) {
-        if (j < nj) acc[j] = fmaf(G[goff[j] + n], Vs[n * d + cg + 4 * j], acc[j]);
+        for (int j = 0; j < 8; ++j)
+          if (j < nj) acc[j] = fmaf(G[goff[j] + n], Vs[n * d + cg + 4 * j], acc[j]);
+      }
+    } else if (nj <= 16) {
+      for (int n = 0; n < cnt; ++n) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j < nj) acc[j] = fmaf(G[goff[j] + n], Vs[n * d + cg + 4 * j], acc[j]);
+      }
+    } else if (nj <= 32) {
+      for (int n = 0; n < cnt; ++n) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (j < nj) acc[j] = fmaf(G[goff[j] + n], Vs[n * d + cg + 4 * j], acc[j]);
+      }
+    } else {
+      for (int n = 0; n < cnt; ++n) {
+#pragma unroll
+        for (int j = 0; j < kStaMaxJ; ++j)
+          if (j < nj) acc[j] = fmaf(G[goff[j] + n], Vs[n * d + cg + 4 * j], acc[j]);
       }
     }
   }
@@ -210,6 +236,8 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
                  const T* __restrict__ cands, const T* __restrict__ Wg, T* __restrict__ z, int U, int L, int d, int H,
                  int S, int Lp, int M, int N, float inv_tau, int* __restrict__ status) {
   extern __shared__ float sm[];
+  chain_wait();
+  chain_release();
   const int cand = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int nwarps = kGstaThreads / 32;
@@ -248,6 +276,7 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
     const T* Wv = Wg + (size_t)(l * 3 + 2) * d * d;
     for (int j = tid; j < d; j += kGstaThreads) {
       float a = 0.f;
+#pragma unroll 8
       for (int i = 0; i < d; ++i) a = fmaf(t[i], to_f32<T>(Wq[(size_t)i * d + j]), a);
       q[j] = a;
     }
@@ -299,6 +328,7 @@ gsta_simt_kernel(const T* __restrict__ Hp, const int* __restrict__ lengths, cons
     for (int col = tid; col < d; col += kGstaThreads) {
       const int h = col / dh;
       float a = 0.f;
+#pragma unroll 8
       for (int i = 0; i < d; ++i) a = fmaf(mh[h * d + i], to_f32<T>(Wv[(size_t)i * d + col]), a);
       q[col] = a;   // o_l
     }
@@ -324,14 +354,16 @@ int simt_project_t(const Plan& p, const T* items, const int32_t* lengths, const 
   {
     dim3 grid((p.N + kProjRows - 1) / kProjRows, 1);
     LaunchScope ls("proj_simt_q", st);
-    proj_simt_kernel<T><<<grid, kProjThreads, proj_smem, st>>>(cands, p.N, nullptr, p.d, Wq, p.dqk, Qf, p.inv_gamma,
-                                                              nullptr, 0, nullptr, nullptr, 0, status);
+    LASER_CUDA_OK(launch_chained(proj_simt_kernel<T>, grid, dim3(kProjThreads), proj_smem, st, cands, p.N,
+                                 (const int*)nullptr, p.d, Wq, p.dqk, Qf, p.inv_gamma, (const T*)nullptr, 0,
+                                 (float*)nullptr, (const int*)nullptr, 0, status));
   }
   {
     dim3 grid((p.L + kProjRows - 1) / kProjRows, p.U);
     LaunchScope ls("proj_simt_kv", st);
-    proj_simt_kernel<T><<<grid, kProjThreads, proj_smem, st>>>(items, p.L, lengths, p.d, Wk, p.dqk, Kf, 1.f, Wv, p.d,
-                                                              Vf, p.item_offsets, p.U, status);
+    LASER_CUDA_OK(launch_chained(proj_simt_kernel<T>, grid, dim3(kProjThreads), proj_smem, st, items, p.L,
+                                 (const int*)lengths, p.d, Wk, p.dqk, Kf, 1.f, Wv, p.d, Vf, (const int*)p.item_offsets,
+                                 p.U, status));
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
@@ -357,13 +389,15 @@ int simt_sta_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     if (softmax) {
       LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<TO, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       LaunchScope ls("sta_simt_softmax", st);
-      sta_simt_kernel<TO, true><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
-                                                               p.H, p.S, p.Lp, p.N, status);
+      LASER_CUDA_OK(launch_chained(sta_simt_kernel<TO, true>, grid, dim3(kStaThreads), smem, st, (const float*)Qf,
+                                   (const float*)Kf, (const float*)Vf, (const int*)lengths, (const int*)cand_offsets, Hp,
+                                   p.L, p.d, p.dqk, p.H, p.S, p.Lp, p.N, status));
     } else {
       LASER_CUDA_OK(cudaFuncSetAttribute(sta_simt_kernel<TO, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       LaunchScope ls("sta_simt", st);
-      sta_simt_kernel<TO, false><<<grid, kStaThreads, smem, st>>>(Qf, Kf, Vf, lengths, cand_offsets, Hp, p.L, p.d, p.dqk,
-                                                                p.H, p.S, p.Lp, p.N, status);
+      LASER_CUDA_OK(launch_chained(sta_simt_kernel<TO, false>, grid, dim3(kStaThreads), smem, st, (const float*)Qf,
+                                   (const float*)Kf, (const float*)Vf, (const int*)lengths, (const int*)cand_offsets, Hp,
+                                   p.L, p.d, p.dqk, p.H, p.S, p.Lp, p.N, status));
     }
   }
   LASER_CUDA_OK(cudaGetLastError());
@@ -380,8 +414,9 @@ int simt_gsta_t(const Plan& p, const T* Hp, const int32_t* lengths, const int32_
   LASER_CUDA_OK(cudaFuncSetAttribute(gsta_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   {
     LaunchScope ls("gsta_simt", st);
-    gsta_simt_kernel<T><<<p.N, kGstaThreads, smem, st>>>(Hp, lengths, cand_offsets, cands, Wg, z, p.U, p.L, p.d, p.H,
-                                                        p.S, p.Lp, p.M, p.N, p.inv_tau, status);
+    LASER_CUDA_OK(launch_chained(gsta_simt_kernel<T>, dim3(p.N), dim3(kGstaThreads), smem, st, Hp, (const int*)lengths,
+                                 (const int*)cand_offsets, cands, Wg, z, p.U, p.L, p.d, p.H, p.S, p.Lp, p.M, p.N,
+                                 p.inv_tau, status));
   }
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
