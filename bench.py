@@ -455,12 +455,19 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
     dz = rng.standard_normal((w.N, s.d)).astype(np.float32)
     dz_d = torch.from_numpy(dz).to(dev)
     bws = torch.empty(need, dtype=torch.uint8, device=dev)
+    P.laser_profile_enable(True)
     try:
         g = P.laser_backward(b.cfg, *b.args(), b.Wg, dz_d, workspace=bws, stream=stream)
+        torch.cuda.synchronize()
+        kernels = {}
+        for name, ms in P.laser_profile_read():
+            kernels[name] = kernels.get(name, 0.0) + ms
     except P.LaserError:
         return None
-    torch.cuda.synchronize()
+    finally:
+        P.laser_profile_enable(False)
     assert P.laser_check_status(bws) == 0
+    tensor = "bwd_sta_mma" in kernels
     users = [u for u in range(s.U) if w.cand_offsets[u + 1] > w.cand_offsets[u]][:2]
     ref = backward_oracle.backward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
                                    dz.astype(np.float64), w.gamma, w.tau, users=users)
@@ -472,7 +479,7 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
             scale = max(float(np.max(np.abs(want))), 1e-30)
             err = max(err, float(np.max(np.abs(got.cpu().numpy().astype(np.float64) - want))) / scale)
         checked += c1 - c0
-    tol = 1e-4
+    tol = 2e-2 if tensor else 1e-4        # bf16 operands on the tensor cores / fp32 throughout (tests/test_gpu_backward.py)
     if not (err <= tol):
         raise SystemExit(f"backward parity failure before timing: error {err:.3e} of the largest entry > {tol}")
     del g
@@ -495,6 +502,8 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
             "bound": "alu", "flops": flops, "achieved": ach, "peak": peak, "achieved_unit": "TFLOP/s", "frac": ach / peak,
             "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
             "parity": {"err_over_max": err, "tol": tol, "users_checked": len(users), "scores_checked": checked},
+            "gate_contractions": "tensor cores (mma.sync, bf16 operands)" if tensor else "FP32 ALUs",
+            "kernel_ms_first_call": {k: round(v, 4) for k, v in sorted(kernels.items())},
             "workspace_bytes": need}
 
 

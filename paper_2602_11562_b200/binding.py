@@ -181,7 +181,7 @@ def laser_profile_enable(on: bool) -> None:
     load_library().laser_profile_enable(1 if on else 0)
 
 
-def laser_profile_read(max_kernels: int = 16):
+def laser_profile_read(max_kernels: int = 256):
     """[(kernel name, milliseconds)] of the last profiled call on this thread, in launch order."""
     ms = (ctypes.c_float * max_kernels)()
     names = (ctypes.c_char_p * max_kernels)()

@@ -16,7 +16,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblaser.so")
-SOURCES = ["laser_api.cu", "laser_simt.cu", "laser_tensor.cu", "laser_gsta.cu", "laser_fusion.cu", "laser_ffn.cu", "laser_stream.cu", "laser_backward.cu", "laser_noalloc.cu"]
+SOURCES = ["laser_api.cu", "laser_simt.cu", "laser_tensor.cu", "laser_gsta.cu", "laser_fusion.cu", "laser_ffn.cu", "laser_stream.cu", "laser_backward.cu", "laser_backward_mma.cu", "laser_noalloc.cu"]
 
 
 def _nvcc() -> str:

@@ -8,7 +8,7 @@
 
 namespace laser {
 
-constexpr int kMaxProfiled = 16;
+constexpr int kMaxProfiled = 256;          // (a backward call launches about a hundred kernels)
 static thread_local int g_launches = 0;
 static thread_local bool g_profile = false;
 static thread_local int g_prof_n = 0;
@@ -307,17 +307,24 @@ int laser_sta_softmax_forward(const laser_config* cfg, const void* items, const 
   return simt_sta_softmax(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Hprime, ws, st);
 }
 
-// The backward pass runs on the FP32 ALUs whatever cfg->path says, on the padded item layout.
-static int backward_plan(const laser_config* cfg, Plan* p) {
+// The backward pass works on the fp32 intermediates and the workspace layout of the FP32-ALU path, on the padded item
+// layout; *tensor says whether its contractions run on the tensor cores (bf16 batches of supported head widths, unless
+// cfg->path asks for the FP32 ALUs; LASER_PATH_TENSOR on anything else is LASER_ERR_UNSUPPORTED).
+static int backward_plan(const laser_config* cfg, Plan* p, bool* tensor) {
   if (!cfg) return LASER_ERR_INVALID_ARG;
   laser_config c = *cfg;
   c.path = LASER_PATH_SIMT;
-  return make_plan(&c, p);
+  const int rc = make_plan(&c, p);
+  if (rc != LASER_OK) return rc;
+  *tensor = cfg->path != LASER_PATH_SIMT && backward_tensor_supported(*p);
+  if (cfg->path == LASER_PATH_TENSOR && !*tensor) return LASER_ERR_UNSUPPORTED;
+  return LASER_OK;
 }
 
 size_t laser_backward_workspace_bytes(const laser_config* cfg) {
   Plan p;
-  if (backward_plan(cfg, &p) != LASER_OK) return 0;
+  bool tensor;
+  if (backward_plan(cfg, &p, &tensor) != LASER_OK) return 0;
   return p.total + backward_scratch_bytes(p);
 }
 
@@ -327,7 +334,8 @@ int laser_backward(const laser_config* cfg, const void* items, const int32_t* le
                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
   reset_launch_count();
   Plan p;
-  int rc = backward_plan(cfg, &p);
+  bool tensor;
+  int rc = backward_plan(cfg, &p, &tensor);
   if (rc != LASER_OK) return rc;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1))) return LASER_ERR_INVALID_ARG;
   if (workspace_bytes < p.total + backward_scratch_bytes(p)) return LASER_ERR_WORKSPACE;
@@ -340,7 +348,7 @@ int laser_backward(const laser_config* cfg, const void* items, const int32_t* le
   char* ws = static_cast<char*>(workspace);
   if ((rc = clear_status(p, ws, st)) != LASER_OK) return rc;
   return backward(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, Wgsta, dz, d_items, d_cands, dWq, dWk, dWv, dWgsta,
-                  ws, st);
+                  ws, st, tensor);
 }
 
 size_t laser_ffn_workspace_bytes(const laser_config* cfg, int32_t d_hidden) {

@@ -520,7 +520,7 @@ BwdScratch carve_scratch(const Plan& p, char* base) {
 template <typename T>
 int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* cands, const int32_t* cand_offsets,
                const T* Wq, const T* Wk, const T* Wv, const T* Wg, const float* dz, float* d_items, float* d_cands,
-               float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st) {
+               float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor) {
   const int N = p.N, d = p.d, H = p.H, Lp = p.Lp, M = p.M, dqk = p.dqk, dvh = p.dvh, U = p.U, L = p.L;
   const size_t UL = (size_t)U * L;
   LASER_CUDA_OK(cudaMemsetAsync(d_items, 0, UL * d * sizeof(float), st));
@@ -610,7 +610,9 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dQf, 0, (size_t)N * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dK, 0, UL * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
-  {
+  if (tensor) {
+    BWD_OK(sta_bwd_mma(p, Qf, Kf, Vf, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, ws + p.total + s.total, st));
+  } else {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
     const int dqh = dqk / H;
     const int variant = (dqh == 16 && dvh == 32) ? 2 : (dqh == 16 && dvh == 16) ? 1 : 0;   // register-resident head slices
@@ -641,19 +643,22 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 
 }  // namespace
 
-size_t backward_scratch_bytes(const Plan& p) { return carve_scratch(p, nullptr).total; }
+size_t backward_scratch_bytes(const Plan& p) { return carve_scratch(p, nullptr).total + sta_bwd_mma_scratch_bytes(p); }
+
+bool backward_tensor_supported(const Plan& p) { return p.dtype == LASER_BF16 && sta_bwd_mma_supported(p); }
 
 int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
              const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,
-             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st) {
+             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor) {
   if ((unsigned long long)p.U * p.L > 0x7fffffffULL) return LASER_ERR_UNSUPPORTED;
+  if (tensor && !backward_tensor_supported(p)) return LASER_ERR_UNSUPPORTED;
   if (p.dtype == LASER_F32)
     return backward_t<float>(p, (const float*)items, lengths, (const float*)cands, cand_offsets, (const float*)Wq,
                              (const float*)Wk, (const float*)Wv, (const float*)Wg, dz, d_items, d_cands, dWq, dWk, dWv,
-                             dWg, ws, st);
+                             dWg, ws, st, false);
   return backward_t<bf16>(p, (const bf16*)items, lengths, (const bf16*)cands, cand_offsets, (const bf16*)Wq,
                           (const bf16*)Wk, (const bf16*)Wv, (const bf16*)Wg, dz, d_items, d_cands, dWq, dWk, dWv, dWg, ws,
-                          st);
+                          st, tensor);
 }
 
 }  // namespace laser

@@ -1,0 +1,384 @@
+// Tensor-core version of the backward pass through the segment aggregation and the sigmoid gates (Eq. 10-12), for bf16
+// batches: the five contractions per (user, head, item tile, candidate tile) run as warp-level mma.sync m16n8k16 with bf16
+// operands and fp32 accumulation.  Operands are bf16 copies of the fp32 intermediates of the recomputed forward (Q / gamma,
+// K, V) and of the upstream gradient dH'; results (dK, dV, the query-side sums dQf) are fp32.
+//
+// With x = q_h . k_n / gamma, g = Sigmoid(x) = (1 + tanh(x / 2)) / 2 and g (1 - g) = (1 - tanh^2(x / 2)) / 4.  The bf16
+// query copy holds Q / (2 gamma), so the score product gives x / 2 directly, and with th = tanh(x / 2), w = 1 - th^2:
+//   dG^T[n, c]  = v_n . ds_i[c, h]                           (i = the segment of item n)
+//   dV[n]      += sum_c g[n, c] ds_i[c, h]
+//   dK[n]       = 1/2 sum_c (dG w)[n, c] Qb[c]               (Qb = Q / (2 gamma), de = dG w / 4, dK = sum de Q / gamma)
+//   dQf[c]     += 1/4 sum_n (dG w)[n, c] k_n
+//
+// One warp = one job (segment i, item tile of 16 MT rows inside it, head h) of one user; it keeps the job's K_h / V_h tiles
+// as A fragments and the dK / dV accumulators in registers and walks the user's candidates 16 at a time.  Everything is
+// formed transposed (items on the MMA rows), so that the gates and the score gradients leave their MMA in the register
+// layout the next one wants as its A operand; only the query-side product contracts over the items and takes its B operand
+// through movmatrix.  The candidate rows of Qb and ds_i (bf16) are staged per warp in shared memory (cp.async, two
+// buffers) and read with ldmatrix, plain for the products that contract over the head width, transposed for those that
+// contract over the candidates.  Rows of the tile past the segment's end or the user's length are zero rows of K and V:
+// they contribute nothing and are not written.  Candidate rows past the user's last are zero-filled: their score
+// gradients vanish with ds.  dK and dV rows are written once, by their job; dQf is summed over the jobs with atomics
+// (eight lanes per 32-byte sector).
+#include "laser_common.cuh"
+#include "laser_mma.cuh"
+
+namespace laser {
+namespace {
+
+using bf16 = __nv_bfloat16;
+using namespace mma;
+
+constexpr int kBwdWarps = 8;
+
+// dst = bf16(scale * src), four elements per thread and step (n4 = number of groups of four; n is a multiple of 4:
+// every array converted here has a row width that is a multiple of 16).
+__global__ void __launch_bounds__(256) cast_bf16_kernel(const float4* __restrict__ src, uint2* __restrict__ dst, size_t n4,
+                                                        float scale) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 v = src[i];
+    dst[i] = make_uint2(pack2(v.x * scale, v.y * scale), pack2(v.z * scale, v.w * scale));
+  }
+}
+
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct BwdMmaParams {
+  const bf16 *Qb, *Kb, *Vb, *dSb;
+  const int32_t *lengths, *cand_offsets;
+  float *dQf, *dK, *dV;
+  int L, d, dqk, H, S, Lp, N, R, jobs;           // R item tiles per segment, jobs = Lp R H per user
+};
+
+template <int MT, int DQ16, int DV16>
+__global__ void __launch_bounds__(kBwdWarps * 32) sta_bwd_mma_kernel(const BwdMmaParams P) {
+  constexpr int DQH = 16 * DQ16, DVH = 16 * DV16;
+  constexpr int QS = 2 * DQH + 16, DS = 2 * DVH + 16;          // bytes per staged row (padding: conflict-free ldmatrix)
+  constexpr int kBuf = 16 * (QS + DS);                         // one staging buffer: 16 candidate rows of Qb_h and ds_i,h
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int u = blockIdx.y, job = blockIdx.x * kBwdWarps + warp;
+  if (job >= P.jobs) return;
+  const int h = job % P.H, r = (job / P.H) % P.R, seg = job / (P.H * P.R);
+  const int len = P.lengths[u], off0 = P.cand_offsets[u], off1 = P.cand_offsets[u + 1];
+  if (len <= 0 || len > P.L || off0 < 0 || off1 <= off0 || off1 > P.N) return;
+  const int C = off1 - off0;
+  const int n0 = seg * P.S + r * 16 * MT, n_end = min(min((seg + 1) * P.S, P.L), len);
+  if (n0 >= n_end) return;
+  const int cnt = min(16 * MT, n_end - n0);
+  const int d = P.d, dqk = P.dqk;
+
+  // ---- the job's K_h and V_h tiles as A fragments (rows = items), zero rows past cnt
+  uint32_t Ka[MT][DQ16][4], Va[MT][DV16][4];
+  {
+    const bf16* Kr = P.Kb + ((size_t)u * P.L + n0) * dqk + h * DQH;
+    const bf16* Vr = P.Vb + ((size_t)u * P.L + n0) * d + h * DVH;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const int r0 = mt * 16 + g, r1 = r0 + 8;
+#pragma unroll
+      for (int k = 0; k < DQ16; ++k) {
+        const int c = k * 16 + 2 * t;
+        Ka[mt][k][0] = r0 < cnt ? *reinterpret_cast<const uint32_t*>(Kr + (size_t)r0 * dqk + c) : 0u;
+        Ka[mt][k][1] = r1 < cnt ? *reinterpret_cast<const uint32_t*>(Kr + (size_t)r1 * dqk + c) : 0u;
+        Ka[mt][k][2] = r0 < cnt ? *reinterpret_cast<const uint32_t*>(Kr + (size_t)r0 * dqk + c + 8) : 0u;
+        Ka[mt][k][3] = r1 < cnt ? *reinterpret_cast<const uint32_t*>(Kr + (size_t)r1 * dqk + c + 8) : 0u;
+      }
+#pragma unroll
+      for (int k = 0; k < DV16; ++k) {
+        const int c = k * 16 + 2 * t;
+        Va[mt][k][0] = r0 < cnt ? *reinterpret_cast<const uint32_t*>(Vr + (size_t)r0 * d + c) : 0u;
+        Va[mt][k][1] = r1 < cnt ? *reinterpret_cast<const uint32_t*>(Vr + (size_t)r1 * d + c) : 0u;
+        Va[mt][k][2] = r0 < cnt ? *reinterpret_cast<const uint32_t*>(Vr + (size_t)r0 * d + c + 8) : 0u;
+        Va[mt][k][3] = r1 < cnt ? *reinterpret_cast<const uint32_t*>(Vr + (size_t)r1 * d + c + 8) : 0u;
+      }
+    }
+  }
+  // K_h^T as A fragments (rows = key components, k = items), from the fragments above: the transposed 8 x 8 blocks
+  uint32_t Kt[DQ16][MT][4];
+#pragma unroll
+  for (int q = 0; q < DQ16; ++q)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      Kt[q][mt][0] = movmatrix_t(Ka[mt][q][0]);
+      Kt[q][mt][1] = movmatrix_t(Ka[mt][q][2]);
+      Kt[q][mt][2] = movmatrix_t(Ka[mt][q][1]);
+      Kt[q][mt][3] = movmatrix_t(Ka[mt][q][3]);
+    }
+
+  float dKacc[MT][2 * DQ16][4], dVacc[MT][2 * DV16][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+    for (int j = 0; j < 2 * DQ16; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) dKacc[mt][j][e] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 2 * DV16; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) dVacc[mt][j][e] = 0.f;
+  }
+
+  // ---- staging of 16 candidate rows: Qb[c, h] (DQH values) and ds_seg[c, h] (DVH values)
+  const uint32_t stage0 = smem_addr(smem) + warp * 2 * kBuf;
+  const bf16* Qg = P.Qb + (size_t)off0 * dqk + h * DQH;
+  const bf16* Sg = P.dSb + ((size_t)off0 * P.Lp + seg) * d + h * DVH;
+  const size_t s_row = (size_t)P.Lp * d;
+  auto stage = [&](int c0, int buf) {
+    const uint32_t base = stage0 + buf * kBuf;
+#pragma unroll
+    for (int k = 0; k < DQ16; ++k) {
+      const int x = lane + 32 * k, row = x / (2 * DQ16), ch = x % (2 * DQ16);
+      const int c = c0 + row;
+      cp16(base + row * QS + ch * 16, Qg + (size_t)min(c, C - 1) * dqk + ch * 8, c < C ? 16u : 0u);
+    }
+#pragma unroll
+    for (int k = 0; k < DV16; ++k) {
+      const int x = lane + 32 * k, row = x / (2 * DV16), ch = x % (2 * DV16);
+      const int c = c0 + row;
+      cp16(base + 16 * QS + row * DS + ch * 16, Sg + (size_t)min(c, C - 1) * s_row + ch * 8, c < C ? 16u : 0u);
+    }
+    cp_commit();
+  };
+  // ldmatrix lane addresses inside a buffer.  Plain (B operand with k = head component, n = candidate): matrices
+  // (cands 0-7, k 0-7), (cands 0-7, k 8-15), (cands 8-15, k 0-7), (cands 8-15, k 8-15) of a 16-component step.
+  // Transposed (k = candidate, n = component): (cands 0-7, n 0-7), (cands 8-15, n 0-7), (cands 0-7, n 8-15), (cands 8-15, n 8-15).
+  const int mi = lane >> 3, lr = lane & 7;
+  const uint32_t q_plain = ((mi >> 1) * 8 + lr) * QS + (mi & 1) * 16;
+  const uint32_t q_trans = ((mi & 1) * 8 + lr) * QS + (mi >> 1) * 16;
+  const uint32_t s_plain = 16 * QS + ((mi >> 1) * 8 + lr) * DS + (mi & 1) * 16;
+  const uint32_t s_trans = 16 * QS + ((mi & 1) * 8 + lr) * DS + (mi >> 1) * 16;
+
+  float* dQg = P.dQf + (size_t)off0 * dqk + h * DQH;
+  const int slabs = (C + 15) >> 4;
+  stage(0, 0);
+  for (int s = 0; s < slabs; ++s) {
+    const int c0 = s * 16;
+    if (s + 1 < slabs) {
+      stage(c0 + 16, (s + 1) & 1);
+      cp_wait<1>();
+    } else {
+      cp_wait<0>();
+    }
+    __syncwarp();
+    const uint32_t base = stage0 + (s & 1) * kBuf;
+
+    // scores^T / 2 and dG^T: [items] x [16 candidates]
+    float E[MT][2][4], G[MT][2][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) E[mt][nt][e] = G[mt][nt][e] = 0.f;
+#pragma unroll
+    for (int k = 0; k < DQ16; ++k) {
+      uint32_t b[4];
+      ldsm_x4(b, base + q_plain + k * 32);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        mma16816(E[mt][0], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], b[0], b[1]);
+        mma16816(E[mt][1], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], b[2], b[3]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < DV16; ++k) {
+      uint32_t b[4];
+      ldsm_x4(b, base + s_plain + k * 32);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        mma16816(G[mt][0], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], b[0], b[1]);
+        mma16816(G[mt][1], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], b[2], b[3]);
+      }
+    }
+    // gates and score gradients, packed as the A operands of the products that contract over the candidates
+    uint32_t gA[MT][4], eA[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        float gg[4], ee[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float th = tanh_fast(E[mt][nt][e]);
+          gg[e] = fmaf(th, 0.5f, 0.5f);
+          ee[e] = G[mt][nt][e] * fmaf(-th, th, 1.f);
+        }
+        gA[mt][2 * nt] = pack2(gg[0], gg[1]);
+        gA[mt][2 * nt + 1] = pack2(gg[2], gg[3]);
+        eA[mt][2 * nt] = pack2(ee[0], ee[1]);
+        eA[mt][2 * nt + 1] = pack2(ee[2], ee[3]);
+      }
+    // dV += g^T ds,  dK += (dG w)^T Qb
+#pragma unroll
+    for (int k = 0; k < DV16; ++k) {
+      uint32_t b[4];
+      ldsm_x4_t(b, base + s_trans + k * 32);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        mma16816(dVacc[mt][2 * k], gA[mt][0], gA[mt][1], gA[mt][2], gA[mt][3], b[0], b[1]);
+        mma16816(dVacc[mt][2 * k + 1], gA[mt][0], gA[mt][1], gA[mt][2], gA[mt][3], b[2], b[3]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < DQ16; ++k) {
+      uint32_t b[4];
+      ldsm_x4_t(b, base + q_trans + k * 32);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        mma16816(dKacc[mt][2 * k], eA[mt][0], eA[mt][1], eA[mt][2], eA[mt][3], b[0], b[1]);
+        mma16816(dKacc[mt][2 * k + 1], eA[mt][0], eA[mt][1], eA[mt][2], eA[mt][3], b[2], b[3]);
+      }
+    }
+    // dQf^T [key components] x [candidates] = K_h^T (dG w)^T: the B operand is the transposed 8 x 8 blocks of eA
+    float dQ[DQ16][2][4];
+#pragma unroll
+    for (int q = 0; q < DQ16; ++q)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dQ[q][nt][e] = 0.f;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const uint32_t b0 = movmatrix_t(eA[mt][2 * nt]), b1 = movmatrix_t(eA[mt][2 * nt + 1]);
+#pragma unroll
+        for (int q = 0; q < DQ16; ++q) mma16816(dQ[q][nt], Kt[q][mt][0], Kt[q][mt][1], Kt[q][mt][2], Kt[q][mt][3], b0, b1);
+      }
+#pragma unroll
+    for (int q = 0; q < DQ16; ++q)
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const int c = c0 + nt * 8 + 2 * t, kq = q * 16 + g;
+        if (c < C) {
+          atomicAdd(dQg + (size_t)c * dqk + kq, 0.25f * dQ[q][nt][0]);
+          atomicAdd(dQg + (size_t)c * dqk + kq + 8, 0.25f * dQ[q][nt][2]);
+        }
+        if (c + 1 < C) {
+          atomicAdd(dQg + (size_t)(c + 1) * dqk + kq, 0.25f * dQ[q][nt][1]);
+          atomicAdd(dQg + (size_t)(c + 1) * dqk + kq + 8, 0.25f * dQ[q][nt][3]);
+        }
+      }
+    __syncwarp();                        // every lane is done with this buffer before the next request overwrites it
+  }
+
+  // ---- this job's rows of dK and dV (valid rows only; the others keep the zeros the caller put there)
+  float* dKr = P.dK + ((size_t)u * P.L + n0) * dqk + h * DQH;
+  float* dVr = P.dV + ((size_t)u * P.L + n0) * d + h * DVH;
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+    const int r0 = mt * 16 + g, r1 = r0 + 8;
+#pragma unroll
+    for (int j = 0; j < 2 * DQ16; ++j) {
+      const int c = j * 8 + 2 * t;
+      if (r0 < cnt) *reinterpret_cast<float2*>(dKr + (size_t)r0 * dqk + c) = make_float2(0.5f * dKacc[mt][j][0], 0.5f * dKacc[mt][j][1]);
+      if (r1 < cnt) *reinterpret_cast<float2*>(dKr + (size_t)r1 * dqk + c) = make_float2(0.5f * dKacc[mt][j][2], 0.5f * dKacc[mt][j][3]);
+    }
+#pragma unroll
+    for (int j = 0; j < 2 * DV16; ++j) {
+      const int c = j * 8 + 2 * t;
+      if (r0 < cnt) *reinterpret_cast<float2*>(dVr + (size_t)r0 * d + c) = make_float2(dVacc[mt][j][0], dVacc[mt][j][1]);
+      if (r1 < cnt) *reinterpret_cast<float2*>(dVr + (size_t)r1 * d + c) = make_float2(dVacc[mt][j][2], dVacc[mt][j][3]);
+    }
+  }
+}
+
+struct MmaShape {
+  int mt, dq16, dv16;
+};
+bool mma_shape(const Plan& p, MmaShape* s) {
+  if (p.dqh % 16 || p.dvh % 16) return false;
+  s->dq16 = p.dqh / 16;
+  s->dv16 = p.dvh / 16;
+  s->mt = (p.S <= 16 || s->dv16 == 4) ? 1 : 2;       // (two row tiles of 64-wide value slices would not fit the registers)
+  return (s->dq16 == 1 || s->dq16 == 2) && (s->dv16 == 1 || s->dv16 == 2 || s->dv16 == 4);
+}
+
+template <int MT, int DQ16, int DV16>
+int launch_mma(const BwdMmaParams& P, int U, cudaStream_t st) {
+  constexpr int smem = kBwdWarps * 2 * 16 * ((2 * 16 * DQ16 + 16) + (2 * 16 * DV16 + 16));
+  auto kernel = sta_bwd_mma_kernel<MT, DQ16, DV16>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  LaunchScope ls("bwd_sta_mma", st);
+  kernel<<<dim3((P.jobs + kBwdWarps - 1) / kBwdWarps, U), kBwdWarps * 32, smem, st>>>(P);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+int cast(const float* src, bf16* dst, size_t n, float scale, cudaStream_t st) {
+  if (n == 0) return LASER_OK;
+  LaunchScope ls("bwd_cast_bf16", st);
+  const size_t n4 = n / 4;
+  const int blocks = (int)std::min<size_t>((n4 + 255) / 256, 148 * 16);
+  cast_bf16_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(src), reinterpret_cast<uint2*>(dst), n4, scale);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+struct MmaScratch {
+  bf16 *Qb, *Kb, *Vb, *dSb;
+  size_t total;
+};
+MmaScratch carve_mma(const Plan& p, char* base) {
+  MmaScratch s;
+  size_t off = 0;
+  auto take = [&](size_t n) {
+    bf16* ptr = base ? reinterpret_cast<bf16*>(base + off) : nullptr;
+    off = align_up(off + n * sizeof(bf16)) + kGuardBytes;
+    return ptr;
+  };
+  const size_t UL = (size_t)p.U * p.L;
+  s.Qb = take((size_t)p.N * p.dqk);
+  s.Kb = take(UL * p.dqk);
+  s.Vb = take(UL * p.d);
+  s.dSb = take((size_t)p.N * p.Lp * p.d);
+  s.total = off;
+  return s;
+}
+
+}  // namespace
+
+bool sta_bwd_mma_supported(const Plan& p) {
+  MmaShape s;
+  if (!mma_shape(p, &s)) return false;
+  const long long R = (std::min(p.S, p.L) + 16 * s.mt - 1) / (16 * s.mt);
+  return p.U <= 65535 && (long long)p.Lp * R * p.H <= 0x7fffffffLL && p.maxC >= 8;
+}
+
+size_t sta_bwd_mma_scratch_bytes(const Plan& p) { return sta_bwd_mma_supported(p) ? carve_mma(p, nullptr).total : 0; }
+
+int sta_bwd_mma(const Plan& p, const float* Qf, const float* Kf, const float* Vf, const float* dHp,
+                const int32_t* lengths, const int32_t* cand_offsets, float* dQf, float* dK, float* dV, char* scratch,
+                cudaStream_t st) {
+  MmaShape sh;
+  if (!mma_shape(p, &sh)) return LASER_ERR_UNSUPPORTED;
+  const MmaScratch s = carve_mma(p, scratch);
+  const size_t UL = (size_t)p.U * p.L;
+  int rc;
+  if ((rc = cast(Qf, s.Qb, (size_t)p.N * p.dqk, 0.5f, st)) != LASER_OK) return rc;
+  if ((rc = cast(Kf, s.Kb, UL * p.dqk, 1.f, st)) != LASER_OK) return rc;
+  if ((rc = cast(Vf, s.Vb, UL * p.d, 1.f, st)) != LASER_OK) return rc;
+  if ((rc = cast(dHp, s.dSb, (size_t)p.N * p.Lp * p.d, 1.f, st)) != LASER_OK) return rc;
+  BwdMmaParams P;
+  P.Qb = s.Qb; P.Kb = s.Kb; P.Vb = s.Vb; P.dSb = s.dSb;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.dQf = dQf; P.dK = dK; P.dV = dV;
+  P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
+  P.R = (std::min(p.S, p.L) + 16 * sh.mt - 1) / (16 * sh.mt);
+  P.jobs = p.Lp * P.R * p.H;
+#define LASER_MMA_CASE(MT, DQ, DV) \
+  if (sh.mt == MT && sh.dq16 == DQ && sh.dv16 == DV) return launch_mma<MT, DQ, DV>(P, p.U, st);
+  LASER_MMA_CASE(1, 1, 1) LASER_MMA_CASE(1, 1, 2) LASER_MMA_CASE(1, 1, 4)
+  LASER_MMA_CASE(1, 2, 1) LASER_MMA_CASE(1, 2, 2) LASER_MMA_CASE(1, 2, 4)
+  LASER_MMA_CASE(2, 1, 1) LASER_MMA_CASE(2, 1, 2)
+  LASER_MMA_CASE(2, 2, 1) LASER_MMA_CASE(2, 2, 2)
+#undef LASER_MMA_CASE
+  return LASER_ERR_UNSUPPORTED;
+}
+
+}  // namespace laser

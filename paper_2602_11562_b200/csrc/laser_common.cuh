@@ -79,11 +79,21 @@ int simt_sta_f32(const Plan& p, const void* items, const int32_t* lengths, const
                  const void* Wq, const void* Wk, const void* Wv, float* Hprime32, char* ws, cudaStream_t st);
 
 // Backward pass (laser_backward.cu): p is a plan of the FP32-ALU path; the workspace holds p.total bytes of the forward
-// plan followed by backward_scratch_bytes(p).  Gradients are fp32.
+// plan followed by backward_scratch_bytes(p).  Gradients are fp32.  tensor: bf16 batches take the tensor-core kernels
+// where backward_tensor_supported(p) says they exist.
 size_t backward_scratch_bytes(const Plan& p);
+bool backward_tensor_supported(const Plan& p);
 int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
              const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,
-             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st);
+             float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor);
+// Tensor-core backward through the segment aggregation and the gates (laser_backward_mma.cu): bf16 copies of Qf (Q / gamma),
+// Kf, Vf and dHp are made in `scratch` (sta_bwd_mma_scratch_bytes), dK / dV rows of valid items are written (the rest must
+// hold zeros), dQf is added to.
+bool sta_bwd_mma_supported(const Plan& p);
+size_t sta_bwd_mma_scratch_bytes(const Plan& p);
+int sta_bwd_mma(const Plan& p, const float* Qf, const float* Kf, const float* Vf, const float* dHp,
+                const int32_t* lengths, const int32_t* cand_offsets, float* dQf, float* dK, float* dV, char* scratch,
+                cudaStream_t st);
 
 bool tensor_supported(const Plan& p);
 void tensor_geometry(const Plan& p, TensorGeom* g);

@@ -24,19 +24,26 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("case", range(len(CASES)))
-def test_backward_matches_oracle(case):
-    kw = dict(CASES[case])
-    w = make_custom(seed=1100 + case, emb_std="one" if kw["d"] <= 32 else "inv_sqrt_d", **kw)
+def _check(case_kw, seed, path, bar, want_kernel=None):
+    kw = dict(case_kw)
+    w = make_custom(seed=seed, emb_std="one" if kw["d"] <= 32 else "inv_sqrt_d", **kw)
     s = w.spec
-    rng = np.random.default_rng(40 + case)
+    rng = np.random.default_rng(seed + 7)
     dz = rng.standard_normal((w.N, s.d)).astype(np.float32)
     ref = backward_oracle.backward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
                                    dz.astype(np.float64), w.gamma, w.tau)
-    b = P.DeviceBatch.from_workload(w)
+    b = P.DeviceBatch.from_workload(w, path=path)
     ws = torch.empty(P.laser_backward_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
-    got = P.laser_backward(b.cfg, *b.args(), b.Wg, torch.from_numpy(dz).cuda(), workspace=ws)
+    P.laser_profile_enable(True)
+    try:
+        got = P.laser_backward(b.cfg, *b.args(), b.Wg, torch.from_numpy(dz).cuda(), workspace=ws)
+        names = [n for n, _ in P.laser_profile_read()]
+    finally:
+        P.laser_profile_enable(False)
     assert P.laser_check_status(ws) == 0
+    if want_kernel is not None:
+        assert ("bwd_sta_mma" in names) == want_kernel, names
+    worst = {}
     for k, r in ref.items():
         g = got[k].cpu().numpy().astype(np.float64)
         assert g.shape == r.shape, k
@@ -44,7 +51,8 @@ def test_backward_matches_oracle(case):
         if r.size == 0:                                       # (no GSTA layer: dWg is empty)
             continue
         scale = max(np.max(np.abs(r)), 1e-30)
-        assert np.max(np.abs(g - r)) <= REL_TO_MAX * scale, (k, np.max(np.abs(g - r)), scale)
+        worst[k] = np.max(np.abs(g - r)) / scale
+        assert worst[k] <= bar, (k, worst[k], scale)
     # padding rows of d_items are exact zeros
     for u in range(s.U):
         assert not got["d_items"][u, int(w.lengths[u]):].any()
@@ -55,6 +63,43 @@ def test_backward_matches_oracle(case):
         if ref[k].size:
             diff = (got[k] - got2[k]).abs().max().item()
             assert diff <= 1e-5 * max(np.max(np.abs(ref[k])), 1e-30), k
+    return worst
+
+
+@pytest.mark.parametrize("case", range(len(CASES)))
+def test_backward_matches_oracle(case):
+    # the FP32-ALU kernels, for either dtype
+    _check(CASES[case], 1100 + case, P.PATH_SIMT, REL_TO_MAX, want_kernel=False)
+
+
+# bf16 batches on the tensor-core kernels.  The operands of the five contractions through the gates are bf16 roundings of
+# fp32 intermediates (Q / gamma, K, V, dH', the gates and the score gradients: relative 2^-9 each, `tanh.approx` 2^-11), the
+# accumulation is fp32; sums of such terms with random signs stay within a few 1e-3 of the largest entry of a gradient
+# (measured: at most 4e-3 on these shapes).  Bar: 2e-2, the forward's bf16 bar.
+TENSOR_BAR = 2e-2
+TENSOR_CASES = [
+    dict(U=3, C=130, L=512, d=64, H=4, S=64, M=2, dtype="bf16", lengths=[512, 300, 77]),   # serving-like (head 16 x 16)
+    dict(U=2, C=50, L=512, d=128, H=4, S=128, M=2, dtype="bf16", lengths=[512, 301]),      # batched-ranking-like (16 x 32)
+    dict(U=2, C=37, L=300, d=128, H=2, S=10, M=2, dtype="bf16", lengths=[300, 137]),       # production-like (16 x 64, 10-item segments)
+    dict(U=2, C=24, L=700, d=64, H=4, S=100, M=1, dtype="bf16", lengths=[700, 455]),       # segments of 100: a 4-row last tile
+    dict(U=1, C=70, L=96, d=16, H=1, S=96, M=3, dtype="bf16", lengths=[90]),               # one head, one segment
+    dict(U=3, C=9, L=64, d=64, H=2, S=16, M=1, dtype="bf16", lengths=[64, 1, 0], d_qh=32), # d_qh = 32, fewer than 16 candidates
+    dict(U=2, C=300, L=128, d=128, H=8, S=32, M=2, dtype="bf16", lengths=[128, 100]),      # eight heads, many candidate tiles
+]
+
+
+@pytest.mark.parametrize("case", range(len(TENSOR_CASES)))
+def test_backward_tensor_path_matches_oracle(case):
+    worst = _check(TENSOR_CASES[case], 1200 + case, P.PATH_AUTO, TENSOR_BAR, want_kernel=True)
+    print("backward tensor path, worst error / largest entry:", {k: f"{v:.2e}" for k, v in worst.items()})
+
+
+def test_backward_tensor_path_on_request_only_where_it_exists():
+    w = make_custom(U=1, C=4, L=32, d=32, H=2, S=8, M=1, dtype="f32", seed=5)
+    b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
+    ws = torch.empty(1 << 24, dtype=torch.uint8, device="cuda")
+    with pytest.raises(P.LaserError):
+        P.laser_backward(b.cfg, *b.args(), b.Wg, torch.zeros((w.N, 32), device="cuda"), workspace=ws)
 
 
 def test_backward_rejects_a_short_workspace():
