@@ -85,21 +85,155 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, cons
   }
 }
 
+// The same product on the tensor cores: mma.sync m16n8k8 with TF32 operands (bf16 inputs are exact in TF32, fp32 ones are
+// rounded to nearest when they are staged), fp32 accumulation.  64 x 64 tiles of C, k-steps of 32, eight warps of 32 x 16.
+// An operand whose contraction index is contiguous in memory is staged row by row ([64][kWK + 4]), the other k-major
+// ([kWK][64 + 8]): both paddings make the fragment reads conflict-free.  Full, aligned tiles are staged with 16-byte (fp32)
+// or 8-byte (bf16) loads, partial or unaligned ones element by element.
+constexpr int kWK = 32, kRowLd = kWK + 4, kColLd = 64 + 8, kStage = 64 * kRowLd;
+static_assert(kWK * kColLd <= kStage, "both layouts fit one staging array");
+
+__device__ __forceinline__ uint32_t tf32_of(float v) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+  return r;
+}
+__device__ __forceinline__ uint4 load4_tf32(const float* p) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  return make_uint4(tf32_of(v.x), tf32_of(v.y), tf32_of(v.z), tf32_of(v.w));
+}
+__device__ __forceinline__ uint4 load4_tf32(const bf16* p) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  return make_uint4(v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u);
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Stages a 64 x kWK tile of an operand X with rows r0 .. (bound R) and contraction indices k0 .. (bound k_hi):
+// X(r, k) = k_major ? X[k ld + r] : X[r ld + k].  Shared layout: k_major ? [k][kColLd] : [r][kRowLd].
+template <typename TX>
+__device__ __forceinline__ void stage_tile(uint32_t* __restrict__ sm, const TX* __restrict__ X, int ld, int k_major, int r0,
+                                           int R, int k0, int k_hi, bool aligned, int tid) {
+  const bool full = aligned && r0 + 64 <= R && k0 + kWK <= k_hi;
+  if (full) {
+    if (k_major) {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int i = tid + kGemmThreads * j, kk = i >> 4, r4 = (i & 15) * 4;
+        *reinterpret_cast<uint4*>(sm + kk * kColLd + r4) = load4_tf32(X + (size_t)(k0 + kk) * ld + r0 + r4);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int i = tid + kGemmThreads * j, rr = i >> 3, k4 = (i & 7) * 4;
+        *reinterpret_cast<uint4*>(sm + rr * kRowLd + k4) = load4_tf32(X + (size_t)(r0 + rr) * ld + k0 + k4);
+      }
+    }
+    return;
+  }
+  for (int i = tid; i < 64 * kWK; i += kGemmThreads) {
+    int rr, kk;
+    if (k_major) { kk = i >> 6; rr = i & 63; } else { rr = i / kWK; kk = i - rr * kWK; }
+    const int r = r0 + rr, k = k0 + kk;
+    float v = 0.f;
+    if (r < R && k < k_hi) v = to_f32<TX>(k_major ? X[(size_t)k * ld + r] : X[(size_t)r * ld + k]);
+    sm[k_major ? kk * kColLd + rr : rr * kRowLd + kk] = tf32_of(v);
+  }
+}
+
 template <typename TA, typename TB>
-int gemm(cudaStream_t st, int M, int N, int K, const TA* A, int lda, bool ta, const TB* B, int ldb, bool tb, float* C,
+__global__ void __launch_bounds__(kGemmThreads)
+gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
+                 float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split, int aligned_a, int aligned_b) {
+  __shared__ __align__(16) uint32_t As[kStage], Bs[kStage];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int m0 = blockIdx.x * 64, n0 = blockIdx.y * 64;
+  const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
+  const int wm = (warp >> 2) * 32, wn = (warp & 3) * 16;
+  // element offsets of this lane's fragment entries: A(m, k) with m = wm + g, k = t;  B(k, n) with k = t, n = wn + g
+  const int a_m = ta ? 1 : kRowLd, a_k = ta ? kColLd : 1, b_n = tb ? kRowLd : 1, b_k = tb ? 1 : kColLd;
+  const int a_off = (wm + g) * a_m + t * a_k, b_off = (wn + g) * b_n + t * b_k;
+  float acc[2][2][4] = {};
+  for (int k0 = k_lo; k0 < k_hi; k0 += kWK) {
+    stage_tile<TA>(As, A, lda, ta, m0, M, k0, k_hi, aligned_a != 0, tid);      // A(m, k): k-major storage when transposed
+    stage_tile<TB>(Bs, B, ldb, !tb, n0, N, k0, k_hi, aligned_b != 0, tid);     // B(k, n): k-major storage when NOT transposed
+    __syncthreads();
+#pragma unroll
+    for (int kb = 0; kb < kWK; kb += 8) {
+      uint32_t a[2][4], b[2][2];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint32_t* pa = As + a_off + mt * 16 * a_m + kb * a_k;
+        a[mt][0] = pa[0];
+        a[mt][1] = pa[8 * a_m];
+        a[mt][2] = pa[4 * a_k];
+        a[mt][3] = pa[8 * a_m + 4 * a_k];
+      }
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        const uint32_t* pb = Bs + b_off + nt * 8 * b_n + kb * b_k;
+        b[nt][0] = pb[0];
+        b[nt][1] = pb[4 * b_k];
+      }
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) mma_tf32(acc[mt][nt], a[mt], b[nt][0], b[nt][1]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int m = m0 + wm + mt * 16 + g + (e >> 1) * 8, n = n0 + wn + nt * 8 + 2 * t + (e & 1);
+        if (m >= M || n >= N) continue;
+        float* c = C + (size_t)m * ldc + n;
+        const float v = alpha * acc[mt][nt][e];
+        if (gridDim.z > 1) atomicAdd(c, v);
+        else *c = accumulate ? *c + v : v;
+      }
+}
+
+// Where a product runs: the stream, and whether on the tensor cores (TF32) or on the FP32 ALUs.
+struct GemmCtx {
+  cudaStream_t st;
+  bool tf32;
+};
+
+template <typename TX>
+bool aligned_for_vector_loads(const TX* X, int ld) {
+  return ld % 4 == 0 && reinterpret_cast<uintptr_t>(X) % (4 * sizeof(TX)) == 0;
+}
+
+template <typename TA, typename TB>
+int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, const TB* B, int ldb, bool tb, float* C,
          int ldc, float alpha, bool accumulate, bool split_k) {
   if (M <= 0 || N <= 0 || K <= 0) return LASER_OK;
+  cudaStream_t st = gx.st;
+  const int kstep = gx.tf32 ? kWK : kTK;
   int splits = 1, per = K;
   if (split_k) {                     // reductions over many rows into a small matrix (C must hold its initial value)
     per = 256;
     splits = (K + per - 1) / per;
-    if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kTK - 1) / kTK * kTK; splits = (K + per - 1) / per; }
+    if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kstep - 1) / kstep * kstep; splits = (K + per - 1) / per; }
   }
   const dim3 grid((M + kTM - 1) / kTM, (N + kTN - 1) / kTN, splits);
   if (grid.y > 65535) return LASER_ERR_UNSUPPORTED;
-  LaunchScope ls("bwd_gemm", st);
-  gemm_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
-                                                    accumulate ? 1 : 0, per);
+  LaunchScope ls(gx.tf32 ? "bwd_gemm_tf32" : "bwd_gemm", st);
+  if (gx.tf32)
+    gemm_tf32_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
+                                                           accumulate ? 1 : 0, per, aligned_for_vector_loads(A, lda) ? 1 : 0,
+                                                           aligned_for_vector_loads(B, ldb) ? 1 : 0);
+  else
+    gemm_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
+                                                      accumulate ? 1 : 0, per);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
 }
@@ -533,6 +667,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   float* Qf = reinterpret_cast<float*>(ws + p.off_q);
   float* Kf = reinterpret_cast<float*>(ws + p.off_k);
   float* Vf = reinterpret_cast<float*>(ws + p.off_v);
+  const GemmCtx gx = {st, tensor};
   int rc;
 #define BWD_OK(...) do { rc = (__VA_ARGS__); if (rc != LASER_OK) return rc; } while (0)
 
@@ -560,9 +695,9 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     const T *Wql = Wg + (size_t)(l * 3) * d * d, *Wkl = Wql + (size_t)d * d, *Wvl = Wkl + (size_t)d * d;
     float *Tl = s.T + l * Nd, *Tn = Tl + Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
           *Ml = s.Mh + l * NHd;
-    BWD_OK(gemm<float, T>(st, N, d, d, Tl, d, false, Wql, d, false, Ql, d, 1.f, false, false));
+    BWD_OK(gemm<float, T>(gx, N, d, d, Tl, d, false, Wql, d, false, Ql, d, 1.f, false, false));
     for (int h = 0; h < H; ++h)
-      BWD_OK(gemm<float, T>(st, N, d, dvh, Ql + h * dvh, d, false, Wkl + h * dvh, d, true, Qtl + (size_t)h * d, H * d,
+      BWD_OK(gemm<float, T>(gx, N, d, dvh, Ql + h * dvh, d, false, Wkl + h * dvh, d, true, Qtl + (size_t)h * d, H * d,
                             p.inv_tau, false, false));
     {
       LaunchScope ls("bwd_attn_fwd", st);
@@ -571,7 +706,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     }
     LASER_CUDA_OK(cudaMemcpyAsync(Tn, Tl, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
     for (int h = 0; h < H; ++h)
-      BWD_OK(gemm<float, T>(st, N, dvh, d, Ml + (size_t)h * d, H * d, false, Wvl + h * dvh, d, false, Tn + h * dvh, d, 1.f,
+      BWD_OK(gemm<float, T>(gx, N, dvh, d, Ml + (size_t)h * d, H * d, false, Wvl + h * dvh, d, false, Tn + h * dvh, d, 1.f,
                             true, false));
   }
 
@@ -585,9 +720,9 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     float *gWq = dWg + (size_t)(l * 3) * d * d, *gWk = gWq + (size_t)d * d, *gWv = gWk + (size_t)d * d;
     for (int h = 0; h < H; ++h) {
       // dW_v[:, h] += m_h^T do_h;  dm_h = do_h W_v[:, h]^T
-      BWD_OK(gemm<float, float>(st, d, dvh, N, Ml + (size_t)h * d, H * d, true, s.dT + h * dvh, d, false, gWv + h * dvh, d,
+      BWD_OK(gemm<float, float>(gx, d, dvh, N, Ml + (size_t)h * d, H * d, true, s.dT + h * dvh, d, false, gWv + h * dvh, d,
                                 1.f, true, true));
-      BWD_OK(gemm<float, T>(st, N, d, dvh, s.dT + h * dvh, d, false, Wvl + h * dvh, d, true, s.dM + (size_t)h * d, H * d,
+      BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT + h * dvh, d, false, Wvl + h * dvh, d, true, s.dM + (size_t)h * d, H * d,
                             1.f, false, false));
     }
     {
@@ -597,13 +732,13 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     }
     for (int h = 0; h < H; ++h) {
       // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau
-      BWD_OK(gemm<float, T>(st, N, dvh, d, s.dQt + (size_t)h * d, H * d, false, Wkl + h * dvh, d, false, s.dQ + h * dvh, d,
+      BWD_OK(gemm<float, T>(gx, N, dvh, d, s.dQt + (size_t)h * d, H * d, false, Wkl + h * dvh, d, false, s.dQ + h * dvh, d,
                             p.inv_tau, false, false));
-      BWD_OK(gemm<float, float>(st, d, dvh, N, s.dQt + (size_t)h * d, H * d, true, Ql + h * dvh, d, false, gWk + h * dvh, d,
+      BWD_OK(gemm<float, float>(gx, d, dvh, N, s.dQt + (size_t)h * d, H * d, true, Ql + h * dvh, d, false, gWk + h * dvh, d,
                                 p.inv_tau, true, true));
     }
-    BWD_OK(gemm<float, float>(st, d, d, N, Tl, d, true, s.dQ, d, false, gWq, d, 1.f, true, true));        // dW_q += T^T dQ
-    BWD_OK(gemm<float, T>(st, N, d, d, s.dQ, d, false, Wql, d, true, s.dT, d, 1.f, true, false));            // dT += dQ W_q^T
+    BWD_OK(gemm<float, float>(gx, d, d, N, Tl, d, true, s.dQ, d, false, gWq, d, 1.f, true, true));        // dW_q += T^T dQ
+    BWD_OK(gemm<float, T>(gx, N, d, d, s.dQ, d, false, Wql, d, true, s.dT, d, 1.f, true, false));            // dT += dQ W_q^T
   }
 
   // ---- backward through the segment aggregation and the gates
@@ -629,12 +764,12 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   }
 
   // ---- backward through the projections (Qf = T W_q / gamma)
-  BWD_OK(gemm<T, float>(st, d, dqk, N, cands, d, true, s.dQf, dqk, false, dWq, dqk, p.inv_gamma, true, true));
-  BWD_OK(gemm<float, T>(st, N, d, dqk, s.dQf, dqk, false, Wq, dqk, true, s.dT, d, p.inv_gamma, true, false));
-  BWD_OK(gemm<T, float>(st, d, dqk, (int)UL, items, d, true, s.dK, dqk, false, dWk, dqk, 1.f, true, true));
-  BWD_OK(gemm<T, float>(st, d, d, (int)UL, items, d, true, s.dV, d, false, dWv, d, 1.f, true, true));
-  BWD_OK(gemm<float, T>(st, (int)UL, d, dqk, s.dK, dqk, false, Wk, dqk, true, d_items, d, 1.f, false, false));
-  BWD_OK(gemm<float, T>(st, (int)UL, d, d, s.dV, d, false, Wv, d, true, d_items, d, 1.f, true, false));
+  BWD_OK(gemm<T, float>(gx, d, dqk, N, cands, d, true, s.dQf, dqk, false, dWq, dqk, p.inv_gamma, true, true));
+  BWD_OK(gemm<float, T>(gx, N, d, dqk, s.dQf, dqk, false, Wq, dqk, true, s.dT, d, p.inv_gamma, true, false));
+  BWD_OK(gemm<T, float>(gx, d, dqk, (int)UL, items, d, true, s.dK, dqk, false, dWk, dqk, 1.f, true, true));
+  BWD_OK(gemm<T, float>(gx, d, d, (int)UL, items, d, true, s.dV, d, false, dWv, d, 1.f, true, true));
+  BWD_OK(gemm<float, T>(gx, (int)UL, d, dqk, s.dK, dqk, false, Wk, dqk, true, d_items, d, 1.f, false, false));
+  BWD_OK(gemm<float, T>(gx, (int)UL, d, d, s.dV, d, false, Wv, d, true, d_items, d, 1.f, true, false));
   LASER_CUDA_OK(cudaMemcpyAsync(d_cands, s.dT, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
 #undef BWD_OK
   LASER_CUDA_OK(cudaGetLastError());

@@ -56,13 +56,16 @@ def _check(case_kw, seed, path, bar, want_kernel=None):
     # padding rows of d_items are exact zeros
     for u in range(s.U):
         assert not got["d_items"][u, int(w.lengths[u]):].any()
-    # a second call on the same workspace agrees (the atomically summed parts to rounding, the rest bit for bit)
+    # a second call on the same workspace agrees (the atomically summed parts to rounding, the rest bit for bit).  On the
+    # tensor-core path an atomically summed intermediate is then rounded to TF32 as a matrix-product operand, so a
+    # last-bit difference of fp32 can become one of 2^-11 in single terms of the weight gradients.
     got2 = P.laser_backward(b.cfg, *b.args(), b.Wg, torch.from_numpy(dz).cuda(), workspace=ws)
     assert torch.equal(got["d_items"], got2["d_items"])
+    repeat_bar = 1e-5 if path == P.PATH_SIMT else 2e-4
     for k in ref:
         if ref[k].size:
             diff = (got[k] - got2[k]).abs().max().item()
-            assert diff <= 1e-5 * max(np.max(np.abs(ref[k])), 1e-30), k
+            assert diff <= repeat_bar * max(np.max(np.abs(ref[k])), 1e-30), k
     return worst
 
 
