@@ -672,7 +672,16 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 #define BWD_OK(...) do { rc = (__VA_ARGS__); if (rc != LASER_OK) return rc; } while (0)
 
   // ---- forward, kept in fp32: projections and H' (the FP32-ALU forward kernels), then the GSTA layers
-  if (p.dqh == 16 && (dvh == 16 || dvh == 32) && p.H <= 32) {
+  char* mma_scratch = ws + p.total + s.total;
+  if (tensor) {
+    LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
+    BWD_OK(simt_project(p, items, lengths, cands, Wq, Wk, Wv, ws, st));
+    BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
+    if (sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, mma_scratch, st));
+    else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
+    else if (p.dqh == 16 && dvh == 32 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
+    else BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
+  } else if (p.dqh == 16 && (dvh == 16 || dvh == 32) && p.H <= 32) {
     // (a candidate tile of a user with more candidates than max_cands_per_user declares would stay unwritten: zero first)
     LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
     BWD_OK(simt_project(p, items, lengths, cands, Wq, Wk, Wv, ws, st));
@@ -746,7 +755,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dK, 0, UL * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
   if (tensor) {
-    BWD_OK(sta_bwd_mma(p, Qf, Kf, Vf, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, ws + p.total + s.total, st));
+    BWD_OK(sta_bwd_mma(p, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, mma_scratch, st));
   } else {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
     const int dqh = dqk / H;

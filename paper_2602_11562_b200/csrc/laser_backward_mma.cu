@@ -288,6 +288,104 @@ __global__ void __launch_bounds__(kBwdWarps * 32) sta_bwd_mma_kernel(const BwdMm
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------------
+// The recomputed forward of the same step, H'[c, seg, h] = sum_n g[c, n] v_n (Eq. 10-12), with the same bf16 operands: one
+// block per (user, segment, head) stages the segment's K_h and V_h rows in shared memory (zero rows up to a multiple of 16)
+// and its warps take the user's candidates 16 at a time: scores = Qb K_h^T per 16 items, gates from the accumulator layout
+// straight into the A operand of g V_h.  Output fp32 (what the GSTA backward reads).
+struct FwdMmaParams {
+  const bf16 *Qb, *Kb, *Vb;
+  const int32_t *lengths, *cand_offsets;
+  float* Hp;
+  int L, d, dqk, H, S, Lp, N, rows;              // rows = staged rows per block (min(S, L) rounded up to 16)
+};
+
+template <int DQ16, int DV16>
+__global__ void __launch_bounds__(kBwdWarps * 32) sta_fwd_mma_kernel(const FwdMmaParams P) {
+  constexpr int DQH = 16 * DQ16, DVH = 16 * DV16;
+  constexpr int KS = 2 * DQH + 16, VS = 2 * DVH + 16;          // bytes per staged row
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int u = blockIdx.y, seg = blockIdx.x / P.H, h = blockIdx.x - seg * P.H;
+  const int len = P.lengths[u], off0 = P.cand_offsets[u], off1 = P.cand_offsets[u + 1];
+  if (len <= 0 || len > P.L || off0 < 0 || off1 <= off0 || off1 > P.N) return;
+  const int C = off1 - off0;
+  const int n0 = seg * P.S, n_end = min(min((seg + 1) * P.S, P.L), len);
+  if (n0 >= n_end) return;
+  const int cnt = n_end - n0, chunks = (cnt + 15) >> 4, d = P.d, dqk = P.dqk;
+  const uint32_t Ksm = smem_addr(smem), Vsm = Ksm + P.rows * KS;
+  {
+    const bf16* Kr = P.Kb + ((size_t)u * P.L + n0) * dqk + h * DQH;
+    const bf16* Vr = P.Vb + ((size_t)u * P.L + n0) * d + h * DVH;
+    for (int x = tid; x < chunks * 16 * 2 * DQ16; x += kBwdWarps * 32) {
+      const int row = x / (2 * DQ16), ch = x - row * (2 * DQ16);
+      cp16(Ksm + row * KS + ch * 16, Kr + (size_t)min(row, cnt - 1) * dqk + ch * 8, row < cnt ? 16u : 0u);
+    }
+    for (int x = tid; x < chunks * 16 * 2 * DV16; x += kBwdWarps * 32) {
+      const int row = x / (2 * DV16), ch = x - row * (2 * DV16);
+      cp16(Vsm + row * VS + ch * 16, Vr + (size_t)min(row, cnt - 1) * d + ch * 8, row < cnt ? 16u : 0u);
+    }
+    cp_commit();
+    cp_wait<0>();
+    __syncthreads();
+  }
+  const int mi = lane >> 3, lr = lane & 7;
+  const uint32_t k_plain = Ksm + ((mi >> 1) * 8 + lr) * KS + (mi & 1) * 16;      // B(k = key component, n = item)
+  const uint32_t v_trans = Vsm + ((mi & 1) * 8 + lr) * VS + (mi >> 1) * 16;      // B(k = item, n = value component)
+  const bf16* Qg = P.Qb + (size_t)off0 * dqk + h * DQH;
+  for (int c0 = warp * 16; c0 < C; c0 += kBwdWarps * 16) {
+    uint32_t Qa[DQ16][4];
+    const int r0 = c0 + g, r1 = r0 + 8;
+#pragma unroll
+    for (int k = 0; k < DQ16; ++k) {
+      const int c = k * 16 + 2 * t;
+      Qa[k][0] = r0 < C ? *reinterpret_cast<const uint32_t*>(Qg + (size_t)r0 * dqk + c) : 0u;
+      Qa[k][1] = r1 < C ? *reinterpret_cast<const uint32_t*>(Qg + (size_t)r1 * dqk + c) : 0u;
+      Qa[k][2] = r0 < C ? *reinterpret_cast<const uint32_t*>(Qg + (size_t)r0 * dqk + c + 8) : 0u;
+      Qa[k][3] = r1 < C ? *reinterpret_cast<const uint32_t*>(Qg + (size_t)r1 * dqk + c + 8) : 0u;
+    }
+    float acc[2 * DV16][4];
+#pragma unroll
+    for (int j = 0; j < 2 * DV16; ++j)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
+    for (int ic = 0; ic < chunks; ++ic) {
+      float E[2][4] = {};
+#pragma unroll
+      for (int k = 0; k < DQ16; ++k) {
+        uint32_t b[4];
+        ldsm_x4(b, k_plain + ic * 16 * KS + k * 32);
+        mma16816(E[0], Qa[k][0], Qa[k][1], Qa[k][2], Qa[k][3], b[0], b[1]);
+        mma16816(E[1], Qa[k][0], Qa[k][1], Qa[k][2], Qa[k][3], b[2], b[3]);
+      }
+      uint32_t gA[4];
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        float gg[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) gg[e] = fmaf(tanh_fast(E[nt][e]), 0.5f, 0.5f);
+        gA[2 * nt] = pack2(gg[0], gg[1]);
+        gA[2 * nt + 1] = pack2(gg[2], gg[3]);
+      }
+#pragma unroll
+      for (int k = 0; k < DV16; ++k) {
+        uint32_t b[4];
+        ldsm_x4_t(b, v_trans + ic * 16 * VS + k * 32);
+        mma16816(acc[2 * k], gA[0], gA[1], gA[2], gA[3], b[0], b[1]);
+        mma16816(acc[2 * k + 1], gA[0], gA[1], gA[2], gA[3], b[2], b[3]);
+      }
+    }
+    float* out = P.Hp + ((size_t)off0 * P.Lp + seg) * d + h * DVH;
+    const size_t row = (size_t)P.Lp * d;
+#pragma unroll
+    for (int j = 0; j < 2 * DV16; ++j) {
+      const int c = j * 8 + 2 * t;
+      if (r0 < C) *reinterpret_cast<float2*>(out + (size_t)r0 * row + c) = make_float2(acc[j][0], acc[j][1]);
+      if (r1 < C) *reinterpret_cast<float2*>(out + (size_t)r1 * row + c) = make_float2(acc[j][2], acc[j][3]);
+    }
+  }
+}
+
 struct MmaShape {
   int mt, dq16, dv16;
 };
@@ -306,6 +404,22 @@ int launch_mma(const BwdMmaParams& P, int U, cudaStream_t st) {
   LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   LaunchScope ls("bwd_sta_mma", st);
   kernel<<<dim3((P.jobs + kBwdWarps - 1) / kBwdWarps, U), kBwdWarps * 32, smem, st>>>(P);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+constexpr size_t kFwdSmemMax = 160 * 1024;
+size_t fwd_smem(const Plan& p) {
+  const size_t rows = (size_t)(std::min(p.S, p.L) + 15) / 16 * 16;
+  return rows * (2 * p.dqh + 16 + 2 * p.dvh + 16);
+}
+
+template <int DQ16, int DV16>
+int launch_fwd(const FwdMmaParams& P, int U, size_t smem, cudaStream_t st) {
+  auto kernel = sta_fwd_mma_kernel<DQ16, DV16>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LaunchScope ls("bwd_sta_fwd_mma", st);
+  kernel<<<dim3(P.Lp * P.H, U), kBwdWarps * 32, smem, st>>>(P);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
 }
@@ -352,17 +466,45 @@ bool sta_bwd_mma_supported(const Plan& p) {
 
 size_t sta_bwd_mma_scratch_bytes(const Plan& p) { return sta_bwd_mma_supported(p) ? carve_mma(p, nullptr).total : 0; }
 
-int sta_bwd_mma(const Plan& p, const float* Qf, const float* Kf, const float* Vf, const float* dHp,
-                const int32_t* lengths, const int32_t* cand_offsets, float* dQf, float* dK, float* dV, char* scratch,
-                cudaStream_t st) {
-  MmaShape sh;
-  if (!mma_shape(p, &sh)) return LASER_ERR_UNSUPPORTED;
+int sta_mma_operands(const Plan& p, const float* Qf, const float* Kf, const float* Vf, char* scratch, cudaStream_t st) {
   const MmaScratch s = carve_mma(p, scratch);
   const size_t UL = (size_t)p.U * p.L;
   int rc;
   if ((rc = cast(Qf, s.Qb, (size_t)p.N * p.dqk, 0.5f, st)) != LASER_OK) return rc;
   if ((rc = cast(Kf, s.Kb, UL * p.dqk, 1.f, st)) != LASER_OK) return rc;
-  if ((rc = cast(Vf, s.Vb, UL * p.d, 1.f, st)) != LASER_OK) return rc;
+  return cast(Vf, s.Vb, UL * p.d, 1.f, st);
+}
+
+bool sta_fwd_mma_supported(const Plan& p) {
+  return sta_bwd_mma_supported(p) && fwd_smem(p) <= kFwdSmemMax && (long long)p.Lp * p.H <= 0x7fffffffLL;
+}
+
+int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, char* scratch,
+                cudaStream_t st) {
+  MmaShape sh;
+  if (!mma_shape(p, &sh) || !sta_fwd_mma_supported(p)) return LASER_ERR_UNSUPPORTED;
+  const MmaScratch s = carve_mma(p, scratch);
+  FwdMmaParams P;
+  P.Qb = s.Qb; P.Kb = s.Kb; P.Vb = s.Vb;
+  P.lengths = lengths; P.cand_offsets = cand_offsets;
+  P.Hp = Hp;
+  P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
+  P.rows = (std::min(p.S, p.L) + 15) / 16 * 16;
+  const size_t smem = fwd_smem(p);
+#define LASER_FWD_CASE(DQ, DV) \
+  if (sh.dq16 == DQ && sh.dv16 == DV) return launch_fwd<DQ, DV>(P, p.U, smem, st);
+  LASER_FWD_CASE(1, 1) LASER_FWD_CASE(1, 2) LASER_FWD_CASE(1, 4)
+  LASER_FWD_CASE(2, 1) LASER_FWD_CASE(2, 2) LASER_FWD_CASE(2, 4)
+#undef LASER_FWD_CASE
+  return LASER_ERR_UNSUPPORTED;
+}
+
+int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const int32_t* cand_offsets, float* dQf,
+                float* dK, float* dV, char* scratch, cudaStream_t st) {
+  MmaShape sh;
+  if (!mma_shape(p, &sh)) return LASER_ERR_UNSUPPORTED;
+  const MmaScratch s = carve_mma(p, scratch);
+  int rc;
   if ((rc = cast(dHp, s.dSb, (size_t)p.N * p.Lp * p.d, 1.f, st)) != LASER_OK) return rc;
   BwdMmaParams P;
   P.Qb = s.Qb; P.Kb = s.Kb; P.Vb = s.Vb; P.dSb = s.dSb;

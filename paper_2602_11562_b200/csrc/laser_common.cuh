@@ -86,14 +86,18 @@ bool backward_tensor_supported(const Plan& p);
 int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
              const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,
              float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor);
-// Tensor-core backward through the segment aggregation and the gates (laser_backward_mma.cu): bf16 copies of Qf (Q / gamma),
-// Kf, Vf and dHp are made in `scratch` (sta_bwd_mma_scratch_bytes), dK / dV rows of valid items are written (the rest must
-// hold zeros), dQf is added to.
+// Tensor-core kernels of the backward pass (laser_backward_mma.cu), all on bf16 copies kept in `scratch`
+// (sta_bwd_mma_scratch_bytes): sta_mma_operands makes the copies of Qf (Q / gamma), Kf and Vf; sta_fwd_mma recomputes H'
+// in fp32 from them (rows of empty segments are left as they are); sta_bwd_mma copies dHp, writes the dK / dV rows of
+// valid items (the rest must hold zeros) and adds to dQf.
 bool sta_bwd_mma_supported(const Plan& p);
+bool sta_fwd_mma_supported(const Plan& p);
 size_t sta_bwd_mma_scratch_bytes(const Plan& p);
-int sta_bwd_mma(const Plan& p, const float* Qf, const float* Kf, const float* Vf, const float* dHp,
-                const int32_t* lengths, const int32_t* cand_offsets, float* dQf, float* dK, float* dV, char* scratch,
+int sta_mma_operands(const Plan& p, const float* Qf, const float* Kf, const float* Vf, char* scratch, cudaStream_t st);
+int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, char* scratch,
                 cudaStream_t st);
+int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const int32_t* cand_offsets, float* dQf,
+                float* dK, float* dV, char* scratch, cudaStream_t st);
 
 bool tensor_supported(const Plan& p);
 void tensor_geometry(const Plan& p, TensorGeom* g);
