@@ -27,16 +27,22 @@ using bf16 = __nv_bfloat16;
 // ------------------------------------------------------------------------------------------------ batched products
 // C[m][n] (+)= alpha * sum_k A(m, k) B(k, n);  A(m, k) = ta ? A[k lda + m] : A[m lda + k],  B(k, n) = tb ? B[n ldb + k]
 // : B[k ldb + n].  64 x 64 tiles of C, k-steps of 16; gridDim.z splits K and the partial sums are added atomically
-// (C then has to hold its initial value before the launch).
+// (C then has to hold its initial value before the launch).  `batch` independent products of the same shape (one per
+// head) go out in one launch: product b reads A + b sa, B + b sb and writes C + b sc.
 constexpr int kTM = 64, kTN = 64, kTK = 16, kGemmThreads = 256;
 
 template <typename TA, typename TB>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
-            float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split) {
+            float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split, int tiles_n, int sa, int sb,
+            int sc) {
   __shared__ __align__(16) float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int m0 = blockIdx.x * kTM, n0 = blockIdx.y * kTN;       // (row tiles on grid.x: there may be millions of rows)
+  const int batch = blockIdx.y / tiles_n;                       // independent products: operands sa, sb, sc elements apart
+  A += (size_t)batch * sa;
+  B += (size_t)batch * sb;
+  C += (size_t)batch * sc;
+  const int m0 = blockIdx.x * kTM, n0 = (blockIdx.y - batch * tiles_n) * kTN;   // (row tiles on grid.x: there may be millions of rows)
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
   float acc[4][4] = {};
   for (int k0 = k_lo; k0 < k_hi; k0 += kTK) {
@@ -148,10 +154,15 @@ __device__ __forceinline__ void stage_tile(uint32_t* __restrict__ sm, const TX* 
 template <typename TA, typename TB>
 __global__ void __launch_bounds__(kGemmThreads)
 gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
-                 float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split, int aligned_a, int aligned_b) {
+                 float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split, int aligned_a, int aligned_b,
+                 int tiles_n, int sa, int sb, int sc) {
   __shared__ __align__(16) uint32_t As[kStage], Bs[kStage];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int m0 = blockIdx.x * 64, n0 = blockIdx.y * 64;
+  const int batch = blockIdx.y / tiles_n;
+  A += (size_t)batch * sa;
+  B += (size_t)batch * sb;
+  C += (size_t)batch * sc;
+  const int m0 = blockIdx.x * 64, n0 = (blockIdx.y - batch * tiles_n) * 64;
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
   const int wm = (warp >> 2) * 32, wn = (warp & 3) * 16;
   // element offsets of this lane's fragment entries: A(m, k) with m = wm + g, k = t;  B(k, n) with k = t, n = wn + g
@@ -214,8 +225,8 @@ bool aligned_for_vector_loads(const TX* X, int ld) {
 
 template <typename TA, typename TB>
 int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, const TB* B, int ldb, bool tb, float* C,
-         int ldc, float alpha, bool accumulate, bool split_k) {
-  if (M <= 0 || N <= 0 || K <= 0) return LASER_OK;
+         int ldc, float alpha, bool accumulate, bool split_k, int batch = 1, int sa = 0, int sb = 0, int sc = 0) {
+  if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return LASER_OK;
   cudaStream_t st = gx.st;
   const int kstep = gx.tf32 ? kWK : kTK;
   int splits = 1, per = K;
@@ -224,16 +235,18 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
     splits = (K + per - 1) / per;
     if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kstep - 1) / kstep * kstep; splits = (K + per - 1) / per; }
   }
-  const dim3 grid((M + kTM - 1) / kTM, (N + kTN - 1) / kTN, splits);
-  if (grid.y > 65535) return LASER_ERR_UNSUPPORTED;
+  const int tiles_n = (N + kTN - 1) / kTN;
+  if ((long long)tiles_n * batch > 65535) return LASER_ERR_UNSUPPORTED;
+  const dim3 grid((M + kTM - 1) / kTM, tiles_n * batch, splits);
   LaunchScope ls(gx.tf32 ? "bwd_gemm_tf32" : "bwd_gemm", st);
   if (gx.tf32)
-    gemm_tf32_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
-                                                           accumulate ? 1 : 0, per, aligned_for_vector_loads(A, lda) ? 1 : 0,
-                                                           aligned_for_vector_loads(B, ldb) ? 1 : 0);
+    gemm_tf32_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(
+        M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha, accumulate ? 1 : 0, per,
+        aligned_for_vector_loads(A, lda) && sa % 4 == 0 ? 1 : 0, aligned_for_vector_loads(B, ldb) && sb % 4 == 0 ? 1 : 0,
+        tiles_n, sa, sb, sc);
   else
     gemm_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(M, N, K, A, lda, ta ? 1 : 0, B, ldb, tb ? 1 : 0, C, ldc, alpha,
-                                                      accumulate ? 1 : 0, per);
+                                                      accumulate ? 1 : 0, per, tiles_n, sa, sb, sc);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
 }
@@ -705,18 +718,16 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     float *Tl = s.T + l * Nd, *Tn = Tl + Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
           *Ml = s.Mh + l * NHd;
     BWD_OK(gemm<float, T>(gx, N, d, d, Tl, d, false, Wql, d, false, Ql, d, 1.f, false, false));
-    for (int h = 0; h < H; ++h)
-      BWD_OK(gemm<float, T>(gx, N, d, dvh, Ql + h * dvh, d, false, Wkl + h * dvh, d, true, Qtl + (size_t)h * d, H * d,
-                            p.inv_tau, false, false));
+    // Qt_h = Q_h W_k[:, h]^T / tau, every head
+    BWD_OK(gemm<float, T>(gx, N, d, dvh, Ql, d, false, Wkl, d, true, Qtl, H * d, p.inv_tau, false, false, H, dvh, dvh, d));
     {
       LaunchScope ls("bwd_attn_fwd", st);
       gsta_attn_fwd_kernel<<<N, kAttnThreads, attn_smem_f, st>>>(s.Hp, Qtl, lengths, cand_offsets, Al, Ml, U, L, p.S, Lp,
                                                                  H, d);
     }
     LASER_CUDA_OK(cudaMemcpyAsync(Tn, Tl, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    for (int h = 0; h < H; ++h)
-      BWD_OK(gemm<float, T>(gx, N, dvh, d, Ml + (size_t)h * d, H * d, false, Wvl + h * dvh, d, false, Tn + h * dvh, d, 1.f,
-                            true, false));
+    // t += o,  o_h = m_h W_v[:, h], every head
+    BWD_OK(gemm<float, T>(gx, N, dvh, d, Ml, H * d, false, Wvl, d, false, Tn, d, 1.f, true, false, H, d, dvh, dvh));
   }
 
   // ---- backward through the GSTA layers
@@ -727,25 +738,17 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     float *Tl = s.T + l * Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
           *Ml = s.Mh + l * NHd;
     float *gWq = dWg + (size_t)(l * 3) * d * d, *gWk = gWq + (size_t)d * d, *gWv = gWk + (size_t)d * d;
-    for (int h = 0; h < H; ++h) {
-      // dW_v[:, h] += m_h^T do_h;  dm_h = do_h W_v[:, h]^T
-      BWD_OK(gemm<float, float>(gx, d, dvh, N, Ml + (size_t)h * d, H * d, true, s.dT + h * dvh, d, false, gWv + h * dvh, d,
-                                1.f, true, true));
-      BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT + h * dvh, d, false, Wvl + h * dvh, d, true, s.dM + (size_t)h * d, H * d,
-                            1.f, false, false));
-    }
+    // dW_v[:, h] += m_h^T do_h;  dm_h = do_h W_v[:, h]^T, every head
+    BWD_OK(gemm<float, float>(gx, d, dvh, N, Ml, H * d, true, s.dT, d, false, gWv, d, 1.f, true, true, H, d, dvh, dvh));
+    BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT, d, false, Wvl, d, true, s.dM, H * d, 1.f, false, false, H, dvh, dvh, d));
     {
       LaunchScope ls("bwd_attn_bwd", st);
       gsta_attn_bwd_kernel<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
                                                                  U, L, p.S, Lp, H, d);
     }
-    for (int h = 0; h < H; ++h) {
-      // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau
-      BWD_OK(gemm<float, T>(gx, N, dvh, d, s.dQt + (size_t)h * d, H * d, false, Wkl + h * dvh, d, false, s.dQ + h * dvh, d,
-                            p.inv_tau, false, false));
-      BWD_OK(gemm<float, float>(gx, d, dvh, N, s.dQt + (size_t)h * d, H * d, true, Ql + h * dvh, d, false, gWk + h * dvh, d,
-                                p.inv_tau, true, true));
-    }
+    // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau, every head
+    BWD_OK(gemm<float, T>(gx, N, dvh, d, s.dQt, H * d, false, Wkl, d, false, s.dQ, d, p.inv_tau, false, false, H, d, dvh, dvh));
+    BWD_OK(gemm<float, float>(gx, d, dvh, N, s.dQt, H * d, true, Ql, d, false, gWk, d, p.inv_tau, true, true, H, d, dvh, dvh));
     BWD_OK(gemm<float, float>(gx, d, d, N, Tl, d, true, s.dQ, d, false, gWq, d, 1.f, true, true));        // dW_q += T^T dQ
     BWD_OK(gemm<float, T>(gx, N, d, d, s.dQ, d, false, Wql, d, true, s.dT, d, 1.f, true, false));            // dT += dQ W_q^T
   }
