@@ -296,13 +296,21 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   const float* s = Hp + (size_t)c * Lp * d;
   for (int i = tid; i < H * d; i += kAttnThreads) qt[i] = Qt[(size_t)c * H * d + i];
   __syncthreads();
-  for (int p = warp; p < nv * H; p += nw) {
-    const int j = p / H, h = p - j * H;
-    float dot = 0.f;
-    for (int x = lane; x < d; x += 32) dot = fmaf(s[(size_t)j * d + x], qt[h * d + x], dot);
-    dot = warp_sum(dot);
-    if (lane == 0) e[h * Lp + j] = dot;
-  }
+  for (int j = warp; j < nv; j += nw)                        // a warp takes segment vector j against four heads at a time
+    for (int h0 = 0; h0 < H; h0 += 4) {
+      float dot[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int x = lane; x < d; x += 32) {
+        const float sv = s[(size_t)j * d + x];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (h0 + k < H) dot[k] = fmaf(sv, qt[(h0 + k) * d + x], dot[k]);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (lane == 0 && h0 + k < H) e[(h0 + k) * Lp + j] = dot[k];
+    }
   __syncthreads();
   for (int h = warp; h < H; h += nw) {
     float mx = -INFINITY;
@@ -340,11 +348,13 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
 }
 
 // One block per candidate: the backward of the kernel above.  dM = dLoss/dm [N, H, d] in; dQt = dLoss/dQt [N, H, d] out;
-// dHp [N, Lp, d] accumulates dLoss/ds_j over the layers.
+// dHp [N, Lp, d] accumulates dLoss/ds_j over the layers: the layer processed first (overwrite != 0) writes every entry
+// (zeros for the empty segments), the others add.
 __global__ void __launch_bounds__(kAttnThreads)
 gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const float* __restrict__ Aw,
                      const float* __restrict__ dM, const int* __restrict__ lengths, const int* __restrict__ cand_offsets,
-                     float* __restrict__ dQt, float* __restrict__ dHp, int U, int L, int S, int Lp, int H, int d) {
+                     float* __restrict__ dQt, float* __restrict__ dHp, int U, int L, int S, int Lp, int H, int d,
+                     int overwrite) {
   extern __shared__ float sm[];
   float* qt = sm;                 // [H][d]
   float* dm = qt + H * d;         // [H][d]
@@ -359,13 +369,21 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   }
   for (int i = tid; i < H * Lp; i += kAttnThreads) a[i] = Aw[(size_t)c * H * Lp + i];
   __syncthreads();
-  for (int p = warp; p < nv * H; p += nw) {
-    const int j = p / H, h = p - j * H;
-    float dot = 0.f;
-    for (int x = lane; x < d; x += 32) dot = fmaf(s[(size_t)j * d + x], dm[h * d + x], dot);
-    dot = warp_sum(dot);
-    if (lane == 0) de[h * Lp + j] = dot;
-  }
+  for (int j = warp; j < nv; j += nw)
+    for (int h0 = 0; h0 < H; h0 += 4) {
+      float dot[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int x = lane; x < d; x += 32) {
+        const float sv = s[(size_t)j * d + x];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (h0 + k < H) dot[k] = fmaf(sv, dm[(h0 + k) * d + x], dot[k]);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (lane == 0 && h0 + k < H) de[(h0 + k) * Lp + j] = dot[k];
+    }
   __syncthreads();
   for (int h = warp; h < H; h += nw) {
     float dotp = 0.f;
@@ -382,6 +400,7 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
         qx[k] = h0 + k < H ? qt[(h0 + k) * d + x] : 0.f;
         mx[k] = h0 + k < H ? dm[(h0 + k) * d + x] : 0.f;
       }
+#pragma unroll 4
       for (int j = 0; j < nv; ++j) {
         const float sv = s[(size_t)j * d + x];
         float g = 0.f;
@@ -393,8 +412,11 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
             g += dej * qx[k] + a[(h0 + k) * Lp + j] * mx[k];
           }
         }
-        dHp[((size_t)c * Lp + j) * d + x] += g;
+        float* out = dHp + ((size_t)c * Lp + j) * d + x;
+        *out = (overwrite && h0 == 0) ? g : *out + g;
       }
+      if (overwrite && h0 == 0)
+        for (int j = nv; j < Lp; ++j) dHp[((size_t)c * Lp + j) * d + x] = 0.f;      // empty segments receive no gradient
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (h0 + k < H) dQt[((size_t)c * H + h0 + k) * d + x] = acc[k];
@@ -732,7 +754,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 
   // ---- backward through the GSTA layers
   LASER_CUDA_OK(cudaMemcpyAsync(s.dT, dz, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
-  LASER_CUDA_OK(cudaMemsetAsync(s.dHp, 0, (size_t)N * Lp * d * sizeof(float), st));
+  if (M == 0) LASER_CUDA_OK(cudaMemsetAsync(s.dHp, 0, (size_t)N * Lp * d * sizeof(float), st));
   for (int l = M - 1; l >= 0; --l) {
     const T *Wql = Wg + (size_t)(l * 3) * d * d, *Wkl = Wql + (size_t)d * d, *Wvl = Wkl + (size_t)d * d;
     float *Tl = s.T + l * Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
@@ -744,7 +766,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     {
       LaunchScope ls("bwd_attn_bwd", st);
       gsta_attn_bwd_kernel<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
-                                                                 U, L, p.S, Lp, H, d);
+                                                                 U, L, p.S, Lp, H, d, l == M - 1 ? 1 : 0);
     }
     // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau, every head
     BWD_OK(gemm<float, T>(gx, N, dvh, d, s.dQt, H * d, false, Wkl, d, false, s.dQ, d, p.inv_tau, false, false, H, d, dvh, dvh));
