@@ -104,14 +104,27 @@ __device__ __forceinline__ uint32_t tf32_of(float v) {
   asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
   return r;
 }
-__device__ __forceinline__ uint4 load4_tf32(const float* p) {
-  const float4 v = *reinterpret_cast<const float4*>(p);
-  return make_uint4(tf32_of(v.x), tf32_of(v.y), tf32_of(v.z), tf32_of(v.w));
-}
-__device__ __forceinline__ uint4 load4_tf32(const bf16* p) {
+// Raw bits of four consecutive elements (fp32: four words; bf16: two words) and of one element, as they come from
+// memory, and their TF32 operand form.  Loading and converting are separate steps so that a tile fetched ahead costs no
+// wait until it is stored to shared memory.
+__device__ __forceinline__ uint4 raw4(const float* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ uint4 raw4(const bf16* p) {
   const uint2 v = *reinterpret_cast<const uint2*>(p);
-  return make_uint4(v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u);
+  return make_uint4(v.x, v.y, 0u, 0u);
 }
+__device__ __forceinline__ uint32_t raw1(const float* p) { return __float_as_uint(*p); }
+__device__ __forceinline__ uint32_t raw1(const bf16* p) { return *reinterpret_cast<const unsigned short*>(p); }
+template <typename TX> __device__ __forceinline__ uint4 tf32_of4(uint4 r);
+template <> __device__ __forceinline__ uint4 tf32_of4<float>(uint4 r) {
+  return make_uint4(tf32_of(__uint_as_float(r.x)), tf32_of(__uint_as_float(r.y)), tf32_of(__uint_as_float(r.z)),
+                    tf32_of(__uint_as_float(r.w)));
+}
+template <> __device__ __forceinline__ uint4 tf32_of4<bf16>(uint4 r) {
+  return make_uint4(r.x << 16, r.x & 0xFFFF0000u, r.y << 16, r.y & 0xFFFF0000u);
+}
+template <typename TX> __device__ __forceinline__ uint32_t tf32_of1(uint32_t r);
+template <> __device__ __forceinline__ uint32_t tf32_of1<float>(uint32_t r) { return tf32_of(__uint_as_float(r)); }
+template <> __device__ __forceinline__ uint32_t tf32_of1<bf16>(uint32_t r) { return r << 16; }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -119,40 +132,57 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Stages a 64 x kWK tile of an operand X with rows r0 .. (bound R) and contraction indices k0 .. (bound k_hi):
-// X(r, k) = k_major ? X[k ld + r] : X[r ld + k].  Shared layout: k_major ? [k][kColLd] : [r][kRowLd].
+// A 64 x kWK tile of an operand X, rows r0 .. (bound R), contraction indices k0 .. (bound k_hi), with
+// X(r, k) = k_major ? X[k ld + r] : X[r ld + k], travels in two steps so that the global loads of the next tile are in
+// flight while the current one is multiplied: fetch_tile brings a thread's eight elements into registers as they are,
+// put_tile rounds them to TF32 and stores them.  Shared layout: k_major ? [k][kColLd] : [r][kRowLd].  Full, aligned tiles move as two
+// 16-byte (fp32) or 8-byte (bf16) loads and two 16-byte stores per thread, the others element by element.
+__device__ __forceinline__ bool tile_is_full(bool aligned, int r0, int R, int k0, int k_hi) {
+  return aligned && r0 + 64 <= R && k0 + kWK <= k_hi;
+}
 template <typename TX>
-__device__ __forceinline__ void stage_tile(uint32_t* __restrict__ sm, const TX* __restrict__ X, int ld, int k_major, int r0,
-                                           int R, int k0, int k_hi, bool aligned, int tid) {
-  const bool full = aligned && r0 + 64 <= R && k0 + kWK <= k_hi;
-  if (full) {
-    if (k_major) {
+__device__ __forceinline__ void fetch_tile(uint32_t (&v)[8], const TX* __restrict__ X, int ld, int k_major, int r0, int R,
+                                           int k0, int k_hi, bool aligned, int tid) {
+  if (tile_is_full(aligned, r0, R, k0, k_hi)) {
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int i = tid + kGemmThreads * j, kk = i >> 4, r4 = (i & 15) * 4;
-        *reinterpret_cast<uint4*>(sm + kk * kColLd + r4) = load4_tf32(X + (size_t)(k0 + kk) * ld + r0 + r4);
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        const int i = tid + kGemmThreads * j, rr = i >> 3, k4 = (i & 7) * 4;
-        *reinterpret_cast<uint4*>(sm + rr * kRowLd + k4) = load4_tf32(X + (size_t)(r0 + rr) * ld + k0 + k4);
-      }
+    for (int j = 0; j < 2; ++j) {
+      const int i = tid + kGemmThreads * j;
+      const TX* src = k_major ? X + (size_t)(k0 + (i >> 4)) * ld + r0 + (i & 15) * 4
+                              : X + (size_t)(r0 + (i >> 3)) * ld + k0 + (i & 7) * 4;
+      const uint4 q = raw4(src);
+      v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
     }
     return;
   }
-  for (int i = tid; i < 64 * kWK; i += kGemmThreads) {
-    int rr, kk;
-    if (k_major) { kk = i >> 6; rr = i & 63; } else { rr = i / kWK; kk = i - rr * kWK; }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int i = tid + kGemmThreads * e;
+    const int rr = k_major ? (i & 63) : (i / kWK), kk = k_major ? (i >> 6) : (i % kWK);
     const int r = r0 + rr, k = k0 + kk;
-    float v = 0.f;
-    if (r < R && k < k_hi) v = to_f32<TX>(k_major ? X[(size_t)k * ld + r] : X[(size_t)r * ld + k]);
-    sm[k_major ? kk * kColLd + rr : rr * kRowLd + kk] = tf32_of(v);
+    v[e] = (r < R && k < k_hi) ? raw1(k_major ? X + (size_t)k * ld + r : X + (size_t)r * ld + k) : 0u;
+  }
+}
+template <typename TX>
+__device__ __forceinline__ void put_tile(uint32_t* __restrict__ sm, const uint32_t (&v)[8], int k_major, bool full, int tid) {
+  if (full) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int i = tid + kGemmThreads * j;
+      uint32_t* dst = k_major ? sm + (i >> 4) * kColLd + (i & 15) * 4 : sm + (i >> 3) * kRowLd + (i & 7) * 4;
+      *reinterpret_cast<uint4*>(dst) = tf32_of4<TX>(make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]));
+    }
+    return;
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int i = tid + kGemmThreads * e;
+    const int rr = k_major ? (i & 63) : (i / kWK), kk = k_major ? (i >> 6) : (i % kWK);
+    sm[k_major ? kk * kColLd + rr : rr * kRowLd + kk] = tf32_of1<TX>(v[e]);
   }
 }
 
 template <typename TA, typename TB>
-__global__ void __launch_bounds__(kGemmThreads)
+__global__ void __launch_bounds__(kGemmThreads, 2)
 gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, const TB* __restrict__ B, int ldb, int tb,
                  float* __restrict__ C, int ldc, float alpha, int accumulate, int k_per_split, int aligned_a, int aligned_b,
                  int tiles_n, int sa, int sb, int sc) {
@@ -169,10 +199,17 @@ gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta,
   const int a_m = ta ? 1 : kRowLd, a_k = ta ? kColLd : 1, b_n = tb ? kRowLd : 1, b_k = tb ? 1 : kColLd;
   const int a_off = (wm + g) * a_m + t * a_k, b_off = (wn + g) * b_n + t * b_k;
   float acc[2][2][4] = {};
+  uint32_t va[8], vb[8];                  // A(m, k): k-major storage when transposed;  B(k, n): k-major when NOT transposed
+  fetch_tile<TA>(va, A, lda, ta, m0, M, k_lo, k_hi, aligned_a != 0, tid);
+  fetch_tile<TB>(vb, B, ldb, !tb, n0, N, k_lo, k_hi, aligned_b != 0, tid);
   for (int k0 = k_lo; k0 < k_hi; k0 += kWK) {
-    stage_tile<TA>(As, A, lda, ta, m0, M, k0, k_hi, aligned_a != 0, tid);      // A(m, k): k-major storage when transposed
-    stage_tile<TB>(Bs, B, ldb, !tb, n0, N, k0, k_hi, aligned_b != 0, tid);     // B(k, n): k-major storage when NOT transposed
+    put_tile<TA>(As, va, ta, tile_is_full(aligned_a != 0, m0, M, k0, k_hi), tid);
+    put_tile<TB>(Bs, vb, !tb, tile_is_full(aligned_b != 0, n0, N, k0, k_hi), tid);
     __syncthreads();
+    if (k0 + kWK < k_hi) {
+      fetch_tile<TA>(va, A, lda, ta, m0, M, k0 + kWK, k_hi, aligned_a != 0, tid);
+      fetch_tile<TB>(vb, B, ldb, !tb, n0, N, k0 + kWK, k_hi, aligned_b != 0, tid);
+    }
 #pragma unroll
     for (int kb = 0; kb < kWK; kb += 8) {
       uint32_t a[2][4], b[2][2];
@@ -231,7 +268,9 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
   const int kstep = gx.tf32 ? kWK : kTK;
   int splits = 1, per = K;
   if (split_k) {                     // reductions over many rows into a small matrix (C must hold its initial value)
-    per = 256;
+    // slices of at least 256 rows, longer when that still leaves about four blocks per SM (fewer atomic adds per product)
+    const long long tiles = (long long)((M + kTM - 1) / kTM) * ((N + kTN - 1) / kTN) * batch;
+    per = (int)std::min<long long>(std::max<long long>(256, ((long long)K * tiles / 592 + 31) / 32 * 32), 1 << 20);
     splits = (K + per - 1) / per;
     if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kstep - 1) / kstep * kstep; splits = (K + per - 1) / per; }
   }
