@@ -38,11 +38,12 @@ gemm_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta, cons
             int sc) {
   __shared__ __align__(16) float As[kTK][kTM + 4], Bs[kTK][kTN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int batch = blockIdx.y / tiles_n;                       // independent products: operands sa, sb, sc elements apart
+  const int batch = blockIdx.y;                                 // independent products: operands sa, sb, sc elements apart
   A += (size_t)batch * sa;
   B += (size_t)batch * sb;
   C += (size_t)batch * sc;
-  const int m0 = blockIdx.x * kTM, n0 = (blockIdx.y - batch * tiles_n) * kTN;   // (row tiles on grid.x: there may be millions of rows)
+  // grid.x enumerates the tiles of C with the column tile running fastest: blocks that share a row tile of A run together
+  const int tile_m = blockIdx.x / tiles_n, m0 = tile_m * kTM, n0 = (blockIdx.x - tile_m * tiles_n) * kTN;
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
   float acc[4][4] = {};
   for (int k0 = k_lo; k0 < k_hi; k0 += kTK) {
@@ -188,11 +189,11 @@ gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta,
                  int tiles_n, int sa, int sb, int sc) {
   __shared__ __align__(16) uint32_t As[kStage], Bs[kStage];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int batch = blockIdx.y / tiles_n;
+  const int batch = blockIdx.y;
   A += (size_t)batch * sa;
   B += (size_t)batch * sb;
   C += (size_t)batch * sc;
-  const int m0 = blockIdx.x * 64, n0 = (blockIdx.y - batch * tiles_n) * 64;
+  const int tile_m = blockIdx.x / tiles_n, m0 = tile_m * 64, n0 = (blockIdx.x - tile_m * tiles_n) * 64;
   const int k_lo = blockIdx.z * k_per_split, k_hi = min(K, k_lo + k_per_split);
   const int wm = (warp >> 2) * 32, wn = (warp & 3) * 16;
   // element offsets of this lane's fragment entries: A(m, k) with m = wm + g, k = t;  B(k, n) with k = t, n = wn + g
@@ -244,8 +245,8 @@ gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta,
         if (m >= M || n >= N) continue;
         float* c = C + (size_t)m * ldc + n;
         const float v = alpha * acc[mt][nt][e];
-        if (gridDim.z > 1) atomicAdd(c, v);
-        else *c = accumulate ? *c + v : v;
+        if (gridDim.z > 1 || accumulate) atomicAdd(c, v);      // (one add per element when K is not split: the result is
+        else *c = v;                                           //  the same, and the thread does not wait for the old value)
       }
 }
 
@@ -275,8 +276,9 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
     if (splits > 65535) { splits = 65535; per = (K + splits - 1) / splits; per = (per + kstep - 1) / kstep * kstep; splits = (K + per - 1) / per; }
   }
   const int tiles_n = (N + kTN - 1) / kTN;
-  if ((long long)tiles_n * batch > 65535) return LASER_ERR_UNSUPPORTED;
-  const dim3 grid((M + kTM - 1) / kTM, tiles_n * batch, splits);
+  const long long tiles = (long long)((M + kTM - 1) / kTM) * tiles_n;
+  if (batch > 65535 || tiles > 0x7fffffffLL) return LASER_ERR_UNSUPPORTED;
+  const dim3 grid((unsigned)tiles, batch, splits);
   LaunchScope ls(gx.tf32 ? "bwd_gemm_tf32" : "bwd_gemm", st);
   if (gx.tf32)
     gemm_tf32_kernel<TA, TB><<<grid, kGemmThreads, 0, st>>>(
