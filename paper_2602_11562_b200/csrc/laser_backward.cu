@@ -751,7 +751,10 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   char* mma_scratch = ws + p.total + s.total;
   if (tensor) {
     LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
-    BWD_OK(simt_project(p, items, lengths, cands, Wq, Wk, Wv, ws, st));
+    // projections as three matrix products over all rows (padding rows included: their K and V are never read)
+    BWD_OK(gemm<T, T>(gx, N, dqk, d, cands, d, false, Wq, dqk, false, Qf, dqk, p.inv_gamma, false, false));
+    BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
+    BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
     BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
     if (sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, mma_scratch, st));
     else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
