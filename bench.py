@@ -467,7 +467,8 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
     finally:
         P.laser_profile_enable(False)
     assert P.laser_check_status(bws) == 0
-    tensor = "bwd_sta_mma" in kernels
+    tensor = "bwd_gemm_tf32" in kernels
+    gates_tensor = "bwd_sta_mma" in kernels
     users = [u for u in range(s.U) if w.cand_offsets[u + 1] > w.cand_offsets[u]][:2]
     ref = backward_oracle.backward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
                                    dz.astype(np.float64), w.gamma, w.tau, users=users)
@@ -502,7 +503,8 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
             "bound": "alu", "flops": flops, "achieved": ach, "peak": peak, "achieved_unit": "TFLOP/s", "frac": ach / peak,
             "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
             "parity": {"err_over_max": err, "tol": tol, "users_checked": len(users), "scores_checked": checked},
-            "gate_contractions": "tensor cores (mma.sync, bf16 operands)" if tensor else "FP32 ALUs",
+            "matrix_products": "tensor cores (mma.sync, TF32 operands)" if tensor else "FP32 ALUs",
+            "gate_contractions": "tensor cores (mma.sync, bf16 operands)" if gates_tensor else "FP32 ALUs",
             "kernel_ms_first_call": {k: round(v, 4) for k, v in sorted(kernels.items())},
             "workspace_bytes": need}
 

@@ -749,14 +749,15 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 
   // ---- forward, kept in fp32: projections and H' (the FP32-ALU forward kernels), then the GSTA layers
   char* mma_scratch = ws + p.total + s.total;
+  const bool mma = tensor && sta_bwd_mma_supported(p);     // (users with very few candidates keep the FP32 gate kernels)
   if (tensor) {
     LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
     // projections as three matrix products over all rows (padding rows included: their K and V are never read)
     BWD_OK(gemm<T, T>(gx, N, dqk, d, cands, d, false, Wq, dqk, false, Qf, dqk, p.inv_gamma, false, false));
     BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
     BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
-    BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
-    if (sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, mma_scratch, st));
+    if (mma) BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
+    if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, mma_scratch, st));
     else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else if (p.dqh == 16 && dvh == 32 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
@@ -823,7 +824,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dQf, 0, (size_t)N * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dK, 0, UL * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
-  if (tensor) {
+  if (mma) {
     BWD_OK(sta_bwd_mma(p, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, mma_scratch, st));
   } else {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
@@ -858,7 +859,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
 
 size_t backward_scratch_bytes(const Plan& p) { return carve_scratch(p, nullptr).total + sta_bwd_mma_scratch_bytes(p); }
 
-bool backward_tensor_supported(const Plan& p) { return p.dtype == LASER_BF16 && sta_bwd_mma_supported(p); }
+bool backward_tensor_supported(const Plan& p) { return p.dtype == LASER_BF16; }
 
 int backward(const Plan& p, const void* items, const int32_t* lengths, const void* cands, const int32_t* cand_offsets,
              const void* Wq, const void* Wk, const void* Wv, const void* Wg, const float* dz, float* d_items,

@@ -97,6 +97,12 @@ def test_backward_tensor_path_matches_oracle(case):
     print("backward tensor path, worst error / largest entry:", {k: f"{v:.2e}" for k, v in worst.items()})
 
 
+def test_backward_of_users_with_few_candidates_keeps_the_fp32_gate_kernels():
+    # one candidate per user (the one-candidate serving shape): the matrix products still run on the tensor cores
+    kw = dict(U=40, C=1, L=128, d=64, H=2, S=32, M=1, dtype="bf16", lengths=[128] * 20 + [77] * 19 + [0])
+    _check(kw, 1300, P.PATH_AUTO, TENSOR_BAR, want_kernel=False)
+
+
 def test_backward_tensor_path_on_request_only_where_it_exists():
     w = make_custom(U=1, C=4, L=32, d=32, H=2, S=8, M=1, dtype="f32", seed=5)
     b = P.DeviceBatch.from_workload(w, path=P.PATH_TENSOR)
