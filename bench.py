@@ -444,7 +444,8 @@ def softmax_row(P, w, b, flush, stream, steps, peaks, dev):
 def backward_row(P, w, b, flush, stream, steps, peaks, dev):
     """Another row of the scope: the backward pass (laser_backward) of this batch for a seeded upstream gradient,
     checked on the first two users with candidates against the backward oracle (their rows of d_cands and d_items
-    depend on no other user), then timed on its own.  FP32-ALU kernels: reported against the derived FP32 peak."""
+    depend on no other user), then timed on its own.  bf16 batches run on the tensor cores (reported against the measured
+    tensor peak scaled to TF32), fp32 batches on the FP32 ALUs (against the derived FP32 peak)."""
     import torch
     from oracle import backward_oracle
     s = w.spec
@@ -497,11 +498,16 @@ def backward_row(P, w, b, flush, stream, steps, peaks, dev):
     work = algorithmic_work(w)
     # forward recomputed once, then about two products per forward product: three times the forward's flops
     flops = 3.0 * (work["proj_flops"] + 2 * w.N * s.d * s.d_qk + work["attn_flops"] + work["gsta_flops"])
-    peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    if tensor:      # matrix products in TF32, gate contractions in bf16: against the TF32 figure (the smaller of the two)
+        peak = peaks["bf16_tflops"] * 1.1 / 2.25
+        bound, source = "tensor", f"{peaks['_source']} bf16 GEMM peak x nominal tf32 : bf16 ratio (1.1 : 2.25)"
+    else:
+        peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        bound, source = "alu", "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"
     ach = flops / (tot * 1e-3) / 1e12
     return {"call": "laser_backward", "ms": tot, "launches": launches, "value": w.N / (tot * 1e-3), "unit": UNIT,
-            "bound": "alu", "flops": flops, "achieved": ach, "peak": peak, "achieved_unit": "TFLOP/s", "frac": ach / peak,
-            "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+            "bound": bound, "flops": flops, "achieved": ach, "peak": peak, "achieved_unit": "TFLOP/s", "frac": ach / peak,
+            "peak_source": source,
             "parity": {"err_over_max": err, "tol": tol, "users_checked": len(users), "scores_checked": checked},
             "matrix_products": "tensor cores (mma.sync, TF32 operands)" if tensor else "FP32 ALUs",
             "gate_contractions": "tensor cores (mma.sync, bf16 operands)" if gates_tensor else "FP32 ALUs",

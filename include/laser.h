@@ -212,8 +212,15 @@ LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* ite
  * segment sums and gates (Eq. 10-12) and the projections (Eq. 8-9).  The paper trains the model (section "Experimental
  * Settings") and prints no backward formulas; readings are those of the forward (an item at or past its user's length
  * receives a zero gradient row, an empty segment passes no gradient).  All gradients are fp32 device arrays, whatever
- * cfg->dtype; the inputs are read in cfg->dtype.  Runs on the FP32 ALUs whatever cfg->path says (a first version: it
- * recomputes the forward in fp32 and keeps every intermediate), padded item layout only.
+ * cfg->dtype; the inputs are read in cfg->dtype.  The forward is recomputed and every intermediate kept in the workspace;
+ * padded item layout only.  Two versions, chosen by cfg->path:
+ *   LASER_PATH_SIMT                 FP32 ALUs throughout, either dtype: every gradient within 1e-4 of its largest entry.
+ *   LASER_PATH_AUTO / _STREAM       fp32 batches as above.  bf16 batches on the tensor cores: every batched matrix product
+ *                                   with TF32 operands and fp32 accumulation, and, when max_cands_per_user >= 8 and the head
+ *                                   widths d_qk / H and d / H are multiples of 16 (d_qk / H at most 32, d / H at most 64), the
+ *                                   five contractions through the gates (and the recomputed H') with bf16 operands, as the
+ *                                   forward's tensor-core path rounds them: every gradient within 2e-2 of its largest entry.
+ *   LASER_PATH_TENSOR               as LASER_PATH_AUTO for bf16 batches; LASER_ERR_UNSUPPORTED for fp32 batches.
  *   dz          [N, d] fp32            IN
  *   d_items     [U, L, d] fp32         OUT (rows of padding are zero)
  *   d_cands     [N, d] fp32            OUT
