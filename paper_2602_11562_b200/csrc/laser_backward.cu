@@ -324,31 +324,66 @@ __device__ __forceinline__ int segments_of(const int* lengths, const int* cand_o
   return min((len + S - 1) / S, Lp);
 }
 
+// VEC consecutive features of a row (VEC = 4 when d is a multiple of 4: one 16-byte access; else 1).
+template <int VEC>
+__device__ __forceinline__ void load_vec(float (&v)[VEC], const float* p) {
+  if constexpr (VEC == 4) {
+    const float4 q = *reinterpret_cast<const float4*>(p);
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+  } else {
+    v[0] = *p;
+  }
+}
+template <int VEC>
+__device__ __forceinline__ void store_vec(float* p, const float (&v)[VEC]) {
+  if constexpr (VEC == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  else *p = v[0];
+}
+
+// dot[k] = s_j . W[h0 + k] for four heads at a time, W = [H][d] in shared memory; lanes split the features.
+template <int VEC>
+__device__ __forceinline__ void row_dots(const float* __restrict__ sj, const float* __restrict__ W, int d, int H, int h0,
+                                         int lane, float (&dot)[4]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) dot[k] = 0.f;
+  for (int x = VEC * lane; x < d; x += 32 * VEC) {
+    float sv[VEC];
+    load_vec<VEC>(sv, sj + x);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (h0 + k < H) {
+        float wv[VEC];
+        load_vec<VEC>(wv, W + (h0 + k) * d + x);
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) dot[k] = fmaf(sv[v], wv[v], dot[k]);
+      }
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+}
+
 // One block per candidate: e_{j,h} = s_j . Qt_h (Qt holds W_k[:, h] Q_h / tau), a = softmax over the non-empty segments,
-// m_h = sum_j a_{j,h} s_j.  Writes a [N, H, Lp] and m [N, H, d].
+// m_h = sum_j a_{j,h} s_j.  Writes a [N, H, Lp] and m [N, H, d].  The warps split the segments (a warp reads a segment
+// vector once for four heads, each lane VEC consecutive features); the per-warp partial sums of m meet in shared memory.
+template <int VEC>
 __global__ void __launch_bounds__(kAttnThreads)
 gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const int* __restrict__ lengths,
                      const int* __restrict__ cand_offsets, float* __restrict__ Aw, float* __restrict__ Mh, int U, int L,
                      int S, int Lp, int H, int d) {
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
+  constexpr int nw = kAttnThreads / 32;
   float* qt = sm;                 // [H][d]
-  float* e = qt + H * d;          // [H][Lp]
-  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = kAttnThreads / 32;
+  float* red = qt + H * d;        // [nw][H][d]: per-warp partial sums of m
+  float* e = red + nw * H * d;    // [H][Lp]
+  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nv = segments_of(lengths, cand_offsets, U, L, S, Lp, c);
   const float* s = Hp + (size_t)c * Lp * d;
   for (int i = tid; i < H * d; i += kAttnThreads) qt[i] = Qt[(size_t)c * H * d + i];
   __syncthreads();
-  for (int j = warp; j < nv; j += nw)                        // a warp takes segment vector j against four heads at a time
+  for (int j = warp; j < nv; j += nw)
     for (int h0 = 0; h0 < H; h0 += 4) {
-      float dot[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int x = lane; x < d; x += 32) {
-        const float sv = s[(size_t)j * d + x];
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) dot[k] = fmaf(sv, qt[(h0 + k) * d + x], dot[k]);
-      }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+      float dot[4];
+      row_dots<VEC>(s + (size_t)j * d, qt, d, H, h0, lane, dot);
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (lane == 0 && h0 + k < H) e[(h0 + k) * Lp + j] = dot[k];
@@ -373,36 +408,55 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
     }
   }
   __syncthreads();
-  for (int x = tid; x < d; x += kAttnThreads) {            // feature x of every head: the segment vectors are read once
+  for (int x = VEC * lane; x < d; x += 32 * VEC)
     for (int h0 = 0; h0 < H; h0 += 4) {
-      float acc[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int j = 0; j < nv; ++j) {
-        const float sv = s[(size_t)j * d + x];
+      float acc[4][VEC];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
+#pragma unroll 2
+      for (int j = warp; j < nv; j += nw) {
+        float sv[VEC];
+        load_vec<VEC>(sv, s + (size_t)j * d + x);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) acc[k] = fmaf(e[(h0 + k) * Lp + j], sv, acc[k]);
+          if (h0 + k < H) {
+            const float a = e[(h0 + k) * Lp + j];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(a, sv[v], acc[k][v]);
+          }
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        if (h0 + k < H) Mh[((size_t)c * H + h0 + k) * d + x] = acc[k];
+        if (h0 + k < H) store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
     }
+  __syncthreads();
+  for (int i = tid; i < H * d; i += kAttnThreads) {
+    float m = 0.f;
+#pragma unroll
+    for (int w = 0; w < nw; ++w) m += red[(size_t)w * H * d + i];
+    Mh[(size_t)c * H * d + i] = m;
   }
 }
 
 // One block per candidate: the backward of the kernel above.  dM = dLoss/dm [N, H, d] in; dQt = dLoss/dQt [N, H, d] out;
 // dHp [N, Lp, d] accumulates dLoss/ds_j over the layers: the layer processed first (overwrite != 0) writes every entry
-// (zeros for the empty segments), the others add.
+// (zeros for the empty segments), the others add.  Same split of the work as in the forward kernel.
+template <int VEC>
 __global__ void __launch_bounds__(kAttnThreads)
 gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const float* __restrict__ Aw,
                      const float* __restrict__ dM, const int* __restrict__ lengths, const int* __restrict__ cand_offsets,
                      float* __restrict__ dQt, float* __restrict__ dHp, int U, int L, int S, int Lp, int H, int d,
                      int overwrite) {
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
+  constexpr int nw = kAttnThreads / 32;
   float* qt = sm;                 // [H][d]
   float* dm = qt + H * d;         // [H][d]
-  float* a = dm + H * d;          // [H][Lp]
+  float* red = dm + H * d;        // [nw][H][d]: per-warp partial sums of dQt
+  float* a = red + nw * H * d;    // [H][Lp]
   float* de = a + H * Lp;         // [H][Lp]: first da, then de
-  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = kAttnThreads / 32;
+  const int c = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nv = segments_of(lengths, cand_offsets, U, L, S, Lp, c);
   const float* s = Hp + (size_t)c * Lp * d;
   for (int i = tid; i < H * d; i += kAttnThreads) {
@@ -413,15 +467,8 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   __syncthreads();
   for (int j = warp; j < nv; j += nw)
     for (int h0 = 0; h0 < H; h0 += 4) {
-      float dot[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int x = lane; x < d; x += 32) {
-        const float sv = s[(size_t)j * d + x];
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) dot[k] = fmaf(sv, dm[(h0 + k) * d + x], dot[k]);
-      }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+      float dot[4];
+      row_dots<VEC>(s + (size_t)j * d, dm, d, H, h0, lane, dot);
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         if (lane == 0 && h0 + k < H) de[(h0 + k) * Lp + j] = dot[k];
@@ -434,35 +481,74 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
     for (int j = lane; j < nv; j += 32) de[h * Lp + j] = a[h * Lp + j] * (de[h * Lp + j] - dotp);
   }
   __syncthreads();
-  for (int x = tid; x < d; x += kAttnThreads) {            // feature x: one pass over the segment vectors for both sums
+  float* dS = dHp + (size_t)c * Lp * d;
+  for (int x = VEC * lane; x < d; x += 32 * VEC) {
     for (int h0 = 0; h0 < H; h0 += 4) {
-      float acc[4] = {0.f, 0.f, 0.f, 0.f}, qx[4], mx[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        qx[k] = h0 + k < H ? qt[(h0 + k) * d + x] : 0.f;
-        mx[k] = h0 + k < H ? dm[(h0 + k) * d + x] : 0.f;
-      }
-#pragma unroll 4
-      for (int j = 0; j < nv; ++j) {
-        const float sv = s[(size_t)j * d + x];
-        float g = 0.f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          if (h0 + k < H) {
-            const float dej = de[(h0 + k) * Lp + j];
-            acc[k] = fmaf(dej, sv, acc[k]);
-            g += dej * qx[k] + a[(h0 + k) * Lp + j] * mx[k];
-          }
-        }
-        float* out = dHp + ((size_t)c * Lp + j) * d + x;
-        *out = (overwrite && h0 == 0) ? g : *out + g;
-      }
-      if (overwrite && h0 == 0)
-        for (int j = nv; j < Lp; ++j) dHp[((size_t)c * Lp + j) * d + x] = 0.f;      // empty segments receive no gradient
+      // dQt_h[x] = sum_j de_{j,h} s_j[x]: this warp's segments
+      float acc[4][VEC];
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        if (h0 + k < H) dQt[((size_t)c * H + h0 + k) * d + x] = acc[k];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
+#pragma unroll 2
+      for (int j = warp; j < nv; j += nw) {
+        float sv[VEC];
+        load_vec<VEC>(sv, s + (size_t)j * d + x);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (h0 + k < H) {
+            const float dej = de[(h0 + k) * Lp + j];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(dej, sv[v], acc[k][v]);
+          }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (h0 + k < H) store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
+      // ds_j[x] += sum_h de_{j,h} Qt_h[x] + a_{j,h} dm_h[x]
+      float qx[4][VEC], mx[4][VEC];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) qx[k][v] = mx[k][v] = 0.f;
+        if (h0 + k < H) {
+          load_vec<VEC>(qx[k], qt + (h0 + k) * d + x);
+          load_vec<VEC>(mx[k], dm + (h0 + k) * d + x);
+        }
+      }
+#pragma unroll 2
+      for (int j = warp; j < nv; j += nw) {
+        float g[VEC];
+        float* out = dS + (size_t)j * d + x;
+        if (overwrite && h0 == 0) {
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) g[v] = 0.f;
+        } else {
+          load_vec<VEC>(g, out);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (h0 + k < H) {
+            const float dej = de[(h0 + k) * Lp + j], aj = a[(h0 + k) * Lp + j];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) g[v] = fmaf(dej, qx[k][v], fmaf(aj, mx[k][v], g[v]));
+          }
+        store_vec<VEC>(out, g);
+      }
     }
+    if (overwrite) {                                        // empty segments receive no gradient
+      float zero[VEC];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) zero[v] = 0.f;
+      for (int j = nv + warp; j < Lp; j += nw) store_vec<VEC>(dS + (size_t)j * d + x, zero);
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < H * d; i += kAttnThreads) {
+    float q = 0.f;
+#pragma unroll
+    for (int w = 0; w < nw; ++w) q += red[(size_t)w * H * d + i];
+    dQt[(size_t)c * H * d + i] = q;
   }
 }
 
@@ -776,11 +862,14 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     LaunchScope ls("bwd_to_f32", st);
     to_f32_kernel<T><<<296, 256, 0, st>>>(cands, s.T, Nd);
   }
-  const size_t attn_smem_f = ((size_t)H * d + (size_t)H * Lp) * sizeof(float);
-  const size_t attn_smem_b = (2 * (size_t)H * d + 2 * (size_t)H * Lp) * sizeof(float);
+  constexpr int attn_warps = kAttnThreads / 32;
+  const size_t attn_smem_f = ((size_t)(1 + attn_warps) * H * d + (size_t)H * Lp) * sizeof(float);
+  const size_t attn_smem_b = ((size_t)(2 + attn_warps) * H * d + 2 * (size_t)H * Lp) * sizeof(float);
   if (attn_smem_b > 200 * 1024) return LASER_ERR_UNSUPPORTED;
-  LASER_CUDA_OK(cudaFuncSetAttribute(gsta_attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_f));
-  LASER_CUDA_OK(cudaFuncSetAttribute(gsta_attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_b));
+  auto attn_fwd = d % 4 == 0 ? gsta_attn_fwd_kernel<4> : gsta_attn_fwd_kernel<1>;      // 16-byte accesses when rows allow
+  auto attn_bwd = d % 4 == 0 ? gsta_attn_bwd_kernel<4> : gsta_attn_bwd_kernel<1>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(attn_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_f));
+  LASER_CUDA_OK(cudaFuncSetAttribute(attn_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_b));
   for (int l = 0; l < M; ++l) {
     const T *Wql = Wg + (size_t)(l * 3) * d * d, *Wkl = Wql + (size_t)d * d, *Wvl = Wkl + (size_t)d * d;
     float *Tl = s.T + l * Nd, *Tn = Tl + Nd, *Ql = s.Q + l * Nd, *Qtl = s.Qt + l * NHd, *Al = s.A + (size_t)l * N * H * Lp,
@@ -790,7 +879,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<float, T>(gx, N, d, dvh, Ql, d, false, Wkl, d, true, Qtl, H * d, p.inv_tau, false, false, H, dvh, dvh, d));
     {
       LaunchScope ls("bwd_attn_fwd", st);
-      gsta_attn_fwd_kernel<<<N, kAttnThreads, attn_smem_f, st>>>(s.Hp, Qtl, lengths, cand_offsets, Al, Ml, U, L, p.S, Lp,
+      attn_fwd<<<N, kAttnThreads, attn_smem_f, st>>>(s.Hp, Qtl, lengths, cand_offsets, Al, Ml, U, L, p.S, Lp,
                                                                  H, d);
     }
     LASER_CUDA_OK(cudaMemcpyAsync(Tn, Tl, Nd * sizeof(float), cudaMemcpyDeviceToDevice, st));
@@ -811,7 +900,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT, d, false, Wvl, d, true, s.dM, H * d, 1.f, false, false, H, dvh, dvh, d));
     {
       LaunchScope ls("bwd_attn_bwd", st);
-      gsta_attn_bwd_kernel<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
+      attn_bwd<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
                                                                  U, L, p.S, Lp, H, d, l == M - 1 ? 1 : 0);
     }
     // dQ_h = dQt_h W_k[:, h] / tau;  dW_k[:, h] += dQt_h^T Q_h / tau, every head

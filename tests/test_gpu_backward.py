@@ -21,6 +21,7 @@ CASES = [
     dict(U=4, C=3, L=64, d=24, H=3, S=1, M=1, dtype="f32", lengths=[64, 1, 0, 17], d_qh=8),  # one-item segments, d_qh = 8
     dict(U=2, C=9, L=40, d=32, H=2, S=8, M=0, dtype="f32", lengths=[40, 13]),              # no GSTA layer: z = t
     dict(U=3, C=130, L=512, d=64, H=4, S=64, M=2, dtype="bf16", lengths=[512, 300, 77]),   # serving-like, more rows
+    dict(U=2, C=5, L=40, d=18, H=3, S=8, M=2, dtype="f32", lengths=[40, 21], d_qh=4),      # a width that is no multiple of 4
 ]
 
 
