@@ -156,8 +156,8 @@ static int run_gsta(const Plan& p, const void* Hp, const int32_t* lengths, const
 
 static int forward_impl(const Plan& p, const void* items, const int32_t* lengths, const void* cands,
                         const int32_t* cand_offsets, const void* Wq, const void* Wk, const void* Wv, const void* Wg,
-                        void* Hprime, void* z, char* ws, cudaStream_t st, bool keep_status = false) {
-  int rc = keep_status ? (int)LASER_OK : clear_status(p, ws, st);   // (a later part of a batch must not erase an earlier report)
+                        void* Hprime, void* z, char* ws, cudaStream_t st) {
+  int rc = clear_status(p, ws, st);
   if (rc != LASER_OK) return rc;
   if (p.N == 0) return LASER_OK;
   void* Hp = Hprime ? Hprime : (void*)(ws + p.off_hp);
@@ -412,9 +412,8 @@ int laser_forward_ffn(const laser_config* cfg, const void* items, const int32_t*
 }
 
 namespace {
-constexpr int kMaxParts = 4;               // parts a large pinned batch is cut into so that transfer and compute overlap
 struct HostStage {
-  size_t items, lengths, cands, offs, item_offs, part_offs, wq, wk, wv, wg, z, total;
+  size_t items, lengths, cands, offs, item_offs, wq, wk, wv, wg, z, total;
   size_t b_items, b_lengths, b_cands, b_offs, b_wq, b_wk, b_wv, b_wg, b_z;
 };
 HostStage host_stage(const Plan& p) {
@@ -432,8 +431,7 @@ HostStage host_stage(const Plan& p) {
   s.lengths = off; off = align_up(off + s.b_lengths);
   s.cands = off; off = align_up(off + s.b_cands);
   s.offs = off; off = align_up(off + s.b_offs);
-  s.item_offs = off; off = align_up(off + s.b_offs + kMaxParts * sizeof(int32_t));     // (one more entry per part)
-  s.part_offs = off; off = align_up(off + s.b_offs + kMaxParts * sizeof(int32_t));     // candidate offsets per part
+  s.item_offs = off; off = align_up(off + s.b_offs);
   s.wq = off; off = align_up(off + s.b_wq);
   s.wk = off; off = align_up(off + s.b_wk);
   s.wv = off; off = align_up(off + s.b_wv);
@@ -538,90 +536,6 @@ __global__ void __launch_bounds__(kGatherThreads) host_gather_kernel(const uint4
 #pragma unroll 4
   for (int i = threadIdx.x; i < n; i += kGatherThreads) d[i] = s[i];
 }
-// Candidate offsets of a part of the batch (users u0 .. u0 + n - 1), counted from the part's first candidate.
-__global__ void __launch_bounds__(256) host_part_offsets_kernel(const int32_t* __restrict__ offs, int u0, int n,
-                                                                int32_t* __restrict__ out) {
-  chain_wait();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i <= n) out[i] = offs[u0 + i] - offs[u0];
-}
-
-// Two side streams (transfers in, results out) and the events that tie them to the caller's stream, per host thread and
-// device, created on first use and kept.
-struct HostPipe {
-  cudaStream_t copy = nullptr, out = nullptr;
-  cudaEvent_t start = nullptr, out_end = nullptr, in[kMaxParts] = {}, done[kMaxParts] = {};
-  bool ok = false, tried = false;
-};
-HostPipe* host_pipe() {
-  constexpr int kMaxDevices = 64;
-  static thread_local HostPipe pipes[kMaxDevices];
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  HostPipe& h = pipes[dev];
-  if (!h.tried) {
-    h.tried = true;
-    bool ok = cudaStreamCreateWithFlags(&h.copy, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaStreamCreateWithFlags(&h.out, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaEventCreateWithFlags(&h.start, cudaEventDisableTiming) == cudaSuccess &&
-              cudaEventCreateWithFlags(&h.out_end, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; ok && i < kMaxParts; ++i)
-      ok = cudaEventCreateWithFlags(&h.in[i], cudaEventDisableTiming) == cudaSuccess &&
-           cudaEventCreateWithFlags(&h.done[i], cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) cudaGetLastError();
-    h.ok = ok;
-  }
-  return h.ok ? &h : nullptr;
-}
-
-// Cuts a batch whose items travel by the gather kernel into parts of about equal item bytes, each a smaller batch of its
-// own (users [u[k], u[k + 1]), candidates [c[k], c[k + 1])), so that part k is computed while part k + 1 crosses the bus.
-// Returns the number of parts (1: not worth it, or the host-side offsets are not a valid partition of [0, N], which the
-// device then reports as for any other call).
-constexpr size_t kPipeWorth = 4u << 20;    // item bytes below which one part is as fast
-struct HostParts {
-  int n, u[kMaxParts + 1], c[kMaxParts + 1];
-  long long row[kMaxParts + 1];            // first row of the part in the gap-free item array
-  Plan plan[kMaxParts];
-};
-int host_parts(const laser_config* cfg, const Plan& p, const HostItemRoute& route, const void* z_h,
-               const int32_t* lengths_h, const int32_t* offs_h, HostParts* hp) {
-  hp->n = 1;
-  if (route.kind != kGather || route.bytes < kPipeWorth || p.U < 2 * kMaxParts || p.N == 0) return 1;
-  cudaPointerAttributes attr;                          // results leave part by part only into pinned memory
-  if (cudaPointerGetAttributes(&attr, z_h) != cudaSuccess) { cudaGetLastError(); return 1; }
-  if (attr.type != cudaMemoryTypeHost) return 1;
-  if (offs_h[0] != 0 || offs_h[p.U] != p.N) return 1;
-  long long rows = 0;
-  for (int u = 0; u < p.U; ++u) {
-    if (offs_h[u + 1] < offs_h[u] || offs_h[u + 1] - offs_h[u] > p.maxC) return 1;
-    rows += std::min(std::max(lengths_h[u], 0), p.L);
-  }
-  int k = 0;
-  long long run = 0;
-  hp->u[0] = 0; hp->c[0] = 0; hp->row[0] = 0;
-  for (int u = 0; u < p.U; ++u) {
-    run += std::min(std::max(lengths_h[u], 0), p.L);
-    // part k ends after user u once it holds its share of the rows (and leaves a user for every later part)
-    if (k + 1 < kMaxParts && run * kMaxParts >= rows * (k + 1) && p.U - (u + 1) >= kMaxParts - (k + 1)) {
-      ++k;
-      hp->u[k] = u + 1; hp->c[k] = offs_h[u + 1]; hp->row[k] = run;
-    }
-  }
-  ++k;
-  hp->u[k] = p.U; hp->c[k] = p.N; hp->row[k] = run;
-  if (k < 2) return 1;
-  for (int i = 0; i < k; ++i) {
-    laser_config c = *cfg;
-    c.num_users = hp->u[i + 1] - hp->u[i];
-    c.total_cands = hp->c[i + 1] - hp->c[i];
-    if (c.num_users <= 0 || c.total_cands <= 0) return 1;      // (a part without candidates would skip its users' checks)
-    c.max_cands_per_user = std::min(cfg->max_cands_per_user, c.total_cands);
-    if (make_plan(&c, &hp->plan[i]) != LASER_OK || hp->plan[i].total > p.total || hp->plan[i].path != p.path) return 1;
-  }
-  hp->n = k;
-  return k;
-}
 }  // namespace
 
 int laser_host_transfer_bytes(const laser_config* cfg, const void* items_h, const int32_t* lengths_h,
@@ -667,75 +581,10 @@ int laser_forward_host(const laser_config* cfg, const void* items_h, const int32
     if (!bytes) return cudaSuccess;
     return cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, st);
   };
-  HostItemRoute route;
-  route.kind = kPadded; route.bytes = 0; route.alias = nullptr;
-  if (p.N > 0) route = host_item_route(p, items_h, lengths_h);
-  HostParts parts;
-  HostPipe* pipe = nullptr;
-  if (host_parts(cfg, p, route, z_h, lengths_h, cand_offsets_h, &parts) > 1) pipe = host_pipe();
-  if (pipe) {
-    // Everything small and the candidates first, on the transfer stream; then part by part: the part's offsets, its valid
-    // item rows (one kernel reading the pinned host array), an event; the caller's stream computes a part as soon as its
-    // event fires, and the result stream sends that part's z home while the next part is computed.
-    auto up = [&](size_t off, const void* src, size_t bytes) -> cudaError_t {
-      if (!bytes) return cudaSuccess;
-      return cudaMemcpyAsync(ws + off, src, bytes, cudaMemcpyHostToDevice, pipe->copy);
-    };
-    LASER_CUDA_OK(cudaEventRecord(pipe->start, st));
-    LASER_CUDA_OK(cudaStreamWaitEvent(pipe->copy, pipe->start, 0));
-    LASER_CUDA_OK(cudaStreamWaitEvent(pipe->out, pipe->start, 0));
-    LASER_CUDA_OK(up(s.lengths, lengths_h, s.b_lengths));
-    LASER_CUDA_OK(up(s.offs, cand_offsets_h, s.b_offs));
-    LASER_CUDA_OK(up(s.wq, Wq_h, s.b_wq));
-    LASER_CUDA_OK(up(s.wk, Wk_h, s.b_wk));
-    LASER_CUDA_OK(up(s.wv, Wv_h, s.b_wv));
-    LASER_CUDA_OK(up(s.wg, Wgsta_h, s.b_wg));
-    LASER_CUDA_OK(up(s.cands, cands_h, s.b_cands));
-    const size_t row = (size_t)p.d * p.esize;
-    const int32_t* lengths_d = reinterpret_cast<const int32_t*>(ws + s.lengths);
-    for (int k = 0; k < parts.n; ++k) {
-      const int u0 = parts.u[k], nu = parts.u[k + 1] - u0;
-      int32_t* item_offs = reinterpret_cast<int32_t*>(ws + s.item_offs) + u0 + k;       // nu + 1 entries per part
-      int32_t* part_offs = reinterpret_cast<int32_t*>(ws + s.part_offs) + u0 + k;
-      {
-        LaunchScope ls("host_part_offsets", pipe->copy);
-        LASER_CUDA_OK(launch_chained(host_part_offsets_kernel, dim3((nu + 256) / 256), dim3(256), 0, pipe->copy,
-                                     reinterpret_cast<const int32_t*>(ws + s.offs), u0, nu, part_offs));
-      }
-      {
-        LaunchScope ls("host_row_offsets", pipe->copy);
-        LASER_CUDA_OK(launch_chained(host_row_offsets_kernel, dim3(1), dim3(1024), 0, pipe->copy, lengths_d + u0, nu, p.L,
-                                     item_offs));
-      }
-      {
-        const int per = std::max(64, (p.L + 65534) / 65535);
-        LaunchScope ls("host_gather", pipe->copy);
-        LASER_CUDA_OK(launch_chained(host_gather_kernel, dim3(nu, (p.L + per - 1) / per), dim3(kGatherThreads), 0, pipe->copy,
-                                     reinterpret_cast<const uint4*>(static_cast<const char*>(route.alias) + (size_t)u0 * p.L * row),
-                                     reinterpret_cast<uint4*>(ws + s.items + (size_t)parts.row[k] * row), lengths_d + u0,
-                                     static_cast<const int32_t*>(item_offs), p.L, (int)(row / 16), per));
-      }
-      LASER_CUDA_OK(cudaEventRecord(pipe->in[k], pipe->copy));
-      LASER_CUDA_OK(cudaStreamWaitEvent(st, pipe->in[k], 0));
-      Plan pk = parts.plan[k];
-      pk.item_offsets = item_offs;
-      const size_t c_bytes = (size_t)parts.c[k] * row;
-      rc = forward_impl(pk, ws + s.items + (size_t)parts.row[k] * row, lengths_d + u0, ws + s.cands + c_bytes, part_offs,
-                        ws + s.wq, ws + s.wk, ws + s.wv, ws + s.wg, nullptr, ws + s.z + c_bytes, ws, st, k > 0);
-      if (rc != LASER_OK) return rc;
-      LASER_CUDA_OK(cudaEventRecord(pipe->done[k], st));
-      LASER_CUDA_OK(cudaStreamWaitEvent(pipe->out, pipe->done[k], 0));
-      LASER_CUDA_OK(cudaMemcpyAsync(static_cast<char*>(z_h) + c_bytes, ws + s.z + c_bytes,
-                                    (size_t)(parts.c[k + 1] - parts.c[k]) * row, cudaMemcpyDeviceToHost, pipe->out));
-    }
-    LASER_CUDA_OK(cudaEventRecord(pipe->out_end, pipe->out));
-    LASER_CUDA_OK(cudaStreamWaitEvent(st, pipe->out_end, 0));
-    if (blocking) return laser_check_status(workspace, cuda_stream);
-    return LASER_OK;
-  }
   LASER_CUDA_OK(h2d(s.lengths, lengths_h, s.b_lengths));
   LASER_CUDA_OK(h2d(s.offs, cand_offsets_h, s.b_offs));
   if (p.N > 0) {
+    const HostItemRoute route = host_item_route(p, items_h, lengths_h);
     if (route.kind == kPadded) LASER_CUDA_OK(h2d(s.items, items_h, s.b_items));
     else {
       {

@@ -379,49 +379,6 @@ def test_host_buffer_entry_point_pageable_memory_copies_runs_of_users():
     assert torch.equal(z_h, z_dev)
 
 
-@pytest.mark.parametrize("path", ["tensor", "simt"])
-def test_host_buffer_entry_point_in_parts_matches_device_entry_point(path):
-    # A pinned batch large enough (4 MB of valid item rows, eight users or more) travels and is computed in parts: part
-    # k + 1 crosses the bus while part k is computed, z goes home part by part.  The bits are those of the device entry
-    # point on the whole batch, call after call on the same workspace, and a bad length in a late part is still reported.
-    rng = np.random.default_rng(77)
-    lengths = [int(x) for x in rng.integers(600, 2049, size=26)]
-    lengths[3], lengths[11], lengths[25] = 0, 2048, 1
-    w = make_custom(U=26, C=7, L=2048, d=64, H=2, S=64, M=2, dtype="bf16", seed=29, lengths=lengths)
-    assert sum(lengths) * 128 >= 4 << 20
-    z_dev = run_forward(w, path, want_hprime=False).cpu()
-    hb = P.DeviceBatch.from_workload(w, path=PATHS[path], device="cpu", pin_host=True)
-    for u, n in enumerate(lengths):
-        hb.items[u, n:] = float("nan")                          # padding never travels
-    ws = torch.empty(P.laser_host_workspace_bytes(hb.cfg), dtype=torch.uint8, device="cuda")
-    z_h = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype).pin_memory()
-    P.laser_profile_enable(True)
-    try:
-        P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
-        names = [n for n, _ in P.laser_profile_read()]
-    finally:
-        P.laser_profile_enable(False)
-    assert names.count("host_gather") == 4, names               # four parts
-    assert torch.equal(z_h, z_dev)
-    z_h.zero_()
-    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws, blocking=False)
-    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws, blocking=False)     # back to back on one workspace
-    torch.cuda.synchronize()
-    assert torch.equal(z_h, z_dev)
-    # pageable output: one part, same bits
-    z_p = torch.empty((hb.cfg.total_cands, hb.cfg.d_model), dtype=hb.items.dtype)
-    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_p, ws)
-    assert torch.equal(z_p, z_dev)
-    bad = hb.lengths.clone()
-    bad[24] = 5000
-    bad = bad.pin_memory()
-    with pytest.raises(P.binding.LaserError) as err:
-        P.laser_forward_host(hb.cfg, hb.items, bad, hb.cands, hb.cand_offsets, hb.Wq, hb.Wk, hb.Wv, hb.Wg, z_h, ws)
-    assert err.value.status == -6
-    P.laser_forward_host(hb.cfg, *hb.args(), hb.Wg, z_h, ws)
-    assert torch.equal(z_h, z_dev)
-
-
 # ------------------------------------------------------------------ full-size configurations, every user
 # Bounds on the maximum absolute error relative to the root mean square of the reference tensor (the signal), asserted
 # beside the pass/fail metric, whose denominator max(1, |r|) never exceeds 1 on these workloads.
