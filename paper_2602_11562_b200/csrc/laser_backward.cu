@@ -137,10 +137,12 @@ __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], 
 // A 64 x kWK tile of an operand X, rows r0 .. (bound R), contraction indices k0 .. (bound k_hi), with
 // X(r, k) = k_major ? X[k ld + r] : X[r ld + k], travels in two steps so that the global loads of the next tile are in
 // flight while the current one is multiplied: fetch_tile brings a thread's eight elements into registers as they are,
-// put_tile rounds them to TF32 and stores them.  Shared layout: k_major ? [k][kColLd] : [r][kRowLd].  Full, aligned tiles move as two
-// 16-byte (fp32) or 8-byte (bf16) loads and two 16-byte stores per thread, the others element by element.
+// put_tile rounds them to TF32 and stores them.  Shared layout: k_major ? [k][kColLd] : [r][kRowLd].  Aligned tiles with
+// all 32 contraction indices in range move as two 16-byte (fp32) or 8-byte (bf16) loads and two 16-byte stores per thread
+// (groups of four past the last row are zeros), the others element by element.
 __device__ __forceinline__ bool tile_is_full(bool aligned, int r0, int R, int k0, int k_hi) {
-  return aligned && r0 + 64 <= R && k0 + kWK <= k_hi;
+  (void)r0;                                // rows past R are left out group by group (R is then a multiple of 4)
+  return aligned && R % 4 == 0 && k0 + kWK <= k_hi;
 }
 template <typename TX>
 __device__ __forceinline__ void fetch_tile(uint32_t (&v)[8], const TX* __restrict__ X, int ld, int k_major, int r0, int R,
@@ -149,9 +151,9 @@ __device__ __forceinline__ void fetch_tile(uint32_t (&v)[8], const TX* __restric
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
       const int i = tid + kGemmThreads * j;
-      const TX* src = k_major ? X + (size_t)(k0 + (i >> 4)) * ld + r0 + (i & 15) * 4
-                              : X + (size_t)(r0 + (i >> 3)) * ld + k0 + (i & 7) * 4;
-      const uint4 q = raw4(src);
+      const int r = r0 + (k_major ? (i & 15) * 4 : (i >> 3));
+      const TX* src = k_major ? X + (size_t)(k0 + (i >> 4)) * ld + r : X + (size_t)r * ld + k0 + (i & 7) * 4;
+      const uint4 q = r < R ? raw4(src) : make_uint4(0u, 0u, 0u, 0u);
       v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
     }
     return;
