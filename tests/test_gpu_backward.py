@@ -98,6 +98,32 @@ def test_backward_tensor_path_matches_oracle(case):
     print("backward tensor path, worst error / largest entry:", {k: f"{v:.2e}" for k, v in worst.items()})
 
 
+@pytest.mark.parametrize("name,users", [("cfg3", (0, 17, 63)), ("cfg2x32", (5, 31)), ("prod", (2, 40))])
+def test_backward_full_size_configs_sampled_users(name, users):
+    # The batches the benchmark times, in its launch configuration: d_cands and d_items of a user depend on no other user,
+    # so the oracle computes those users alone (seconds each); the weight gradients sum over all users and are checked on
+    # the small shapes above.
+    from workloads import make_workload
+    w = make_workload(name)
+    s = w.spec
+    dz = np.random.default_rng(4242).standard_normal((w.N, s.d)).astype(np.float32)
+    ref = backward_oracle.backward(w.items, w.lengths, w.cands, w.cand_offsets, w.Wq, w.Wk, w.Wv, w.Wg, s.S, s.H,
+                                   dz.astype(np.float64), w.gamma, w.tau, users=list(users))
+    b = P.DeviceBatch.from_workload(w)
+    ws = torch.empty(P.laser_backward_workspace_bytes(b.cfg), dtype=torch.uint8, device="cuda")
+    got = P.laser_backward(b.cfg, *b.args(), b.Wg, torch.from_numpy(dz).cuda(), workspace=ws)
+    assert P.laser_check_status(ws) == 0
+    for u in users:
+        c0, c1 = int(w.cand_offsets[u]), int(w.cand_offsets[u + 1])
+        for g, r, what in ((got["d_cands"][c0:c1], ref["d_cands"][c0:c1], "d_cands"),
+                           (got["d_items"][u], ref["d_items"][u], "d_items")):
+            g = g.cpu().numpy().astype(np.float64)
+            scale = max(float(np.max(np.abs(r))), 1e-30)
+            assert np.isfinite(g).all()
+            assert np.max(np.abs(g - r)) <= TENSOR_BAR * scale, (name, u, what, float(np.max(np.abs(g - r))), scale)
+        assert not got["d_items"][u, int(w.lengths[u]):].any()
+
+
 def test_backward_of_users_with_few_candidates_keeps_the_fp32_gate_kernels():
     # one candidate per user (the one-candidate serving shape): the matrix products still run on the tensor cores
     kw = dict(U=40, C=1, L=128, d=64, H=2, S=32, M=1, dtype="bf16", lengths=[128] * 20 + [77] * 19 + [0])
