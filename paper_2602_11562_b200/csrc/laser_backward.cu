@@ -19,6 +19,7 @@
 // Sums over candidates that end in one weight matrix are split over blocks and finished with floating-point atomics, so
 // the last bits of the weight gradients and of d_cands' STA part depend on the order in which blocks finish.
 #include "laser_common.cuh"
+#include "laser_mma.cuh"
 
 namespace laser {
 namespace {
@@ -253,6 +254,140 @@ gemm_tf32_kernel(int M, int N, int K, const TA* __restrict__ A, int lda, int ta,
       }
 }
 
+// Products with very many rows and a small second operand, C[M x N] (+)= alpha A[M x K] B(K, N) with N, K <= 128: what
+// the generic kernel above does badly (a block lives for K / 32 steps, reads B again for every tile of rows and never has
+// more than one step in flight).  Here a block stays: it stages B once (TF32, k-major, pitch N + 8), then walks tiles of
+// 128 rows, whose A rows arrive by cp.async as they are (fp32 or bf16, row pitch of K + 4 words or K + 8 halves) into one
+// of two buffers while the previous tile is multiplied; A is rounded to TF32 when a fragment is read.  Eight warps of
+// 32 rows x N / 2 columns.
+constexpr int kRowsTile = 128;
+template <typename TA> struct RowsPitch;
+template <> struct RowsPitch<float> { static __host__ __device__ int elems(int K) { return K + 4; } };
+template <> struct RowsPitch<bf16> { static __host__ __device__ int elems(int K) { return K + 8; } };
+__device__ __forceinline__ uint32_t frag_of(const float* p) { return tf32_of(*p); }
+__device__ __forceinline__ uint32_t frag_of(const bf16* p) {
+  return static_cast<uint32_t>(*reinterpret_cast<const unsigned short*>(p)) << 16;
+}
+
+template <typename TA, typename TB, int N>
+__global__ void __launch_bounds__(kGemmThreads)
+rows_gemm_kernel(int M, int K, const TA* __restrict__ A, int lda, const TB* __restrict__ B, int ldb, int tb,
+                 float* __restrict__ C, int ldc, float alpha, int accumulate, int n_tiles) {
+  constexpr int WN = N / 2, NTW = WN / 8, BP = N + 8;
+  extern __shared__ __align__(16) unsigned char rg_smem[];
+  uint32_t* Bs = reinterpret_cast<uint32_t*>(rg_smem);                       // [K][BP]
+  const int ap = RowsPitch<TA>::elems(K);
+  TA* As = reinterpret_cast<TA*>(rg_smem + (size_t)K * BP * sizeof(uint32_t));    // [2][128][ap]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  constexpr int kPer16 = 16 / (int)sizeof(TA);                               // elements per 16-byte copy
+  const int chunks_per_row = K / kPer16, chunks = kRowsTile * chunks_per_row;
+  auto stage = [&](int tile, int buf) {
+    TA* dst = As + (size_t)buf * kRowsTile * ap;
+    const int r0 = tile * kRowsTile;
+    for (int x = tid; x < chunks; x += kGemmThreads) {
+      const int rr = x / chunks_per_row, ch = x - rr * chunks_per_row;
+      const int r = r0 + rr;
+      mma::cp16(mma::smem_addr(dst + (size_t)rr * ap + ch * kPer16), A + (size_t)min(r, M - 1) * lda + ch * kPer16,
+                r < M ? 16u : 0u);
+    }
+    mma::cp_commit();
+  };
+  int tile = blockIdx.x;
+  if (tile < n_tiles) stage(tile, 0);
+  for (int i = tid; i < K * N; i += kGemmThreads) {
+    const int k = i / N, n = i - k * N;
+    Bs[k * BP + n] = tf32_of(to_f32<TB>(tb ? B[(size_t)n * ldb + k] : B[(size_t)k * ldb + n]));
+  }
+  const int wr = (warp >> 1) * 32, wc = (warp & 1) * WN;
+  int buf = 0;
+  for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
+    const int next = tile + gridDim.x;
+    if (next < n_tiles) {
+      stage(next, buf ^ 1);
+      mma::cp_wait<1>();
+    } else {
+      mma::cp_wait<0>();
+    }
+    __syncthreads();
+    const TA* At = As + (size_t)buf * kRowsTile * ap;
+    float acc[2][NTW][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
+    for (int kb = 0; kb < K; kb += 8) {
+      uint32_t a[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const TA* pa = At + (size_t)(wr + mt * 16 + g) * ap + kb + t;
+        a[mt][0] = frag_of(pa);
+        a[mt][1] = frag_of(pa + 8 * ap);
+        a[mt][2] = frag_of(pa + 4);
+        a[mt][3] = frag_of(pa + 8 * ap + 4);
+      }
+      const uint32_t* pb = Bs + (kb + t) * BP + wc + g;
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const uint32_t b0 = pb[nt * 8], b1 = pb[4 * BP + nt * 8];
+        mma_tf32(acc[0][nt], a[0], b0, b1);
+        mma_tf32(acc[1][nt], a[1], b0, b1);
+      }
+    }
+    const int r0 = tile * kRowsTile + wr;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int r = r0 + mt * 16 + g + h * 8;
+        if (r >= M) continue;
+        float* c = C + (size_t)r * ldc + wc + 2 * t;
+#pragma unroll
+        for (int nt = 0; nt < NTW; ++nt) {
+          const float v0 = alpha * acc[mt][nt][2 * h], v1 = alpha * acc[mt][nt][2 * h + 1];
+          if (accumulate) {
+            atomicAdd(c + nt * 8, v0);
+            atomicAdd(c + nt * 8 + 1, v1);
+          } else {
+            *reinterpret_cast<float2*>(c + nt * 8) = make_float2(v0, v1);
+          }
+        }
+      }
+    __syncthreads();                     // the buffer just read is the next one to be filled
+  }
+}
+
+int bwd_sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  return n;
+}
+
+template <typename TA, typename TB>
+bool rows_gemm_fits(int M, int N, int K, const TA* A, int lda, const float* C, int ldc) {
+  constexpr int per16 = 16 / (int)sizeof(TA);
+  return M >= 32768 && (N == 32 || N == 64 || N == 128) && K >= 8 && K <= 128 && K % per16 == 0 && K % 8 == 0 &&
+         lda % per16 == 0 && reinterpret_cast<uintptr_t>(A) % 16 == 0 && ldc % 2 == 0 &&
+         reinterpret_cast<uintptr_t>(C) % 8 == 0;
+}
+
+template <typename TA, typename TB, int N>
+int launch_rows_gemm(cudaStream_t st, int M, int K, const TA* A, int lda, const TB* B, int ldb, bool tb, float* C, int ldc,
+                     float alpha, bool accumulate) {
+  const size_t smem = (size_t)K * (N + 8) * sizeof(uint32_t) + 2 * (size_t)kRowsTile * RowsPitch<TA>::elems(K) * sizeof(TA);
+  auto kernel = rows_gemm_kernel<TA, TB, N>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int n_tiles = (M + kRowsTile - 1) / kRowsTile;
+  const int per_sm = smem <= 100 * 1024 ? 2 : 1;
+  LaunchScope ls("bwd_gemm_rows", st);
+  kernel<<<std::min(n_tiles, per_sm * bwd_sm_count()), kGemmThreads, smem, st>>>(M, K, A, lda, B, ldb, tb ? 1 : 0, C, ldc, alpha,
+                                                                              accumulate ? 1 : 0, n_tiles);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
 // Where a product runs: the stream, and whether on the tensor cores (TF32) or on the FP32 ALUs.
 struct GemmCtx {
   cudaStream_t st;
@@ -269,6 +404,11 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
          int ldc, float alpha, bool accumulate, bool split_k, int batch = 1, int sa = 0, int sb = 0, int sc = 0) {
   if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return LASER_OK;
   cudaStream_t st = gx.st;
+  if (gx.tf32 && !ta && !split_k && batch == 1 && rows_gemm_fits<TA, TB>(M, N, K, A, lda, C, ldc)) {
+    if (N == 32) return launch_rows_gemm<TA, TB, 32>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
+    if (N == 64) return launch_rows_gemm<TA, TB, 64>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
+    return launch_rows_gemm<TA, TB, 128>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
+  }
   const int kstep = gx.tf32 ? kWK : kTK;
   int splits = 1, per = K;
   if (split_k) {                     // reductions over many rows into a small matrix (C must hold its initial value)
