@@ -388,6 +388,119 @@ int launch_rows_gemm(cudaStream_t st, int M, int K, const TA* A, int lda, const 
   return LASER_OK;
 }
 
+// Reductions over very many rows into a small matrix, C[MO x N] += alpha sum_r A[r][m] B[r][n] (the weight gradients
+// dW = X^T dY): a block stays, takes one contiguous slice of the rows, streams 32 rows of A and of B at a time (cp.async,
+// two buffers, as they are: the row index is the contraction index, so both land k-major) and keeps its MO x N partial
+// sum in registers until the end: one atomic add per element and block instead of one per element and 256 rows.
+template <typename TA, typename TB, int MO, int N>
+__global__ void __launch_bounds__(kGemmThreads)
+cols_gemm_kernel(int R, const TA* __restrict__ A, int lda, const TB* __restrict__ B, int ldb, float* __restrict__ C, int ldc,
+                 float alpha, int rows_per_block) {
+  constexpr int WARPS_M = MO / 32, WARPS_N = 8 / WARPS_M, WN = N / WARPS_N, NTW = WN / 8;
+  constexpr int AP = MO + 16 / (int)sizeof(TA) * 2, BPT = N + 32 / (int)sizeof(TB);     // pitches in elements
+  static_assert(WN % 8 == 0 && NTW >= 1, "warp tiles of whole 8-column MMA tiles");
+  extern __shared__ __align__(16) unsigned char cg_smem[];
+  TA* As = reinterpret_cast<TA*>(cg_smem);                                    // [2][32][AP]
+  TB* Bs = reinterpret_cast<TB*>(cg_smem + 2 * 32 * AP * sizeof(TA));         // [2][32][BPT]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  const int r_lo = blockIdx.x * rows_per_block, r_hi = min(R, r_lo + rows_per_block);
+  constexpr int a16 = 16 / (int)sizeof(TA), b16 = 16 / (int)sizeof(TB);
+  constexpr int a_chunks = 32 * MO / a16, b_chunks = 32 * N / b16;
+  auto stage = [&](int r0, int buf) {
+    TA* da = As + buf * 32 * AP;
+    TB* db = Bs + buf * 32 * BPT;
+    for (int x = tid; x < a_chunks; x += kGemmThreads) {
+      const int rr = x / (MO / a16), ch = x - rr * (MO / a16), r = r0 + rr;
+      mma::cp16(mma::smem_addr(da + rr * AP + ch * a16), A + (size_t)min(r, R - 1) * lda + ch * a16, r < r_hi ? 16u : 0u);
+    }
+    for (int x = tid; x < b_chunks; x += kGemmThreads) {
+      const int rr = x / (N / b16), ch = x - rr * (N / b16), r = r0 + rr;
+      mma::cp16(mma::smem_addr(db + rr * BPT + ch * b16), B + (size_t)min(r, R - 1) * ldb + ch * b16, r < r_hi ? 16u : 0u);
+    }
+    mma::cp_commit();
+  };
+  const int wm = (warp / WARPS_N) * 32, wn = (warp % WARPS_N) * WN;
+  float acc[2][NTW][4];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
+  if (r_lo < r_hi) stage(r_lo, 0);
+  int buf = 0;
+  for (int r0 = r_lo; r0 < r_hi; r0 += 32, buf ^= 1) {
+    if (r0 + 32 < r_hi) {
+      stage(r0 + 32, buf ^ 1);
+      mma::cp_wait<1>();
+    } else {
+      mma::cp_wait<0>();
+    }
+    __syncthreads();
+    const TA* Ak = As + buf * 32 * AP;
+    const TB* Bk = Bs + buf * 32 * BPT;
+#pragma unroll
+    for (int kb = 0; kb < 32; kb += 8) {
+      uint32_t a[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const TA* pa = Ak + (kb + t) * AP + wm + mt * 16 + g;
+        a[mt][0] = frag_of(pa);
+        a[mt][1] = frag_of(pa + 8);
+        a[mt][2] = frag_of(pa + 4 * AP);
+        a[mt][3] = frag_of(pa + 4 * AP + 8);
+      }
+      const TB* pb = Bk + (kb + t) * BPT + wn + g;
+#pragma unroll
+      for (int nt = 0; nt < NTW; ++nt) {
+        const uint32_t b0 = frag_of(pb + nt * 8), b1 = frag_of(pb + 4 * BPT + nt * 8);
+        mma_tf32(acc[0][nt], a[0], b0, b1);
+        mma_tf32(acc[1][nt], a[1], b0, b1);
+      }
+    }
+    __syncthreads();
+  }
+  if (r_lo >= r_hi) return;
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NTW; ++nt)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int m = wm + mt * 16 + g + (e >> 1) * 8, n = wn + nt * 8 + 2 * t + (e & 1);
+        atomicAdd(C + (size_t)m * ldc + n, alpha * acc[mt][nt][e]);
+      }
+}
+
+template <typename TA, typename TB>
+bool cols_gemm_fits(int M, int N, int K, const TA* A, int lda, const TB* B, int ldb) {
+  return K >= 32768 && (M == 64 || M == 128) && (N == 32 || N == 64 || N == 128) &&
+         lda % (16 / (int)sizeof(TA)) == 0 && ldb % (16 / (int)sizeof(TB)) == 0 &&
+         reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+}
+
+template <typename TA, typename TB, int MO, int N>
+int launch_cols_gemm(cudaStream_t st, int R, const TA* A, int lda, const TB* B, int ldb, float* C, int ldc, float alpha) {
+  constexpr int AP = MO + 16 / (int)sizeof(TA) * 2, BPT = N + 32 / (int)sizeof(TB);
+  const size_t smem = 2 * 32 * ((size_t)AP * sizeof(TA) + (size_t)BPT * sizeof(TB));
+  auto kernel = cols_gemm_kernel<TA, TB, MO, N>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int blocks_max = 2 * bwd_sm_count();
+  const int per = ((R + blocks_max - 1) / blocks_max + 31) / 32 * 32;
+  LaunchScope ls("bwd_gemm_cols", st);
+  kernel<<<(R + per - 1) / per, kGemmThreads, smem, st>>>(R, A, lda, B, ldb, C, ldc, alpha, per);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+template <typename TA, typename TB, int MO>
+int launch_cols_gemm_n(cudaStream_t st, int N, int R, const TA* A, int lda, const TB* B, int ldb, float* C, int ldc,
+                       float alpha) {
+  if (N == 32) return launch_cols_gemm<TA, TB, MO, 32>(st, R, A, lda, B, ldb, C, ldc, alpha);
+  if (N == 64) return launch_cols_gemm<TA, TB, MO, 64>(st, R, A, lda, B, ldb, C, ldc, alpha);
+  return launch_cols_gemm<TA, TB, MO, 128>(st, R, A, lda, B, ldb, C, ldc, alpha);
+}
+
 // Where a product runs: the stream, and whether on the tensor cores (TF32) or on the FP32 ALUs.
 struct GemmCtx {
   cudaStream_t st;
@@ -408,6 +521,10 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
     if (N == 32) return launch_rows_gemm<TA, TB, 32>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
     if (N == 64) return launch_rows_gemm<TA, TB, 64>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
     return launch_rows_gemm<TA, TB, 128>(st, M, K, A, lda, B, ldb, tb, C, ldc, alpha, accumulate);
+  }
+  if (gx.tf32 && ta && !tb && split_k && batch == 1 && cols_gemm_fits<TA, TB>(M, N, K, A, lda, B, ldb)) {
+    if (M == 64) return launch_cols_gemm_n<TA, TB, 64>(st, N, K, A, lda, B, ldb, C, ldc, alpha);
+    return launch_cols_gemm_n<TA, TB, 128>(st, N, K, A, lda, B, ldb, C, ldc, alpha);
   }
   const int kstep = gx.tf32 ? kWK : kTK;
   int splits = 1, per = K;
