@@ -1079,7 +1079,8 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
                float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor) {
   const int N = p.N, d = p.d, H = p.H, Lp = p.Lp, M = p.M, dqk = p.dqk, dvh = p.dvh, U = p.U, L = p.L;
   const size_t UL = (size_t)U * L;
-  LASER_CUDA_OK(cudaMemsetAsync(d_items, 0, UL * d * sizeof(float), st));
+  // (d_items: with candidates present its first matrix product writes every row, padding included)
+  if (N == 0 || U == 0) LASER_CUDA_OK(cudaMemsetAsync(d_items, 0, UL * d * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(dWq, 0, (size_t)d * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(dWk, 0, (size_t)d * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(dWv, 0, (size_t)d * d * sizeof(float), st));
@@ -1097,7 +1098,8 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   char* mma_scratch = ws + p.total + s.total;
   const bool mma = tensor && sta_bwd_mma_supported(p);     // (users with very few candidates keep the FP32 gate kernels)
   if (tensor) {
-    LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
+    // (sta_fwd_mma writes every row of H' that is read later: all candidates of every non-empty segment)
+    if (!(mma && sta_fwd_mma_supported(p))) LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
     // projections as three matrix products over all rows (padding rows included: their K and V are never read)
     BWD_OK(gemm<T, T>(gx, N, dqk, d, cands, d, false, Wq, dqk, false, Qf, dqk, p.inv_gamma, false, false));
     BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
