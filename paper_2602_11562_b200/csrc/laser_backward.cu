@@ -674,14 +674,17 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
       for (int k = 0; k < 4; ++k)
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
+      const float* sp = s + (size_t)warp * d + x;          // row j of the segment vectors, and column j of the weights
+      const float* ep = e + h0 * Lp + warp;
+      const int heads = min(4, H - h0);
 #pragma unroll 2
-      for (int j = warp; j < nv; j += nw) {
+      for (int j = warp; j < nv; j += nw, sp += nw * d, ep += nw) {
         float sv[VEC];
-        load_vec<VEC>(sv, s + (size_t)j * d + x);
+        load_vec<VEC>(sv, sp);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) {
-            const float a = e[(h0 + k) * Lp + j];
+          if (k < heads) {
+            const float a = ep[k * Lp];
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(a, sv[v], acc[k][v]);
           }
@@ -749,14 +752,17 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
       for (int k = 0; k < 4; ++k)
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
+      const int heads = min(4, H - h0);
+      const float* sp = s + (size_t)warp * d + x;
+      const float* dep = de + h0 * Lp + warp;
 #pragma unroll 2
-      for (int j = warp; j < nv; j += nw) {
+      for (int j = warp; j < nv; j += nw, sp += nw * d, dep += nw) {
         float sv[VEC];
-        load_vec<VEC>(sv, s + (size_t)j * d + x);
+        load_vec<VEC>(sv, sp);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) {
-            const float dej = de[(h0 + k) * Lp + j];
+          if (k < heads) {
+            const float dej = dep[k * Lp];
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(dej, sv[v], acc[k][v]);
           }
@@ -775,11 +781,14 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
           load_vec<VEC>(mx[k], dm + (h0 + k) * d + x);
         }
       }
+      float* out = dS + (size_t)warp * d + x;
+      const float* ap = a + h0 * Lp + warp;
+      dep = de + h0 * Lp + warp;
+      const bool fresh = overwrite && h0 == 0;
 #pragma unroll 2
-      for (int j = warp; j < nv; j += nw) {
+      for (int j = warp; j < nv; j += nw, out += nw * d, dep += nw, ap += nw) {
         float g[VEC];
-        float* out = dS + (size_t)j * d + x;
-        if (overwrite && h0 == 0) {
+        if (fresh) {
 #pragma unroll
           for (int v = 0; v < VEC; ++v) g[v] = 0.f;
         } else {
@@ -787,8 +796,8 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          if (h0 + k < H) {
-            const float dej = de[(h0 + k) * Lp + j], aj = a[(h0 + k) * Lp + j];
+          if (k < heads) {
+            const float dej = dep[k * Lp], aj = ap[k * Lp];
 #pragma unroll
             for (int v = 0; v < VEC; ++v) g[v] = fmaf(dej, qx[k][v], fmaf(aj, mx[k][v], g[v]));
           }
