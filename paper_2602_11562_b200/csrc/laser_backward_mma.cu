@@ -55,7 +55,7 @@ struct BwdMmaParams {
 };
 
 template <int MT, int DQ16, int DV16>
-__global__ void __launch_bounds__(kBwdWarps * 32) sta_bwd_mma_kernel(const BwdMmaParams P) {
+__global__ void __launch_bounds__(kBwdWarps * 32, 2) sta_bwd_mma_kernel(const BwdMmaParams P) {
   constexpr int DQH = 16 * DQ16, DVH = 16 * DV16;
   constexpr int QS = 2 * DQH + 16, DS = 2 * DVH + 16;          // bytes per staged row (padding: conflict-free ldmatrix)
   constexpr int kBuf = 16 * (QS + DS);                         // one staging buffer: 16 candidate rows of Qb_h and ds_i,h
@@ -167,52 +167,46 @@ __global__ void __launch_bounds__(kBwdWarps * 32) sta_bwd_mma_kernel(const BwdMm
     __syncwarp();
     const uint32_t base = stage0 + (s & 1) * kBuf;
 
-    // scores^T / 2 and dG^T: [items] x [16 candidates]
-    float E[MT][2][4], G[MT][2][4];
+    // scores^T / 2 and dG^T ([items] x [16 candidates]), one 16-item row tile at a time, then its gates and score
+    // gradients packed as the A operands of the products that contract over the candidates
+    uint32_t qb[DQ16][4], sb[DV16][4];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int k = 0; k < DQ16; ++k) ldsm_x4(qb[k], base + q_plain + k * 32);
+#pragma unroll
+    for (int k = 0; k < DV16; ++k) ldsm_x4(sb[k], base + s_plain + k * 32);
+    uint32_t gA[MT][4], eA[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      float E[2][4], G[2][4];
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) E[mt][nt][e] = G[mt][nt][e] = 0.f;
+        for (int e = 0; e < 4; ++e) E[nt][e] = G[nt][e] = 0.f;
 #pragma unroll
-    for (int k = 0; k < DQ16; ++k) {
-      uint32_t b[4];
-      ldsm_x4(b, base + q_plain + k * 32);
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        mma16816(E[mt][0], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], b[0], b[1]);
-        mma16816(E[mt][1], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], b[2], b[3]);
+      for (int k = 0; k < DQ16; ++k) {
+        mma16816(E[0], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], qb[k][0], qb[k][1]);
+        mma16816(E[1], Ka[mt][k][0], Ka[mt][k][1], Ka[mt][k][2], Ka[mt][k][3], qb[k][2], qb[k][3]);
       }
-    }
 #pragma unroll
-    for (int k = 0; k < DV16; ++k) {
-      uint32_t b[4];
-      ldsm_x4(b, base + s_plain + k * 32);
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        mma16816(G[mt][0], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], b[0], b[1]);
-        mma16816(G[mt][1], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], b[2], b[3]);
+      for (int k = 0; k < DV16; ++k) {
+        mma16816(G[0], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], sb[k][0], sb[k][1]);
+        mma16816(G[1], Va[mt][k][0], Va[mt][k][1], Va[mt][k][2], Va[mt][k][3], sb[k][2], sb[k][3]);
       }
-    }
-    // gates and score gradients, packed as the A operands of the products that contract over the candidates
-    uint32_t gA[MT][4], eA[MT][4];
-#pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         float gg[4], ee[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float th = tanh_fast(E[mt][nt][e]);
+          const float th = tanh_fast(E[nt][e]);
           gg[e] = fmaf(th, 0.5f, 0.5f);
-          ee[e] = G[mt][nt][e] * fmaf(-th, th, 1.f);
+          ee[e] = G[nt][e] * fmaf(-th, th, 1.f);
         }
         gA[mt][2 * nt] = pack2(gg[0], gg[1]);
         gA[mt][2 * nt + 1] = pack2(gg[2], gg[3]);
         eA[mt][2 * nt] = pack2(ee[0], ee[1]);
         eA[mt][2 * nt + 1] = pack2(ee[2], ee[3]);
       }
+    }
     // dV += g^T ds,  dK += (dG w)^T Qb
 #pragma unroll
     for (int k = 0; k < DV16; ++k) {
