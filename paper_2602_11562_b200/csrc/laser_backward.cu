@@ -599,32 +599,32 @@ __device__ __forceinline__ void store_vec(float* p, const float (&v)[VEC]) {
   else *p = v[0];
 }
 
-// dot[k] = s_j . W[h0 + k] for four heads at a time, W = [H][d] in shared memory; lanes split the features.
-template <int VEC>
+// dot[k] = s_j . W[h0 + k] for HG heads at a time (HG = 4, 2 or 1 divides H: no head of a group is ever missing),
+// W = [H][d] in shared memory; lanes split the features.
+template <int VEC, int HG>
 __device__ __forceinline__ void row_dots(const float* __restrict__ sj, const float* __restrict__ W, int d, int H, int h0,
-                                         int lane, float (&dot)[4]) {
+                                         int lane, float (&dot)[HG]) {
 #pragma unroll
-  for (int k = 0; k < 4; ++k) dot[k] = 0.f;
+  for (int k = 0; k < HG; ++k) dot[k] = 0.f;
   for (int x = VEC * lane; x < d; x += 32 * VEC) {
     float sv[VEC];
     load_vec<VEC>(sv, sj + x);
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
-      if (h0 + k < H) {
-        float wv[VEC];
-        load_vec<VEC>(wv, W + (h0 + k) * d + x);
+    for (int k = 0; k < HG; ++k) {
+      float wv[VEC];
+      load_vec<VEC>(wv, W + (h0 + k) * d + x);
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) dot[k] = fmaf(sv[v], wv[v], dot[k]);
-      }
+      for (int v = 0; v < VEC; ++v) dot[k] = fmaf(sv[v], wv[v], dot[k]);
+    }
   }
 #pragma unroll
-  for (int k = 0; k < 4; ++k) dot[k] = warp_sum(dot[k]);
+  for (int k = 0; k < HG; ++k) dot[k] = warp_sum(dot[k]);
 }
 
 // One block per candidate: e_{j,h} = s_j . Qt_h (Qt holds W_k[:, h] Q_h / tau), a = softmax over the non-empty segments,
 // m_h = sum_j a_{j,h} s_j.  Writes a [N, H, Lp] and m [N, H, d].  The warps split the segments (a warp reads a segment
-// vector once for four heads, each lane VEC consecutive features); the per-warp partial sums of m meet in shared memory.
-template <int VEC>
+// vector once for HG heads, each lane VEC consecutive features); the per-warp partial sums of m meet in shared memory.
+template <int VEC, int HG>
 __global__ void __launch_bounds__(kAttnThreads)
 gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const int* __restrict__ lengths,
                      const int* __restrict__ cand_offsets, float* __restrict__ Aw, float* __restrict__ Mh, int U, int L,
@@ -640,12 +640,12 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   for (int i = tid; i < H * d; i += kAttnThreads) qt[i] = Qt[(size_t)c * H * d + i];
   __syncthreads();
   for (int j = warp; j < nv; j += nw)
-    for (int h0 = 0; h0 < H; h0 += 4) {
-      float dot[4];
-      row_dots<VEC>(s + (size_t)j * d, qt, d, H, h0, lane, dot);
+    for (int h0 = 0; h0 < H; h0 += HG) {
+      float dot[HG];
+      row_dots<VEC, HG>(s + (size_t)j * d, qt, d, H, h0, lane, dot);
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (lane == 0 && h0 + k < H) e[(h0 + k) * Lp + j] = dot[k];
+      for (int k = 0; k < HG; ++k)
+        if (lane == 0) e[(h0 + k) * Lp + j] = dot[k];
     }
   __syncthreads();
   for (int h = warp; h < H; h += nw) {
@@ -668,30 +668,28 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   }
   __syncthreads();
   for (int x = VEC * lane; x < d; x += 32 * VEC)
-    for (int h0 = 0; h0 < H; h0 += 4) {
-      float acc[4][VEC];
+    for (int h0 = 0; h0 < H; h0 += HG) {
+      float acc[HG][VEC];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
+      for (int k = 0; k < HG; ++k)
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
       const float* sp = s + (size_t)warp * d + x;          // row j of the segment vectors, and column j of the weights
       const float* ep = e + h0 * Lp + warp;
-      const int heads = min(4, H - h0);
 #pragma unroll 2
       for (int j = warp; j < nv; j += nw, sp += nw * d, ep += nw) {
         float sv[VEC];
         load_vec<VEC>(sv, sp);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (k < heads) {
-            const float a = ep[k * Lp];
+        for (int k = 0; k < HG; ++k) {
+          const float a = ep[k * Lp];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(a, sv[v], acc[k][v]);
-          }
+          for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(a, sv[v], acc[k][v]);
+        }
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (h0 + k < H) store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
+      for (int k = 0; k < HG; ++k)
+        store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
     }
   __syncthreads();
   for (int i = tid; i < H * d; i += kAttnThreads) {
@@ -705,7 +703,7 @@ gsta_attn_fwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
 // One block per candidate: the backward of the kernel above.  dM = dLoss/dm [N, H, d] in; dQt = dLoss/dQt [N, H, d] out;
 // dHp [N, Lp, d] accumulates dLoss/ds_j over the layers: the layer processed first (overwrite != 0) writes every entry
 // (zeros for the empty segments), the others add.  Same split of the work as in the forward kernel.
-template <int VEC>
+template <int VEC, int HG>
 __global__ void __launch_bounds__(kAttnThreads)
 gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt, const float* __restrict__ Aw,
                      const float* __restrict__ dM, const int* __restrict__ lengths, const int* __restrict__ cand_offsets,
@@ -728,12 +726,12 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   for (int i = tid; i < H * Lp; i += kAttnThreads) a[i] = Aw[(size_t)c * H * Lp + i];
   __syncthreads();
   for (int j = warp; j < nv; j += nw)
-    for (int h0 = 0; h0 < H; h0 += 4) {
-      float dot[4];
-      row_dots<VEC>(s + (size_t)j * d, dm, d, H, h0, lane, dot);
+    for (int h0 = 0; h0 < H; h0 += HG) {
+      float dot[HG];
+      row_dots<VEC, HG>(s + (size_t)j * d, dm, d, H, h0, lane, dot);
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (lane == 0 && h0 + k < H) de[(h0 + k) * Lp + j] = dot[k];
+      for (int k = 0; k < HG; ++k)
+        if (lane == 0) de[(h0 + k) * Lp + j] = dot[k];
     }
   __syncthreads();
   for (int h = warp; h < H; h += nw) {
@@ -745,14 +743,13 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
   __syncthreads();
   float* dS = dHp + (size_t)c * Lp * d;
   for (int x = VEC * lane; x < d; x += 32 * VEC) {
-    for (int h0 = 0; h0 < H; h0 += 4) {
+    for (int h0 = 0; h0 < H; h0 += HG) {
       // dQt_h[x] = sum_j de_{j,h} s_j[x]: this warp's segments
-      float acc[4][VEC];
+      float acc[HG][VEC];
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
+      for (int k = 0; k < HG; ++k)
 #pragma unroll
         for (int v = 0; v < VEC; ++v) acc[k][v] = 0.f;
-      const int heads = min(4, H - h0);
       const float* sp = s + (size_t)warp * d + x;
       const float* dep = de + h0 * Lp + warp;
 #pragma unroll 2
@@ -760,26 +757,21 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
         float sv[VEC];
         load_vec<VEC>(sv, sp);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (k < heads) {
-            const float dej = dep[k * Lp];
+        for (int k = 0; k < HG; ++k) {
+          const float dej = dep[k * Lp];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(dej, sv[v], acc[k][v]);
-          }
+          for (int v = 0; v < VEC; ++v) acc[k][v] = fmaf(dej, sv[v], acc[k][v]);
+        }
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (h0 + k < H) store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
+      for (int k = 0; k < HG; ++k)
+        store_vec<VEC>(red + ((size_t)warp * H + h0 + k) * d + x, acc[k]);
       // ds_j[x] += sum_h de_{j,h} Qt_h[x] + a_{j,h} dm_h[x]
-      float qx[4][VEC], mx[4][VEC];
+      float qx[HG][VEC], mx[HG][VEC];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) qx[k][v] = mx[k][v] = 0.f;
-        if (h0 + k < H) {
-          load_vec<VEC>(qx[k], qt + (h0 + k) * d + x);
-          load_vec<VEC>(mx[k], dm + (h0 + k) * d + x);
-        }
+      for (int k = 0; k < HG; ++k) {
+        load_vec<VEC>(qx[k], qt + (h0 + k) * d + x);
+        load_vec<VEC>(mx[k], dm + (h0 + k) * d + x);
       }
       float* out = dS + (size_t)warp * d + x;
       const float* ap = a + h0 * Lp + warp;
@@ -795,12 +787,11 @@ gsta_attn_bwd_kernel(const float* __restrict__ Hp, const float* __restrict__ Qt,
           load_vec<VEC>(g, out);
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (k < heads) {
-            const float dej = dep[k * Lp], aj = ap[k * Lp];
+        for (int k = 0; k < HG; ++k) {
+          const float dej = dep[k * Lp], aj = ap[k * Lp];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) g[v] = fmaf(dej, qx[k][v], fmaf(aj, mx[k][v], g[v]));
-          }
+          for (int v = 0; v < VEC; ++v) g[v] = fmaf(dej, qx[k][v], fmaf(aj, mx[k][v], g[v]));
+        }
         store_vec<VEC>(out, g);
       }
     }
@@ -1136,8 +1127,14 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   const size_t attn_smem_f = ((size_t)(1 + attn_warps) * H * d + (size_t)H * Lp) * sizeof(float);
   const size_t attn_smem_b = ((size_t)(2 + attn_warps) * H * d + 2 * (size_t)H * Lp) * sizeof(float);
   if (attn_smem_b > 200 * 1024) return LASER_ERR_UNSUPPORTED;
-  auto attn_fwd = d % 4 == 0 ? gsta_attn_fwd_kernel<4> : gsta_attn_fwd_kernel<1>;      // 16-byte accesses when rows allow
-  auto attn_bwd = d % 4 == 0 ? gsta_attn_bwd_kernel<4> : gsta_attn_bwd_kernel<1>;
+  // 16-byte accesses when rows allow; heads in groups of four, two or one, whichever divides H
+  const bool v4 = d % 4 == 0;
+  auto attn_fwd = H % 4 == 0 ? (v4 ? gsta_attn_fwd_kernel<4, 4> : gsta_attn_fwd_kernel<1, 4>)
+                  : H % 2 == 0 ? (v4 ? gsta_attn_fwd_kernel<4, 2> : gsta_attn_fwd_kernel<1, 2>)
+                               : (v4 ? gsta_attn_fwd_kernel<4, 1> : gsta_attn_fwd_kernel<1, 1>);
+  auto attn_bwd = H % 4 == 0 ? (v4 ? gsta_attn_bwd_kernel<4, 4> : gsta_attn_bwd_kernel<1, 4>)
+                  : H % 2 == 0 ? (v4 ? gsta_attn_bwd_kernel<4, 2> : gsta_attn_bwd_kernel<1, 2>)
+                               : (v4 ? gsta_attn_bwd_kernel<4, 1> : gsta_attn_bwd_kernel<1, 1>);
   LASER_CUDA_OK(cudaFuncSetAttribute(attn_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_f));
   LASER_CUDA_OK(cudaFuncSetAttribute(attn_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_b));
   for (int l = 0; l < M; ++l) {
