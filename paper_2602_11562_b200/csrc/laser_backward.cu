@@ -1097,6 +1097,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   // ---- forward, kept in fp32: projections and H' (the FP32-ALU forward kernels), then the GSTA layers
   char* mma_scratch = ws + p.total + s.total;
   const bool mma = tensor && sta_bwd_mma_supported(p);     // (users with very few candidates keep the FP32 gate kernels)
+  const bool attn_mma = mma && gsta_attn_mma_supported(p); // the recomputed GSTA attention on the MMAs as well
   if (tensor) {
     // (sta_fwd_mma writes every row of H' that is read later: all candidates of every non-empty segment)
     if (!(mma && sta_fwd_mma_supported(p))) LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
@@ -1105,7 +1106,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
     BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
     if (mma) BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
-    if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, mma_scratch, st));
+    if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, attn_mma, mma_scratch, st));
     else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else if (p.dqh == 16 && dvh == 32 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
@@ -1144,7 +1145,9 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<float, T>(gx, N, d, d, Tl, d, false, Wql, d, false, Ql, d, 1.f, false, false));
     // Qt_h = Q_h W_k[:, h]^T / tau, every head
     BWD_OK(gemm<float, T>(gx, N, d, dvh, Ql, d, false, Wkl, d, true, Qtl, H * d, p.inv_tau, false, false, H, dvh, dvh, d));
-    {
+    if (attn_mma) {
+      BWD_OK(gsta_attn_fwd_mma(p, Qtl, lengths, cand_offsets, Al, Ml, mma_scratch, st));
+    } else {
       LaunchScope ls("bwd_attn_fwd", st);
       attn_fwd<<<N, kAttnThreads, attn_smem_f, st>>>(s.Hp, Qtl, lengths, cand_offsets, Al, Ml, U, L, p.S, Lp,
                                                                  H, d);

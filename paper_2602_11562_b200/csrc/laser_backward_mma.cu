@@ -293,7 +293,8 @@ __global__ void __launch_bounds__(kBwdWarps * 32, 2) sta_bwd_mma_kernel(const Bw
 struct FwdMmaParams {
   const bf16 *Qb, *Kb, *Vb;
   const int32_t *lengths, *cand_offsets;
-  float* Hp;
+  float* Hp;                                     // fp32 H' (null: not wanted)
+  bf16* Hb;                                      // bf16 H' for the attention kernels below (null: not wanted)
   int L, d, dqk, H, S, Lp, N, rows;              // rows = staged rows per block (min(S, L) rounded up to 16)
 };
 
@@ -372,13 +373,193 @@ __global__ void __launch_bounds__(kBwdWarps * 32) sta_fwd_mma_kernel(const FwdMm
         mma16816(acc[2 * k + 1], gA[0], gA[1], gA[2], gA[3], b[2], b[3]);
       }
     }
-    float* out = P.Hp + ((size_t)off0 * P.Lp + seg) * d + h * DVH;
-    const size_t row = (size_t)P.Lp * d;
+    const size_t at = ((size_t)off0 * P.Lp + seg) * d + h * DVH, row = (size_t)P.Lp * d;
 #pragma unroll
     for (int j = 0; j < 2 * DV16; ++j) {
       const int c = j * 8 + 2 * t;
-      if (r0 < C) *reinterpret_cast<float2*>(out + (size_t)r0 * row + c) = make_float2(acc[j][0], acc[j][1]);
-      if (r1 < C) *reinterpret_cast<float2*>(out + (size_t)r1 * row + c) = make_float2(acc[j][2], acc[j][3]);
+      if (P.Hp) {
+        if (r0 < C) *reinterpret_cast<float2*>(P.Hp + at + (size_t)r0 * row + c) = make_float2(acc[j][0], acc[j][1]);
+        if (r1 < C) *reinterpret_cast<float2*>(P.Hp + at + (size_t)r1 * row + c) = make_float2(acc[j][2], acc[j][3]);
+      }
+      if (P.Hb) {
+        if (r0 < C) *reinterpret_cast<uint32_t*>(P.Hb + at + (size_t)r0 * row + c) = pack2(acc[j][0], acc[j][1]);
+        if (r1 < C) *reinterpret_cast<uint32_t*>(P.Hb + at + (size_t)r1 * row + c) = pack2(acc[j][2], acc[j][3]);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------------------
+// The attention of a recomputed GSTA layer on the same MMAs: per candidate e_{j,h} = s_j . Qt_h, a = softmax over the
+// non-empty segments, m_h = sum_j a_{j,h} s_j, with the segment vectors in bf16 (the copy sta_fwd_mma_kernel writes), Qt
+// and the weights a rounded to bf16, fp32 accumulation.  One warp per candidate: it stages 32 segment vectors at a time
+// in its own shared memory (cp.async; rows past the candidate's last non-empty segment are zero rows) and Qt as eight head
+// rows (heads past H are zero rows); scores = S Qt^T (segments on the MMA rows, heads on the eight columns), the softmax
+// over the rows with lane-group reductions, then m^T = S^T a with S^T read by transposing ldmatrix and a taken from the
+// accumulator layout through movmatrix.  More than 32 segments: the scores of all chunks first (they stay in registers),
+// then a second pass over the chunks for m.
+constexpr int kAttnWarps = 4;
+
+__device__ __forceinline__ int nonempty_segments(const int32_t* lengths, const int32_t* cand_offsets, int U, int L, int S,
+                                                 int Lp, int c) {
+  int lo = 0, hi = U - 1;
+  while (lo < hi) {                               // the last user whose first candidate is <= c
+    const int mid = (lo + hi + 1) >> 1;
+    if (cand_offsets[mid] <= c) lo = mid; else hi = mid - 1;
+  }
+  const int len = lengths[lo];
+  if (len <= 0 || len > L) return 0;
+  return min((len + S - 1) / S, Lp);
+}
+
+struct AttnFwdParams {
+  const bf16* Hb;
+  const float* Qt;
+  const int32_t *lengths, *cand_offsets;
+  float *Aw, *Mh;
+  int N, U, L, S, Lp, H;
+};
+
+template <int D16, int NCH>
+__global__ void __launch_bounds__(kAttnWarps * 32) gsta_attn_fwd_mma_kernel(const AttnFwdParams P) {
+  constexpr int d = 16 * D16, SP = 2 * d + 16, kS = 32 * SP, kQ = 8 * SP;      // bytes: row pitch, S chunk, Qt rows
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int c = blockIdx.x * kAttnWarps + warp;
+  if (c >= P.N) return;
+  const int H = P.H, Lp = P.Lp;
+  unsigned char* mine = smem + warp * (kS + kQ);
+  const uint32_t Ssm = smem_addr(mine), Qsm = Ssm + kS;
+  for (int i = lane; i < 8 * (d / 2); i += 32) {                   // Qt rows as bf16 pairs; heads past H: zeros
+    const int h = i / (d / 2), x2 = i - h * (d / 2);
+    uint32_t v = 0u;
+    if (h < H) {
+      const float2 q = *reinterpret_cast<const float2*>(P.Qt + ((size_t)c * H + h) * d + 2 * x2);
+      v = pack2(q.x, q.y);
+    }
+    *reinterpret_cast<uint32_t*>(mine + kS + h * SP + x2 * 4) = v;
+  }
+  const int nv = nonempty_segments(P.lengths, P.cand_offsets, P.U, P.L, P.S, Lp, c);
+  const int nch = (nv + 31) >> 5;
+  const bf16* Sg = P.Hb + (size_t)c * Lp * d;
+  auto stage = [&](int ch) {
+#pragma unroll
+    for (int k = 0; k < 2 * D16; ++k) {
+      const int x = lane + 32 * k, r = x / (2 * D16), cc = x - r * (2 * D16), j = 32 * ch + r;
+      cp16(Ssm + r * SP + cc * 16, Sg + (size_t)min(j, Lp - 1) * d + cc * 8, j < nv ? 16u : 0u);
+    }
+    cp_commit();
+    cp_wait<0>();
+    __syncwarp();
+  };
+  const int mi = lane >> 3, lr = lane & 7;
+  const uint32_t a_plain = Ssm + ((mi & 1) * 8 + lr) * SP + (mi >> 1) * 16;      // A = S:   + mt 16 SP + k 32
+  const uint32_t a_trans = Ssm + ((mi >> 1) * 8 + lr) * SP + (mi & 1) * 16;      // A = S^T: + mt 16 SP + mf 32
+  const uint32_t q_rows = Qsm + lr * SP + (mi & 1) * 16;                         // B = Qt (x2): + k 32
+  float e[NCH][2][4];
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch) {
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) e[ch][mt][x] = 0.f;
+    if (ch < nch) {
+      stage(ch);
+#pragma unroll
+      for (int k = 0; k < D16; ++k) {
+        uint32_t b[2];
+        ldsm_x2(b, q_rows + k * 32);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          uint32_t a[4];
+          ldsm_x4(a, a_plain + mt * 16 * SP + k * 32);
+          mma16816(e[ch][mt], a[0], a[1], a[2], a[3], b[0], b[1]);
+        }
+      }
+      __syncwarp();
+    }
+  }
+  // softmax over the non-empty segments (rows), per head (columns 2t, 2t + 1)
+  float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const bool in = 32 * ch + 16 * mt + 8 * hf + g < nv;
+        if (!in) e[ch][mt][2 * hf] = e[ch][mt][2 * hf + 1] = -INFINITY;
+        mx0 = fmaxf(mx0, e[ch][mt][2 * hf]);
+        mx1 = fmaxf(mx1, e[ch][mt][2 * hf + 1]);
+      }
+  mx0 = group_max(mx0);
+  mx1 = group_max(mx1);
+  float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const float p0 = nv > 0 ? expf(e[ch][mt][2 * hf] - mx0) : 0.f, p1 = nv > 0 ? expf(e[ch][mt][2 * hf + 1] - mx1) : 0.f;
+        e[ch][mt][2 * hf] = p0;
+        e[ch][mt][2 * hf + 1] = p1;
+        sum0 += p0;
+        sum1 += p1;
+      }
+  sum0 = group_sum(sum0);
+  sum1 = group_sum(sum1);
+  const float inv0 = sum0 > 0.f ? 1.f / sum0 : 0.f, inv1 = sum1 > 0.f ? 1.f / sum1 : 0.f;
+  float* Aw = P.Aw + (size_t)c * H * Lp;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int j = 32 * ch + 16 * mt + 8 * hf + g;
+        const float a0 = e[ch][mt][2 * hf] * inv0, a1 = e[ch][mt][2 * hf + 1] * inv1;
+        e[ch][mt][2 * hf] = a0;
+        e[ch][mt][2 * hf + 1] = a1;
+        if (j < Lp) {
+          if (2 * t < H) Aw[(size_t)(2 * t) * Lp + j] = a0;
+          if (2 * t + 1 < H) Aw[(size_t)(2 * t + 1) * Lp + j] = a1;
+        }
+      }
+  // m^T [features] x [heads] = S^T a
+  float macc[D16][4];
+#pragma unroll
+  for (int mf = 0; mf < D16; ++mf)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) macc[mf][x] = 0.f;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch) {
+    if (ch < nch) {
+      if (nch > 1) stage(ch);                                    // (a single chunk is still there)
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint32_t b0 = movmatrix_t(pack2(e[ch][mt][0], e[ch][mt][1])), b1 = movmatrix_t(pack2(e[ch][mt][2], e[ch][mt][3]));
+#pragma unroll
+        for (int mf = 0; mf < D16; ++mf) {
+          uint32_t a[4];
+          ldsm_x4_t(a, a_trans + mt * 16 * SP + mf * 32);
+          mma16816(macc[mf], a[0], a[1], a[2], a[3], b0, b1);
+        }
+      }
+      __syncwarp();
+    }
+  }
+  float* Mh = P.Mh + (size_t)c * H * d;
+#pragma unroll
+  for (int mf = 0; mf < D16; ++mf) {
+    const int f0 = mf * 16 + g, f1 = f0 + 8;
+    if (2 * t < H) {
+      Mh[(size_t)(2 * t) * d + f0] = macc[mf][0];
+      Mh[(size_t)(2 * t) * d + f1] = macc[mf][2];
+    }
+    if (2 * t + 1 < H) {
+      Mh[(size_t)(2 * t + 1) * d + f0] = macc[mf][1];
+      Mh[(size_t)(2 * t + 1) * d + f1] = macc[mf][3];
     }
   }
 }
@@ -432,7 +613,7 @@ int cast(const float* src, bf16* dst, size_t n, float scale, cudaStream_t st) {
 }
 
 struct MmaScratch {
-  bf16 *Qb, *Kb, *Vb, *dSb;
+  bf16 *Qb, *Kb, *Vb, *dSb, *Hb;
   size_t total;
 };
 MmaScratch carve_mma(const Plan& p, char* base) {
@@ -448,6 +629,7 @@ MmaScratch carve_mma(const Plan& p, char* base) {
   s.Kb = take(UL * p.dqk);
   s.Vb = take(UL * p.d);
   s.dSb = take((size_t)p.N * p.Lp * p.d);
+  s.Hb = take((size_t)p.N * p.Lp * p.d);
   s.total = off;
   return s;
 }
@@ -476,7 +658,35 @@ bool sta_fwd_mma_supported(const Plan& p) {
   return sta_bwd_mma_supported(p) && fwd_smem(p) <= kFwdSmemMax && (long long)p.Lp * p.H <= 0x7fffffffLL;
 }
 
-int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, char* scratch,
+bool gsta_attn_mma_supported(const Plan& p) {
+  return sta_fwd_mma_supported(p) && (p.d == 32 || p.d == 64 || p.d == 128) && p.H <= 8 && p.Lp <= 128;
+}
+
+template <int D16>
+int launch_attn_fwd(const AttnFwdParams& P, cudaStream_t st) {
+  constexpr size_t smem = (size_t)kAttnWarps * 40 * (2 * 16 * D16 + 16);
+  const int nch = (P.Lp + 31) / 32;
+  auto kernel = nch <= 1 ? gsta_attn_fwd_mma_kernel<D16, 1> : nch <= 2 ? gsta_attn_fwd_mma_kernel<D16, 2> : gsta_attn_fwd_mma_kernel<D16, 4>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LaunchScope ls("bwd_attn_fwd_mma", st);
+  kernel<<<(P.N + kAttnWarps - 1) / kAttnWarps, kAttnWarps * 32, smem, st>>>(P);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+int gsta_attn_fwd_mma(const Plan& p, const float* Qt, const int32_t* lengths, const int32_t* cand_offsets, float* Aw,
+                      float* Mh, char* scratch, cudaStream_t st) {
+  const MmaScratch s = carve_mma(p, scratch);
+  AttnFwdParams P;
+  P.Hb = s.Hb; P.Qt = Qt; P.lengths = lengths; P.cand_offsets = cand_offsets; P.Aw = Aw; P.Mh = Mh;
+  P.N = p.N; P.U = p.U; P.L = p.L; P.S = p.S; P.Lp = p.Lp; P.H = p.H;
+  if (p.d == 32) return launch_attn_fwd<2>(P, st);
+  if (p.d == 64) return launch_attn_fwd<4>(P, st);
+  if (p.d == 128) return launch_attn_fwd<8>(P, st);
+  return LASER_ERR_UNSUPPORTED;
+}
+
+int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, bool bf16_copy, char* scratch,
                 cudaStream_t st) {
   MmaShape sh;
   if (!mma_shape(p, &sh) || !sta_fwd_mma_supported(p)) return LASER_ERR_UNSUPPORTED;
@@ -485,6 +695,7 @@ int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offse
   P.Qb = s.Qb; P.Kb = s.Kb; P.Vb = s.Vb;
   P.lengths = lengths; P.cand_offsets = cand_offsets;
   P.Hp = Hp;
+  P.Hb = bf16_copy ? s.Hb : nullptr;
   P.L = p.L; P.d = p.d; P.dqk = p.dqk; P.H = p.H; P.S = p.S; P.Lp = p.Lp; P.N = p.N;
   P.rows = (std::min(p.S, p.L) + 15) / 16 * 16;
   const size_t smem = fwd_smem(p);

@@ -94,8 +94,13 @@ bool sta_bwd_mma_supported(const Plan& p);
 bool sta_fwd_mma_supported(const Plan& p);
 size_t sta_bwd_mma_scratch_bytes(const Plan& p);
 int sta_mma_operands(const Plan& p, const float* Qf, const float* Kf, const float* Vf, char* scratch, cudaStream_t st);
-int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, char* scratch,
+int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, bool bf16_copy, char* scratch,
                 cudaStream_t st);
+// The attention of a recomputed GSTA layer on the bf16 copy of H' that sta_fwd_mma keeps (bf16_copy): writes the weights
+// Aw [N, H, Lp] and the weighted sums Mh [N, H, d] (fp32) from Qt [N, H, d].
+bool gsta_attn_mma_supported(const Plan& p);
+int gsta_attn_fwd_mma(const Plan& p, const float* Qt, const int32_t* lengths, const int32_t* cand_offsets, float* Aw,
+                      float* Mh, char* scratch, cudaStream_t st);
 int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const int32_t* cand_offsets, float* dQf,
                 float* dK, float* dV, char* scratch, cudaStream_t st);
 
