@@ -1168,7 +1168,9 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     // dW_v[:, h] += m_h^T do_h;  dm_h = do_h W_v[:, h]^T, every head
     BWD_OK(gemm<float, float>(gx, d, dvh, N, Ml, H * d, true, s.dT, d, false, gWv, d, 1.f, true, true, H, d, dvh, dvh));
     BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT, d, false, Wvl, d, true, s.dM, H * d, 1.f, false, false, H, dvh, dvh, d));
-    {
+    if (attn_mma) {
+      BWD_OK(gsta_attn_bwd_mma(p, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp, l == M - 1, mma_scratch, st));
+    } else {
       LaunchScope ls("bwd_attn_bwd", st);
       attn_bwd<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
                                                                  U, L, p.S, Lp, H, d, l == M - 1 ? 1 : 0);

@@ -564,6 +564,182 @@ __global__ void __launch_bounds__(kAttnWarps * 32) gsta_attn_fwd_mma_kernel(cons
   }
 }
 
+// The backward of the kernel above, same layout of the work: da_{j,h} = s_j . dm_h (S dm^T), de = a (da - sum_j a da),
+// dQt_h = sum_j de_{j,h} s_j (S^T de, de through movmatrix), and the update of dH', ds_j += sum_h de_{j,h} Qt_h + a_{j,h} dm_h,
+// as one product [de | a] [Qt ; dm] per 16 segments: its A operand is the two accumulator-layout tiles side by side
+// (eight de heads, eight a heads), its B operand Qt and dm read by transposing ldmatrix.  The layer processed first
+// writes dH' (zeros for the empty segments), the others add.
+struct AttnBwdParams {
+  const bf16* Hb;
+  const float *Qt, *dM, *Aw;
+  const int32_t *lengths, *cand_offsets;
+  float *dQt, *dHp;
+  int N, U, L, S, Lp, H, overwrite;
+};
+
+template <int D16, int NCH>
+__global__ void __launch_bounds__(kAttnWarps * 32) gsta_attn_bwd_mma_kernel(const AttnBwdParams P) {
+  constexpr int d = 16 * D16, SP = 2 * d + 16, kS = 32 * SP, kQ = 8 * SP;
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int c = blockIdx.x * kAttnWarps + warp;
+  if (c >= P.N) return;
+  const int H = P.H, Lp = P.Lp;
+  unsigned char* mine = smem + warp * (kS + 2 * kQ);
+  const uint32_t Ssm = smem_addr(mine), Qsm = Ssm + kS, Msm = Qsm + kQ;
+  for (int i = lane; i < 8 * (d / 2); i += 32) {                   // Qt and dm rows as bf16 pairs; heads past H: zeros
+    const int h = i / (d / 2), x2 = i - h * (d / 2);
+    uint32_t vq = 0u, vm = 0u;
+    if (h < H) {
+      const float2 q = *reinterpret_cast<const float2*>(P.Qt + ((size_t)c * H + h) * d + 2 * x2);
+      const float2 m = *reinterpret_cast<const float2*>(P.dM + ((size_t)c * H + h) * d + 2 * x2);
+      vq = pack2(q.x, q.y);
+      vm = pack2(m.x, m.y);
+    }
+    *reinterpret_cast<uint32_t*>(mine + kS + h * SP + x2 * 4) = vq;
+    *reinterpret_cast<uint32_t*>(mine + kS + kQ + h * SP + x2 * 4) = vm;
+  }
+  const int nv = nonempty_segments(P.lengths, P.cand_offsets, P.U, P.L, P.S, Lp, c);
+  const int nch = (nv + 31) >> 5;
+  const bf16* Sg = P.Hb + (size_t)c * Lp * d;
+  auto stage = [&](int ch) {
+#pragma unroll
+    for (int k = 0; k < 2 * D16; ++k) {
+      const int x = lane + 32 * k, r = x / (2 * D16), cc = x - r * (2 * D16), j = 32 * ch + r;
+      cp16(Ssm + r * SP + cc * 16, Sg + (size_t)min(j, Lp - 1) * d + cc * 8, j < nv ? 16u : 0u);
+    }
+    cp_commit();
+    cp_wait<0>();
+    __syncwarp();
+  };
+  const int mi = lane >> 3, lr = lane & 7;
+  const uint32_t a_plain = Ssm + ((mi & 1) * 8 + lr) * SP + (mi >> 1) * 16;
+  const uint32_t a_trans = Ssm + ((mi >> 1) * 8 + lr) * SP + (mi & 1) * 16;
+  const uint32_t m_rows = Msm + lr * SP + (mi & 1) * 16;                          // B = dm (x2): + k 32
+  const uint32_t qm_trans = ((mi & 1) ? Msm : Qsm) + lr * SP + (mi >> 1) * 16;    // B = [Qt ; dm]^T: + 32 per 16 features
+  // the weights a in the accumulator layout (rows = segments g, g + 8; columns = heads 2t, 2t + 1)
+  float a[NCH][2][4], de[NCH][2][4];
+  const float* Aw = P.Aw + (size_t)c * H * Lp;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int j = 32 * ch + 16 * mt + 8 * (x >> 1) + g, h = 2 * t + (x & 1);
+        a[ch][mt][x] = (j < nv && h < H) ? Aw[(size_t)h * Lp + j] : 0.f;
+        de[ch][mt][x] = 0.f;
+      }
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+    if (ch < nch) {
+      stage(ch);
+#pragma unroll
+      for (int k = 0; k < D16; ++k) {
+        uint32_t b[2];
+        ldsm_x2(b, m_rows + k * 32);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          uint32_t af[4];
+          ldsm_x4(af, a_plain + mt * 16 * SP + k * 32);
+          mma16816(de[ch][mt], af[0], af[1], af[2], af[3], b[0], b[1]);        // (da for now)
+        }
+      }
+      __syncwarp();
+    }
+  float dot0 = 0.f, dot1 = 0.f;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        dot0 = fmaf(a[ch][mt][2 * hf], de[ch][mt][2 * hf], dot0);
+        dot1 = fmaf(a[ch][mt][2 * hf + 1], de[ch][mt][2 * hf + 1], dot1);
+      }
+  dot0 = group_sum(dot0);
+  dot1 = group_sum(dot1);
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        de[ch][mt][2 * hf] = a[ch][mt][2 * hf] * (de[ch][mt][2 * hf] - dot0);
+        de[ch][mt][2 * hf + 1] = a[ch][mt][2 * hf + 1] * (de[ch][mt][2 * hf + 1] - dot1);
+      }
+  float qacc[D16][4];
+#pragma unroll
+  for (int mf = 0; mf < D16; ++mf)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) qacc[mf][x] = 0.f;
+  float* dS = P.dHp + (size_t)c * Lp * d;
+#pragma unroll
+  for (int ch = 0; ch < NCH; ++ch)
+    if (ch < nch) {
+      if (nch > 1) stage(ch);
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint32_t e0 = pack2(de[ch][mt][0], de[ch][mt][1]), e1 = pack2(de[ch][mt][2], de[ch][mt][3]);
+        const uint32_t w0 = pack2(a[ch][mt][0], a[ch][mt][1]), w1 = pack2(a[ch][mt][2], a[ch][mt][3]);
+        const uint32_t b0 = movmatrix_t(e0), b1 = movmatrix_t(e1);
+#pragma unroll
+        for (int mf = 0; mf < D16; ++mf) {
+          uint32_t af[4];
+          ldsm_x4_t(af, a_trans + mt * 16 * SP + mf * 32);
+          mma16816(qacc[mf], af[0], af[1], af[2], af[3], b0, b1);
+        }
+        // ds rows of these 16 segments: [de | a] [Qt ; dm]
+        const int j0 = 32 * ch + 16 * mt + g, j1 = j0 + 8;
+#pragma unroll
+        for (int nf = 0; nf < D16; ++nf) {
+          uint32_t b[4];
+          ldsm_x4_t(b, qm_trans + nf * 32);
+          float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
+          mma16816(c0, e0, e1, w0, w1, b[0], b[1]);
+          mma16816(c1, e0, e1, w0, w1, b[2], b[3]);
+          float* o0 = dS + (size_t)j0 * d + nf * 16 + 2 * t;
+          float* o1 = dS + (size_t)j1 * d + nf * 16 + 2 * t;
+          if (j0 < nv) {
+            float2 u = make_float2(c0[0], c0[1]), v = make_float2(c1[0], c1[1]);
+            if (!P.overwrite) {
+              const float2 pu = *reinterpret_cast<const float2*>(o0), pv = *reinterpret_cast<const float2*>(o0 + 8);
+              u.x += pu.x; u.y += pu.y; v.x += pv.x; v.y += pv.y;
+            }
+            *reinterpret_cast<float2*>(o0) = u;
+            *reinterpret_cast<float2*>(o0 + 8) = v;
+          }
+          if (j1 < nv) {
+            float2 u = make_float2(c0[2], c0[3]), v = make_float2(c1[2], c1[3]);
+            if (!P.overwrite) {
+              const float2 pu = *reinterpret_cast<const float2*>(o1), pv = *reinterpret_cast<const float2*>(o1 + 8);
+              u.x += pu.x; u.y += pu.y; v.x += pv.x; v.y += pv.y;
+            }
+            *reinterpret_cast<float2*>(o1) = u;
+            *reinterpret_cast<float2*>(o1 + 8) = v;
+          }
+        }
+      }
+      __syncwarp();
+    }
+  if (P.overwrite)                                                 // empty segments receive no gradient
+    for (int i = nv * (d / 4) + lane; i < Lp * (d / 4); i += 32)
+      *reinterpret_cast<float4*>(dS + (size_t)i * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+  float* dQt = P.dQt + (size_t)c * H * d;
+#pragma unroll
+  for (int mf = 0; mf < D16; ++mf) {
+    const int f0 = mf * 16 + g, f1 = f0 + 8;
+    if (2 * t < H) {
+      dQt[(size_t)(2 * t) * d + f0] = qacc[mf][0];
+      dQt[(size_t)(2 * t) * d + f1] = qacc[mf][2];
+    }
+    if (2 * t + 1 < H) {
+      dQt[(size_t)(2 * t + 1) * d + f0] = qacc[mf][1];
+      dQt[(size_t)(2 * t + 1) * d + f1] = qacc[mf][3];
+    }
+  }
+}
+
 struct MmaShape {
   int mt, dq16, dv16;
 };
@@ -683,6 +859,30 @@ int gsta_attn_fwd_mma(const Plan& p, const float* Qt, const int32_t* lengths, co
   if (p.d == 32) return launch_attn_fwd<2>(P, st);
   if (p.d == 64) return launch_attn_fwd<4>(P, st);
   if (p.d == 128) return launch_attn_fwd<8>(P, st);
+  return LASER_ERR_UNSUPPORTED;
+}
+
+template <int D16>
+int launch_attn_bwd(const AttnBwdParams& P, cudaStream_t st) {
+  constexpr size_t smem = (size_t)kAttnWarps * 48 * (2 * 16 * D16 + 16);
+  const int nch = (P.Lp + 31) / 32;
+  auto kernel = nch <= 1 ? gsta_attn_bwd_mma_kernel<D16, 1> : nch <= 2 ? gsta_attn_bwd_mma_kernel<D16, 2> : gsta_attn_bwd_mma_kernel<D16, 4>;
+  LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LaunchScope ls("bwd_attn_bwd_mma", st);
+  kernel<<<(P.N + kAttnWarps - 1) / kAttnWarps, kAttnWarps * 32, smem, st>>>(P);
+  LASER_CUDA_OK(cudaGetLastError());
+  return LASER_OK;
+}
+
+int gsta_attn_bwd_mma(const Plan& p, const float* Qt, const float* Aw, const float* dM, const int32_t* lengths,
+                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, char* scratch, cudaStream_t st) {
+  const MmaScratch s = carve_mma(p, scratch);
+  AttnBwdParams P;
+  P.Hb = s.Hb; P.Qt = Qt; P.dM = dM; P.Aw = Aw; P.lengths = lengths; P.cand_offsets = cand_offsets; P.dQt = dQt; P.dHp = dHp;
+  P.N = p.N; P.U = p.U; P.L = p.L; P.S = p.S; P.Lp = p.Lp; P.H = p.H; P.overwrite = overwrite ? 1 : 0;
+  if (p.d == 32) return launch_attn_bwd<2>(P, st);
+  if (p.d == 64) return launch_attn_bwd<4>(P, st);
+  if (p.d == 128) return launch_attn_bwd<8>(P, st);
   return LASER_ERR_UNSUPPORTED;
 }
 

@@ -101,6 +101,9 @@ int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offse
 bool gsta_attn_mma_supported(const Plan& p);
 int gsta_attn_fwd_mma(const Plan& p, const float* Qt, const int32_t* lengths, const int32_t* cand_offsets, float* Aw,
                       float* Mh, char* scratch, cudaStream_t st);
+// Its backward: dQt [N, H, d] from Qt, Aw and dM [N, H, d]; dHp [N, Lp, d] written (overwrite) or added to.
+int gsta_attn_bwd_mma(const Plan& p, const float* Qt, const float* Aw, const float* dM, const int32_t* lengths,
+                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, char* scratch, cudaStream_t st);
 int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const int32_t* cand_offsets, float* dQf,
                 float* dK, float* dV, char* scratch, cudaStream_t st);
 
