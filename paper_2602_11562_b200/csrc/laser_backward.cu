@@ -1106,7 +1106,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
     BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
     if (mma) BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
-    if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, s.Hp, attn_mma, mma_scratch, st));
+    if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, attn_mma ? nullptr : s.Hp, attn_mma, mma_scratch, st));
     else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else if (p.dqh == 16 && dvh == 32 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else BWD_OK(simt_sta_f32(p, items, lengths, cands, cand_offsets, Wq, Wk, Wv, s.Hp, ws, st));
@@ -1169,7 +1169,7 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     BWD_OK(gemm<float, float>(gx, d, dvh, N, Ml, H * d, true, s.dT, d, false, gWv, d, 1.f, true, true, H, d, dvh, dvh));
     BWD_OK(gemm<float, T>(gx, N, d, dvh, s.dT, d, false, Wvl, d, true, s.dM, H * d, 1.f, false, false, H, dvh, dvh, d));
     if (attn_mma) {
-      BWD_OK(gsta_attn_bwd_mma(p, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp, l == M - 1, mma_scratch, st));
+      BWD_OK(gsta_attn_bwd_mma(p, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp, l == M - 1, l == 0, mma_scratch, st));
     } else {
       LaunchScope ls("bwd_attn_bwd", st);
       attn_bwd<<<N, kAttnThreads, attn_smem_b, st>>>(s.Hp, Qtl, Al, s.dM, lengths, cand_offsets, s.dQt, s.dHp,
@@ -1187,7 +1187,8 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
   LASER_CUDA_OK(cudaMemsetAsync(s.dK, 0, UL * dqk * sizeof(float), st));
   LASER_CUDA_OK(cudaMemsetAsync(s.dV, 0, UL * d * sizeof(float), st));
   if (mma) {
-    BWD_OK(sta_bwd_mma(p, s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, mma_scratch, st));
+    // (with the attention on the MMAs and at least one layer, dH' has arrived in bf16 already)
+    BWD_OK(sta_bwd_mma(p, attn_mma && M > 0 ? nullptr : s.dHp, lengths, cand_offsets, s.dQf, s.dK, s.dV, mma_scratch, st));
   } else {
     const int cps = (min(p.S, L) + kChunk - 1) / kChunk;
     const int dqh = dqk / H;

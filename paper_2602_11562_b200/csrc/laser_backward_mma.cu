@@ -574,6 +574,7 @@ struct AttnBwdParams {
   const float *Qt, *dM, *Aw;
   const int32_t *lengths, *cand_offsets;
   float *dQt, *dHp;
+  bf16* dSb;                                     // non-null for the layer processed last: dH' leaves as this bf16 array only
   int N, U, L, S, Lp, H, overwrite;
 };
 
@@ -674,6 +675,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) gsta_attn_bwd_mma_kernel(cons
 #pragma unroll
     for (int x = 0; x < 4; ++x) qacc[mf][x] = 0.f;
   float* dS = P.dHp + (size_t)c * Lp * d;
+  bf16* dSb = P.dSb ? P.dSb + (size_t)c * Lp * d : nullptr;
 #pragma unroll
   for (int ch = 0; ch < NCH; ++ch)
     if (ch < nch) {
@@ -698,31 +700,29 @@ __global__ void __launch_bounds__(kAttnWarps * 32) gsta_attn_bwd_mma_kernel(cons
           float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};
           mma16816(c0, e0, e1, w0, w1, b[0], b[1]);
           mma16816(c1, e0, e1, w0, w1, b[2], b[3]);
-          float* o0 = dS + (size_t)j0 * d + nf * 16 + 2 * t;
-          float* o1 = dS + (size_t)j1 * d + nf * 16 + 2 * t;
-          if (j0 < nv) {
-            float2 u = make_float2(c0[0], c0[1]), v = make_float2(c1[0], c1[1]);
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const int j = hf ? j1 : j0;
+            if (j >= nv) continue;
+            const size_t at = (size_t)j * d + nf * 16 + 2 * t;
+            float2 u = make_float2(c0[2 * hf], c0[2 * hf + 1]), v = make_float2(c1[2 * hf], c1[2 * hf + 1]);
             if (!P.overwrite) {
-              const float2 pu = *reinterpret_cast<const float2*>(o0), pv = *reinterpret_cast<const float2*>(o0 + 8);
+              const float2 pu = *reinterpret_cast<const float2*>(dS + at), pv = *reinterpret_cast<const float2*>(dS + at + 8);
               u.x += pu.x; u.y += pu.y; v.x += pv.x; v.y += pv.y;
             }
-            *reinterpret_cast<float2*>(o0) = u;
-            *reinterpret_cast<float2*>(o0 + 8) = v;
-          }
-          if (j1 < nv) {
-            float2 u = make_float2(c0[2], c0[3]), v = make_float2(c1[2], c1[3]);
-            if (!P.overwrite) {
-              const float2 pu = *reinterpret_cast<const float2*>(o1), pv = *reinterpret_cast<const float2*>(o1 + 8);
-              u.x += pu.x; u.y += pu.y; v.x += pv.x; v.y += pv.y;
+            if (dSb) {
+              *reinterpret_cast<uint32_t*>(dSb + at) = pack2(u.x, u.y);
+              *reinterpret_cast<uint32_t*>(dSb + at + 8) = pack2(v.x, v.y);
+            } else {
+              *reinterpret_cast<float2*>(dS + at) = u;
+              *reinterpret_cast<float2*>(dS + at + 8) = v;
             }
-            *reinterpret_cast<float2*>(o1) = u;
-            *reinterpret_cast<float2*>(o1 + 8) = v;
           }
         }
       }
       __syncwarp();
     }
-  if (P.overwrite)                                                 // empty segments receive no gradient
+  if (P.overwrite && !dSb)                                         // empty segments receive no gradient (their bf16 rows are never read)
     for (int i = nv * (d / 4) + lane; i < Lp * (d / 4); i += 32)
       *reinterpret_cast<float4*>(dS + (size_t)i * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
   float* dQt = P.dQt + (size_t)c * H * d;
@@ -875,9 +875,11 @@ int launch_attn_bwd(const AttnBwdParams& P, cudaStream_t st) {
 }
 
 int gsta_attn_bwd_mma(const Plan& p, const float* Qt, const float* Aw, const float* dM, const int32_t* lengths,
-                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, char* scratch, cudaStream_t st) {
+                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, bool last, char* scratch,
+                      cudaStream_t st) {
   const MmaScratch s = carve_mma(p, scratch);
   AttnBwdParams P;
+  P.dSb = last ? s.dSb : nullptr;
   P.Hb = s.Hb; P.Qt = Qt; P.dM = dM; P.Aw = Aw; P.lengths = lengths; P.cand_offsets = cand_offsets; P.dQt = dQt; P.dHp = dHp;
   P.N = p.N; P.U = p.U; P.L = p.L; P.S = p.S; P.Lp = p.Lp; P.H = p.H; P.overwrite = overwrite ? 1 : 0;
   if (p.d == 32) return launch_attn_bwd<2>(P, st);
@@ -913,7 +915,7 @@ int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const i
   if (!mma_shape(p, &sh)) return LASER_ERR_UNSUPPORTED;
   const MmaScratch s = carve_mma(p, scratch);
   int rc;
-  if ((rc = cast(dHp, s.dSb, (size_t)p.N * p.Lp * p.d, 1.f, st)) != LASER_OK) return rc;
+  if (dHp && (rc = cast(dHp, s.dSb, (size_t)p.N * p.Lp * p.d, 1.f, st)) != LASER_OK) return rc;
   BwdMmaParams P;
   P.Qb = s.Qb; P.Kb = s.Kb; P.Vb = s.Vb; P.dSb = s.dSb;
   P.lengths = lengths; P.cand_offsets = cand_offsets;

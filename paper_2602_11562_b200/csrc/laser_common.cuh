@@ -88,8 +88,8 @@ int backward(const Plan& p, const void* items, const int32_t* lengths, const voi
              float* d_cands, float* dWq, float* dWk, float* dWv, float* dWg, char* ws, cudaStream_t st, bool tensor);
 // Tensor-core kernels of the backward pass (laser_backward_mma.cu), all on bf16 copies kept in `scratch`
 // (sta_bwd_mma_scratch_bytes): sta_mma_operands makes the copies of Qf (Q / gamma), Kf and Vf; sta_fwd_mma recomputes H'
-// in fp32 from them (rows of empty segments are left as they are); sta_bwd_mma copies dHp, writes the dK / dV rows of
-// valid items (the rest must hold zeros) and adds to dQf.
+// in fp32 from them (rows of empty segments are left as they are); sta_bwd_mma copies dHp (null: the bf16 copy is there
+// already), writes the dK / dV rows of valid items (the rest must hold zeros) and adds to dQf.
 bool sta_bwd_mma_supported(const Plan& p);
 bool sta_fwd_mma_supported(const Plan& p);
 size_t sta_bwd_mma_scratch_bytes(const Plan& p);
@@ -101,9 +101,12 @@ int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offse
 bool gsta_attn_mma_supported(const Plan& p);
 int gsta_attn_fwd_mma(const Plan& p, const float* Qt, const int32_t* lengths, const int32_t* cand_offsets, float* Aw,
                       float* Mh, char* scratch, cudaStream_t st);
-// Its backward: dQt [N, H, d] from Qt, Aw and dM [N, H, d]; dHp [N, Lp, d] written (overwrite) or added to.
+// Its backward: dQt [N, H, d] from Qt, Aw and dM [N, H, d]; dHp [N, Lp, d] written (overwrite) or added to; for the
+// layer processed last the sum leaves as the bf16 array sta_bwd_mma reads (which then takes dHp = null) and dHp stays
+// as it was.
 int gsta_attn_bwd_mma(const Plan& p, const float* Qt, const float* Aw, const float* dM, const int32_t* lengths,
-                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, char* scratch, cudaStream_t st);
+                      const int32_t* cand_offsets, float* dQt, float* dHp, bool overwrite, bool last, char* scratch,
+                      cudaStream_t st);
 int sta_bwd_mma(const Plan& p, const float* dHp, const int32_t* lengths, const int32_t* cand_offsets, float* dQf,
                 float* dK, float* dV, char* scratch, cudaStream_t st);
 
