@@ -218,8 +218,9 @@ LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* ite
  *   LASER_PATH_AUTO / _STREAM       fp32 batches as above.  bf16 batches on the tensor cores: every batched matrix product
  *                                   with TF32 operands and fp32 accumulation, and, when max_cands_per_user >= 8 and the head
  *                                   widths d_qk / H and d / H are multiples of 16 (d_qk / H at most 32, d / H at most 64), the
- *                                   five contractions through the gates (and the recomputed H') with bf16 operands, as the
- *                                   forward's tensor-core path rounds them: every gradient within 2e-2 of its largest entry.
+ *                                   five contractions through the gates, the recomputed H' and (d in {32, 64, 128}, at most 8
+ *                                   heads and 128 segments) the GSTA attention with bf16 operands, as the forward's
+ *                                   tensor-core path rounds them: every gradient within 2e-2 of its largest entry.
  *   LASER_PATH_TENSOR               as LASER_PATH_AUTO for bf16 batches; LASER_ERR_UNSUPPORTED for fp32 batches.
  *   dz          [N, d] fp32            IN
  *   d_items     [U, L, d] fp32         OUT (rows of padding are zero)

@@ -4,7 +4,7 @@
 //
 // Inputs are read in their dtype, everything else is fp32.  Two versions: FP32 ALUs throughout (either dtype), and, for
 // bf16 batches, the batched matrix products on the tensor cores with TF32 operands (gemm_tf32_kernel) plus the gate
-// contractions and the recomputed H' with bf16 operands (laser_backward_mma.cu).  The forward intermediates are recomputed and kept (projections, H', and per GSTA layer
+// contractions, the recomputed H' and the GSTA attention with bf16 operands (laser_backward_mma.cu).  The forward intermediates are recomputed and kept (projections, H', and per GSTA layer
 // the running target, Q, the key-folded query Qt_h = W_k[:, h] Q_h / tau, the attention weights and the weighted sums
 // m_h = sum_j a_j s_j), all dense steps are batched matrix products over the N candidates (or the U L item rows), and
 // three kernels do what is not a matrix product:
