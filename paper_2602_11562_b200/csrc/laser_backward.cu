@@ -272,7 +272,7 @@ __device__ __forceinline__ uint32_t frag_of(const bf16* p) {
 template <typename TA, typename TB, int N>
 __global__ void __launch_bounds__(kGemmThreads)
 rows_gemm_kernel(int M, int K, const TA* __restrict__ A, int lda, const TB* __restrict__ B, int ldb, int tb,
-                 float* __restrict__ C, int ldc, float alpha, int accumulate, int n_tiles) {
+                 float* __restrict__ C, bf16* __restrict__ C16, int ldc, float alpha, int accumulate, int n_tiles) {
   constexpr int WN = N / 2, NTW = WN / 8, BP = N + 8;
   extern __shared__ __align__(16) unsigned char rg_smem[];
   uint32_t* Bs = reinterpret_cast<uint32_t*>(rg_smem);                       // [K][BP]
@@ -342,11 +342,14 @@ rows_gemm_kernel(int M, int K, const TA* __restrict__ A, int lda, const TB* __re
       for (int h = 0; h < 2; ++h) {
         const int r = r0 + mt * 16 + g + h * 8;
         if (r >= M) continue;
-        float* c = C + (size_t)r * ldc + wc + 2 * t;
+        const size_t at = (size_t)r * ldc + wc + 2 * t;
+        float* c = C + at;
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) {
           const float v0 = alpha * acc[mt][nt][2 * h], v1 = alpha * acc[mt][nt][2 * h + 1];
-          if (accumulate) {
+          if (C16) {                               // (the result is wanted as bf16 only)
+            *reinterpret_cast<uint32_t*>(C16 + at + nt * 8) = mma::pack2(v0, v1);
+          } else if (accumulate) {
             atomicAdd(c + nt * 8, v0);
             atomicAdd(c + nt * 8 + 1, v1);
           } else {
@@ -375,15 +378,15 @@ bool rows_gemm_fits(int M, int N, int K, const TA* A, int lda, const float* C, i
 
 template <typename TA, typename TB, int N>
 int launch_rows_gemm(cudaStream_t st, int M, int K, const TA* A, int lda, const TB* B, int ldb, bool tb, float* C, int ldc,
-                     float alpha, bool accumulate) {
+                     float alpha, bool accumulate, bf16* C16 = nullptr) {
   const size_t smem = (size_t)K * (N + 8) * sizeof(uint32_t) + 2 * (size_t)kRowsTile * RowsPitch<TA>::elems(K) * sizeof(TA);
   auto kernel = rows_gemm_kernel<TA, TB, N>;
   LASER_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const int n_tiles = (M + kRowsTile - 1) / kRowsTile;
   const int per_sm = smem <= 100 * 1024 ? 2 : 1;
   LaunchScope ls("bwd_gemm_rows", st);
-  kernel<<<std::min(n_tiles, per_sm * bwd_sm_count()), kGemmThreads, smem, st>>>(M, K, A, lda, B, ldb, tb ? 1 : 0, C, ldc, alpha,
-                                                                              accumulate ? 1 : 0, n_tiles);
+  kernel<<<std::min(n_tiles, per_sm * bwd_sm_count()), kGemmThreads, smem, st>>>(M, K, A, lda, B, ldb, tb ? 1 : 0, C, C16, ldc,
+                                                                              alpha, accumulate ? 1 : 0, n_tiles);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
 }
@@ -550,6 +553,18 @@ int gemm(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, bool ta, 
                                                       accumulate ? 1 : 0, per, tiles_n, sa, sb, sc);
   LASER_CUDA_OK(cudaGetLastError());
   return LASER_OK;
+}
+
+// C16 [M x N] (bf16) = A [M x K] B [K x N] on the persistent rows kernel, for results that are only ever read as bf16 MMA
+// operands; LASER_ERR_UNSUPPORTED when the shape does not fit that kernel (the caller then takes the fp32 product and a copy).
+template <typename TA, typename TB>
+int gemm_rows_bf16(const GemmCtx& gx, int M, int N, int K, const TA* A, int lda, const TB* B, int ldb, bf16* C16, int ldc) {
+  if (!gx.tf32 || !rows_gemm_fits<TA, TB>(M, N, K, A, lda, reinterpret_cast<const float*>(C16), ldc) ||
+      reinterpret_cast<uintptr_t>(C16) % 4 != 0)
+    return LASER_ERR_UNSUPPORTED;
+  if (N == 32) return launch_rows_gemm<TA, TB, 32>(gx.st, M, K, A, lda, B, ldb, false, nullptr, ldc, 1.f, false, C16);
+  if (N == 64) return launch_rows_gemm<TA, TB, 64>(gx.st, M, K, A, lda, B, ldb, false, nullptr, ldc, 1.f, false, C16);
+  return launch_rows_gemm<TA, TB, 128>(gx.st, M, K, A, lda, B, ldb, false, nullptr, ldc, 1.f, false, C16);
 }
 
 template <typename T>
@@ -1103,9 +1118,21 @@ int backward_t(const Plan& p, const T* items, const int32_t* lengths, const T* c
     if (!(mma && sta_fwd_mma_supported(p))) LASER_CUDA_OK(cudaMemsetAsync(s.Hp, 0, (size_t)N * Lp * d * sizeof(float), st));
     // projections as three matrix products over all rows (padding rows included: their K and V are never read)
     BWD_OK(gemm<T, T>(gx, N, dqk, d, cands, d, false, Wq, dqk, false, Qf, dqk, p.inv_gamma, false, false));
-    BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
-    BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
-    if (mma) BWD_OK(sta_mma_operands(p, Qf, Kf, Vf, mma_scratch, st));
+    // K and V: as bf16 straight into the MMA kernels' operand arrays when nothing reads them in fp32
+    bool kv_ready = false;
+    if (mma && sta_fwd_mma_supported(p)) {
+      bf16 *Kb, *Vb;
+      sta_mma_operand_arrays(p, mma_scratch, &Kb, &Vb);
+      const int r1 = gemm_rows_bf16<T, T>(gx, (int)UL, dqk, d, items, d, Wk, dqk, Kb, dqk);
+      const int r2 = r1 == LASER_OK ? gemm_rows_bf16<T, T>(gx, (int)UL, d, d, items, d, Wv, d, Vb, d) : r1;
+      if (r2 != LASER_OK && r2 != LASER_ERR_UNSUPPORTED) return r2;
+      kv_ready = r2 == LASER_OK;
+    }
+    if (!kv_ready) {
+      BWD_OK(gemm<T, T>(gx, (int)UL, dqk, d, items, d, false, Wk, dqk, false, Kf, dqk, 1.f, false, false));
+      BWD_OK(gemm<T, T>(gx, (int)UL, d, d, items, d, false, Wv, d, false, Vf, d, 1.f, false, false));
+    }
+    if (mma) BWD_OK(sta_mma_operands(p, Qf, kv_ready ? nullptr : Kf, kv_ready ? nullptr : Vf, mma_scratch, st));
     if (mma && sta_fwd_mma_supported(p)) BWD_OK(sta_fwd_mma(p, lengths, cand_offsets, attn_mma ? nullptr : s.Hp, attn_mma, mma_scratch, st));
     else if (p.dqh == 16 && dvh == 16 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 16>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));
     else if (p.dqh == 16 && dvh == 32 && p.H <= 32) BWD_OK(launch_sta_fwd32<16, 32>(p, Qf, Kf, Vf, lengths, cand_offsets, s.Hp, st));

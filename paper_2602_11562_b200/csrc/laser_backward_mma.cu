@@ -826,8 +826,14 @@ int sta_mma_operands(const Plan& p, const float* Qf, const float* Kf, const floa
   const size_t UL = (size_t)p.U * p.L;
   int rc;
   if ((rc = cast(Qf, s.Qb, (size_t)p.N * p.dqk, 0.5f, st)) != LASER_OK) return rc;
-  if ((rc = cast(Kf, s.Kb, UL * p.dqk, 1.f, st)) != LASER_OK) return rc;
-  return cast(Vf, s.Vb, UL * p.d, 1.f, st);
+  if (Kf && (rc = cast(Kf, s.Kb, UL * p.dqk, 1.f, st)) != LASER_OK) return rc;
+  return Vf ? cast(Vf, s.Vb, UL * p.d, 1.f, st) : (int)LASER_OK;
+}
+
+void sta_mma_operand_arrays(const Plan& p, char* scratch, __nv_bfloat16** Kb, __nv_bfloat16** Vb) {
+  const MmaScratch s = carve_mma(p, scratch);
+  *Kb = s.Kb;
+  *Vb = s.Vb;
 }
 
 bool sta_fwd_mma_supported(const Plan& p) {

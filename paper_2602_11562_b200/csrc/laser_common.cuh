@@ -94,6 +94,9 @@ bool sta_bwd_mma_supported(const Plan& p);
 bool sta_fwd_mma_supported(const Plan& p);
 size_t sta_bwd_mma_scratch_bytes(const Plan& p);
 int sta_mma_operands(const Plan& p, const float* Qf, const float* Kf, const float* Vf, char* scratch, cudaStream_t st);
+// The bf16 K [U L, d_qk] and V [U L, d] arrays inside `scratch`, for a producer that writes them directly (it then passes
+// Kf = Vf = null to sta_mma_operands).
+void sta_mma_operand_arrays(const Plan& p, char* scratch, __nv_bfloat16** Kb, __nv_bfloat16** Vb);
 int sta_fwd_mma(const Plan& p, const int32_t* lengths, const int32_t* cand_offsets, float* Hp, bool bf16_copy, char* scratch,
                 cudaStream_t st);
 // The attention of a recomputed GSTA layer on the bf16 copy of H' that sta_fwd_mma keeps (bf16_copy): writes the weights
