@@ -98,7 +98,7 @@ def test_backward_tensor_path_matches_oracle(case):
     print("backward tensor path, worst error / largest entry:", {k: f"{v:.2e}" for k, v in worst.items()})
 
 
-@pytest.mark.parametrize("name,users", [("cfg3", (0, 17, 63)), ("cfg2x32", (5, 31)), ("prod", (2, 40))])
+@pytest.mark.parametrize("name,users", [("cfg3", (0, 17, 63)), ("cfg2x32", (5, 31)), ("prod", (2, 40)), ("cfg4", (3,))])
 def test_backward_full_size_configs_sampled_users(name, users):
     # The batches the benchmark times, in its launch configuration: d_cands and d_items of a user depend on no other user,
     # so the oracle computes those users alone (seconds each); the weight gradients sum over all users and are checked on
