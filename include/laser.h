@@ -220,7 +220,9 @@ LASER_API int laser_sta_softmax_forward(const laser_config* cfg, const void* ite
  *                                   widths d_qk / H and d / H are multiples of 16 (d_qk / H at most 32, d / H at most 64), the
  *                                   five contractions through the gates, the recomputed H' and (d in {32, 64, 128}, at most 8
  *                                   heads and 128 segments) the GSTA attention with bf16 operands, as the forward's
- *                                   tensor-core path rounds them: every gradient within 2e-2 of its largest entry.
+ *                                   tensor-core path rounds them: every gradient within 2e-2 of its largest entry while the
+ *                                   attention logits stay within a few nats (at tens of nats the bf16 rounding of a
+ *                                   segment vector alone moves a softmax weight by several per cent: ask for the FP32 ALUs).
  *   LASER_PATH_TENSOR               as LASER_PATH_AUTO for bf16 batches; LASER_ERR_UNSUPPORTED for fp32 batches.
  *   dz          [N, d] fp32            IN
  *   d_items     [U, L, d] fp32         OUT (rows of padding are zero)

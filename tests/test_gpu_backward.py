@@ -27,7 +27,8 @@ CASES = [
 
 def _check(case_kw, seed, path, bar, want_kernel=None):
     kw = dict(case_kw)
-    w = make_custom(seed=seed, emb_std="one" if kw["d"] <= 32 else "inv_sqrt_d", **kw)
+    std = kw.pop("emb_std", "one" if kw["d"] <= 32 else "inv_sqrt_d")
+    w = make_custom(seed=seed, emb_std=std, **kw)
     s = w.spec
     rng = np.random.default_rng(seed + 7)
     dz = rng.standard_normal((w.N, s.d)).astype(np.float32)
@@ -96,6 +97,22 @@ TENSOR_CASES = [
 def test_backward_tensor_path_matches_oracle(case):
     worst = _check(TENSOR_CASES[case], 1200 + case, P.PATH_AUTO, TENSOR_BAR, want_kernel=True)
     print("backward tensor path, worst error / largest entry:", {k: f"{v:.2e}" for k, v in worst.items()})
+
+
+# many segments per user: the attention kernels walk them in chunks of 32 (two and four chunks, ragged last chunk)
+MANY_SEGMENTS = [
+    dict(U=2, C=9, L=200, d=64, H=4, S=2, M=2, dtype="bf16", lengths=[200, 67]),           # 100 segments, 34 non-empty
+    dict(U=2, C=12, L=640, d=128, H=8, S=5, M=1, dtype="bf16", lengths=[640, 333]),        # 128 segments, eight heads
+    # (embeddings of variance 1 / d here: with unit variance at this width the GSTA logits reach tens of nats, where the
+    # bf16 rounding of the segment vectors alone moves a softmax weight by several per cent)
+    dict(U=3, C=8, L=330, d=32, H=2, S=10, M=3, dtype="bf16", lengths=[330, 1, 0], emb_std="inv_sqrt_d"),   # 33 segments
+    dict(U=1, C=17, L=1040, d=128, H=2, S=16, M=2, dtype="bf16", lengths=[1029]),          # 65 segments, wide heads
+]
+
+
+@pytest.mark.parametrize("case", range(len(MANY_SEGMENTS)))
+def test_backward_tensor_path_many_segments(case):
+    _check(MANY_SEGMENTS[case], 1400 + case, P.PATH_AUTO, TENSOR_BAR, want_kernel=True)
 
 
 @pytest.mark.parametrize("name,users", [("cfg3", (0, 17, 63)), ("cfg2x32", (5, 31)), ("prod", (2, 40)), ("cfg4", (3,))])
